@@ -1,0 +1,80 @@
+"""Seeded synthetic inputs shared by the tests, the smoke check and the benchmark.
+
+This module only draws random tensors and runs the router (Eq. 1 of the paper: logits,
+softmax, top-k) that produces the layer's inputs `topk_ids` / `topk_weights`.  It holds
+none of the layer's own arithmetic (no quantiser, no expert MLP, no cache logic), so both
+the CUDA path and the CPU oracle can be fed from it without sharing code.
+
+Recipe (stand-in for the OLMoE checkpoint and prompts the paper measures on):
+  expert weights  N(0, 0.02) rounded to BF16          W_g, W_u: [E, I, H]   W_d: [E, H, I]
+  hidden states   N(0, 1)    rounded to BF16          [T, H]
+  router          N(0, 0.02) rounded to BF16          [E, H]
+  routing         fp32 logits (+ optional per-expert bias), softmax over all E experts,
+                  top-k by descending probability, ties to the lower expert id,
+                  weights NOT renormalised over the selected k.
+  Zipf skew       bias_e = alpha * (-1.1 * ln rank_e), rank a seeded permutation of 1..E.
+"""
+from dataclasses import dataclass
+
+import torch
+
+
+@dataclass(frozen=True)
+class Shape:
+    d_model: int
+    d_ff: int
+    num_experts: int
+    top_k: int
+    group_size: int = 128
+
+
+TINY = Shape(d_model=256, d_ff=128, num_experts=8, top_k=2)        # config 1
+OLMOE = Shape(d_model=2048, d_ff=1024, num_experts=64, top_k=8)    # configs 2-5
+MID = Shape(d_model=512, d_ff=256, num_experts=16, top_k=4)        # parity size between the two
+
+
+def _gen(seed, device="cpu"):
+    g = torch.Generator(device=device)
+    g.manual_seed(int(seed))
+    return g
+
+
+def normal_bf16(shape, std, seed, device="cpu"):
+    x = torch.randn(*shape, generator=_gen(seed, device), device=device, dtype=torch.float32)
+    return (x * std).to(torch.bfloat16)
+
+
+def expert_weights(shape: Shape, seed, device="cpu", std=0.02):
+    """(W_g [E,I,H], W_u [E,I,H], W_d [E,H,I]) in BF16."""
+    E, I, H = shape.num_experts, shape.d_ff, shape.d_model
+    wg = normal_bf16((E, I, H), std, 3 * seed + 0, device)
+    wu = normal_bf16((E, I, H), std, 3 * seed + 1, device)
+    wd = normal_bf16((E, H, I), std, 3 * seed + 2, device)
+    return wg, wu, wd
+
+
+def hidden_states(shape: Shape, T, seed, device="cpu"):
+    return normal_bf16((T, shape.d_model), 1.0, seed, device)
+
+
+def router_weights(shape: Shape, seed, device="cpu"):
+    return normal_bf16((shape.num_experts, shape.d_model), 0.02, seed, device)
+
+
+def zipf_bias(num_experts, alpha, seed):
+    """alpha * (-1.1 * ln rank_e) with rank a seeded permutation of 1..E (fp32, CPU)."""
+    perm = torch.randperm(num_experts, generator=_gen(seed))
+    rank = torch.empty(num_experts, dtype=torch.float32)
+    rank[perm] = torch.arange(1, num_experts + 1, dtype=torch.float32)
+    return alpha * (-1.1 * torch.log(rank))
+
+
+def route(hidden, w_router, top_k, bias=None):
+    """Eq. 1: logits -> softmax over all experts -> top-k.  Returns (ids int32 [T,k], p fp32 [T,k])."""
+    logits = hidden.float() @ w_router.float().t()
+    if bias is not None:
+        logits = logits + bias.to(logits.device)
+    p = torch.softmax(logits, dim=-1)
+    order = torch.sort(-p, dim=-1, stable=True).indices[:, :top_k]     # ties -> lower id
+    w = torch.gather(p, 1, order)
+    return order.to(torch.int32).contiguous(), w.contiguous()
