@@ -1,0 +1,147 @@
+/*
+ * exmoe.h - C ABI of the B200 (sm_100a) complete-expert sparse-MoE layer forward.
+ *
+ * What the library computes (ExactMoE paper, Section 3):
+ *   Eq. 2    y_t = sum_{e in TopK_t} p_{t,e} * W_d,e [ silu(W_g,e h_t) (.) W_u,e h_t ]
+ *   Eq. 3    routed expert weights are symmetric group-128 int4: s = absmax/7,
+ *            q = clip(round(W/s), -8, 7), W^ = s*q defines the arithmetic; FP16 scales.
+ *   Sec. 3.3 every layer owns C expert slots (k <= C <= E) holding the packed bytes; the same
+ *            bytes live in a pinned host bank; a miss is one asynchronous copy; LRU replacement
+ *            among slots the current wave does not use; C = E preloads and bypasses lookups.
+ *   Sec. 3.4 the active expert set is cut into waves of at most `wave_cap` experts; per wave:
+ *            resolve/load, expert map with sentinel, fused grouped gate/up GEMM + SwiGLU and down
+ *            GEMM over the complete token matrix, accumulate, completion event.
+ *
+ * Conventions
+ *   - Every entry point returns an int status: EXMOE_OK (0) or a negative EXMOE_ERR_* code.
+ *     Nothing throws, aborts or traps the device.  exmoe_strerror() names a code.
+ *   - "dev" pointers are device memory of the current CUDA device, "host" pointers are host
+ *     memory.  `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).
+ *   - The caller owns every buffer it passes (tensors, slot memory, workspace, host bank) and
+ *     must keep them alive while the cache exists.  The library owns only its host bookkeeping,
+ *     one copy stream, its events and a small pinned staging buffer.
+ *   - BF16 tensors are row-major, dense.  ids are int32, mixture weights are float32.
+ *   - All calls on one cache must come from one host thread at a time.
+ */
+#ifndef EXMOE_H
+#define EXMOE_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+enum {
+    EXMOE_OK = 0,
+    EXMOE_ERR_ARG = -1,           /* null pointer, negative size, T > max_tokens, layer out of range */
+    EXMOE_ERR_SHAPE = -2,         /* d_model or d_ff not a multiple of 128, group_size != 128,
+                                     top_k > num_slots, num_slots > num_experts, ... (Sec. 3.3, Sec. 7) */
+    EXMOE_ERR_NOT_PINNED = -3,    /* a host bank pointer is not page-locked host memory (Sec. 3.3) */
+    EXMOE_ERR_CUDA = -4,          /* a CUDA runtime call failed */
+    EXMOE_ERR_NONFINITE = -5,     /* exmoe_pack: a weight is NaN/Inf or a scale overflows FP16 */
+    EXMOE_ERR_BAD_EXPERT_ID = -6, /* a top-k id was outside [0, E); that pair contributed nothing */
+    EXMOE_ERR_TIMEOUT = -7,       /* a bounded device-side wait expired */
+    EXMOE_ERR_STATE = -8          /* call order: e.g. debug plan asked for a layer that did not run last */
+};
+
+/* Geometry of one sparse layer (Sec. 4.1 gives OLMoE's: 2048, 1024, 64, 8).  group_size must be 128. */
+typedef struct {
+    int d_model;      /* H: hidden size, K of gate/up, N of down */
+    int d_ff;         /* I: expert intermediate size */
+    int num_experts;  /* E */
+    int top_k;        /* k */
+    int group_size;   /* 128 (Eq. 3) */
+} exmoe_shape;
+
+/* Runtime counters of one layer's cache (Sec. 4.2 "cache events, transferred bytes").
+ * All zero while the layer is fully resident (C = E): lookup accounting is bypassed (Sec. 5.1). */
+typedef struct {
+    uint64_t lookups;    /* active experts looked up, summed over calls */
+    uint64_t hits;
+    uint64_t misses;
+    uint64_t waves;
+    uint64_t h2d_bytes;  /* misses * bytes of one packed expert */
+    uint64_t forwards;   /* layer calls */
+} exmoe_stats;
+
+typedef struct exmoe_cache exmoe_cache; /* opaque */
+
+const char* exmoe_strerror(int code);
+
+/* Eq. 4: bytes of one packed expert = 3*I*H * (4/8 + 16/(128*8)); 3,244,032 for OLMoE.
+ * This is also the size of one GPU slot and of one entry of the host bank. */
+int exmoe_packed_bytes(const exmoe_shape* shape, size_t* bytes_per_expert);
+
+/* Offline conversion of ONE expert (Eq. 3 + this library's packed layout, Sec. 3.2).
+ *   w_gate_bf16, w_up_bf16 : dev, BF16 [I, H]     w_down_bf16 : dev, BF16 [H, I]
+ *   packed_out             : dev, bytes_per_expert, 16-byte aligned
+ * Layout: 16-row panels x 128-wide blocks of 1056 bytes (1024 bytes of offset-binary nibbles in
+ * the register order of the kernels, then 16 FP16 scales); gate and up panels alternate, the down
+ * matrix follows.  Quantiser: binary32 absmax, s = fp16(absmax/7), q = clip(rint(W/s), -8, 7) with
+ * IEEE division and round-half-even; a zero (or FP16-underflowing) group has s = 0, q = 0.
+ * Runs on `stream` and waits for it, so the status covers the data: EXMOE_ERR_NONFINITE if any
+ * weight is NaN/Inf or a scale overflows FP16 (the output is then unspecified). */
+int exmoe_pack(const exmoe_shape* shape, const void* w_gate_bf16, const void* w_up_bf16,
+               const void* w_down_bf16, void* packed_out, void* stream);
+
+/* Sizes of the two device buffers the caller must allocate for exmoe_cache_create (Sec. 3.3):
+ *   slot_bytes_total = num_layers * num_slots * bytes_per_expert
+ *   workspace_bytes  = cache state + plan + token grouping + intermediate activations for
+ *                      up to max_tokens tokens per call. */
+int exmoe_cache_workspace_bytes(const exmoe_shape* shape, int num_layers, int num_slots,
+                                int max_tokens, size_t* slot_bytes_total, size_t* workspace_bytes);
+
+/* Create the slot caches of `num_layers` sparse layers, C = num_slots slots each (Sec. 3.3).
+ *   host_bank[l] : host, pinned, E * bytes_per_expert bytes: expert e of layer l at offset
+ *                  e * bytes_per_expert, exactly as exmoe_pack wrote it.
+ *   slot_mem     : dev, slot_bytes_total, 256-byte aligned.   workspace : dev, workspace_bytes, 256-aligned.
+ *   wave_cap     : experts per wave, 1..num_slots; 0 means num_slots (Sec. 3.4 "at most C").
+ * C = E: all experts are copied into their slots here (slot = expert id) and later calls do no
+ * lookups.  C < E: the cache starts empty.  Synchronous. */
+int exmoe_cache_create(exmoe_cache** out, const exmoe_shape* shape, int num_layers, int num_slots,
+                       const void* const* host_bank, void* slot_mem, void* workspace,
+                       int max_tokens, int wave_cap);
+
+/* One sparse-layer forward (Eq. 2 through Sec. 3.4's waves).
+ *   hidden_bf16  : dev, BF16 [T, H]        topk_ids : dev, int32 [T, k]
+ *   topk_weights : dev, float32 [T, k]     out_bf16 : dev, BF16 [T, H], fully overwritten
+ * Mixture weights are used as given (no renormalisation, Sec. 3.4).  Pair contributions are
+ * accumulated in binary32 in the order j = 0..k-1 and rounded once to BF16, so the result does not
+ * depend on C, wave_cap or cache history.  T = 0 is a no-op.  An id outside [0, E) contributes
+ * nothing and sets the sticky status EXMOE_ERR_BAD_EXPERT_ID (see exmoe_status).
+ * C = E: fully asynchronous on `stream`.  C < E: the resolution kernel's miss plan is read back
+ * once (the paper's single batched id transfer) and the host waits for it; miss copies run on the
+ * library's copy stream, ordered against the compute stream by events, and return before they finish. */
+int exmoe_moe_forward(exmoe_cache* cache, int layer, const void* hidden_bf16, const int32_t* topk_ids,
+                      const float* topk_weights, int T, void* out_bf16, void* stream);
+
+/* Test hooks (synchronise).  Sec. 3.3 state of one layer: expert_slot [E] (-1 = not resident),
+ * slot_expert [C] (-1 = empty), slot_stamp [C], all host pointers, any may be NULL. */
+int exmoe_cache_get_state(exmoe_cache* cache, int layer, int32_t* expert_slot, int32_t* slot_expert,
+                          uint64_t* slot_stamp, uint64_t* tick);
+
+/* Plan of the most recent exmoe_moe_forward, which must have been for `layer` (Sec. 3.4 steps 1-2
+ * and the token grouping): wave_of [E], slot_of [E] (-1 = inactive sentinel), counts [n_keys],
+ * offsets [n_keys + 1], perm [T*k] (first offsets[n_keys] entries valid), misses [3*E] as
+ * (expert, slot, wave) triples; n_keys = ceil(E / wave_cap) * C.  Any output pointer may be NULL. */
+int exmoe_debug_last_plan(exmoe_cache* cache, int layer, int32_t* n_active, int32_t* n_waves,
+                          int32_t* n_misses, int32_t* wave_of, int32_t* slot_of, int32_t* counts,
+                          int32_t* offsets, int32_t* perm, int32_t* misses);
+
+/* Copy one slot's bytes back to the host (test hook for the miss-copy path; synchronises). */
+int exmoe_debug_read_slot(exmoe_cache* cache, int layer, int slot, void* host_out);
+
+int exmoe_cache_stats(exmoe_cache* cache, int layer, exmoe_stats* out);   /* synchronises */
+int exmoe_cache_reset(exmoe_cache* cache, int layer);                     /* empty cache, zero counters */
+int exmoe_status(exmoe_cache* cache);   /* synchronises; returns and clears the sticky device status */
+int exmoe_cache_destroy(exmoe_cache* cache);
+
+/* Kernels launched by this library since it was loaded (all streams, all caches). */
+uint64_t exmoe_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* EXMOE_H */

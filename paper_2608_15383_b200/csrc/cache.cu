@@ -1,0 +1,415 @@
+// Host side of the C ABI: slot caches (Section 3.3), the wave executor (Section 3.4), miss copies on a
+// side stream ordered by events, and the test hooks.  All arithmetic of the path runs in kernels;
+// this file only validates, carves the caller's workspace, launches and orders.
+#include <atomic>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "common.cuh"
+
+namespace exmoe {
+
+static std::atomic<uint64_t> g_launches{0};
+void count_launch(int n) { g_launches.fetch_add((uint64_t)n, std::memory_order_relaxed); }
+
+static inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+static int check_shape(const exmoe_shape* s) {
+    if (!s) return EXMOE_ERR_ARG;
+    if (s->group_size != kGroup) return EXMOE_ERR_SHAPE;
+    if (s->d_model <= 0 || s->d_ff <= 0 || s->d_model % kGroup || s->d_ff % kGroup) return EXMOE_ERR_SHAPE;
+    if (s->num_experts <= 0 || s->num_experts > 4096) return EXMOE_ERR_SHAPE;
+    if (s->top_k <= 0 || s->top_k > s->num_experts) return EXMOE_ERR_SHAPE;
+    return EXMOE_OK;
+}
+
+static size_t packed_bytes(const exmoe_shape& s) {
+    return matrix_bytes(2 * s.d_ff, s.d_model) + matrix_bytes(s.d_model, s.d_ff);
+}
+
+struct Carve {                      // bump allocator over the caller's workspace (256-byte aligned pieces)
+    uint8_t* base;
+    size_t off = 0;
+    template <typename T> T* take(size_t n) {
+        T* p = base ? reinterpret_cast<T*>(base + off) : nullptr;
+        off += align_up(n * sizeof(T), 256);
+        return p;
+    }
+};
+
+constexpr int kEventRing = 64;
+constexpr int kMaxKeys = 8192;      // ceil(E / wave_cap) * C: bounds the grouping kernels' shared memory
+
+}  // namespace exmoe
+
+using namespace exmoe;
+
+struct exmoe_cache {
+    exmoe_shape shape;
+    int L, C, Cw, max_tokens, max_pairs, n_keys, max_waves;
+    size_t bpe;                               // bytes per packed expert = slot stride
+    std::vector<const uint8_t*> bank;
+    uint8_t* slot_mem;
+    int* d_status;
+    std::vector<LayerState> state;
+    PlanPtrs plan;
+    size_t plan_d2h_bytes;                    // header | wave_of | slot_of | misses, contiguous
+    __nv_bfloat16* act;                       // [max_pairs, I] SwiGLU output, grouped row order
+    float* y;                                 // [max_pairs, H] weighted expert outputs, pair order
+    int32_t* h_plan;                          // pinned staging of the plan
+    cudaStream_t copy_stream;
+    cudaEvent_t ev_plan;
+    cudaEvent_t ev_compute[kEventRing];       // completion of a wave's kernels (Section 3.4 step 5)
+    cudaEvent_t ev_copy[kEventRing];          // completion of a wave's miss copies
+    uint64_t seq;                             // last recorded compute event
+    uint64_t copy_seq;
+    std::vector<std::vector<uint64_t>> slot_last_seq;   // [L][C] compute event that last read the slot
+    int last_layer;
+    int last_T;
+};
+
+static void carve_workspace(exmoe_cache* c, uint8_t* ws, size_t* total) {
+    const exmoe_shape& s = c->shape;
+    const int E = s.num_experts, C = c->C;
+    Carve k{ws};
+    c->d_status = k.take<int>(64);
+    c->state.resize(c->L);
+    for (int l = 0; l < c->L; ++l) {
+        c->state[l].expert_slot = k.take<int32_t>(E);
+        c->state[l].slot_expert = k.take<int32_t>(C);
+        c->state[l].slot_stamp = k.take<uint64_t>(C);
+        c->state[l].tick = k.take<uint64_t>(1);
+        c->state[l].stats = k.take<uint64_t>(6);
+    }
+    int32_t* p = k.take<int32_t>(HDR_WORDS + 5 * (size_t)E);
+    c->plan.header = p;
+    c->plan.wave_of = p ? p + HDR_WORDS : nullptr;
+    c->plan.slot_of = p ? p + HDR_WORDS + E : nullptr;
+    c->plan.misses = p ? p + HDR_WORDS + 2 * E : nullptr;
+    c->plan_d2h_bytes = (HDR_WORDS + 5 * (size_t)E) * 4;
+    c->plan.counts = k.take<int32_t>(c->n_keys);
+    c->plan.offsets = k.take<int32_t>(c->n_keys + 1);
+    c->plan.group_keys = k.take<int32_t>(c->n_keys);
+    c->plan.wave_start = k.take<int32_t>(c->max_waves + 1);
+    c->plan.perm = k.take<int32_t>(c->max_pairs);
+    c->act = k.take<__nv_bfloat16>((size_t)c->max_pairs * s.d_ff);
+    c->y = k.take<float>((size_t)c->max_pairs * s.d_model);
+    *total = k.off;
+}
+
+static int fill_dims(exmoe_cache* c, const exmoe_shape* shape, int num_layers, int num_slots, int max_tokens,
+                     int wave_cap) {
+    int rc = check_shape(shape);
+    if (rc) return rc;
+    if (num_layers <= 0 || max_tokens <= 0) return EXMOE_ERR_ARG;
+    if (num_slots < shape->top_k || num_slots > shape->num_experts) return EXMOE_ERR_SHAPE;
+    if (wave_cap < 0 || wave_cap > num_slots) return EXMOE_ERR_SHAPE;
+    if ((long long)max_tokens * shape->top_k > (1ll << 30)) return EXMOE_ERR_ARG;
+    c->shape = *shape;
+    c->L = num_layers;
+    c->C = num_slots;
+    c->Cw = wave_cap ? wave_cap : num_slots;
+    c->max_tokens = max_tokens;
+    c->max_pairs = max_tokens * shape->top_k;
+    c->max_waves = (shape->num_experts + c->Cw - 1) / c->Cw;
+    c->n_keys = c->max_waves * c->C;
+    if (c->n_keys > kMaxKeys) return EXMOE_ERR_SHAPE;
+    c->bpe = packed_bytes(*shape);
+    return EXMOE_OK;
+}
+
+static int reset_layer(exmoe_cache* c, int layer) {
+    const int E = c->shape.num_experts, C = c->C;
+    std::vector<int32_t> es(E, -1), se(C, -1);
+    if (C == E)
+        for (int e = 0; e < E; ++e) es[e] = se[e] = e;
+    std::vector<uint64_t> zeros(C > 8 ? C : 8, 0);
+    LayerState& st = c->state[layer];
+    if (cudaMemcpy(st.expert_slot, es.data(), E * 4, cudaMemcpyHostToDevice) != cudaSuccess) return EXMOE_ERR_CUDA;
+    if (cudaMemcpy(st.slot_expert, se.data(), C * 4, cudaMemcpyHostToDevice) != cudaSuccess) return EXMOE_ERR_CUDA;
+    if (cudaMemcpy(st.slot_stamp, zeros.data(), C * 8, cudaMemcpyHostToDevice) != cudaSuccess) return EXMOE_ERR_CUDA;
+    if (cudaMemcpy(st.tick, zeros.data(), 8, cudaMemcpyHostToDevice) != cudaSuccess) return EXMOE_ERR_CUDA;
+    if (cudaMemcpy(st.stats, zeros.data(), 48, cudaMemcpyHostToDevice) != cudaSuccess) return EXMOE_ERR_CUDA;
+    std::fill(c->slot_last_seq[layer].begin(), c->slot_last_seq[layer].end(), 0);
+    return EXMOE_OK;
+}
+
+extern "C" {
+
+const char* exmoe_strerror(int code) {
+    switch (code) {
+        case EXMOE_OK: return "ok";
+        case EXMOE_ERR_ARG: return "invalid argument";
+        case EXMOE_ERR_SHAPE: return "unsupported shape (dims must be multiples of 128, k <= C <= E)";
+        case EXMOE_ERR_NOT_PINNED: return "host bank is not pinned host memory";
+        case EXMOE_ERR_CUDA: return "CUDA runtime error";
+        case EXMOE_ERR_NONFINITE: return "non-finite weight or scale overflow";
+        case EXMOE_ERR_BAD_EXPERT_ID: return "expert id out of range";
+        case EXMOE_ERR_TIMEOUT: return "bounded device wait expired";
+        case EXMOE_ERR_STATE: return "call order";
+        default: return "unknown error";
+    }
+}
+
+uint64_t exmoe_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
+
+int exmoe_packed_bytes(const exmoe_shape* shape, size_t* bytes_per_expert) {
+    int rc = check_shape(shape);
+    if (rc) return rc;
+    if (!bytes_per_expert) return EXMOE_ERR_ARG;
+    *bytes_per_expert = packed_bytes(*shape);
+    return EXMOE_OK;
+}
+
+int exmoe_pack(const exmoe_shape* shape, const void* w_gate, const void* w_up, const void* w_down, void* packed_out,
+               void* stream) {
+    int rc = check_shape(shape);
+    if (rc) return rc;
+    if (!w_gate || !w_up || !w_down || !packed_out) return EXMOE_ERR_ARG;
+    if ((reinterpret_cast<uintptr_t>(packed_out) | reinterpret_cast<uintptr_t>(w_gate) |
+         reinterpret_cast<uintptr_t>(w_up) | reinterpret_cast<uintptr_t>(w_down)) & 15)
+        return EXMOE_ERR_ARG;
+    cudaStream_t st = (cudaStream_t)stream;
+    int* d_flag = nullptr;
+    if (cudaMalloc(&d_flag, sizeof(int)) != cudaSuccess) return EXMOE_ERR_CUDA;
+    int flag = 0;
+    rc = EXMOE_OK;
+    if (cudaMemsetAsync(d_flag, 0, sizeof(int), st) != cudaSuccess) rc = EXMOE_ERR_CUDA;
+    if (!rc) rc = launch_pack(*shape, w_gate, w_up, w_down, packed_out, d_flag, st);
+    if (!rc && cudaMemcpyAsync(&flag, d_flag, sizeof(int), cudaMemcpyDeviceToHost, st) != cudaSuccess) rc = EXMOE_ERR_CUDA;
+    if (cudaStreamSynchronize(st) != cudaSuccess) rc = EXMOE_ERR_CUDA;
+    cudaFree(d_flag);
+    if (!rc && flag) rc = EXMOE_ERR_NONFINITE;
+    return rc;
+}
+
+int exmoe_cache_workspace_bytes(const exmoe_shape* shape, int num_layers, int num_slots, int max_tokens,
+                                size_t* slot_bytes_total, size_t* workspace_bytes) {
+    exmoe_cache tmp{};
+    int rc = check_shape(shape);
+    if (rc) return rc;
+    int wc = 1;                                         // smallest wave_cap allowed = largest key space
+    while (wc < num_slots && (long long)((shape->num_experts + wc - 1) / wc) * num_slots > kMaxKeys) ++wc;
+    rc = fill_dims(&tmp, shape, num_layers, num_slots, max_tokens, wc);
+    if (rc) return rc;
+    if (!slot_bytes_total || !workspace_bytes) return EXMOE_ERR_ARG;
+    *slot_bytes_total = (size_t)num_layers * num_slots * tmp.bpe;
+    carve_workspace(&tmp, nullptr, workspace_bytes);
+    return EXMOE_OK;
+}
+
+int exmoe_cache_create(exmoe_cache** out, const exmoe_shape* shape, int num_layers, int num_slots,
+                       const void* const* host_bank, void* slot_mem, void* workspace, int max_tokens, int wave_cap) {
+    if (!out || !host_bank || !slot_mem || !workspace) return EXMOE_ERR_ARG;
+    if ((reinterpret_cast<uintptr_t>(slot_mem) | reinterpret_cast<uintptr_t>(workspace)) & 255) return EXMOE_ERR_ARG;
+    exmoe_cache* c = new (std::nothrow) exmoe_cache{};
+    if (!c) return EXMOE_ERR_ARG;
+    int rc = fill_dims(c, shape, num_layers, num_slots, max_tokens, wave_cap);
+    if (rc) { delete c; return rc; }
+    for (int l = 0; l < num_layers; ++l) {
+        cudaPointerAttributes attr{};
+        if (!host_bank[l] || cudaPointerGetAttributes(&attr, host_bank[l]) != cudaSuccess ||
+            attr.type != cudaMemoryTypeHost) {
+            cudaGetLastError();
+            delete c;
+            return host_bank[l] ? EXMOE_ERR_NOT_PINNED : EXMOE_ERR_ARG;
+        }
+        c->bank.push_back(static_cast<const uint8_t*>(host_bank[l]));
+    }
+    c->slot_mem = static_cast<uint8_t*>(slot_mem);
+    size_t total = 0;
+    carve_workspace(c, static_cast<uint8_t*>(workspace), &total);
+    c->slot_last_seq.assign(num_layers, std::vector<uint64_t>(num_slots, 0));
+    c->last_layer = -1;
+    c->last_T = 0;
+    bool ok = cudaMallocHost(&c->h_plan, c->plan_d2h_bytes) == cudaSuccess;
+    ok = ok && cudaStreamCreateWithFlags(&c->copy_stream, cudaStreamNonBlocking) == cudaSuccess;
+    ok = ok && cudaEventCreateWithFlags(&c->ev_plan, cudaEventDisableTiming) == cudaSuccess;
+    for (int i = 0; i < kEventRing && ok; ++i) {
+        ok = ok && cudaEventCreateWithFlags(&c->ev_compute[i], cudaEventDisableTiming) == cudaSuccess;
+        ok = ok && cudaEventCreateWithFlags(&c->ev_copy[i], cudaEventDisableTiming) == cudaSuccess;
+    }
+    ok = ok && cudaMemset(c->d_status, 0, 256) == cudaSuccess;
+    ok = ok && cudaMemset(c->plan.header, 0, c->plan_d2h_bytes) == cudaSuccess;
+    for (int l = 0; l < num_layers && ok; ++l) ok = reset_layer(c, l) == EXMOE_OK;
+    if (ok && c->C == c->shape.num_experts) {            // full residency: preload, slot = expert id
+        for (int l = 0; l < num_layers && ok; ++l)
+            ok = cudaMemcpy(c->slot_mem + (size_t)l * c->C * c->bpe, c->bank[l], (size_t)c->C * c->bpe,
+                            cudaMemcpyHostToDevice) == cudaSuccess;
+    }
+    if (!ok) {
+        cudaGetLastError();
+        exmoe_cache_destroy(c);
+        return EXMOE_ERR_CUDA;
+    }
+    *out = c;
+    return EXMOE_OK;
+}
+
+int exmoe_moe_forward(exmoe_cache* c, int layer, const void* hidden, const int32_t* topk_ids,
+                      const float* topk_weights, int T, void* out, void* stream) {
+    if (!c || layer < 0 || layer >= c->L || T < 0 || T > c->max_tokens) return EXMOE_ERR_ARG;
+    if (T == 0) return EXMOE_OK;
+    if (!hidden || !topk_ids || !topk_weights || !out) return EXMOE_ERR_ARG;
+    if ((reinterpret_cast<uintptr_t>(hidden) | reinterpret_cast<uintptr_t>(out)) & 15) return EXMOE_ERR_ARG;
+    cudaStream_t st = (cudaStream_t)stream;
+    const exmoe_shape& s = c->shape;
+    const int E = s.num_experts, C = c->C, k = s.top_k, P = T * k;
+    const bool identity = (C == E);
+    c->last_layer = layer;
+    c->last_T = T;
+
+    if (!identity) {
+        launch_resolve(s, C, c->Cw, c->bpe, topk_ids, P, c->state[layer], c->plan, c->d_status, st);
+        if (cudaMemcpyAsync(c->h_plan, c->plan.header, c->plan_d2h_bytes, cudaMemcpyDeviceToHost, st) != cudaSuccess)
+            return EXMOE_ERR_CUDA;
+        if (cudaEventRecord(c->ev_plan, st) != cudaSuccess) return EXMOE_ERR_CUDA;
+    }
+    launch_group(s, C, c->n_keys, c->max_waves, identity, topk_ids, P, c->plan, c->d_status, st);
+
+    int n_waves = 1;
+    const int32_t *h_wave_of = nullptr, *h_slot_of = nullptr, *h_miss = nullptr;
+    int n_miss = 0;
+    if (!identity) {
+        if (cudaEventSynchronize(c->ev_plan) != cudaSuccess) return EXMOE_ERR_CUDA;   // the one batched id transfer
+        n_waves = c->h_plan[HDR_N_WAVES];
+        n_miss = c->h_plan[HDR_N_MISSES];
+        h_wave_of = c->h_plan + HDR_WORDS;
+        h_slot_of = h_wave_of + E;
+        h_miss = h_slot_of + E;
+    }
+
+    GemmArgs a{};
+    a.slots = c->slot_mem + (size_t)layer * C * c->bpe;
+    a.slot_stride = c->bpe;
+    a.counts = c->plan.counts;
+    a.offsets = c->plan.offsets;
+    a.group_keys = c->plan.group_keys;
+    a.perm = c->plan.perm;
+    a.num_slots = C;
+    a.top_k = k;
+    a.H = s.d_model;
+    a.I = s.d_ff;
+
+    int mi = 0;
+    for (int w = 0; w < n_waves; ++w) {
+        int groups = identity ? (E < P ? E : P) : 0;
+        if (!identity) {
+            bool copied = false;
+            for (; mi < n_miss && h_miss[3 * mi + 2] == w; ++mi) {
+                const int e = h_miss[3 * mi], v = h_miss[3 * mi + 1];
+                const uint64_t last = c->slot_last_seq[layer][v];
+                if (last) cudaStreamWaitEvent(c->copy_stream, c->ev_compute[last % kEventRing], 0);
+                if (cudaMemcpyAsync(const_cast<uint8_t*>(a.slots) + (size_t)v * c->bpe, c->bank[layer] + (size_t)e * c->bpe,
+                                    c->bpe, cudaMemcpyHostToDevice, c->copy_stream) != cudaSuccess)
+                    return EXMOE_ERR_CUDA;
+                copied = true;
+            }
+            if (copied) {
+                cudaEvent_t ev = c->ev_copy[(++c->copy_seq) % kEventRing];
+                cudaEventRecord(ev, c->copy_stream);
+                cudaStreamWaitEvent(st, ev, 0);
+            }
+            for (int e = 0; e < E; ++e) groups += (h_wave_of[e] == w);
+        }
+        a.wave_start = c->plan.wave_start + w;
+        launch_decode_gateup(a, (const __nv_bfloat16*)hidden, c->act, T, groups, st);
+        launch_decode_down(a, c->act, topk_weights, c->y, T, groups, st);
+        if (!identity) {
+            ++c->seq;
+            cudaEventRecord(c->ev_compute[c->seq % kEventRing], st);                  // completion event of the wave
+            for (int e = 0; e < E; ++e)
+                if (h_wave_of[e] == w) c->slot_last_seq[layer][h_slot_of[e]] = c->seq;
+        }
+    }
+    launch_combine(c->y, topk_ids, E, T, k, s.d_model, (__nv_bfloat16*)out, st);
+    return cudaGetLastError() == cudaSuccess ? EXMOE_OK : EXMOE_ERR_CUDA;
+}
+
+int exmoe_cache_get_state(exmoe_cache* c, int layer, int32_t* expert_slot, int32_t* slot_expert, uint64_t* slot_stamp,
+                          uint64_t* tick) {
+    if (!c || layer < 0 || layer >= c->L) return EXMOE_ERR_ARG;
+    if (cudaDeviceSynchronize() != cudaSuccess) return EXMOE_ERR_CUDA;
+    const LayerState& st = c->state[layer];
+    bool ok = true;
+    if (expert_slot) ok = ok && cudaMemcpy(expert_slot, st.expert_slot, c->shape.num_experts * 4, cudaMemcpyDeviceToHost) == cudaSuccess;
+    if (slot_expert) ok = ok && cudaMemcpy(slot_expert, st.slot_expert, c->C * 4, cudaMemcpyDeviceToHost) == cudaSuccess;
+    if (slot_stamp) ok = ok && cudaMemcpy(slot_stamp, st.slot_stamp, c->C * 8, cudaMemcpyDeviceToHost) == cudaSuccess;
+    if (tick) ok = ok && cudaMemcpy(tick, st.tick, 8, cudaMemcpyDeviceToHost) == cudaSuccess;
+    return ok ? EXMOE_OK : EXMOE_ERR_CUDA;
+}
+
+int exmoe_debug_last_plan(exmoe_cache* c, int layer, int32_t* n_active, int32_t* n_waves, int32_t* n_misses,
+                          int32_t* wave_of, int32_t* slot_of, int32_t* counts, int32_t* offsets, int32_t* perm,
+                          int32_t* misses) {
+    if (!c || layer < 0 || layer >= c->L) return EXMOE_ERR_ARG;
+    if (layer != c->last_layer) return EXMOE_ERR_STATE;
+    if (cudaDeviceSynchronize() != cudaSuccess) return EXMOE_ERR_CUDA;
+    const int E = c->shape.num_experts;
+    std::vector<int32_t> hdr(HDR_WORDS + 5 * (size_t)E);
+    bool ok = cudaMemcpy(hdr.data(), c->plan.header, hdr.size() * 4, cudaMemcpyDeviceToHost) == cudaSuccess;
+    std::vector<int32_t> cnt(c->n_keys);
+    ok = ok && cudaMemcpy(cnt.data(), c->plan.counts, cnt.size() * 4, cudaMemcpyDeviceToHost) == cudaSuccess;
+    if (!ok) return EXMOE_ERR_CUDA;
+    if (n_active) *n_active = hdr[HDR_N_ACTIVE];
+    if (n_waves) *n_waves = hdr[HDR_N_WAVES];
+    if (n_misses) *n_misses = hdr[HDR_N_MISSES];
+    const bool identity = (c->C == E);
+    if (wave_of)
+        for (int e = 0; e < E; ++e) wave_of[e] = identity ? (cnt[e] > 0 ? 0 : -1) : hdr[HDR_WORDS + e];
+    if (slot_of)
+        for (int e = 0; e < E; ++e) slot_of[e] = identity ? (cnt[e] > 0 ? e : -1) : hdr[HDR_WORDS + E + e];
+    if (misses) std::memcpy(misses, hdr.data() + HDR_WORDS + 2 * E, 3 * (size_t)E * 4);
+    if (counts) std::memcpy(counts, cnt.data(), cnt.size() * 4);
+    if (offsets) ok = ok && cudaMemcpy(offsets, c->plan.offsets, (c->n_keys + 1) * 4, cudaMemcpyDeviceToHost) == cudaSuccess;
+    if (perm) ok = ok && cudaMemcpy(perm, c->plan.perm, (size_t)c->last_T * c->shape.top_k * 4, cudaMemcpyDeviceToHost) == cudaSuccess;
+    return ok ? EXMOE_OK : EXMOE_ERR_CUDA;
+}
+
+int exmoe_debug_read_slot(exmoe_cache* c, int layer, int slot, void* host_out) {
+    if (!c || layer < 0 || layer >= c->L || slot < 0 || slot >= c->C || !host_out) return EXMOE_ERR_ARG;
+    if (cudaDeviceSynchronize() != cudaSuccess) return EXMOE_ERR_CUDA;
+    return cudaMemcpy(host_out, c->slot_mem + ((size_t)layer * c->C + slot) * c->bpe, c->bpe, cudaMemcpyDeviceToHost) ==
+                   cudaSuccess ? EXMOE_OK : EXMOE_ERR_CUDA;
+}
+
+int exmoe_cache_stats(exmoe_cache* c, int layer, exmoe_stats* out) {
+    if (!c || layer < 0 || layer >= c->L || !out) return EXMOE_ERR_ARG;
+    if (cudaDeviceSynchronize() != cudaSuccess) return EXMOE_ERR_CUDA;
+    uint64_t v[6];
+    if (cudaMemcpy(v, c->state[layer].stats, 48, cudaMemcpyDeviceToHost) != cudaSuccess) return EXMOE_ERR_CUDA;
+    out->lookups = v[0]; out->hits = v[1]; out->misses = v[2]; out->waves = v[3]; out->h2d_bytes = v[4]; out->forwards = v[5];
+    return EXMOE_OK;
+}
+
+int exmoe_cache_reset(exmoe_cache* c, int layer) {
+    if (!c || layer < 0 || layer >= c->L) return EXMOE_ERR_ARG;
+    if (cudaDeviceSynchronize() != cudaSuccess) return EXMOE_ERR_CUDA;
+    return reset_layer(c, layer);
+}
+
+int exmoe_status(exmoe_cache* c) {
+    if (!c) return EXMOE_ERR_ARG;
+    if (cudaDeviceSynchronize() != cudaSuccess) return EXMOE_ERR_CUDA;
+    int v = 0;
+    if (cudaMemcpy(&v, c->d_status, 4, cudaMemcpyDeviceToHost) != cudaSuccess) return EXMOE_ERR_CUDA;
+    if (v && cudaMemset(c->d_status, 0, 4) != cudaSuccess) return EXMOE_ERR_CUDA;
+    return v;
+}
+
+int exmoe_cache_destroy(exmoe_cache* c) {
+    if (!c) return EXMOE_ERR_ARG;
+    cudaDeviceSynchronize();
+    if (c->h_plan) cudaFreeHost(c->h_plan);
+    if (c->copy_stream) cudaStreamDestroy(c->copy_stream);
+    if (c->ev_plan) cudaEventDestroy(c->ev_plan);
+    for (int i = 0; i < kEventRing; ++i) {
+        if (c->ev_compute[i]) cudaEventDestroy(c->ev_compute[i]);
+        if (c->ev_copy[i]) cudaEventDestroy(c->ev_copy[i]);
+    }
+    delete c;
+    return EXMOE_OK;
+}
+
+}  // extern "C"

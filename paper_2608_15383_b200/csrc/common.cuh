@@ -1,0 +1,78 @@
+// Shared declarations of the exmoe CUDA library (sm_100a only).
+#pragma once
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <cuda_fp16.h>
+#include <stdint.h>
+#include <stddef.h>
+#include "../../include/exmoe.h"
+
+namespace exmoe {
+
+// ---- packed layout (Eq. 3 / Eq. 4): 16-row panels x 128-wide blocks of 1056 bytes -------------
+constexpr int kGroup = 128;          // scale group along K
+constexpr int kPanelRows = 16;       // rows per panel (one m16 MMA tile)
+constexpr int kBlockBytes = 1056;    // 1024 code bytes + 16 FP16 scales
+constexpr int kCodeBytes = 1024;
+
+// bytes of a packed [rows, K] matrix
+__host__ __device__ inline size_t matrix_bytes(int rows, int K) {
+    return (size_t)(rows / kPanelRows) * (K / kGroup) * kBlockBytes;
+}
+
+// ---- plan buffers shared by the resolution, grouping and GEMM kernels ------------------------
+// header words
+enum { HDR_N_ACTIVE = 0, HDR_N_WAVES = 1, HDR_N_MISSES = 2, HDR_BAD_ID = 3, HDR_N_GROUPS = 4, HDR_N_VALID = 5,
+       HDR_WORDS = 8 };
+
+struct PlanPtrs {
+    int32_t* header;        // [HDR_WORDS]
+    int32_t* wave_of;       // [E]
+    int32_t* slot_of;       // [E]
+    int32_t* misses;        // [3*E] (expert, slot, wave)
+    int32_t* counts;        // [n_keys]
+    int32_t* offsets;       // [n_keys + 1]
+    int32_t* group_keys;    // [n_keys] active keys, ascending
+    int32_t* wave_start;    // [max_waves + 1] index into group_keys
+    int32_t* perm;          // [max_pairs]
+};
+
+struct LayerState {         // Section 3.3 state of one layer, device memory
+    int32_t* expert_slot;   // [E]
+    int32_t* slot_expert;   // [C]
+    uint64_t* slot_stamp;   // [C]
+    uint64_t* tick;         // [1]
+    uint64_t* stats;        // [6] lookups, hits, misses, waves, h2d_bytes, forwards
+};
+
+struct GemmArgs {
+    const uint8_t* slots;       // slot memory of the layer
+    size_t slot_stride;         // bytes per slot
+    const int32_t* counts;
+    const int32_t* offsets;
+    const int32_t* group_keys;
+    const int32_t* wave_start;  // already offset to the wave: [0] first group, [1] end
+    const int32_t* perm;
+    int num_slots;              // C (key % C = slot)
+    int top_k;
+    int H, I;
+};
+
+// launch accounting (exmoe_launch_count)
+void count_launch(int n = 1);
+
+// ---- kernel launchers (defined in the .cu files) ------------------------------------------------
+int launch_pack(const exmoe_shape& s, const void* wg, const void* wu, const void* wd, void* out,
+                int* d_flag, cudaStream_t st);
+void launch_resolve(const exmoe_shape& s, int C, int Cw, size_t bytes_per_expert, const int32_t* ids, int n_pairs,
+                    LayerState state, PlanPtrs plan, int* d_status, cudaStream_t st);
+void launch_group(const exmoe_shape& s, int C, int n_keys, int max_waves, bool identity, const int32_t* ids,
+                  int n_pairs, PlanPtrs plan, int* d_status, cudaStream_t st);
+void launch_decode_gateup(const GemmArgs& a, const __nv_bfloat16* hidden, __nv_bfloat16* act, int max_rows,
+                          int max_groups, cudaStream_t st);
+void launch_decode_down(const GemmArgs& a, const __nv_bfloat16* act, const float* topk_w, float* y, int max_rows,
+                        int max_groups, cudaStream_t st);
+void launch_combine(const float* y, const int32_t* ids, int E, int T, int k, int H, __nv_bfloat16* out,
+                    cudaStream_t st);
+
+}  // namespace exmoe

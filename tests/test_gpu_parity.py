@@ -1,0 +1,309 @@
+"""GPU parity: the CUDA library (through the C ABI) against the CPU oracle on the same seeded inputs.
+
+Bit-exact: packed bytes, slot maps, waves, miss lists, counters, token grouping, slot contents.
+Toleranced (spec bound): BF16 layer output, max|err| <= 2e-2*max|ref| and rel. Frobenius <= 5e-3.
+"""
+import numpy as np
+import pytest
+import torch
+
+from oracle import cache as ocache
+from paper_2608_15383_b200 import synth
+
+import helpers
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def B():
+    from paper_2608_15383_b200 import binding, build
+    build.build()
+    binding.lib()
+    return binding
+
+
+@pytest.fixture(scope="module")
+def tiny_layer(B):
+    return helpers.make_layer(synth.TINY, seed=0)
+
+
+@pytest.fixture(scope="module")
+def mid_layer(B):
+    return helpers.make_layer(synth.MID, seed=5)
+
+
+@pytest.fixture(scope="module")
+def olmoe_layer(B):
+    return helpers.make_layer(synth.OLMOE, seed=2000)
+
+
+# ------------------------------------------------------------------------------------ a0: pack
+def test_pack_bytes_tiny_all_experts(B, tiny_layer):
+    ora, bank = tiny_layer
+    assert B.exmoe_packed_bytes(synth.TINY) == 50688 == bank.shape[1]
+    for e in range(synth.TINY.num_experts):
+        assert np.array_equal(bank[e].numpy(), ora.packed(e)), e
+
+
+def test_pack_bytes_olmoe_shape(B, olmoe_layer):
+    ora, bank = olmoe_layer
+    assert B.exmoe_packed_bytes(synth.OLMOE) == 3244032
+    for e in (0, 37):
+        assert np.array_equal(bank[e].numpy(), ora.packed(e)), e
+
+
+def test_pack_special_groups_and_errors(B):
+    s = synth.Shape(d_model=256, d_ff=128, num_experts=1, top_k=1)
+    wg, wu, wd = synth.expert_weights(s, seed=3)
+    wg[0, 3, 128:] = 0                               # zero group
+    wg[0, 5, :128] = 0
+    wg[0, 5, 17] = 0.0123                            # one-nonzero group
+    wu[0, 2, :128] = 2.0 ** -30                      # FP16-underflowing scale
+    wd[0, 0, :128] = 0
+    wd[0, 0, :8] = torch.tensor([1.5, 0.5, -0.5, 2.5, -2.5, 3.5, 7, -7]) * 2.0 ** -6   # s = 2^-6: exact ties
+    ora = helpers.OracleLayer(s, wg, wu, wd)
+    got = B.exmoe_pack(s, wg[0].cuda(), wu[0].cuda(), wd[0].cuda()).cpu().numpy()
+    assert np.array_equal(got, ora.packed(0))
+    bad = wg[0].clone()
+    bad[1, 1] = float("nan")
+    with pytest.raises(B.ExmoeError) as ei:
+        B.exmoe_pack(s, bad.cuda(), wu[0].cuda(), wd[0].cuda())
+    assert ei.value.code == B.EXMOE_ERR_NONFINITE
+    bad = wg[0].clone()
+    bad[1, 1] = 3e38                                 # absmax/7 overflows FP16
+    with pytest.raises(B.ExmoeError) as ei:
+        B.exmoe_pack(s, bad.cuda(), wu[0].cuda(), wd[0].cuda())
+    assert ei.value.code == B.EXMOE_ERR_NONFINITE
+    with pytest.raises(B.ExmoeError) as ei:
+        B.exmoe_packed_bytes(synth.Shape(d_model=200, d_ff=128, num_experts=4, top_k=2))
+    assert ei.value.code == B.EXMOE_ERR_SHAPE
+
+
+# ------------------------------------------------------------------------------------ a1/a2: plan
+def compare_plan(cache, sc, ids, layer=0):
+    plan, counts, offsets, perm = helpers.oracle_plan(sc, ids.numpy())
+    got = cache.last_plan(layer, ids.numel())
+    assert got["n_active"] == plan.n_active and got["n_waves"] == plan.n_waves
+    assert np.array_equal(got["wave_of"], plan.wave_of)
+    assert np.array_equal(got["slot_of"], plan.slot_of)
+    assert got["misses"] == plan.misses
+    assert np.array_equal(got["counts"], counts)
+    assert np.array_equal(got["offsets"], offsets)
+    assert np.array_equal(got["perm"], perm)
+    if sc.C < sc.E:
+        es, se, stamp, tick = cache.state(layer)
+        assert np.array_equal(es, sc.expert_slot) and np.array_equal(se, sc.slot_expert)
+        assert np.array_equal(stamp, sc.slot_stamp) and tick == sc.tick
+    st = cache.stats(layer)
+    assert st == {"lookups": sc.stats.lookups, "hits": sc.stats.hits, "misses": sc.stats.misses,
+                  "waves": sc.stats.waves, "h2d_bytes": sc.stats.h2d_bytes, "forwards": sc.stats.forwards}
+    return plan
+
+
+@pytest.mark.parametrize("C,Cw,T,alpha", [(8, 0, 16, 0.0), (2, 0, 5, 0.0), (4, 2, 16, 1.0), (3, 0, 1, 0.0), (5, 3, 40, 0.5)])
+def test_plan_bit_exact_tiny(B, tiny_layer, C, Cw, T, alpha):
+    ora, bank = tiny_layer
+    s = synth.TINY
+    cache = B.Cache(s, [bank], C, max_tokens=64, wave_cap=Cw)
+    sc = ocache.SlotCache(s.num_experts, C, Cw, bytes_per_expert=cache.bytes_per_expert)
+    for step in range(12):
+        hidden, ids, p = helpers.routed_inputs(s, T, seed=100 + step, alpha=alpha)
+        cache.forward(0, hidden.cuda(), ids.cuda(), p.cuda())
+        compare_plan(cache, sc, ids)
+    assert cache.status() == 0
+    cache.close()
+
+
+@pytest.mark.parametrize("C,Cw,T,alpha", [(16, 0, 16, 1.0), (16, 8, 16, 0.5), (32, 0, 4, 1.0), (8, 0, 1, 0.0),
+                                          (64, 0, 16, 1.0), (16, 0, 200, 0.0), (64, 0, 300, 1.0)])
+def test_plan_bit_exact_olmoe(B, olmoe_layer, C, Cw, T, alpha):
+    """Resolution, LRU, waves and grouping on OLMoE geometry, incl. the multi-CTA grouping path (T*k > 1024)."""
+    ora, bank = olmoe_layer
+    s = synth.OLMOE
+    cache = B.Cache(s, [bank], C, max_tokens=max(T, 16), wave_cap=Cw)
+    sc = ocache.SlotCache(s.num_experts, C, Cw, bytes_per_expert=cache.bytes_per_expert)
+    for step in range(4 if T > 64 else 10):
+        hidden, ids, p = helpers.routed_inputs(s, T, seed=300 + step, alpha=alpha)
+        cache.forward(0, hidden.cuda(), ids.cuda(), p.cuda())
+        compare_plan(cache, sc, ids)
+    cache.close()
+
+
+def test_slot_bytes_after_miss_copies(B, olmoe_layer):
+    """After misses, every occupied slot holds exactly the host bank's bytes of its expert (Section 3.3)."""
+    ora, bank = olmoe_layer
+    s = synth.OLMOE
+    cache = B.Cache(s, [bank], 16, max_tokens=16)
+    for step in range(3):
+        hidden, ids, p = helpers.routed_inputs(s, 16, seed=400 + step, alpha=0.5)
+        cache.forward(0, hidden.cuda(), ids.cuda(), p.cuda())
+    _, slot_expert, _, _ = cache.state(0)
+    assert (slot_expert >= 0).all()
+    for slot in (0, 7, 15):
+        assert np.array_equal(cache.read_slot(0, slot), bank[int(slot_expert[slot])].numpy())
+    cache.close()
+
+
+# ------------------------------------------------------------------------------------ a4-a6: output
+def test_config1_tiny_output(B, tiny_layer):
+    """Config 1: d_model 256, d_ff 128, 8 experts, top-2, 16 tokens, all resident, seed 0."""
+    ora, bank = tiny_layer
+    s = synth.TINY
+    hidden, ids, p = helpers.routed_inputs(s, 16, seed=0)
+    y, ref = ora.forward(hidden, ids, p)
+    outs = {}
+    for C, Cw in [(8, 0), (2, 0), (4, 2), (5, 3)]:
+        cache = B.Cache(s, [bank], C, max_tokens=16, wave_cap=Cw)
+        out = cache.forward(0, hidden.cuda(), ids.cuda(), p.cuda())
+        helpers.check_output(out, y, ref, f"C={C}")
+        outs[(C, Cw)] = out.cpu()
+        assert cache.status() == 0
+        cache.close()
+    base = outs[(8, 0)]
+    for key, o in outs.items():                      # independent of slot count and wave partition, bit for bit
+        assert torch.equal(o.view(torch.int16), base.view(torch.int16)), key
+
+
+@pytest.mark.parametrize("T", [1, 3, 8, 9, 33, 100])
+def test_mid_shape_ragged_groups(B, mid_layer, T):
+    ora, bank = mid_layer
+    s = synth.MID
+    hidden, ids, p = helpers.routed_inputs(s, T, seed=50 + T, alpha=1.0)
+    y, ref = ora.forward(hidden, ids, p)
+    cache = B.Cache(s, [bank], s.num_experts, max_tokens=128)
+    out = cache.forward(0, hidden.cuda(), ids.cuda(), p.cuda())
+    helpers.check_output(out, y, ref, f"T={T}")
+    cache2 = B.Cache(s, [bank], 6, max_tokens=128, wave_cap=3)
+    out2 = cache2.forward(0, hidden.cuda(), ids.cuda(), p.cuda())
+    assert torch.equal(out2.view(torch.int16), out.view(torch.int16))
+    cache.close()
+    cache2.close()
+
+
+def test_config2_decode_olmoe(B, olmoe_layer):
+    """Config 2: OLMoE shape, 1 token per step, 64 slots, fresh hidden state per step."""
+    ora, bank = olmoe_layer
+    s = synth.OLMOE
+    cache = B.Cache(s, [bank], 64, max_tokens=16)
+    for step in range(4):
+        hidden, ids, p = helpers.routed_inputs(s, 1, seed=2000 + step)
+        y, ref = ora.forward(hidden, ids, p)
+        out = cache.forward(0, hidden.cuda(), ids.cuda(), p.cuda())
+        helpers.check_output(out, y, ref, f"step {step}")
+    st = cache.stats(0)
+    assert all(v == 0 for v in st.values())          # full residency bypasses the accounting
+    cache.close()
+
+
+def test_config3_offload_matches_resident(B, olmoe_layer):
+    """Config 3: 16 slots over the 64-expert host bank, 16 tokens per step, Zipf-biased routing:
+    1-4 waves with LRU misses; output equals the 64-slot run bit for bit and the oracle within tolerance."""
+    ora, bank = olmoe_layer
+    s = synth.OLMOE
+    full = B.Cache(s, [bank], 64, max_tokens=16)
+    small = B.Cache(s, [bank], 16, max_tokens=16)
+    half = B.Cache(s, [bank], 16, max_tokens=16, wave_cap=8)
+    sc = ocache.SlotCache(64, 16, 0, bytes_per_expert=small.bytes_per_expert)
+    waves = set()
+    for step, alpha in enumerate([2.0, 1.0, 0.5, 0.0, 2.0, 0.0]):
+        hidden, ids, p = helpers.routed_inputs(s, 16, seed=3000 + step, alpha=alpha)
+        h, i, w = hidden.cuda(), ids.cuda(), p.cuda()
+        o_full = full.forward(0, h, i, w)
+        o_small = small.forward(0, h, i, w)
+        o_half = half.forward(0, h, i, w)
+        plan = compare_plan(small, sc, ids)
+        waves.add(plan.n_waves)
+        assert torch.equal(o_small.view(torch.int16), o_full.view(torch.int16)), step
+        assert torch.equal(o_half.view(torch.int16), o_full.view(torch.int16)), step
+        if step in (1, 3):
+            y, ref = ora.forward(hidden, ids, p)
+            helpers.check_output(o_small, y, ref, f"step {step}")
+    assert len(waves) >= 3 and max(waves) == 4
+    for c in (full, small, half):
+        assert c.status() == 0
+        c.close()
+
+
+@pytest.mark.parametrize("M", [1, 2, 3, 4, 7, 8, 15, 16, 17, 31, 32, 33, 63, 64, 65, 127, 128])
+def test_group_size_sweep_single_expert(B, M):
+    """Kernel check in the paper's style (Section 5.3): token-group sizes 1..128 on one expert of OLMoE's
+    gate/up and down shapes, against the dequantised reference."""
+    s = synth.Shape(d_model=2048, d_ff=1024, num_experts=2, top_k=1)
+    if not hasattr(test_group_size_sweep_single_expert, "layer"):
+        test_group_size_sweep_single_expert.layer = helpers.make_layer(s, seed=77)
+    ora, bank = test_group_size_sweep_single_expert.layer
+    hidden = synth.hidden_states(s, M, seed=900 + M)
+    ids = torch.ones((M, 1), dtype=torch.int32)
+    p = torch.rand((M, 1), generator=torch.Generator().manual_seed(M)) + 0.5
+    y, ref = ora.forward(hidden, ids, p)
+    cache = B.Cache(s, [bank], 2, max_tokens=128)
+    out = cache.forward(0, hidden.cuda(), ids.cuda(), p.cuda())
+    helpers.check_output(out, y, ref, f"M={M}")
+    cache.close()
+
+
+# ------------------------------------------------------------------------------------ edge cases
+def test_edge_cases(B, tiny_layer):
+    ora, bank = tiny_layer
+    s = synth.TINY
+    cache = B.Cache(s, [bank], 4, max_tokens=16)
+    # T = 0 is a no-op
+    empty = torch.empty((0, s.d_model), dtype=torch.bfloat16, device="cuda")
+    cache.forward(0, empty, torch.empty((0, 2), dtype=torch.int32, device="cuda"),
+                  torch.empty((0, 2), dtype=torch.float32, device="cuda"))
+    # invalid ids contribute nothing and raise the sticky status
+    hidden, ids, p = helpers.routed_inputs(s, 6, seed=9)
+    bad = ids.clone()
+    bad[2, 1] = 99
+    bad[4, 0] = -1
+    y, ref = ora.forward(hidden, bad, p)
+    out = cache.forward(0, hidden.cuda(), bad.cuda(), p.cuda())
+    helpers.check_output(out, y, ref, "bad ids")
+    assert cache.status() == B.EXMOE_ERR_BAD_EXPERT_ID
+    assert cache.status() == 0                       # cleared by the read
+    # too many tokens, bad layer
+    big = synth.hidden_states(s, 17, seed=1).cuda()
+    with pytest.raises(B.ExmoeError):
+        cache.forward(0, big, torch.zeros((17, 2), dtype=torch.int32, device="cuda"),
+                      torch.zeros((17, 2), dtype=torch.float32, device="cuda"))
+    with pytest.raises(B.ExmoeError):
+        cache.forward(3, hidden.cuda(), ids.cuda(), p.cuda())
+    # same input twice -> identical bits; zero weights -> zero output
+    o1 = cache.forward(0, hidden.cuda(), ids.cuda(), p.cuda()).clone()
+    o2 = cache.forward(0, hidden.cuda(), ids.cuda(), p.cuda())
+    assert torch.equal(o1.view(torch.int16), o2.view(torch.int16))
+    oz = cache.forward(0, hidden.cuda(), ids.cuda(), torch.zeros_like(p).cuda())
+    assert not oz.float().abs().max().item()
+    cache.close()
+
+
+def test_create_rejects_bad_arguments(B, tiny_layer):
+    ora, bank = tiny_layer
+    s = synth.TINY
+    with pytest.raises(B.ExmoeError) as ei:
+        B.Cache(s, [bank], 1, max_tokens=4)           # C < k
+    assert ei.value.code == B.EXMOE_ERR_SHAPE
+    with pytest.raises(B.ExmoeError) as ei:
+        B.Cache(s, [bank], 9, max_tokens=4)           # C > E
+    assert ei.value.code == B.EXMOE_ERR_SHAPE
+    unpinned = bank.clone()                           # pageable copy
+    with pytest.raises(B.ExmoeError) as ei:
+        B.Cache(s, [unpinned], 4, max_tokens=4)
+    assert ei.value.code == B.EXMOE_ERR_NOT_PINNED
+
+
+def test_multi_layer_caches_are_independent(B, tiny_layer):
+    ora, bank = tiny_layer
+    s = synth.TINY
+    ora2, bank2 = helpers.make_layer(s, seed=1)
+    cache = B.Cache(s, [bank, bank2], 3, max_tokens=16)
+    hidden, ids, p = helpers.routed_inputs(s, 8, seed=21)
+    for layer, o in ((0, ora), (1, ora2), (0, ora)):
+        out = cache.forward(layer, hidden.cuda(), ids.cuda(), p.cuda())
+        y, ref = o.forward(hidden, ids, p)
+        helpers.check_output(out, y, ref, f"layer {layer}")
+    assert cache.stats(0)["forwards"] == 2 and cache.stats(1)["forwards"] == 1
+    cache.reset(0)
+    assert cache.stats(0)["forwards"] == 0 and (cache.state(0)[0] == -1).all()
+    cache.close()
