@@ -1,0 +1,383 @@
+#!/usr/bin/env python
+"""Benchmark of the complete-expert MoE layer forward on B200 (one process per GPU).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload NAME]
+
+A step is one pass of the whole hot path (grouping, gate/up GEMM + SwiGLU, down GEMM, combine; plus
+resolution and miss copies when slots < experts) over one batch of synthetic tokens of one
+OLMoE-shaped sparse layer.  Default workload: decode, 1 token per step, 64 slots (fully resident),
+fresh seeded hidden state per step, rotating over 16 independent layer banks (3.3 GB of packed
+experts) so that every step's weights come from HBM, not from the 126 MB L2.
+
+Prints ONE JSON line: MoE-layer tokens/s (inputs resident in HBM, CUDA-graph replay, CUDA events),
+the end-to-end number through host buffers, the roofline of the dominant kernel (gate/up GEMM;
+packed weight + scale bytes it must read / its CUDA-event time / measured HBM copy rate), the CPU
+oracle timed on the host cores on a bounded sample, SM clocks sampled during the timed region and
+the number of kernels launched.  `--impl reference` times the CPU oracle alone.
+"""
+import argparse
+import json
+import os
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np
+import torch
+
+from paper_2608_15383_b200 import synth
+
+WORKLOADS = {
+    # name: (tokens per step, slots, layers rotated over, Zipf alpha, description)
+    "decode": (1, 64, 16, 0.0, "config2: OLMoE-shaped decode, T=1, 64 slots resident, top-8 of 64, int4 g128"),
+    "decode16": (16, 64, 16, 1.0, "OLMoE-shaped batched decode, T=16, 64 slots resident, Zipf(1.1) routing"),
+    "offload": (16, 16, 1, 1.0, "config3: T=16, 16 slots over a 64-expert pinned host bank, Zipf(1.1) routing"),
+    "prefill": (2048, 64, 1, 0.0, "config4: OLMoE-shaped prefill, T=2048, 64 slots resident, uniform routing"),
+}
+METRIC = "moe_layer_tokens_per_s"
+UNIT = "tokens/s"
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return {"hbm_gbs": float(p["hbm_gbs"]), "bf16_tflops": float(p["bf16_tflops"]),
+                "bf16_tflops_sustained": float(p.get("bf16_tflops_sustained", p["bf16_tflops"])), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+class ClockSampler:
+    """nvidia-smi clocks and throttle reasons of this rank's GPU while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.f = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+        try:
+            self.p = subprocess.Popen(["nvidia-smi", "-i", str(index), f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                                       "-lms", "100"], stdout=self.f, stderr=subprocess.DEVNULL)
+        except Exception:
+            self.p = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.p is None:
+            return out
+        self.p.terminate()
+        try:
+            self.p.wait(timeout=5)
+        except Exception:
+            self.p.kill()
+        self.f.flush()
+        self.f.seek(0)
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in self.f.read().splitlines():
+            parts = [x.strip() for x in line.split(",")]
+            if len(parts) < 7:
+                continue
+            try:
+                sm.append(float(parts[0]))
+                mx.append(float(parts[1]))
+            except ValueError:
+                continue
+            for n, v in zip(names, parts[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        self.f.close()
+        os.unlink(self.f.name)
+        if sm:
+            out.update(sm_mhz=float(np.median(sm)), sm_max_mhz=float(max(mx)), reasons=sorted(reasons), samples=len(sm))
+        return out
+
+
+def make_inputs(shape, T, n_sets, alpha, seed0, device):
+    """n_sets independent (hidden, ids, weights) batches, generated on the device, routed by Eq. 1."""
+    wr = synth.router_weights(shape, seed0 + 1, device=device)
+    bias = synth.zipf_bias(shape.num_experts, alpha, seed0 + 2).to(device) if alpha else None
+    hs, ids, ws = [], [], []
+    for i in range(n_sets):
+        h = synth.hidden_states(shape, T, seed0 + 10 + i, device=device)
+        a, b = synth.route(h, wr, shape.top_k, bias)
+        hs.append(h)
+        ids.append(a)
+        ws.append(b)
+    return hs, ids, ws
+
+
+def build_banks(shape, layers, seed0, device, keep_layer0=False):
+    """Per layer: draw BF16 expert weights on the device, pack them with exmoe_pack into a pinned host bank."""
+    from paper_2608_15383_b200 import binding
+    banks, kept = [], None
+    for l in range(layers):
+        wg, wu, wd = synth.expert_weights(shape, seed0 + l, device=device)
+        banks.append(binding.pack_bank(shape, wg, wu, wd, device=device))
+        if l == 0 and keep_layer0:
+            kept = (wg.cpu(), wu.cpu(), wd.cpu())
+        del wg, wu, wd
+    return banks, kept
+
+
+def oracle_leg(shape, T, weights_cpu, hs, ids, ws, budget_s):
+    """Time the CPU oracle as it stands on batches of the same workload until ~budget_s of work is done."""
+    from oracle import moe as omoe, quant as oquant
+    try:
+        from threadpoolctl import threadpool_info
+        cores = max([p.get("num_threads", 1) for p in threadpool_info()] + [1])
+    except Exception:
+        cores = 1
+    wg, wu, wd = weights_cpu
+    cache = {}
+
+    def expert(e):
+        if e not in cache:
+            if len(cache) >= 24:
+                cache.pop(next(iter(cache)))
+            cache[e] = tuple(oquant.dequantize_g128(*oquant.quantize_g128(w[e].float().numpy())) for w in (wg, wu, wd))
+        return cache[e]
+
+    done_tokens, t0, steps = 0, time.perf_counter(), 0
+    t_rows = min(T, 8)                                   # a bounded sample of each batch's tokens
+    while steps < len(hs):
+        h = hs[steps][:t_rows].float().cpu().numpy()
+        i = ids[steps][:t_rows].cpu().numpy()
+        w = ws[steps][:t_rows].cpu().numpy()
+        omoe.moe_layer_forward(h, i, w, expert, shape.num_experts)
+        done_tokens += t_rows
+        steps += 1
+        if time.perf_counter() - t0 > budget_s:
+            break
+    dt = time.perf_counter() - t0
+    return {"value": done_tokens / dt, "unit": UNIT, "cores": int(cores), "kind": "oracle",
+            "sample": f"{steps} steps x {t_rows} tokens of layer 0 ({done_tokens} tokens, {dt:.1f} s), dequantising on the fly"}
+
+
+def run_reference(args, rank, world):
+    if rank != 0:
+        return
+    T, C, L, alpha, desc = WORKLOADS[args.workload]
+    shape = synth.OLMOE
+    wg, wu, wd = synth.expert_weights(shape, 2000, device="cpu")
+    hs, ids, ws = make_inputs(shape, T, max(args.steps + args.warmup, 4), alpha, 2000, "cpu")
+    per_step_budget = max(2.0, 120.0 / max(args.steps + args.warmup, 1))
+    from oracle import moe as omoe, quant as oquant
+    leg = None
+    for _ in range(args.warmup):
+        oracle_leg(shape, T, (wg, wu, wd), hs[:1], ids[:1], ws[:1], 0.0)
+    t0 = time.perf_counter()
+    tokens = 0
+    for s in range(args.steps):
+        leg = oracle_leg(shape, T, (wg, wu, wd), hs[s:s + 1], ids[s:s + 1], ws[s:s + 1], per_step_budget)
+        tokens += min(T, 8)
+    dt = time.perf_counter() - t0
+    value = tokens / dt
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": 1e3 * dt / max(args.steps, 1), "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": desc, "note": "CPU oracle on a bounded sample: first min(T,8) tokens of each step"},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": leg["cores"] if leg else 1, "kind": "oracle",
+                             "sample": f"{args.steps} steps x {min(T, 8)} tokens"},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=1000)
+    ap.add_argument("--warmup", type=int, default=50)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="decode", choices=sorted(WORKLOADS))
+    ap.add_argument("--cpu-budget", type=float, default=15.0, help="seconds of CPU oracle work for cpu_baseline")
+    args = ap.parse_args()
+
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+
+    if args.impl == "reference":
+        if args.steps > 50:
+            args.steps = 50
+        args.warmup = min(args.warmup, 3)
+        run_reference(args, rank, world)
+        return
+
+    import torch.distributed as dist
+    from paper_2608_15383_b200 import binding, build
+    if rank == 0:
+        build.build()
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+        dist.barrier()
+    binding.lib()
+
+    T, C, L, alpha, desc = WORKLOADS[args.workload]
+    shape = synth.OLMOE
+    K, W = args.steps, max(args.warmup, 3)
+    peaks = load_peaks()
+
+    # ---- data: replicas only, every rank holds the same workload with its own seed offset
+    seed0 = 2000 + 100000 * rank
+    banks, w_cpu = build_banks(shape, L, seed0, dev, keep_layer0=(rank == 0))
+    cache = binding.Cache(shape, banks, C, max_tokens=T, device=dev)
+    n_sets = min(K + W, 1024) if T <= 64 else 4
+    hs, ids, ws = make_inputs(shape, T, n_sets, alpha, seed0, dev)
+    outs = [torch.empty_like(hs[0]) for _ in range(2)]
+    stream = torch.cuda.Stream(device=dev)
+    identity = (C == shape.num_experts)
+
+    def step(i, out):
+        cache.forward(i % L, hs[i % n_sets], ids[i % n_sets], ws[i % n_sets], out=out, stream=stream)
+
+    with torch.cuda.stream(stream):
+        for i in range(3):
+            step(i, outs[0])
+    stream.synchronize()
+
+    # ---- device-timed region: CUDA-graph replay when the layer is fully resident (no host sync inside)
+    launches0 = binding.exmoe_launch_count()
+    graph_w = graph_k = None
+    if identity:
+        graph_w, graph_k = torch.cuda.CUDAGraph(), torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph_w, stream=stream):
+            for i in range(W):
+                step(i, outs[i & 1])
+        launches0 = binding.exmoe_launch_count()
+        with torch.cuda.graph(graph_k, stream=stream):
+            for i in range(W, W + K):
+                step(i, outs[i & 1])
+        launches = binding.exmoe_launch_count() - launches0
+        with torch.cuda.stream(stream):
+            graph_w.replay()
+    else:
+        with torch.cuda.stream(stream):
+            for i in range(W):
+                step(i, outs[i & 1])
+    stream.synchronize()
+    if world > 1:
+        dist.barrier()
+    torch.cuda.synchronize()
+    sampler = ClockSampler(local_rank)
+    time.sleep(0.15)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    stats0 = cache.stats(0) if not identity else None
+    with torch.cuda.stream(stream):
+        e0.record(stream)
+        if identity:
+            graph_k.replay()
+        else:
+            launches0 = binding.exmoe_launch_count()
+            for i in range(W, W + K):
+                step(i, outs[i & 1])
+            launches = binding.exmoe_launch_count() - launches0
+        e1.record(stream)
+    stream.synchronize()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1)
+    clocks = sampler.stop()
+    if world > 1:
+        dist.barrier()
+        t = torch.tensor([ms], device=dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms = float(t.item())
+    value = world * K * T / (ms * 1e-3)
+
+    # ---- per-kernel CUDA-event times of the same steps (roofline of the dominant kernel)
+    cache.profile_enable(True)
+    n_prof = min(K, 200)
+    with torch.cuda.stream(stream):
+        for i in range(W, W + n_prof):
+            step(i, outs[i & 1])
+    stream.synchronize()
+    kinds = {}
+    for kind, name in enumerate(["plan", "gate_up", "down", "combine"]):
+        tot, n = cache.profile_read(kind)
+        kinds[name] = {"us_per_launch": 1e3 * tot / max(n, 1), "launches": n}
+    cache.profile_enable(False)
+    bpe = cache.bytes_per_expert
+    w13_bytes = bpe * 2 // 3
+    active = float(np.mean([len(torch.unique(ids[i % n_sets])) for i in range(W, W + n_prof)]))
+    if args.workload == "prefill":
+        flops = 2.0 * T * shape.top_k * 2 * shape.d_ff * shape.d_model          # gate/up GEMM of one step
+        achieved = flops / (kinds["gate_up"]["us_per_launch"] * 1e-6) / 1e12
+        roof = {"bound": "tensor", "achieved": achieved, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
+                "frac": achieved / peaks["bf16_tflops"], "traffic": None, "kernel": "gate_up", "peak_source": peaks["source"]}
+    else:
+        gu_bytes = active * w13_bytes                                            # packed gate/up codes + scales
+        achieved = gu_bytes / (kinds["gate_up"]["us_per_launch"] * 1e-6) / 1e9
+        roof = {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                "frac": achieved / peaks["hbm_gbs"], "traffic": None, "kernel": "gate_up (decode_gemm_kernel)",
+                "bytes_per_launch": gu_bytes, "peak_source": peaks["source"] + " copy rate, burst"}
+    step_gbs = active * bpe / (ms * 1e-3 / K) / 1e9
+
+    # ---- end to end: host buffers in, host buffer out, copies inside the timed region
+    n_e2e = min(K, 300)
+    h_h = [h.cpu().pin_memory() for h in hs[:8]]
+    h_i = [x.cpu().pin_memory() for x in ids[:8]]
+    h_w = [x.cpu().pin_memory() for x in ws[:8]]
+    h_out = torch.empty_like(h_h[0]).pin_memory()
+    d_h, d_i, d_w, d_o = torch.empty_like(hs[0]), torch.empty_like(ids[0]), torch.empty_like(ws[0]), torch.empty_like(hs[0])
+
+    def e2e_step(i):
+        j = i % 8
+        with torch.cuda.stream(stream):
+            d_h.copy_(h_h[j], non_blocking=True)
+            d_i.copy_(h_i[j], non_blocking=True)
+            d_w.copy_(h_w[j], non_blocking=True)
+            cache.forward(i % L, d_h, d_i, d_w, out=d_o, stream=stream)
+            h_out.copy_(d_o, non_blocking=True)
+        stream.synchronize()
+
+    for i in range(3):
+        e2e_step(i)
+    if world > 1:
+        dist.barrier()
+    t0 = time.perf_counter()
+    for i in range(n_e2e):
+        e2e_step(i)
+    dt = time.perf_counter() - t0
+    if world > 1:
+        t = torch.tensor([dt], device=dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        dt = float(t.item())
+    h2d = h_h[0].numel() * 2 + h_i[0].numel() * 4 + h_w[0].numel() * 4
+    e2e = {"value": world * n_e2e * T / dt, "unit": UNIT, "h2d_bytes_per_step": int(h2d),
+           "d2h_bytes_per_step": int(h_out.numel() * 2), "steps": n_e2e}
+
+    status = cache.status()
+    extra = {}
+    if not identity:
+        st = cache.stats(0)
+        extra = {"hit_rate": st["hits"] / max(st["lookups"], 1), "h2d_expert_bytes_per_token":
+                 st["h2d_bytes"] / max(st["forwards"] * T, 1), "waves_per_step": st["waves"] / max(st["forwards"], 1)}
+
+    if rank == 0:
+        cpu = oracle_leg(shape, T, w_cpu, hs, ids, ws, args.cpu_budget)
+        line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
+                "ms_per_step": ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+                "dtype": "int4 weights x bf16 activations, fp32 accumulate", "data": "synthetic",
+                "config": {"workload": desc, "tokens_per_step": T, "slots": C, "layers_rotated": L,
+                           "l2": "inputs larger than L2: steps rotate over %d layer banks (%.2f GB packed)" % (L, L * 64 * bpe / 1e9)
+                           if L > 1 else "single layer bank (%.0f MB packed) vs 126 MB L2" % (64 * bpe / 1e6),
+                           "timing": "CUDA graph replay of all steps" if identity else "host-driven loop (one plan read-back per step)",
+                           "active_experts_per_step": active, "packed_gb_per_s_whole_step": step_gbs,
+                           "kernel_us": kinds, "parallelism": "replicas only (no collective)", "status": status, **extra},
+                "roofline": roof, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": int(launches), "clocks": clocks}
+        print(json.dumps(line), flush=True)
+    cache.close()
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -138,6 +138,14 @@ int exmoe_cache_reset(exmoe_cache* cache, int layer);                     /* emp
 int exmoe_status(exmoe_cache* cache);   /* synchronises; returns and clears the sticky device status */
 int exmoe_cache_destroy(exmoe_cache* cache);
 
+/* Measurement hooks (the paper has no counterpart).  While enabled, every exmoe_moe_forward brackets
+ * its kernels with CUDA events on the caller's stream, per kind: 0 = resolution + grouping,
+ * 1 = gate/up GEMM + SwiGLU, 2 = down GEMM, 3 = combine.  exmoe_profile_read synchronises and returns
+ * the summed event time and the number of bracketed launches of one kind since the last enable.
+ * Not for use during stream capture. */
+int exmoe_profile_enable(exmoe_cache* cache, int on);
+int exmoe_profile_read(exmoe_cache* cache, int kind, double* total_ms, uint64_t* launches);
+
 /* Kernels launched by this library since it was loaded (all streams, all caches). */
 uint64_t exmoe_launch_count(void);
 

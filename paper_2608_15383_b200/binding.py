@@ -54,6 +54,8 @@ _SIGNATURES = {
     "exmoe_cache_reset": (c_int, [c_void_p, c_int]),
     "exmoe_status": (c_int, [c_void_p]),
     "exmoe_cache_destroy": (c_int, [c_void_p]),
+    "exmoe_profile_enable": (c_int, [c_void_p, c_int]),
+    "exmoe_profile_read": (c_int, [c_void_p, c_int, POINTER(ctypes.c_double), POINTER(c_uint64)]),
     "exmoe_launch_count": (c_uint64, []),
 }
 
@@ -226,6 +228,15 @@ class Cache:
 
     def status(self):
         return int(lib().exmoe_status(self.handle))
+
+    def profile_enable(self, on=True):
+        _check(lib().exmoe_profile_enable(self.handle, int(bool(on))), "exmoe_profile_enable")
+
+    def profile_read(self, kind):
+        """(total event ms, bracketed launches) of kind 0 plan, 1 gate/up, 2 down, 3 combine."""
+        ms, n = ctypes.c_double(), c_uint64()
+        _check(lib().exmoe_profile_read(self.handle, int(kind), byref(ms), byref(n)), "exmoe_profile_read")
+        return ms.value, int(n.value)
 
     def close(self):
         if getattr(self, "handle", None):

@@ -67,6 +67,30 @@ struct exmoe_cache {
     std::vector<std::vector<uint64_t>> slot_last_seq;   // [L][C] compute event that last read the slot
     int last_layer;
     int last_T;
+    bool prof_on;                             // per-kernel CUDA-event timing (exmoe_profile_*)
+    std::vector<cudaEvent_t> prof_ev[4];      // begin/end pairs per kernel kind
+    size_t prof_used[4];
+};
+
+enum { PROF_PLAN = 0, PROF_GATEUP = 1, PROF_DOWN = 2, PROF_COMBINE = 3 };
+
+// Brackets one launch (or launch group) with a pair of events on its own stream when profiling is on.
+struct ProfScope {
+    exmoe_cache* c;
+    int kind;
+    cudaStream_t st;
+    ProfScope(exmoe_cache* c_, int kind_, cudaStream_t st_) : c(c_), kind(kind_), st(st_) { mark(); }
+    ~ProfScope() { mark(); }
+    void mark() {
+        if (!c->prof_on) return;
+        std::vector<cudaEvent_t>& v = c->prof_ev[kind];
+        if (c->prof_used[kind] == v.size()) {
+            cudaEvent_t e;
+            if (cudaEventCreate(&e) != cudaSuccess) return;
+            v.push_back(e);
+        }
+        cudaEventRecord(v[c->prof_used[kind]++], st);
+    }
 };
 
 static void carve_workspace(exmoe_cache* c, uint8_t* ws, size_t* total) {
@@ -261,12 +285,16 @@ int exmoe_moe_forward(exmoe_cache* c, int layer, const void* hidden, const int32
     c->last_T = T;
 
     if (!identity) {
+        ProfScope ps(c, PROF_PLAN, st);
         launch_resolve(s, C, c->Cw, c->bpe, topk_ids, P, c->state[layer], c->plan, c->d_status, st);
         if (cudaMemcpyAsync(c->h_plan, c->plan.header, c->plan_d2h_bytes, cudaMemcpyDeviceToHost, st) != cudaSuccess)
             return EXMOE_ERR_CUDA;
         if (cudaEventRecord(c->ev_plan, st) != cudaSuccess) return EXMOE_ERR_CUDA;
     }
-    launch_group(s, C, c->n_keys, c->max_waves, identity, topk_ids, P, c->plan, c->d_status, st);
+    {
+        ProfScope ps(c, PROF_PLAN, st);
+        launch_group(s, C, c->n_keys, c->max_waves, identity, topk_ids, P, c->plan, c->d_status, st);
+    }
 
     int n_waves = 1;
     const int32_t *h_wave_of = nullptr, *h_slot_of = nullptr, *h_miss = nullptr;
@@ -314,8 +342,14 @@ int exmoe_moe_forward(exmoe_cache* c, int layer, const void* hidden, const int32
             for (int e = 0; e < E; ++e) groups += (h_wave_of[e] == w);
         }
         a.wave_start = c->plan.wave_start + w;
-        launch_decode_gateup(a, (const __nv_bfloat16*)hidden, c->act, T, groups, st);
-        launch_decode_down(a, c->act, topk_weights, c->y, T, groups, st);
+        {
+            ProfScope ps(c, PROF_GATEUP, st);
+            launch_decode_gateup(a, (const __nv_bfloat16*)hidden, c->act, T, groups, st);
+        }
+        {
+            ProfScope ps(c, PROF_DOWN, st);
+            launch_decode_down(a, c->act, topk_weights, c->y, T, groups, st);
+        }
         if (!identity) {
             ++c->seq;
             cudaEventRecord(c->ev_compute[c->seq % kEventRing], st);                  // completion event of the wave
@@ -323,7 +357,10 @@ int exmoe_moe_forward(exmoe_cache* c, int layer, const void* hidden, const int32
                 if (h_wave_of[e] == w) c->slot_last_seq[layer][h_slot_of[e]] = c->seq;
         }
     }
-    launch_combine(c->y, topk_ids, E, T, k, s.d_model, (__nv_bfloat16*)out, st);
+    {
+        ProfScope ps(c, PROF_COMBINE, st);
+        launch_combine(c->y, topk_ids, E, T, k, s.d_model, (__nv_bfloat16*)out, st);
+    }
     return cudaGetLastError() == cudaSuccess ? EXMOE_OK : EXMOE_ERR_CUDA;
 }
 
@@ -398,9 +435,35 @@ int exmoe_status(exmoe_cache* c) {
     return v;
 }
 
+int exmoe_profile_enable(exmoe_cache* c, int on) {
+    if (!c) return EXMOE_ERR_ARG;
+    if (cudaDeviceSynchronize() != cudaSuccess) return EXMOE_ERR_CUDA;
+    c->prof_on = on != 0;
+    for (int k = 0; k < 4; ++k) c->prof_used[k] = 0;
+    return EXMOE_OK;
+}
+
+int exmoe_profile_read(exmoe_cache* c, int kind, double* total_ms, uint64_t* launches) {
+    if (!c || kind < 0 || kind > 3 || !total_ms || !launches) return EXMOE_ERR_ARG;
+    if (cudaDeviceSynchronize() != cudaSuccess) return EXMOE_ERR_CUDA;
+    double sum = 0.0;
+    const size_t n = c->prof_used[kind] / 2;
+    for (size_t i = 0; i < n; ++i) {
+        float ms = 0.f;
+        if (cudaEventElapsedTime(&ms, c->prof_ev[kind][2 * i], c->prof_ev[kind][2 * i + 1]) != cudaSuccess)
+            return EXMOE_ERR_CUDA;
+        sum += ms;
+    }
+    *total_ms = sum;
+    *launches = n;
+    return EXMOE_OK;
+}
+
 int exmoe_cache_destroy(exmoe_cache* c) {
     if (!c) return EXMOE_ERR_ARG;
     cudaDeviceSynchronize();
+    for (int k = 0; k < 4; ++k)
+        for (cudaEvent_t e : c->prof_ev[k]) cudaEventDestroy(e);
     if (c->h_plan) cudaFreeHost(c->h_plan);
     if (c->copy_stream) cudaStreamDestroy(c->copy_stream);
     if (c->ev_plan) cudaEventDestroy(c->ev_plan);
