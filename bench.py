@@ -196,6 +196,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="decode", choices=sorted(WORKLOADS))
     ap.add_argument("--cpu-budget", type=float, default=15.0, help="seconds of CPU oracle work for cpu_baseline")
+    ap.add_argument("--layers", type=int, default=0, help="layer banks to rotate over (0 = the workload's default)")
     args = ap.parse_args()
 
     rank = int(os.environ.get("RANK", "0"))
@@ -221,6 +222,7 @@ def main():
     binding.lib()
 
     T, C, L, alpha, desc = WORKLOADS[args.workload]
+    L = args.layers or L
     shape = synth.OLMOE
     K, W = args.steps, max(args.warmup, 3)
     peaks = load_peaks()
@@ -258,6 +260,7 @@ def main():
         launches = binding.exmoe_launch_count() - launches0
         with torch.cuda.stream(stream):
             graph_w.replay()
+            graph_k.replay()          # untimed first replay: uploads the instantiated graph to the device
     else:
         with torch.cuda.stream(stream):
             for i in range(W):
@@ -291,17 +294,36 @@ def main():
         ms = float(t.item())
     value = world * K * T / (ms * 1e-3)
 
-    # ---- per-kernel CUDA-event times of the same steps (roofline of the dominant kernel)
-    cache.profile_enable(True)
+    # ---- per-kernel times (roofline of the dominant kernel): the same steps with ONLY one kernel kind
+    # launched, timed with CUDA events on the launching stream (graph replay when fully resident)
     n_prof = min(K, 200)
-    with torch.cuda.stream(stream):
-        for i in range(W, W + n_prof):
-            step(i, outs[i & 1])
-    stream.synchronize()
     kinds = {}
-    for kind, name in enumerate(["plan", "gate_up", "down", "combine"]):
-        tot, n = cache.profile_read(kind)
-        kinds[name] = {"us_per_launch": 1e3 * tot / max(n, 1), "launches": n}
+    for kind, name in ((1, "gate_up"), (2, "down")):
+        cache.profile_enable(False, only=kind)
+        a0, a1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        if identity:
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.stream(stream):
+                step(0, outs[0])
+            stream.synchronize()
+            with torch.cuda.graph(g, stream=stream):
+                for i in range(W, W + n_prof):
+                    step(i, outs[i & 1])
+            with torch.cuda.stream(stream):
+                g.replay()
+                a0.record(stream)
+                g.replay()
+                a1.record(stream)
+        else:
+            with torch.cuda.stream(stream):
+                for i in range(3):
+                    step(i, outs[0])
+                a0.record(stream)
+                for i in range(W, W + n_prof):
+                    step(i, outs[i & 1])
+                a1.record(stream)
+        stream.synchronize()
+        kinds[name] = {"us_per_launch": 1e3 * a0.elapsed_time(a1) / n_prof, "launches": n_prof}
     cache.profile_enable(False)
     bpe = cache.bytes_per_expert
     w13_bytes = bpe * 2 // 3

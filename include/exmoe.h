@@ -142,7 +142,11 @@ int exmoe_cache_destroy(exmoe_cache* cache);
  * its kernels with CUDA events on the caller's stream, per kind: 0 = resolution + grouping,
  * 1 = gate/up GEMM + SwiGLU, 2 = down GEMM, 3 = combine.  exmoe_profile_read synchronises and returns
  * the summed event time and the number of bracketed launches of one kind since the last enable.
- * Not for use during stream capture. */
+ * Not for use during stream capture.
+ * `on` bit 0 switches the event bracketing; bits 4-5, if non-zero, make later forwards launch ONLY
+ * the kernels of that kind (1 gate/up, 2 down, 3 combine) so that one kernel can be timed alone, e.g.
+ * in a CUDA-graph replay; the layer output is then meaningless.  exmoe_profile_enable(cache, 0)
+ * restores normal operation. */
 int exmoe_profile_enable(exmoe_cache* cache, int on);
 int exmoe_profile_read(exmoe_cache* cache, int kind, double* total_ms, uint64_t* launches);
 

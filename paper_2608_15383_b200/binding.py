@@ -229,8 +229,9 @@ class Cache:
     def status(self):
         return int(lib().exmoe_status(self.handle))
 
-    def profile_enable(self, on=True):
-        _check(lib().exmoe_profile_enable(self.handle, int(bool(on))), "exmoe_profile_enable")
+    def profile_enable(self, on=True, only=0):
+        """on: bracket kernels with events; only: 0 all kernels, 1 gate/up, 2 down, 3 combine (timing runs)."""
+        _check(lib().exmoe_profile_enable(self.handle, int(bool(on)) | (int(only) << 4)), "exmoe_profile_enable")
 
     def profile_read(self, kind):
         """(total event ms, bracketed launches) of kind 0 plan, 1 gate/up, 2 down, 3 combine."""

@@ -57,6 +57,11 @@ struct exmoe_cache {
     size_t plan_d2h_bytes;                    // header | wave_of | slot_of | misses, contiguous
     __nv_bfloat16* act;                       // [max_pairs, I] SwiGLU output, grouped row order
     float* y;                                 // [max_pairs, H] weighted expert outputs, pair order
+    int* arrive;                              // fused-combine arrival counters of the small path
+    size_t arrive_words;
+    bool last_small;
+    bool last_pair;
+    int32_t* saved_ids;                       // ids of the last pairwise call (plan materialised on request)
     int32_t* h_plan;                          // pinned staging of the plan
     cudaStream_t copy_stream;
     cudaEvent_t ev_plan;
@@ -68,6 +73,7 @@ struct exmoe_cache {
     int last_layer;
     int last_T;
     bool prof_on;                             // per-kernel CUDA-event timing (exmoe_profile_*)
+    int prof_only;                            // 0 = all kernels; 1..3 = launch only that kind (timing runs)
     std::vector<cudaEvent_t> prof_ev[4];      // begin/end pairs per kernel kind
     size_t prof_used[4];
 };
@@ -119,6 +125,9 @@ static void carve_workspace(exmoe_cache* c, uint8_t* ws, size_t* total) {
     c->plan.perm = k.take<int32_t>(c->max_pairs);
     c->act = k.take<__nv_bfloat16>((size_t)c->max_pairs * s.d_ff);
     c->y = k.take<float>((size_t)c->max_pairs * s.d_model);
+    c->arrive_words = (size_t)(kSmallMaxPairs / s.top_k + 1) * (s.d_model / kPanelRows);
+    c->arrive = k.take<int>(c->arrive_words);
+    c->saved_ids = k.take<int32_t>(kPairMaxPairs);
     *total = k.off;
 }
 
@@ -256,6 +265,7 @@ int exmoe_cache_create(exmoe_cache** out, const exmoe_shape* shape, int num_laye
     }
     ok = ok && cudaMemset(c->d_status, 0, 256) == cudaSuccess;
     ok = ok && cudaMemset(c->plan.header, 0, c->plan_d2h_bytes) == cudaSuccess;
+    ok = ok && cudaMemset(c->arrive, 0, c->arrive_words * 4) == cudaSuccess;
     for (int l = 0; l < num_layers && ok; ++l) ok = reset_layer(c, l) == EXMOE_OK;
     if (ok && c->C == c->shape.num_experts) {            // full residency: preload, slot = expert id
         for (int l = 0; l < num_layers && ok; ++l)
@@ -284,6 +294,8 @@ int exmoe_moe_forward(exmoe_cache* c, int layer, const void* hidden, const int32
     c->last_layer = layer;
     c->last_T = T;
 
+    const bool small = (P <= kSmallMaxPairs && C <= kSmallMaxSlots);   // decode: grouping fused into the GEMM kernels
+    c->last_small = small;
     if (!identity) {
         ProfScope ps(c, PROF_PLAN, st);
         launch_resolve(s, C, c->Cw, c->bpe, topk_ids, P, c->state[layer], c->plan, c->d_status, st);
@@ -291,7 +303,7 @@ int exmoe_moe_forward(exmoe_cache* c, int layer, const void* hidden, const int32
             return EXMOE_ERR_CUDA;
         if (cudaEventRecord(c->ev_plan, st) != cudaSuccess) return EXMOE_ERR_CUDA;
     }
-    {
+    if (!small) {
         ProfScope ps(c, PROF_PLAN, st);
         launch_group(s, C, c->n_keys, c->max_waves, identity, topk_ids, P, c->plan, c->d_status, st);
     }
@@ -320,6 +332,10 @@ int exmoe_moe_forward(exmoe_cache* c, int layer, const void* hidden, const int32
     a.H = s.d_model;
     a.I = s.d_ff;
 
+    const bool pairwise = small && P <= kPairMaxPairs && n_waves == 1;
+    c->last_pair = pairwise;
+    if (small && n_waves == 0)                           // no valid id at all: the output is zero
+        cudaMemsetAsync(out, 0, (size_t)T * s.d_model * 2, st);
     int mi = 0;
     for (int w = 0; w < n_waves; ++w) {
         int groups = identity ? (E < P ? E : P) : 0;
@@ -342,13 +358,43 @@ int exmoe_moe_forward(exmoe_cache* c, int layer, const void* hidden, const int32
             for (int e = 0; e < E; ++e) groups += (h_wave_of[e] == w);
         }
         a.wave_start = c->plan.wave_start + w;
-        {
-            ProfScope ps(c, PROF_GATEUP, st);
-            launch_decode_gateup(a, (const __nv_bfloat16*)hidden, c->act, T, groups, st);
-        }
-        {
-            ProfScope ps(c, PROF_DOWN, st);
-            launch_decode_down(a, c->act, topk_weights, c->y, T, groups, st);
+        if (small) {
+            SmallWave sw{};
+            sw.ids = topk_ids;
+            sw.wave_of = identity ? nullptr : c->plan.wave_of;
+            sw.slot_of = identity ? nullptr : c->plan.slot_of;
+            sw.n_pairs = P;
+            sw.E = E;
+            sw.wave = w;
+            sw.plan = c->plan;
+            sw.status = c->d_status;
+            sw.arrive = c->arrive;
+            sw.hidden = (const __nv_bfloat16*)hidden;
+            sw.act = c->act;
+            sw.topk_w = topk_weights;
+            sw.y = c->y;
+            sw.out = (__nv_bfloat16*)out;
+            sw.max_rows = T;
+            sw.max_groups = groups;
+            sw.pairwise = pairwise;
+            sw.saved_ids = c->saved_ids;
+            if (!c->prof_only || c->prof_only == PROF_GATEUP) {
+                ProfScope ps(c, PROF_GATEUP, st);
+                launch_small_wave(a, sw, st, true, false);
+            }
+            if (!c->prof_only || c->prof_only == PROF_DOWN) {
+                ProfScope ps(c, PROF_DOWN, st);
+                launch_small_wave(a, sw, st, false, true);
+            }
+        } else {
+            if (!c->prof_only || c->prof_only == PROF_GATEUP) {
+                ProfScope ps(c, PROF_GATEUP, st);
+                launch_decode_gateup(a, (const __nv_bfloat16*)hidden, c->act, T, groups, st);
+            }
+            if (!c->prof_only || c->prof_only == PROF_DOWN) {
+                ProfScope ps(c, PROF_DOWN, st);
+                launch_decode_down(a, c->act, topk_weights, c->y, T, groups, st);
+            }
         }
         if (!identity) {
             ++c->seq;
@@ -357,7 +403,7 @@ int exmoe_moe_forward(exmoe_cache* c, int layer, const void* hidden, const int32
                 if (h_wave_of[e] == w) c->slot_last_seq[layer][h_slot_of[e]] = c->seq;
         }
     }
-    {
+    if (!small && (!c->prof_only || c->prof_only == PROF_COMBINE)) {
         ProfScope ps(c, PROF_COMBINE, st);
         launch_combine(c->y, topk_ids, E, T, k, s.d_model, (__nv_bfloat16*)out, st);
     }
@@ -384,11 +430,29 @@ int exmoe_debug_last_plan(exmoe_cache* c, int layer, int32_t* n_active, int32_t*
     if (layer != c->last_layer) return EXMOE_ERR_STATE;
     if (cudaDeviceSynchronize() != cudaSuccess) return EXMOE_ERR_CUDA;
     const int E = c->shape.num_experts;
+    if (c->last_pair) {
+        // the pairwise path never groups: run the grouping kernel now on the ids it kept
+        launch_group(c->shape, c->C, c->n_keys, c->max_waves, c->C == E, c->saved_ids, c->last_T * c->shape.top_k,
+                     c->plan, c->d_status, nullptr);
+        if (cudaDeviceSynchronize() != cudaSuccess) return EXMOE_ERR_CUDA;
+        c->last_pair = false;
+        c->last_small = false;
+    }
     std::vector<int32_t> hdr(HDR_WORDS + 5 * (size_t)E);
     bool ok = cudaMemcpy(hdr.data(), c->plan.header, hdr.size() * 4, cudaMemcpyDeviceToHost) == cudaSuccess;
     std::vector<int32_t> cnt(c->n_keys);
     ok = ok && cudaMemcpy(cnt.data(), c->plan.counts, cnt.size() * 4, cudaMemcpyDeviceToHost) == cudaSuccess;
     if (!ok) return EXMOE_ERR_CUDA;
+    std::vector<int32_t> off(c->n_keys + 1);
+    ok = cudaMemcpy(off.data(), c->plan.offsets, off.size() * 4, cudaMemcpyDeviceToHost) == cudaSuccess;
+    if (!ok) return EXMOE_ERR_CUDA;
+    if (c->last_small) {                                 // each wave's kernel published its own part only
+        const int first = hdr[HDR_N_WAVES] * c->C;
+        int total = 0;
+        for (int i = 0; i < first; ++i) total += cnt[i];
+        for (int i = first; i < c->n_keys; ++i) cnt[i] = 0;
+        for (int i = first; i <= c->n_keys; ++i) off[i] = total;
+    }
     if (n_active) *n_active = hdr[HDR_N_ACTIVE];
     if (n_waves) *n_waves = hdr[HDR_N_WAVES];
     if (n_misses) *n_misses = hdr[HDR_N_MISSES];
@@ -399,7 +463,7 @@ int exmoe_debug_last_plan(exmoe_cache* c, int layer, int32_t* n_active, int32_t*
         for (int e = 0; e < E; ++e) slot_of[e] = identity ? (cnt[e] > 0 ? e : -1) : hdr[HDR_WORDS + E + e];
     if (misses) std::memcpy(misses, hdr.data() + HDR_WORDS + 2 * E, 3 * (size_t)E * 4);
     if (counts) std::memcpy(counts, cnt.data(), cnt.size() * 4);
-    if (offsets) ok = ok && cudaMemcpy(offsets, c->plan.offsets, (c->n_keys + 1) * 4, cudaMemcpyDeviceToHost) == cudaSuccess;
+    if (offsets) std::memcpy(offsets, off.data(), off.size() * 4);
     if (perm) ok = ok && cudaMemcpy(perm, c->plan.perm, (size_t)c->last_T * c->shape.top_k * 4, cudaMemcpyDeviceToHost) == cudaSuccess;
     return ok ? EXMOE_OK : EXMOE_ERR_CUDA;
 }
@@ -438,7 +502,8 @@ int exmoe_status(exmoe_cache* c) {
 int exmoe_profile_enable(exmoe_cache* c, int on) {
     if (!c) return EXMOE_ERR_ARG;
     if (cudaDeviceSynchronize() != cudaSuccess) return EXMOE_ERR_CUDA;
-    c->prof_on = on != 0;
+    c->prof_on = (on & 1) != 0;
+    c->prof_only = (on >> 4) & 3;
     for (int k = 0; k < 4; ++k) c->prof_used[k] = 0;
     return EXMOE_OK;
 }

@@ -58,6 +58,28 @@ struct GemmArgs {
     int H, I;
 };
 
+// One wave of the small-problem path (decode): the GEMM kernels rebuild the grouping themselves.
+struct SmallWave {
+    const int32_t* ids;         // [n_pairs] top-k ids
+    const int32_t* wave_of;     // null when C = E (slot = expert id, single wave)
+    const int32_t* slot_of;
+    int n_pairs, E, wave;
+    PlanPtrs plan;              // published for the test hooks
+    int* status;
+    int* arrive;                // [T * H/16] zero-initialised arrival counters of the fused combine
+    const __nv_bfloat16* hidden;
+    __nv_bfloat16* act;
+    const float* topk_w;
+    float* y;
+    __nv_bfloat16* out;
+    int max_rows, max_groups;
+    bool pairwise;              // T*k <= kPairMaxPairs and a single wave: per-pair gate/up, by-token down
+    int32_t* saved_ids;         // [kPairMaxPairs]
+};
+constexpr int kPairMaxPairs = 32;
+constexpr int kSmallMaxPairs = 512;
+constexpr int kSmallMaxSlots = 1024;
+
 // launch accounting (exmoe_launch_count)
 void count_launch(int n = 1);
 
@@ -72,6 +94,7 @@ void launch_decode_gateup(const GemmArgs& a, const __nv_bfloat16* hidden, __nv_b
                           int max_groups, cudaStream_t st);
 void launch_decode_down(const GemmArgs& a, const __nv_bfloat16* act, const float* topk_w, float* y, int max_rows,
                         int max_groups, cudaStream_t st);
+void launch_small_wave(const GemmArgs& a, const SmallWave& w, cudaStream_t st, bool gateup, bool down);
 void launch_combine(const float* y, const int32_t* ids, int E, int T, int k, int H, __nv_bfloat16* out,
                     cudaStream_t st);
 

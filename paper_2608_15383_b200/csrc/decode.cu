@@ -11,6 +11,15 @@
 // round trip touches the weights.  Per 128-wide group the integer-valued partial sums are scaled
 // in binary32 by the FP16 group scale (post-scaling: codes and activations enter the MMA exactly).
 // K-split partials are reduced through shared memory in a fixed order.
+//
+// Two flavours share the body:
+//   SMALL (T*k <= 512): a decode step is launch-latency bound, so the chain of dependent global
+//     loads is cut to two levels: every CTA rebuilds the wave's token grouping (histogram, prefix
+//     sum, stable permutation) in shared memory straight from topk_ids; CTA 0 also publishes it.
+//     The down kernel is launched with programmatic dependent launch: it prefetches its weights
+//     while the gate/up kernel still runs, and it folds the fixed-order combine in: the last CTA
+//     to finish a (token, column tile) sums the k pair rows in order j = 0..k-1 (no spin wait).
+//   otherwise: the grouping kernels' global plan is used and a separate combine kernel follows.
 #include "common.cuh"
 
 namespace exmoe {
@@ -31,28 +40,131 @@ __device__ __forceinline__ uint32_t ldg_stream32(const void* p) {
 }
 __device__ __forceinline__ void mma_m16n8k16(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
                                              uint32_t b0, uint32_t b1) {
-    asm volatile(
-        "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+    asm("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
         : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
         : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
-// two offset-binary nibbles (bits s..s+3 of each 16-bit half) -> bf16x2 of the signed codes:
-// 0x4300 | u is BF16 128+u exactly; subtracting 136 leaves q = u - 8.
-__device__ __forceinline__ uint32_t dequant_pair(uint32_t w, int s) {
-    uint32_t v = ((w >> s) & 0x000f000fu) | 0x43004300u;
-    uint32_t bias = 0x43084308u;                         // BF16 136.0 twice
-    __nv_bfloat162 r = __hsub2(*reinterpret_cast<__nv_bfloat162*>(&v), *reinterpret_cast<__nv_bfloat162*>(&bias));
-    return *reinterpret_cast<uint32_t*>(&r);
+// two offset-binary nibbles (bits s..s+3 of each 16-bit half) -> bf16x2 of 128 + u = 136 + q:
+// 0x4300 | u is that BF16 value exactly (one shift and one lop3 per pair of codes).
+__device__ __forceinline__ uint32_t code_pair(uint32_t w, int s) {
+    uint32_t r;
+    asm("lop3.b32 %0, %1, 0x000f000f, 0x43004300, 0xea;" : "=r"(r) : "r"(w >> s));   // (a & b) | c
+    return r;
+}
+// sum of the 8 BF16 values of a 16-byte chunk, in binary32
+__device__ __forceinline__ float sum8_bf16(const uint4& v) {
+    const uint32_t r[4] = {v.x, v.y, v.z, v.w};
+    float s = 0.f;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) s += __uint_as_float(r[i] << 16) + __uint_as_float(r[i] & 0xffff0000u);
+    return s;
+}
+__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void grid_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+// Shared-memory plan of ONE wave, rebuilt by every CTA of the SMALL kernels.
+struct SmallPlan {
+    int* cnt;     // [C] pairs per slot in this wave
+    int* off;     // [C + 1] exclusive prefix sum (rows local to the wave)
+    int* gkeys;   // [C] slots with cnt > 0, ascending
+    int* lkey;    // [P] slot of the pair in this wave, -1 other wave, -2 invalid id
+    int* perm;    // [P] pair indices of this wave ordered by (slot, pair)
+    int n_groups;
+    int row_base; // valid pairs in earlier waves = first grouped row of this wave
+};
+
+struct SmallArgs {
+    const int32_t* ids;
+    const int32_t* wave_of;   // null in identity mode (C = E: slot = expert id, one wave)
+    const int32_t* slot_of;
+    int n_pairs, E, wave;
+    int32_t* pub_counts;      // global plan arrays published by CTA 0 of the gate/up kernel
+    int32_t* pub_offsets;
+    int32_t* pub_perm;
+    int32_t* header;
+    int* status;
+    int* arrive;              // [T * tiles] arrival counters of the fused combine (zero between calls)
+    __nv_bfloat16* out;       // [T, H]
+    int32_t* saved_ids;       // [kPairMaxPairs] copy of the ids kept by the pairwise path
+};
+
+__device__ __forceinline__ void build_small_plan(const SmallArgs& sa, int C, SmallPlan& sp, int* s_scalars) {
+    const int tid = threadIdx.x, P = sa.n_pairs;
+    for (int i = tid; i < C; i += blockDim.x) sp.cnt[i] = 0;
+    if (tid < 4) s_scalars[tid] = 0;                      // [0] rows before this wave, [1] n_groups, [2] bad id
+    __syncthreads();
+    for (int p = tid; p < P; p += blockDim.x) {
+        const int id = sa.ids[p];
+        int lk = -2;
+        if (id >= 0 && id < sa.E) {
+            const int w = sa.wave_of ? sa.wave_of[id] : 0;
+            const int s = sa.slot_of ? sa.slot_of[id] : id;
+            if (w < sa.wave) atomicAdd(&s_scalars[0], 1);
+            lk = (w == sa.wave) ? s : -1;
+            if (lk >= 0) atomicAdd(&sp.cnt[lk], 1);
+        } else {
+            s_scalars[2] = 1;
+        }
+        sp.lkey[p] = lk;
+    }
+    __syncthreads();
+    if (tid < 32) {
+        const unsigned lt = (1u << tid) - 1u;
+        int running = 0, ng = 0;
+        for (int base = 0; base < C; base += 32) {
+            const int kx = base + tid;
+            const int v = kx < C ? sp.cnt[kx] : 0;
+            int incl = v;
+#pragma unroll
+            for (int d = 1; d < 32; d <<= 1) {
+                const int o = __shfl_up_sync(0xffffffffu, incl, d);
+                if (tid >= d) incl += o;
+            }
+            if (kx < C) sp.off[kx] = running + incl - v;
+            const unsigned b = __ballot_sync(0xffffffffu, v > 0);
+            if (v > 0) sp.gkeys[ng + __popc(b & lt)] = kx;
+            ng += __popc(b);
+            running += __shfl_sync(0xffffffffu, incl, 31);
+        }
+        if (tid == 0) {
+            sp.off[C] = running;
+            s_scalars[1] = ng;
+        }
+    }
+    __syncthreads();
+    for (int p = tid; p < P; p += blockDim.x) {
+        const int lk = sp.lkey[p];
+        if (lk < 0) continue;
+        int r = 0;
+        for (int j = 0; j < p; ++j) r += (sp.lkey[j] == lk);
+        sp.perm[sp.off[lk] + r] = p;
+    }
+    __syncthreads();
+    sp.row_base = s_scalars[0];
+    sp.n_groups = s_scalars[1];
 }
 
 // NB  = 128-wide blocks held in registers per warp and matrix
 // NCH = 8-row activation chunks per pass (rows per pass = 8*NCH)
-template <int NB, int NCH, bool GATEUP>
-__global__ void __launch_bounds__(256)
-decode_gemm_kernel(GemmArgs a, const __nv_bfloat16* __restrict__ x_src, __nv_bfloat16* __restrict__ act_out,
-                   const float* __restrict__ topk_w, float* __restrict__ y_out, int KS, int blocks_per_warp) {
+enum { MODE_PLAN = 0, MODE_SMALL = 1, MODE_PAIR = 2 };
+
+// MODE_PLAN  : groups come from the grouping kernels' global plan
+// MODE_SMALL : every CTA rebuilds the wave's grouping in shared memory (T*k <= 512)
+// MODE_PAIR  : one item per token-expert pair, no grouping at all (T*k <= 32, gate/up only)
+#ifndef EXMOE_MINB_NB2
+#define EXMOE_MINB_NB2 1
+#endif
+#ifndef EXMOE_MINB_NB4
+#define EXMOE_MINB_NB4 1
+#endif
+template <int NB, int NCH, bool GATEUP, int MODE>
+__global__ void __launch_bounds__(256, (NCH == 1 && NB == 2) ? EXMOE_MINB_NB2 : (NCH == 1 && NB == 4) ? EXMOE_MINB_NB4 : 1)
+decode_gemm_kernel(GemmArgs a, SmallArgs sa, const __nv_bfloat16* __restrict__ x_src,
+                   __nv_bfloat16* __restrict__ act_out, const float* __restrict__ topk_w, float* __restrict__ y_out,
+                   int KS, int blocks_per_warp) {
     constexpr int NM = GATEUP ? 2 : 1;
     extern __shared__ __align__(16) unsigned char smem[];
+    __shared__ int s_scalars[4];
     const int K = GATEUP ? a.H : a.I;                  // reduction length
     const int NR = GATEUP ? a.I : a.H;                 // output rows of the weight matrix
     const int KB = K / kGroup;
@@ -61,20 +173,81 @@ decode_gemm_kernel(GemmArgs a, const __nv_bfloat16* __restrict__ x_src, __nv_bfl
     const int x_stride = K * 2 + 64;                   // bytes; +64 keeps 128-bit fragment loads conflict-free
     unsigned char* xs = smem;
     float* red = reinterpret_cast<float*>(smem + (size_t)8 * NCH * x_stride);   // [KS-1][PP][NM][NCH][32][4]
+    float* adj = red + (size_t)(KS - 1) * PP * NM * NCH * 128;                  // [KB][8*NCH]
+    int* plan_mem = reinterpret_cast<int*>(adj + (size_t)KB * 8 * NCH);
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int q = lane >> 2, c = lane & 3;
     const int ks = warp % KS, pp = warp / KS;
-    const int g0 = a.wave_start[0], g1 = a.wave_start[1];
-    const int n_items = (g1 - g0) * tiles;
     const size_t w13_bytes = matrix_bytes(2 * a.I, a.H);
     const bool single_chunk = (blocks_per_warp == NB);
+    const int C = a.num_slots;
 
+    constexpr bool SMALL = (MODE == MODE_SMALL);
+    constexpr bool PAIR = (MODE == MODE_PAIR);
+    SmallPlan sp{};
+    int g0 = 0, n_items;
+    if (PAIR) {
+        grid_launch_dependents();
+        n_items = sa.n_pairs * tiles;
+        if (blockIdx.x == 0 && tid < sa.n_pairs) {     // keep the ids so the plan can be materialised on request
+            const int id = sa.ids[tid];
+            sa.saved_ids[tid] = id;
+            if (id < 0 || id >= sa.E) atomicExch(sa.status, EXMOE_ERR_BAD_EXPERT_ID);
+        }
+    } else if (SMALL) {
+        if (GATEUP) grid_launch_dependents();          // let the down kernel start prefetching its weights
+        sp.cnt = plan_mem;
+        sp.off = sp.cnt + C;
+        sp.gkeys = sp.off + C + 1;
+        sp.lkey = sp.gkeys + C;
+        sp.perm = sp.lkey + sa.n_pairs;
+        build_small_plan(sa, C, sp, s_scalars);
+        n_items = sp.n_groups * tiles;
+        if (GATEUP && blockIdx.x == 0) {               // publish the wave's part of the plan (test hook, stats)
+            for (int i = tid; i < C; i += 256) {
+                sa.pub_counts[sa.wave * C + i] = sp.cnt[i];
+                sa.pub_offsets[sa.wave * C + i] = sp.row_base + sp.off[i];
+            }
+            for (int i = tid; i < sp.off[C]; i += 256) sa.pub_perm[sp.row_base + i] = sp.perm[i];
+            if (tid == 0) {
+                sa.pub_offsets[sa.wave * C + C] = sp.row_base + sp.off[C];
+                if (!sa.wave_of) {                     // identity mode: no resolution kernel wrote the header
+                    sa.header[HDR_N_ACTIVE] = sp.n_groups;
+                    sa.header[HDR_N_WAVES] = sp.n_groups ? 1 : 0;
+                    sa.header[HDR_N_MISSES] = 0;
+                    sa.header[HDR_BAD_ID] = s_scalars[2];
+                }
+                if (s_scalars[2]) atomicExch(sa.status, EXMOE_ERR_BAD_EXPERT_ID);
+            }
+        }
+    } else {
+        g0 = a.wave_start[0];
+        n_items = (a.wave_start[1] - g0) * tiles;
+    }
+
+    bool waited = false;
     for (int item = blockIdx.x; item < n_items; item += gridDim.x) {
-        const int key = a.group_keys[g0 + item / tiles];
         const int tile = item % tiles;
-        const int slot = key % a.num_slots;
-        const int m_rows = a.counts[key], row0 = a.offsets[key];
+        int slot, m_rows, row0, lrow0 = 0;
+        if (PAIR) {
+            const int p = item / tiles;                // activation row = pair index, one row per item
+            const int id = sa.ids[p];
+            if (id < 0 || id >= sa.E) continue;        // uniform over the CTA
+            slot = sa.slot_of ? sa.slot_of[id] : id;
+            m_rows = 1;
+            row0 = p;
+        } else if (SMALL) {
+            slot = sp.gkeys[item / tiles];
+            m_rows = sp.cnt[slot];
+            lrow0 = sp.off[slot];
+            row0 = sp.row_base + lrow0;
+        } else {
+            const int key = a.group_keys[g0 + item / tiles];
+            slot = key % C;
+            m_rows = a.counts[key];
+            row0 = a.offsets[key];
+        }
         const uint8_t* wbase = a.slots + (size_t)slot * a.slot_stride + (GATEUP ? 0 : w13_bytes);
         const int panel = tile * PP + pp;              // panel (pair) index inside the matrix
         const uint8_t* mat[NM];
@@ -109,29 +282,46 @@ decode_gemm_kernel(GemmArgs a, const __nv_bfloat16* __restrict__ x_src, __nv_bfl
                 }
                 if (b0 == 0) {
                     // stage this pass's activation rows (zero rows beyond the group) while the weights fly
+                    if (SMALL && !GATEUP && !waited) {
+                        grid_dependency_wait();        // the gate/up kernel's activations are complete and visible
+                        waited = true;
+                    }
                     __syncthreads();                   // previous readers of xs / red are done
+                    // also: adj[kb][n] = -136 * sum_k x[n][k] over each 128-wide block (see the block loop)
                     const int chunks_per_row = K / 8;
-                    for (int idx = tid; idx < 8 * NCH * chunks_per_row; idx += 256) {
+                    const int rows_here = min(8 * NCH, m_rows - pass0);   // rows beyond are zero registers, not staged
+                    const int total = rows_here * chunks_per_row;
+                    for (int base = warp * 32; base < total; base += 256) {
+                        const int idx = base + lane;
                         const int n = idx / chunks_per_row, ck = idx % chunks_per_row;
                         uint4 v = make_uint4(0, 0, 0, 0);
-                        if (pass0 + n < m_rows) {
-                            const int r = row0 + pass0 + n;
-                            const size_t src_row = GATEUP ? (size_t)(a.perm[r] / a.top_k) : (size_t)r;
+                        if (idx < total) {
+                            size_t src_row;
+                            if (PAIR) src_row = (size_t)(row0 / a.top_k);
+                            else if (GATEUP) src_row = (size_t)((SMALL ? sp.perm[lrow0 + pass0 + n] : a.perm[row0 + pass0 + n]) / a.top_k);
+                            else src_row = (size_t)(row0 + pass0 + n);
                             v = *reinterpret_cast<const uint4*>(x_src + src_row * K + ck * 8);
+                            *reinterpret_cast<uint4*>(xs + (size_t)n * x_stride + ck * 16) = v;
                         }
-                        *reinterpret_cast<uint4*>(xs + (size_t)n * x_stride + ck * 16) = v;
+                        float sx = sum8_bf16(v);
+#pragma unroll
+                        for (int m = 8; m >= 1; m >>= 1) sx += __shfl_xor_sync(0xffffffffu, sx, m);   // 16 chunks = one block
+                        if (idx < total && (ck & 15) == 0) adj[(ck >> 4) * (8 * NCH) + n] = -136.f * sx;
                     }
                     __syncthreads();
                 }
+                const int rows_here = min(8 * NCH, m_rows - pass0);
 #pragma unroll
                 for (int b = 0; b < NB; ++b) {
+                    // acc = sum (136 + q) x over the block's 128 columns (codes enter the MMA as 128 + u,
+                    // exact in BF16); adj = -136 * sum x was formed while staging; acc + adj = sum q x.
                     float acc[NM][NCH][4];
 #pragma unroll
-                    for (int m = 0; m < NM; ++m)
+                    for (int ch = 0; ch < NCH; ++ch)
 #pragma unroll
-                        for (int ch = 0; ch < NCH; ++ch)
+                        for (int i = 0; i < 4; ++i)
 #pragma unroll
-                            for (int i = 0; i < 4; ++i) acc[m][ch][i] = 0.f;
+                            for (int m = 0; m < NM; ++m) acc[m][ch][i] = 0.f;
 #pragma unroll
                     for (int h = 0; h < 2; ++h) {
 #pragma unroll
@@ -139,33 +329,40 @@ decode_gemm_kernel(GemmArgs a, const __nv_bfloat16* __restrict__ x_src, __nv_bfl
                             const int k0 = (kb0 + b) * kGroup + 64 * h + 32 * set + 8 * c;
                             uint4 xb[NCH];
 #pragma unroll
-                            for (int ch = 0; ch < NCH; ++ch)
-                                xb[ch] = *reinterpret_cast<const uint4*>(xs + (size_t)(8 * ch + q) * x_stride + k0 * 2);
+                            for (int ch = 0; ch < NCH; ++ch) {
+                                xb[ch] = make_uint4(0, 0, 0, 0);
+                                if (8 * ch + q < rows_here)
+                                    xb[ch] = *reinterpret_cast<const uint4*>(xs + (size_t)(8 * ch + q) * x_stride + k0 * 2);
+                            }
 #pragma unroll
                             for (int m = 0; m < NM; ++m) {
                                 const uint32_t wq = set ? wreg[m][b][h].z : wreg[m][b][h].x;    // row q
                                 const uint32_t wq8 = set ? wreg[m][b][h].w : wreg[m][b][h].y;   // row q + 8
-                                uint32_t a0 = dequant_pair(wq, 0), a1 = dequant_pair(wq8, 0);
-                                uint32_t a2 = dequant_pair(wq, 4), a3 = dequant_pair(wq8, 4);
+                                uint32_t a0 = code_pair(wq, 0), a1 = code_pair(wq8, 0);
+                                uint32_t a2 = code_pair(wq, 4), a3 = code_pair(wq8, 4);
 #pragma unroll
                                 for (int ch = 0; ch < NCH; ++ch) mma_m16n8k16(acc[m][ch], a0, a1, a2, a3, xb[ch].x, xb[ch].y);
-                                a0 = dequant_pair(wq, 8), a1 = dequant_pair(wq8, 8);
-                                a2 = dequant_pair(wq, 12), a3 = dequant_pair(wq8, 12);
+                                a0 = code_pair(wq, 8), a1 = code_pair(wq8, 8);
+                                a2 = code_pair(wq, 12), a3 = code_pair(wq8, 12);
 #pragma unroll
                                 for (int ch = 0; ch < NCH; ++ch) mma_m16n8k16(acc[m][ch], a0, a1, a2, a3, xb[ch].z, xb[ch].w);
                             }
                         }
                     }
+                    float2 cr[NCH];
+#pragma unroll
+                    for (int ch = 0; ch < NCH; ++ch)
+                        cr[ch] = *reinterpret_cast<const float2*>(adj + (size_t)(kb0 + b) * (8 * NCH) + 8 * ch + 2 * c);
 #pragma unroll
                     for (int m = 0; m < NM; ++m) {     // post-scale the group's integer-valued sums
                         const __half2 sc = *reinterpret_cast<const __half2*>(&sreg[m][b]);
                         const float s_lo = __low2float(sc), s_hi = __high2float(sc);
 #pragma unroll
                         for (int ch = 0; ch < NCH; ++ch) {
-                            tot[m][ch][0] = fmaf(s_lo, acc[m][ch][0], tot[m][ch][0]);
-                            tot[m][ch][1] = fmaf(s_lo, acc[m][ch][1], tot[m][ch][1]);
-                            tot[m][ch][2] = fmaf(s_hi, acc[m][ch][2], tot[m][ch][2]);
-                            tot[m][ch][3] = fmaf(s_hi, acc[m][ch][3], tot[m][ch][3]);
+                            tot[m][ch][0] = fmaf(s_lo, acc[m][ch][0] + cr[ch].x, tot[m][ch][0]);
+                            tot[m][ch][1] = fmaf(s_lo, acc[m][ch][1] + cr[ch].y, tot[m][ch][1]);
+                            tot[m][ch][2] = fmaf(s_hi, acc[m][ch][2] + cr[ch].x, tot[m][ch][2]);
+                            tot[m][ch][3] = fmaf(s_hi, acc[m][ch][3] + cr[ch].y, tot[m][ch][3]);
                         }
                     }
                 }
@@ -197,20 +394,311 @@ decode_gemm_kernel(GemmArgs a, const __nv_bfloat16* __restrict__ x_src, __nv_bfl
                     for (int i = 0; i < 4; ++i) {
                         const int n = pass0 + 8 * ch + 2 * c + (i & 1);
                         if (n >= m_rows) continue;
-                        const int r = row0 + n;
                         const int orow = (tile * PP + pp) * kPanelRows + q + 8 * (i >> 1);
                         if (GATEUP) {
                             const float g = tot[0][ch][i], u = tot[NM - 1][ch][i];
                             const float act = g / (1.f + __expf(-g)) * u;
-                            act_out[(size_t)r * a.I + orow] = __float2bfloat16_rn(act);
+                            act_out[(size_t)(row0 + n) * a.I + orow] = __float2bfloat16_rn(act);
                         } else {
-                            const int pair = a.perm[r];
+                            const int pair = SMALL ? sp.perm[lrow0 + n] : a.perm[row0 + n];
                             y_out[(size_t)pair * a.H + orow] = topk_w[pair] * tot[0][ch][i];
                         }
                     }
             }
         }
+
+        if (SMALL && !GATEUP) {
+            // Fused combine (Eq. 2's sum over the selected experts): the CTA that completes the last
+            // pair of a token for this column tile adds the k rows in the fixed order j = 0..k-1.
+            const int cols = kPanelRows * PP, col0 = tile * cols, k = a.top_k;
+            __threadfence();
+            __syncthreads();
+            for (int i = 0; i < m_rows; ++i) {
+                const int t = sp.perm[lrow0 + i] / k;
+                __shared__ int s_last;
+                if (tid == 0) {
+                    int need = 0;
+                    for (int j = 0; j < k; ++j) need += (sp.lkey[t * k + j] != -2);
+                    const int old = atomicAdd(&sa.arrive[t * tiles + tile], 1);
+                    s_last = (old == need - 1);
+                    if (s_last) sa.arrive[t * tiles + tile] = 0;          // self-cleaning for the next call
+                }
+                __syncthreads();
+                if (s_last) {
+                    __threadfence();
+                    for (int col = tid; col < cols; col += 256) {
+                        float sum = 0.f;
+                        for (int j = 0; j < k; ++j)
+                            if (sp.lkey[t * k + j] != -2) sum += __ldcg(y_out + (size_t)(t * k + j) * a.H + col0 + col);
+                        sa.out[(size_t)t * a.H + col0 + col] = __float2bfloat16_rn(sum);
+                    }
+                }
+                __syncthreads();
+            }
+        }
     }
+    if (SMALL && !GATEUP && !waited) grid_dependency_wait();
+    if (SMALL && GATEUP && blockIdx.x == 0) {
+        // tokens whose ids are all invalid get no contribution: their output row is zero
+        const int k = a.top_k, T = sa.n_pairs / k;
+        if (sa.wave == 0 && s_scalars[2])
+            for (int t = 0; t < T; ++t) {
+                int need = 0;
+                for (int j = 0; j < k; ++j) need += (sp.lkey[t * k + j] != -2);
+                if (need == 0)
+                    for (int col = tid; col < a.H; col += 256) sa.out[(size_t)t * a.H + col] = __float2bfloat16_rn(0.f);
+            }
+    }
+}
+
+
+// Down projection + routing weight + combine for tiny batches (T*k <= 32, one wave): one CTA per
+// (token, 16-column panel), one warp per selected expert.  Each warp streams its expert's panel over
+// the whole K (all loads in flight at once), the k results are summed in the fixed order j = 0..k-1
+// through shared memory and the BF16 output row is written directly: no pair buffer, no atomics.
+// Launched as a programmatic dependent of the gate/up kernel: weights are prefetched before the
+// dependency wait.  `KSg`/`bpwg` replay the grouped kernel's K-split order so that both paths round
+// identically.
+template <int NBT>
+__global__ void __launch_bounds__(256)
+token_down_kernel(GemmArgs a, SmallArgs sa, const __nv_bfloat16* __restrict__ act, const float* __restrict__ topk_w,
+                  int bpwg) {
+    extern __shared__ __align__(16) unsigned char smem[];
+    const int K = a.I, KB = K / kGroup, k = a.top_k;
+    const int x_stride = K * 2 + 64;
+    unsigned char* xs = smem;                                          // [k][x_stride]
+    float* ys = reinterpret_cast<float*>(smem + (size_t)k * x_stride); // [k][16]
+    int* s_valid = reinterpret_cast<int*>(ys + k * 16);                // [k]
+    float* adj = reinterpret_cast<float*>(s_valid + k);                // [KB][k]  -136 * block sums of the activations
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int q = lane >> 2, c = lane & 3;
+    const int panels = a.H / kPanelRows;
+    const int t = blockIdx.x / panels, panel = blockIdx.x % panels;
+    const size_t w13_bytes = matrix_bytes(2 * a.I, a.H);
+    bool staged = false;
+
+    for (int j0 = 0; j0 < k; j0 += 8) {
+        const int j = j0 + warp;
+        const int pair = t * k + j;
+        int id = -1;
+        if (j < k) id = sa.ids[pair];
+        const bool valid = (j < k) && id >= 0 && id < sa.E;
+        const float rw = valid ? topk_w[pair] : 0.f;   // requested early: it is needed only in the epilogue
+        float result[2] = {0.f, 0.f};
+        float total[2] = {0.f, 0.f};
+        for (int b0 = 0; b0 < KB; b0 += NBT) {
+            uint4 wreg[NBT][2];
+            uint32_t sreg[NBT];
+            if (valid) {
+                const int slot = sa.slot_of ? sa.slot_of[id] : id;
+                const uint8_t* mat = a.slots + (size_t)slot * a.slot_stride + w13_bytes + (size_t)panel * KB * kBlockBytes;
+#pragma unroll
+                for (int b = 0; b < NBT; ++b) {
+                    const uint8_t* blk = mat + (size_t)(b0 + b) * kBlockBytes;
+                    wreg[b][0] = ldg_stream128(blk + lane * 16);
+                    wreg[b][1] = ldg_stream128(blk + 512 + lane * 16);
+                    sreg[b] = ldg_stream32(blk + kCodeBytes + q * 4);
+                }
+            }
+            if (!staged) {                          // first chunk: the activations arrive after the weights were requested
+                grid_dependency_wait();
+                const int chunks_per_row = K / 8, total = k * chunks_per_row;
+                for (int base = warp * 32; base < total; base += 256) {
+                    const int idx = base + lane;
+                    const int n = idx / chunks_per_row, ck = idx % chunks_per_row;
+                    uint4 v = make_uint4(0, 0, 0, 0);
+                    if (idx < total) {
+                        v = *reinterpret_cast<const uint4*>(act + (size_t)(t * k + n) * K + ck * 8);
+                        *reinterpret_cast<uint4*>(xs + (size_t)n * x_stride + ck * 16) = v;
+                    }
+                    float sx = sum8_bf16(v);
+#pragma unroll
+                    for (int m = 8; m >= 1; m >>= 1) sx += __shfl_xor_sync(0xffffffffu, sx, m);
+                    if (idx < total && (ck & 15) == 0) adj[(ck >> 4) * k + n] = -136.f * sx;
+                }
+                __syncthreads();
+                staged = true;
+            }
+            if (valid) {
+#pragma unroll
+                for (int b = 0; b < NBT; ++b) {
+                    float acc[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+                    for (int h = 0; h < 2; ++h)
+#pragma unroll
+                        for (int set = 0; set < 2; ++set) {
+                            const int k0 = (b0 + b) * kGroup + 64 * h + 32 * set + 8 * c;
+                            uint4 xb = make_uint4(0, 0, 0, 0);
+                            if (q == 0) xb = *reinterpret_cast<const uint4*>(xs + (size_t)j * x_stride + k0 * 2);
+                            const uint32_t wq = set ? wreg[b][h].z : wreg[b][h].x;
+                            const uint32_t wq8 = set ? wreg[b][h].w : wreg[b][h].y;
+                            mma_m16n8k16(acc, code_pair(wq, 0), code_pair(wq8, 0), code_pair(wq, 4), code_pair(wq8, 4), xb.x, xb.y);
+                            mma_m16n8k16(acc, code_pair(wq, 8), code_pair(wq8, 8), code_pair(wq, 12), code_pair(wq8, 12), xb.z, xb.w);
+                        }
+                    const __half2 sc = *reinterpret_cast<const __half2*>(&sreg[b]);
+                    const float cr = adj[(b0 + b) * k + j];
+                    total[0] = fmaf(__low2float(sc), acc[0] + cr, total[0]);
+                    total[1] = fmaf(__high2float(sc), acc[2] + cr, total[1]);
+                    if ((b0 + b + 1) % bpwg == 0) {            // end of one K-split range of the grouped kernel
+                        const bool first = (b0 + b + 1 == bpwg);
+                        result[0] = first ? total[0] : result[0] + total[0];
+                        result[1] = first ? total[1] : result[1] + total[1];
+                        total[0] = total[1] = 0.f;
+                    }
+                }
+            }
+        }
+        if (j < k) {
+            if (lane == 0) s_valid[j] = valid ? 1 : 0;
+            if (c == 0) {
+                ys[j * 16 + q] = rw * result[0];
+                ys[j * 16 + q + 8] = rw * result[1];
+            }
+        }
+    }
+    if (!staged) grid_dependency_wait();
+    __syncthreads();
+    if (tid < 16) {
+        float sum = 0.f;
+        for (int j = 0; j < k; ++j)
+            if (s_valid[j]) sum += ys[j * 16 + tid];
+        sa.out[(size_t)t * a.H + panel * kPanelRows + tid] = __float2bfloat16_rn(sum);
+    }
+}
+
+
+// Gate/up + SwiGLU for tiny batches (T*k <= 32, one wave): one CTA per (token-expert pair, tile of
+// 8/KS panel pairs), one activation row, every weight load of a warp issued before anything else.
+// Straight-line code (no item, pass or chunk loops) so that two CTAs fit an SM and the whole grid is
+// one resident wave; the arithmetic and its order are those of decode_gemm_kernel.
+template <int NB>
+__global__ void __launch_bounds__(256, 2)
+pair_gateup_kernel(GemmArgs a, SmallArgs sa, const __nv_bfloat16* __restrict__ hidden,
+                   __nv_bfloat16* __restrict__ act_out, int KS) {
+    extern __shared__ __align__(16) unsigned char smem[];
+    grid_launch_dependents();
+    const int K = a.H, KB = K / kGroup, PP = 8 / KS;
+    const int tiles = a.I / (kPanelRows * PP);
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int q = lane >> 2, c = lane & 3;
+    const int ks = warp % KS, pp = warp / KS;
+    const int p = blockIdx.x / tiles, tile = blockIdx.x % tiles;
+    unsigned char* xs = smem;                                            // one activation row
+    float* red = reinterpret_cast<float*>(smem + K * 2 + 64);            // [KS-1][PP][2][32][4]
+    float* adj = red + (size_t)(KS - 1) * PP * 2 * 128;                  // [KB]
+
+    // The hidden row does not depend on the ids: request it first so that it is not queued behind the weights.
+    const __nv_bfloat16* xrow = hidden + (size_t)(p / a.top_k) * K;
+    uint4 xpre = make_uint4(0, 0, 0, 0);
+    if (tid < K / 8) xpre = *reinterpret_cast<const uint4*>(xrow + tid * 8);
+    const int id = sa.ids[p];
+    if (blockIdx.x == 0 && tid < sa.n_pairs) {         // keep the ids so the plan can be materialised on request
+        const int v = sa.ids[tid];
+        sa.saved_ids[tid] = v;
+        if (v < 0 || v >= sa.E) atomicExch(sa.status, EXMOE_ERR_BAD_EXPERT_ID);
+    }
+    if (id < 0 || id >= sa.E) return;                  // uniform over the CTA; the pair contributes nothing
+    const int slot = sa.slot_of ? sa.slot_of[id] : id;
+    const int panel = tile * PP + pp;
+    const uint8_t* wbase = a.slots + (size_t)slot * a.slot_stride;
+    uint4 wreg[2][NB][2];
+    uint32_t sreg[2][NB];
+#pragma unroll
+    for (int m = 0; m < 2; ++m)
+#pragma unroll
+        for (int b = 0; b < NB; ++b) {
+            const uint8_t* blk = wbase + ((size_t)(2 * panel + m) * KB + ks * NB + b) * kBlockBytes;
+            wreg[m][b][0] = ldg_stream128(blk + lane * 16);
+            wreg[m][b][1] = ldg_stream128(blk + 512 + lane * 16);
+            sreg[m][b] = ldg_stream32(blk + kCodeBytes + q * 4);
+        }
+    // stage the token's hidden row; adj[kb] = -136 * (sum of the row over block kb)
+    const int total = K / 8;
+    for (int base = warp * 32; base < total; base += 256) {
+        const int ck = base + lane;
+        uint4 v = make_uint4(0, 0, 0, 0);
+        if (ck < total) {
+            v = (base < 256) ? xpre : *reinterpret_cast<const uint4*>(xrow + ck * 8);
+            *reinterpret_cast<uint4*>(xs + ck * 16) = v;
+        }
+        float sx = sum8_bf16(v);
+#pragma unroll
+        for (int m = 8; m >= 1; m >>= 1) sx += __shfl_xor_sync(0xffffffffu, sx, m);
+        if (ck < total && (ck & 15) == 0) adj[ck >> 4] = -136.f * sx;
+    }
+    __syncthreads();
+
+    float tot[2][4];
+#pragma unroll
+    for (int m = 0; m < 2; ++m)
+#pragma unroll
+        for (int i = 0; i < 4; ++i) tot[m][i] = 0.f;
+#pragma unroll
+    for (int b = 0; b < NB; ++b) {
+        float acc[2][4];
+#pragma unroll
+        for (int m = 0; m < 2; ++m)
+#pragma unroll
+            for (int i = 0; i < 4; ++i) acc[m][i] = 0.f;
+#pragma unroll
+        for (int h = 0; h < 2; ++h)
+#pragma unroll
+            for (int set = 0; set < 2; ++set) {
+                const int k0 = (ks * NB + b) * kGroup + 64 * h + 32 * set + 8 * c;
+                uint4 xb = make_uint4(0, 0, 0, 0);
+                if (q == 0) xb = *reinterpret_cast<const uint4*>(xs + k0 * 2);
+#pragma unroll
+                for (int m = 0; m < 2; ++m) {
+                    const uint32_t wq = set ? wreg[m][b][h].z : wreg[m][b][h].x;
+                    const uint32_t wq8 = set ? wreg[m][b][h].w : wreg[m][b][h].y;
+                    mma_m16n8k16(acc[m], code_pair(wq, 0), code_pair(wq8, 0), code_pair(wq, 4), code_pair(wq8, 4), xb.x, xb.y);
+                    mma_m16n8k16(acc[m], code_pair(wq, 8), code_pair(wq8, 8), code_pair(wq, 12), code_pair(wq8, 12), xb.z, xb.w);
+                }
+            }
+        const float cr = adj[ks * NB + b];             // column 0 is the only live one; others are discarded
+#pragma unroll
+        for (int m = 0; m < 2; ++m) {
+            const __half2 sc = *reinterpret_cast<const __half2*>(&sreg[m][b]);
+            const float s_lo = __low2float(sc), s_hi = __high2float(sc);
+            tot[m][0] = fmaf(s_lo, acc[m][0] + cr, tot[m][0]);
+            tot[m][2] = fmaf(s_hi, acc[m][2] + cr, tot[m][2]);
+        }
+    }
+    if (ks > 0 && c == 0) {
+        red[(((ks - 1) * PP + pp) * 2 + 0) * 16 + q] = tot[0][0];
+        red[(((ks - 1) * PP + pp) * 2 + 0) * 16 + q + 8] = tot[0][2];
+        red[(((ks - 1) * PP + pp) * 2 + 1) * 16 + q] = tot[1][0];
+        red[(((ks - 1) * PP + pp) * 2 + 1) * 16 + q + 8] = tot[1][2];
+    }
+    __syncthreads();
+    if (ks == 0 && c == 0) {
+        for (int s = 1; s < KS; ++s) {
+            tot[0][0] += red[(((s - 1) * PP + pp) * 2 + 0) * 16 + q];
+            tot[0][2] += red[(((s - 1) * PP + pp) * 2 + 0) * 16 + q + 8];
+            tot[1][0] += red[(((s - 1) * PP + pp) * 2 + 1) * 16 + q];
+            tot[1][2] += red[(((s - 1) * PP + pp) * 2 + 1) * 16 + q + 8];
+        }
+#pragma unroll
+        for (int i = 0; i < 4; i += 2) {
+            const float g = tot[0][i], u = tot[1][i];
+            act_out[(size_t)p * a.I + panel * kPanelRows + q + 4 * i] = __float2bfloat16_rn(g / (1.f + __expf(-g)) * u);
+        }
+    }
+}
+
+template <int NB>
+void launch_pair_gateup(const GemmArgs& a, const SmallArgs& sa, const __nv_bfloat16* hidden, __nv_bfloat16* act, int KS,
+                        cudaStream_t st) {
+    auto kern = pair_gateup_kernel<NB>;
+    const int PP = 8 / KS, tiles = a.I / (kPanelRows * PP);
+    const size_t smem = (size_t)a.H * 2 + 64 + (size_t)(KS - 1) * PP * 2 * 128 * 4 + (size_t)(a.H / kGroup) * 4;
+    static bool attr_done = false;
+    if (!attr_done) {
+        cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 100 * 1024);
+        attr_done = true;
+    }
+    kern<<<sa.n_pairs * tiles, 256, smem, st>>>(a, sa, hidden, act, KS);
+    count_launch();
 }
 
 // K split over KS warps (KS in {1,2,4,8}, 8/KS panels per CTA) and register depth NB; aims at
@@ -231,15 +719,18 @@ DecodeCfg pick_cfg(int K, int rows) {
     return {1, 1, KB};                                  // rows % 128 == 0 always makes KS = 1 feasible
 }
 
-template <int NB, int NCH, bool GATEUP>
-void launch_cfg(const GemmArgs& a, const __nv_bfloat16* x, __nv_bfloat16* act, const float* w, float* y,
-                const DecodeCfg& cfg, int max_groups, cudaStream_t st) {
+template <int NB, int NCH, bool GATEUP, int MODE>
+void launch_cfg(const GemmArgs& a, const SmallArgs& sa, const __nv_bfloat16* x, __nv_bfloat16* act, const float* w,
+                float* y, const DecodeCfg& cfg, int max_groups, cudaStream_t st) {
     constexpr int NM = GATEUP ? 2 : 1;
     const int K = GATEUP ? a.H : a.I, NR = GATEUP ? a.I : a.H;
     const int PP = 8 / cfg.KS;
     const int tiles = NR / (kPanelRows * PP);
-    const size_t smem = (size_t)8 * NCH * (K * 2 + 64) + (size_t)(cfg.KS - 1) * PP * NM * NCH * 128 * 4;
-    auto kern = decode_gemm_kernel<NB, NCH, GATEUP>;
+    size_t smem = (size_t)8 * NCH * (K * 2 + 64) + (size_t)(cfg.KS - 1) * PP * NM * NCH * 128 * 4 +
+                  (size_t)(K / kGroup) * 8 * NCH * 4;
+    constexpr bool SMALL = (MODE == MODE_SMALL);
+    if (SMALL) smem += (size_t)(3 * a.num_slots + 1 + 2 * sa.n_pairs) * 4;
+    auto kern = decode_gemm_kernel<NB, NCH, GATEUP, MODE>;
     static bool attr_done = false;                      // per instantiation
     if (!attr_done) {
         cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
@@ -247,22 +738,42 @@ void launch_cfg(const GemmArgs& a, const __nv_bfloat16* x, __nv_bfloat16* act, c
     }
     long long items = (long long)max_groups * tiles;
     const int grid = (int)(items < 148 * 8 ? (items < 1 ? 1 : items) : 148 * 8);
-    kern<<<grid, 256, smem, st>>>(a, x, act, w, y, cfg.KS, cfg.bpw);
+    cudaLaunchConfig_t lc{};
+    lc.gridDim = dim3(grid);
+    lc.blockDim = dim3(256);
+    lc.dynamicSmemBytes = smem;
+    lc.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    lc.attrs = attr;
+    lc.numAttrs = (SMALL && !GATEUP) ? 1 : 0;           // only the down kernel overlaps its predecessor
+#ifdef EXMOE_DISABLE_PDL
+    lc.numAttrs = 0;
+#endif
+    cudaLaunchKernelEx(&lc, kern, a, sa, x, act, w, y, cfg.KS, cfg.bpw);
     count_launch();
 }
 
-template <bool GATEUP>
-void launch_decode(const GemmArgs& a, const __nv_bfloat16* x, __nv_bfloat16* act, const float* w, float* y,
-                   int max_rows, int max_groups, cudaStream_t st) {
+template <bool GATEUP, int MODE>
+void launch_decode(const GemmArgs& a, const SmallArgs& sa, const __nv_bfloat16* x, __nv_bfloat16* act, const float* w,
+                   float* y, int max_rows, int max_groups, cudaStream_t st) {
     const int K = GATEUP ? a.H : a.I, NR = GATEUP ? a.I : a.H;
-    const DecodeCfg cfg = pick_cfg(K, NR);
+    DecodeCfg cfg = pick_cfg(K, NR);
+#ifdef EXMOE_PAIR_KS
+    if (MODE == MODE_PAIR && (K / kGroup) % EXMOE_PAIR_KS == 0) {
+        const int bpw = K / kGroup / EXMOE_PAIR_KS;
+        cfg = {(bpw % 4 == 0) ? 4 : (bpw % 2 == 0) ? 2 : 1, EXMOE_PAIR_KS, bpw};
+    }
+#endif
     // rows per pass: one 8-row chunk covers decode; more chunks amortise the dequantisation
     int nch = max_rows <= 8 ? 1 : (max_rows <= 16 ? 2 : 4);
     while (nch > 1 && (size_t)8 * nch * (K * 2 + 64) > 150 * 1024) nch >>= 1;
-#define EXMOE_DISPATCH(NBv)                                                                     \
-    if (nch == 1) launch_cfg<NBv, 1, GATEUP>(a, x, act, w, y, cfg, max_groups, st);             \
-    else if (nch == 2) launch_cfg<NBv, 2, GATEUP>(a, x, act, w, y, cfg, max_groups, st);        \
-    else launch_cfg<NBv, 4, GATEUP>(a, x, act, w, y, cfg, max_groups, st);
+#define EXMOE_DISPATCH(NBv)                                                                                   \
+    if (nch == 1) launch_cfg<NBv, 1, GATEUP, MODE>(a, sa, x, act, w, y, cfg, max_groups, st);                 \
+    else if (MODE == MODE_PAIR) return;                                                                       \
+    else if (nch == 2) launch_cfg<NBv, 2, GATEUP, MODE>(a, sa, x, act, w, y, cfg, max_groups, st);            \
+    else launch_cfg<NBv, 4, GATEUP, MODE>(a, sa, x, act, w, y, cfg, max_groups, st);
     if (cfg.NB == 4) { EXMOE_DISPATCH(4) }
     else if (cfg.NB == 2) { EXMOE_DISPATCH(2) }
     else { EXMOE_DISPATCH(1) }
@@ -295,17 +806,85 @@ combine_kernel(const float* __restrict__ y, const int32_t* __restrict__ ids, int
 
 void launch_decode_gateup(const GemmArgs& a, const __nv_bfloat16* hidden, __nv_bfloat16* act, int max_rows,
                           int max_groups, cudaStream_t st) {
-    launch_decode<true>(a, hidden, act, nullptr, nullptr, max_rows, max_groups, st);
+    launch_decode<true, MODE_PLAN>(a, SmallArgs{}, hidden, act, nullptr, nullptr, max_rows, max_groups, st);
 }
 void launch_decode_down(const GemmArgs& a, const __nv_bfloat16* act, const float* topk_w, float* y, int max_rows,
                         int max_groups, cudaStream_t st) {
-    launch_decode<false>(a, act, nullptr, topk_w, y, max_rows, max_groups, st);
+    launch_decode<false, MODE_PLAN>(a, SmallArgs{}, act, nullptr, topk_w, y, max_rows, max_groups, st);
 }
 void launch_combine(const float* y, const int32_t* ids, int E, int T, int k, int H, __nv_bfloat16* out,
                     cudaStream_t st) {
     const long long n = (long long)T * (H / 4);
     combine_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(y, ids, E, T, k, H, out);
     count_launch();
+}
+
+
+template <int NBT>
+void launch_token_down(const GemmArgs& a, const SmallArgs& sa, const __nv_bfloat16* act, const float* w, int T,
+                       int bpwg, cudaStream_t st) {
+    auto kern = token_down_kernel<NBT>;
+    const size_t smem = (size_t)a.top_k * (a.I * 2 + 64) + (size_t)a.top_k * 17 * 4 + (size_t)(a.I / kGroup) * a.top_k * 4;
+    static bool attr_done = false;
+    if (!attr_done) {
+        cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+        attr_done = true;
+    }
+    cudaLaunchConfig_t lc{};
+    lc.gridDim = dim3(T * (a.H / kPanelRows));
+    lc.blockDim = dim3(256);
+    lc.dynamicSmemBytes = smem;
+    lc.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    lc.attrs = attr;
+    lc.numAttrs = 1;
+#ifdef EXMOE_DISABLE_PDL
+    lc.numAttrs = 0;
+#endif
+    cudaLaunchKernelEx(&lc, kern, a, sa, act, w, bpwg);
+    count_launch();
+}
+
+// One wave of the SMALL path: gate/up kernel, then the down kernel with the fused combine.
+void launch_small_wave(const GemmArgs& a, const SmallWave& w, cudaStream_t st, bool gateup, bool down) {
+    SmallArgs sa{};
+    sa.ids = w.ids;
+    sa.wave_of = w.wave_of;
+    sa.slot_of = w.slot_of;
+    sa.n_pairs = w.n_pairs;
+    sa.E = w.E;
+    sa.wave = w.wave;
+    sa.pub_counts = w.plan.counts;
+    sa.pub_offsets = w.plan.offsets;
+    sa.pub_perm = w.plan.perm;
+    sa.header = w.plan.header;
+    sa.status = w.status;
+    sa.arrive = w.arrive;
+    sa.out = w.out;
+    sa.saved_ids = w.saved_ids;
+    if (w.pairwise) {                                   // T*k <= 32, one wave: no grouping, by-token down + combine
+        if (gateup) {
+            const DecodeCfg cfg = pick_cfg(a.H, a.I);
+            if (cfg.bpw == 4) launch_pair_gateup<4>(a, sa, w.hidden, w.act, cfg.KS, st);
+            else if (cfg.bpw == 2) launch_pair_gateup<2>(a, sa, w.hidden, w.act, cfg.KS, st);
+            else if (cfg.bpw == 1) launch_pair_gateup<1>(a, sa, w.hidden, w.act, cfg.KS, st);
+            else launch_decode<true, MODE_PAIR>(a, sa, w.hidden, w.act, nullptr, nullptr, 1, w.n_pairs, st);
+        }
+        if (down) {
+            const int KB = a.I / kGroup;
+            const int bpwg = pick_cfg(a.I, a.H).bpw;    // the grouped kernel's K-split range, replayed for rounding
+            const int T = w.n_pairs / a.top_k;
+            if (KB % 8 == 0) launch_token_down<8>(a, sa, w.act, w.topk_w, T, bpwg, st);
+            else if (KB % 4 == 0) launch_token_down<4>(a, sa, w.act, w.topk_w, T, bpwg, st);
+            else if (KB % 2 == 0) launch_token_down<2>(a, sa, w.act, w.topk_w, T, bpwg, st);
+            else launch_token_down<1>(a, sa, w.act, w.topk_w, T, bpwg, st);
+        }
+        return;
+    }
+    if (gateup) launch_decode<true, MODE_SMALL>(a, sa, w.hidden, w.act, nullptr, nullptr, w.max_rows, w.max_groups, st);
+    if (down) launch_decode<false, MODE_SMALL>(a, sa, w.act, nullptr, w.topk_w, w.y, w.max_rows, w.max_groups, st);
 }
 
 }  // namespace exmoe
