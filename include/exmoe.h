@@ -117,6 +117,33 @@ int exmoe_cache_create(exmoe_cache** out, const exmoe_shape* shape, int num_laye
 int exmoe_moe_forward(exmoe_cache* cache, int layer, const void* hidden_bf16, const int32_t* topk_ids,
                       const float* topk_weights, int T, void* out_bf16, void* stream);
 
+/* Tiny-batch forward that allocates nothing and needs no cache object (the paper has no counterpart: this
+ * is a service for one kind of caller, not a step of the method).
+ *
+ * Who it is for: code that cannot get device memory at the moment it needs this layer - a serving loop that
+ * handed all device memory to its own pool at start-up, a plug-in living under a host framework that owns the
+ * allocator, or a latency-critical path that must not pay the device-wide synchronisation a cudaMalloc or
+ * cudaFree brings.  exmoe_moe_forward needs a caller-allocated workspace for the activations that travel from
+ * the gate/up kernel to the down kernel; here that scratch is a fixed 262,400-byte `__device__` array inside
+ * the library (held by every GPU that loads the library until the process exits), so the caller passes inputs
+ * and outputs only.  The function calls no cudaMalloc, cudaFree or other allocating routine.
+ *
+ *   experts_dev  : dev, num_experts packed experts back to back (expert e at e * bytes_per_expert), i.e. a
+ *                  fully resident layer exactly as exmoe_pack wrote it (slot = expert id, one wave).
+ *   hidden_bf16, topk_ids, topk_weights, out_bf16 : as for exmoe_moe_forward.  Same kernels, same result.
+ *
+ * Limits (fixed by the size of the scratch): T * top_k <= 32 and d_ff <= 4096; anything larger is refused
+ * with EXMOE_ERR_SHAPE before any work is queued.  T = 0 is a no-op.
+ * First call on a device: looks up the device address of the scratch array (cudaGetSymbolAddress, with that
+ * device current) and keeps it; make this first call outside any stream capture.
+ * The scratch is shared by all calls and keeps the previous call's contents; the function clears the one word
+ * that must start at zero.  Calls on one device that may overlap on the GPU (different streams without
+ * ordering between them) race on it: order them, or use exmoe_moe_forward with separate workspaces.
+ * An id outside [0, E) contributes nothing; it is not reported by this entry point. */
+int exmoe_moe_forward_static(const exmoe_shape* shape, const void* experts_dev, const void* hidden_bf16,
+                             const int32_t* topk_ids, const float* topk_weights, int T, void* out_bf16,
+                             void* stream);
+
 /* Test hooks (synchronise).  Sec. 3.3 state of one layer: expert_slot [E] (-1 = not resident),
  * slot_expert [C] (-1 = empty), slot_stamp [C], all host pointers, any may be NULL. */
 int exmoe_cache_get_state(exmoe_cache* cache, int layer, int32_t* expert_slot, int32_t* slot_expert,

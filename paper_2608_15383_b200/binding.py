@@ -47,6 +47,7 @@ _SIGNATURES = {
     "exmoe_cache_create": (c_int, [POINTER(c_void_p), POINTER(exmoe_shape), c_int, c_int, POINTER(c_void_p), c_void_p,
                                    c_void_p, c_int, c_int]),
     "exmoe_moe_forward": (c_int, [c_void_p, c_int, c_void_p, c_void_p, c_void_p, c_int, c_void_p, c_void_p]),
+    "exmoe_moe_forward_static": (c_int, [POINTER(exmoe_shape), c_void_p, c_void_p, c_void_p, c_void_p, c_int, c_void_p, c_void_p]),
     "exmoe_cache_get_state": (c_int, [c_void_p, c_int, c_void_p, c_void_p, c_void_p, c_void_p]),
     "exmoe_debug_last_plan": (c_int, [c_void_p, c_int] + [c_void_p] * 9),
     "exmoe_debug_read_slot": (c_int, [c_void_p, c_int, c_int, c_void_p]),
@@ -129,6 +130,18 @@ def exmoe_cache_workspace_bytes(shape, num_layers, num_slots, max_tokens):
     _check(lib().exmoe_cache_workspace_bytes(byref(_shape(shape)), num_layers, num_slots, max_tokens, byref(a), byref(b)),
            "exmoe_cache_workspace_bytes")
     return a.value, b.value
+
+
+def exmoe_moe_forward_static(shape, experts_dev, hidden, topk_ids, topk_weights, out, stream=None):
+    """Tiny-batch forward through the library's built-in scratch: no cache object, no workspace, nothing is
+    allocated by the call (the caller passes `out`).  For callers that cannot obtain device memory when they
+    need the layer; limits: T * top_k <= 32, d_ff <= 4096, fully resident experts."""
+    rc = lib().exmoe_moe_forward_static(byref(_shape(shape)), _dev(experts_dev, torch.uint8, "experts_dev"),
+                                        _dev(hidden, torch.bfloat16, "hidden"), _dev(topk_ids, torch.int32, "topk_ids"),
+                                        _dev(topk_weights, torch.float32, "topk_weights"), int(hidden.shape[0]),
+                                        _dev(out, torch.bfloat16, "out"), _stream_ptr(stream))
+    _check(rc, "exmoe_moe_forward_static")
+    return out
 
 
 def exmoe_launch_count():

@@ -887,4 +887,88 @@ void launch_small_wave(const GemmArgs& a, const SmallWave& w, cudaStream_t st, b
     if (down) launch_decode<false, MODE_SMALL>(a, sa, w.act, nullptr, w.topk_w, w.y, w.max_rows, w.max_groups, st);
 }
 
+// ------------------------------------------------------------------------------------------------
+// Allocation-free tiny-batch forward (exmoe_moe_forward_static).
+//
+// The pairwise kernels need scratch: the BF16 SwiGLU activations handed from the gate/up kernel to
+// the down kernel, plus a status word and the kept ids.  exmoe_moe_forward takes that scratch from
+// the workspace the caller allocated for the cache.  This entry point serves callers that can hand
+// over no scratch at all: it lives in the fixed array below, which every GPU that loads this
+// library holds until the process exits.
+// ------------------------------------------------------------------------------------------------
+constexpr int kStaticMaxPairs = kPairMaxPairs;           // T * top_k <= 32
+constexpr int kStaticMaxDff = 4096;                      // d_ff <= 4096
+constexpr size_t kStaticCtrlBytes = 256;                 // [0,4) status word, [64,192) kept ids
+constexpr size_t kStaticScratchBytes = kStaticCtrlBytes + (size_t)kStaticMaxPairs * kStaticMaxDff * 2;   // 262,400 B
+
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
+
 }  // namespace exmoe
+
+#include <mutex>
+
+extern "C" int exmoe_moe_forward_static(const exmoe_shape* shape, const void* experts_dev, const void* hidden_bf16,
+                                        const int32_t* topk_ids, const float* topk_weights, int T, void* out_bf16,
+                                        void* stream) {
+    using namespace exmoe;
+    if (!shape || T < 0) return EXMOE_ERR_ARG;
+    if (shape->group_size != kGroup || shape->d_model <= 0 || shape->d_ff <= 0 || shape->d_model % kGroup ||
+        shape->d_ff % kGroup || shape->num_experts <= 0 || shape->top_k <= 0 || shape->top_k > shape->num_experts)
+        return EXMOE_ERR_SHAPE;
+    // the fixed scratch bounds the problem: reject anything larger instead of overrunning it
+    if ((long long)T * shape->top_k > kStaticMaxPairs || shape->d_ff > kStaticMaxDff) return EXMOE_ERR_SHAPE;
+    if (T == 0) return EXMOE_OK;
+    if (!experts_dev || !hidden_bf16 || !topk_ids || !topk_weights || !out_bf16) return EXMOE_ERR_ARG;
+    if ((reinterpret_cast<uintptr_t>(experts_dev) | reinterpret_cast<uintptr_t>(hidden_bf16) |
+         reinterpret_cast<uintptr_t>(out_bf16)) & 15)
+        return EXMOE_ERR_ARG;
+
+    // Set-up, once per device, with that device current: in host code `g_static_scratch` is only a
+    // stand-in for the symbol, not a device address; the address a kernel may use comes from
+    // cudaGetSymbolAddress.
+    static std::mutex mu;
+    static unsigned char* dev_ptr[64] = {};
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return EXMOE_ERR_CUDA;
+    unsigned char* scratch = nullptr;
+    {
+        std::lock_guard<std::mutex> lock(mu);
+        if (!dev_ptr[dev]) {
+            void* p = nullptr;
+            if (cudaGetSymbolAddress(&p, g_static_scratch) != cudaSuccess || !p) {
+                cudaGetLastError();
+                return EXMOE_ERR_CUDA;
+            }
+            dev_ptr[dev] = static_cast<unsigned char*>(p);
+        }
+        scratch = dev_ptr[dev];
+    }
+
+    cudaStream_t st = (cudaStream_t)stream;
+    // the array keeps the previous call's contents: the status word must start at zero
+    if (cudaMemsetAsync(scratch, 0, kStaticCtrlBytes, st) != cudaSuccess) return EXMOE_ERR_CUDA;
+
+    GemmArgs a{};
+    a.slots = static_cast<const uint8_t*>(experts_dev);
+    a.slot_stride = matrix_bytes(2 * shape->d_ff, shape->d_model) + matrix_bytes(shape->d_model, shape->d_ff);
+    a.num_slots = shape->num_experts;
+    a.top_k = shape->top_k;
+    a.H = shape->d_model;
+    a.I = shape->d_ff;
+    SmallWave w{};
+    w.ids = topk_ids;
+    w.n_pairs = T * shape->top_k;
+    w.E = shape->num_experts;
+    w.wave = 0;
+    w.status = reinterpret_cast<int*>(scratch);
+    w.saved_ids = reinterpret_cast<int32_t*>(scratch + 64);
+    w.hidden = static_cast<const __nv_bfloat16*>(hidden_bf16);
+    w.act = reinterpret_cast<__nv_bfloat16*>(scratch + kStaticCtrlBytes);
+    w.topk_w = topk_weights;
+    w.out = static_cast<__nv_bfloat16*>(out_bf16);
+    w.max_rows = T;
+    w.max_groups = w.n_pairs;
+    w.pairwise = true;
+    launch_small_wave(a, w, st, true, true);
+    return cudaGetLastError() == cudaSuccess ? EXMOE_OK : EXMOE_ERR_CUDA;
+}
