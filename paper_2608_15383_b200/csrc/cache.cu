@@ -62,6 +62,7 @@ struct exmoe_cache {
     bool last_small;
     bool last_pair;
     int32_t* saved_ids;                       // ids of the last pairwise call (plan materialised on request)
+    void* tc_scratch;                         // tile list of the tensor-core path
     int32_t* h_plan;                          // pinned staging of the plan
     cudaStream_t copy_stream;
     cudaEvent_t ev_plan;
@@ -128,6 +129,7 @@ static void carve_workspace(exmoe_cache* c, uint8_t* ws, size_t* total) {
     c->arrive_words = (size_t)(kSmallMaxPairs / s.top_k + 1) * (s.d_model / kPanelRows);
     c->arrive = k.take<int>(c->arrive_words);
     c->saved_ids = k.take<int32_t>(kPairMaxPairs);
+    c->tc_scratch = k.take<uint8_t>(prefill_scratch_bytes(c->max_pairs, E));
     *total = k.off;
 }
 
@@ -387,13 +389,16 @@ int exmoe_moe_forward(exmoe_cache* c, int layer, const void* hidden, const int32
                 launch_small_wave(a, sw, st, false, true);
             }
         } else {
+            // many rows per expert: dense contraction on the tensor cores (tcgen05 / TMEM)
             if (!c->prof_only || c->prof_only == PROF_GATEUP) {
                 ProfScope ps(c, PROF_GATEUP, st);
-                launch_decode_gateup(a, (const __nv_bfloat16*)hidden, c->act, T, groups, st);
+                launch_prefill_wave(a, a.wave_start, c->tc_scratch, c->d_status, (const __nv_bfloat16*)hidden, c->act,
+                                    topk_weights, c->y, 1, st);
             }
             if (!c->prof_only || c->prof_only == PROF_DOWN) {
                 ProfScope ps(c, PROF_DOWN, st);
-                launch_decode_down(a, c->act, topk_weights, c->y, T, groups, st);
+                launch_prefill_wave(a, a.wave_start, c->tc_scratch, c->d_status, (const __nv_bfloat16*)hidden, c->act,
+                                    topk_weights, c->y, 2, st);
             }
         }
         if (!identity) {

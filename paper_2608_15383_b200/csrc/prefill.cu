@@ -1,0 +1,461 @@
+// Large-M grouped W4A16 GEMMs on the 5th-generation tensor cores (prefill; the two grouped expert
+// GEMMs per wave of Section 3.4 / Eq. 2 when every expert has many rows).
+//
+// Swap-AB: the WEIGHTS are the UMMA A operand (M = 128 rows = 8 consecutive 16-row panels of the
+// packed matrix), the TOKENS are the B operand (N <= 256 grouped rows), the accumulator D[128 x N]
+// lives in TMEM (fp32, lane = weight row, column = token).  For gate/up the 8 panels are
+// gate p, up p, gate p+1, ... so one accumulator holds 64 intermediates' gate rows and up rows
+// 16 lanes apart: SwiGLU is one shuffle away in the epilogue.
+//
+// A persistent CTA (one per SM, 16 warps) is specialised by warp:
+//   warp 0        allocates TMEM, then one elected thread issues tcgen05.mma (8 x K16 per 128-wide
+//                 block) and tcgen05.commit to the stage-empty / accumulator-full mbarriers.
+//   warps 4-7     epilogue: tcgen05.ld the accumulator (warp w reads TMEM lanes 32(w%4)..), SwiGLU
+//                 -> BF16 activations, or routing weight -> fp32 pair buffer; two accumulators
+//                 (2 x 256 columns) let the epilogue of tile i overlap the MMAs of tile i+1.
+//   warps 8-11    A producers: stream packed int4 (128-bit loads, one block ahead in registers),
+//                 dequantise to BF16 (shift/lop3 -> 128+u, subtract 136, multiply by the group
+//                 scale) and store the canonical no-swizzle K-major core-matrix layout.
+//   warps 12-15   B producers: gather the tile's token rows with 16-byte cp.async into the same
+//                 canonical layout, two stages in flight.
+// Producers -> MMA through full[stage] mbarriers (generic-proxy writes are fenced with
+// fence.proxy.async before the arrive), MMA -> producers through tcgen05.commit on empty[stage].
+// Every wait is bounded: on expiry the CTA raises EXMOE_ERR_TIMEOUT, all roles drain, TMEM is freed.
+#include "common.cuh"
+
+namespace exmoe {
+
+namespace {
+
+constexpr int BM = 128;            // weight rows per tile
+constexpr int BN = 256;            // max grouped rows (tokens) per tile
+constexpr int BK = 128;            // K per stage = one packed block / one scale group
+constexpr int STAGES = 2;
+constexpr int A_STAGE_BYTES = BM * BK * 2;     // 32 KB
+constexpr int B_STAGE_BYTES = BN * BK * 2;     // 64 KB
+constexpr int SBO = 16 * 128;      // bytes between 8-row groups (16 k-chunks of one 8-row group are contiguous)
+constexpr int LBO = 128;           // bytes between the two 16-byte k-chunks of one K16 step
+constexpr int NUM_THREADS = 512;
+constexpr long long kWaitBudget = 2000000000ll;   // clock64 ticks (~1 s) before a wait gives up
+
+struct Tile { int key, n0, nrows, pad; };
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void mbar_init(uint64_t* bar, int count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
+}
+__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ bool mbar_try(uint64_t* bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(smem_u32(bar)), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+// bounded wait; returns false when the CTA is aborting (and raises the abort on expiry)
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag, int* status) {
+    if (mbar_try(bar, parity)) return true;
+    const long long t0 = clock64();
+    while (!mbar_try(bar, parity)) {
+        if (*abort_flag) return false;
+        if (clock64() - t0 > kWaitBudget) {
+            *abort_flag = 1;
+            atomicExch(status, EXMOE_ERR_TIMEOUT);
+            return false;
+        }
+    }
+    return true;
+}
+__device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_commit(uint64_t* bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void tc_mma(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+__device__ __forceinline__ void tc_ld32(uint32_t taddr, uint32_t (&r)[32]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+          "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+          "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+          "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr));
+}
+__device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// shared-memory matrix descriptor: no swizzle, K-major, version 1 (sm_100)
+__device__ __forceinline__ uint64_t make_desc(uint32_t saddr) {
+    uint64_t d = 0;
+    d |= (uint64_t)((saddr >> 4) & 0x3fff);
+    d |= (uint64_t)((LBO >> 4) & 0x3fff) << 16;
+    d |= (uint64_t)((SBO >> 4) & 0x3fff) << 32;
+    d |= (uint64_t)1 << 46;
+    return d;
+}
+// instruction descriptor: D fp32, A/B BF16, both K-major, M = 128, N = n
+__device__ __forceinline__ uint32_t make_idesc(int n) {
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+}
+__device__ __forceinline__ uint4 ldg_stream128(const void* p) {
+    uint4 v;
+    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+                 : "l"(p));
+    return v;
+}
+__device__ __forceinline__ uint32_t ldg_stream32(const void* p) {
+    uint32_t v;
+    asm volatile("ld.global.nc.L1::no_allocate.u32 %0, [%1];" : "=r"(v) : "l"(p));
+    return v;
+}
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src, int src_bytes) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(src_bytes) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+
+// eight codes of one word -> eight BF16 weights (q * s), K order, as one 16-byte value
+__device__ __forceinline__ uint4 dequant_word(uint32_t w, __nv_bfloat162 scale2) {
+    uint32_t bias = 0x43084308u;                                   // BF16 136 twice
+    const __nv_bfloat162 b2 = *reinterpret_cast<__nv_bfloat162*>(&bias);
+    uint32_t out[4];
+#pragma unroll
+    for (int s = 0; s < 4; ++s) {
+        uint32_t v;
+        asm("lop3.b32 %0, %1, 0x000f000f, 0x43004300, 0xea;" : "=r"(v) : "r"(w >> (4 * s)));   // (128+u, 128+u')
+        __nv_bfloat162 q2 = __hsub2(*reinterpret_cast<__nv_bfloat162*>(&v), b2);               // exact small integers
+        q2 = __hmul2(q2, scale2);                                                               // one rounding to BF16
+        out[s] = *reinterpret_cast<uint32_t*>(&q2);
+    }
+    return make_uint4(out[0], out[1], out[2], out[3]);
+}
+
+struct PrefillArgs {
+    const uint8_t* slots;
+    size_t slot_stride;
+    const int32_t* perm;
+    const Tile* tiles;         // n-tiles of this wave
+    const int32_t* n_tiles;    // device scalar
+    int num_slots, top_k, H, I;
+    int* status;
+};
+
+template <bool GATEUP>
+__global__ void __launch_bounds__(NUM_THREADS, 1)
+prefill_gemm_kernel(PrefillArgs a, const __nv_bfloat16* __restrict__ x_src, __nv_bfloat16* __restrict__ act_out,
+                    const float* __restrict__ topk_w, const int32_t* __restrict__ offsets, float* __restrict__ y_out) {
+    extern __shared__ __align__(1024) unsigned char smem[];
+    unsigned char* sA = smem;                                     // [STAGES][32 KB]
+    unsigned char* sB = smem + STAGES * A_STAGE_BYTES;            // [STAGES][64 KB]
+    uint64_t* bars = reinterpret_cast<uint64_t*>(sB + STAGES * B_STAGE_BYTES);
+    uint64_t* full = bars;              // [STAGES]  producers -> MMA (8 warp arrivals)
+    uint64_t* empty = bars + 2;         // [STAGES]  MMA -> producers (tcgen05.commit)
+    uint64_t* acc_full = bars + 4;      // [2]       MMA -> epilogue
+    uint64_t* acc_empty = bars + 6;     // [2]       epilogue -> MMA (4 warp arrivals)
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 8);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int K = GATEUP ? a.H : a.I;
+    const int KB = K / BK;
+    const int MT = (GATEUP ? 2 * a.I : a.H) / BM;                 // m-tiles of the packed matrix
+    const size_t w13_bytes = matrix_bytes(2 * a.I, a.H);
+    const int total_tiles = (*a.n_tiles) * MT;
+
+    if (tid == 0) {
+        for (int s = 0; s < STAGES; ++s) {
+            mbar_init(&full[s], 8);
+            mbar_init(&empty[s], 1);
+        }
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(&acc_full[b], 1);
+            mbar_init(&acc_empty[b], 4);
+        }
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 0) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(512));
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::);
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    if (warp == 0) {
+        // ------------------------------------------------------------------ MMA issuer
+        // the whole warp walks the loop (so it stays converged for the block-wide teardown); lane 0 issues
+        int it = 0;                                                // running k-block counter (stage/phase)
+        int tcount = 0;
+        bool ok = true;
+        for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x, ++tcount) {
+            const Tile tl = a.tiles[t / MT];
+            const int n_mma = (tl.nrows + 15) & ~15;
+            const uint32_t idesc = make_idesc(n_mma);
+            const int buf = tcount & 1;
+            ok = mbar_wait(&acc_empty[buf], ((tcount >> 1) & 1) ^ 1, abort_flag, a.status);
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) break;
+            tc_fence_after();
+            const uint32_t d_tmem = tmem_base + buf * BN;
+            for (int kb = 0; kb < KB; ++kb, ++it) {
+                const int s = it % STAGES;
+                ok = mbar_wait(&full[s], (it / STAGES) & 1, abort_flag, a.status);
+                ok = __all_sync(0xffffffffu, ok);
+                if (!ok) break;
+                tc_fence_after();
+                if (lane == 0) {
+                    const uint64_t da = make_desc(smem_u32(sA + s * A_STAGE_BYTES));
+                    const uint64_t db = make_desc(smem_u32(sB + s * B_STAGE_BYTES));
+#pragma unroll
+                    for (int j = 0; j < BK / 16; ++j)              // K16 step j: two 16-byte k-chunks = 256 bytes on
+                        tc_mma(d_tmem, da + (uint64_t)(j * 2 * LBO >> 4), db + (uint64_t)(j * 2 * LBO >> 4), idesc,
+                               (kb | j) ? 1u : 0u);
+                    tc_commit(&empty[s]);                          // stage reusable once these MMAs have read it
+                }
+                __syncwarp();
+            }
+            if (ok && lane == 0) tc_commit(&acc_full[buf]);        // accumulator complete
+            __syncwarp();
+        }
+    } else if (warp >= 4 && warp < 8) {
+        // ------------------------------------------------------------------ epilogue
+        const int e = warp & 3;                                    // TMEM lane quarter
+        int tcount = 0;
+        bool ok = true;
+        for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x, ++tcount) {
+            const Tile tl = a.tiles[t / MT];
+            const int mt = t % MT;
+            const int buf = tcount & 1;
+            ok = mbar_wait(&acc_full[buf], (tcount >> 1) & 1, abort_flag, a.status);
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) break;
+            tc_fence_after();
+            const int row0 = offsets[tl.key] + tl.n0;
+            const uint32_t taddr = tmem_base + buf * BN + ((uint32_t)(32 * e) << 16);
+            for (int c0 = 0; c0 < tl.nrows; c0 += 32) {
+                uint32_t v[32];
+                tc_ld32(taddr + c0, v);
+                tc_wait_ld();
+                if (GATEUP) {
+                    // lanes 0-15: gate rows, lanes 16-31: up rows of the same 16 intermediates
+                    const int interm = (mt * 4 + e) * 16 + (lane & 15);
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) {
+                        const uint32_t send = (lane < 16) ? v[j + 16] : v[j];
+                        const uint32_t recv = __shfl_xor_sync(0xffffffffu, send, 16);
+                        const int col = (lane < 16) ? j : j + 16;
+                        const float g = __uint_as_float((lane < 16) ? v[j] : recv);
+                        const float u = __uint_as_float((lane < 16) ? recv : v[j + 16]);
+                        const int n = c0 + col;
+                        if (n < tl.nrows)
+                            act_out[(size_t)(row0 + n) * a.I + interm] = __float2bfloat16_rn(g / (1.f + __expf(-g)) * u);
+                    }
+                } else {
+                    const int h = mt * BM + 32 * e + lane;
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) {
+                        const int n = c0 + j;
+                        if (n < tl.nrows) {
+                            const int pair = a.perm[row0 + n];
+                            y_out[(size_t)pair * a.H + h] = topk_w[pair] * __uint_as_float(v[j]);
+                        }
+                    }
+                }
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&acc_empty[buf]);
+        }
+    } else if (warp >= 8 && warp < 12) {
+        // ------------------------------------------------------------------ A producers (dequantise)
+        const int pw = warp - 8;                                   // handles panels 2*pw, 2*pw+1 of the tile
+        const int q = lane >> 2, c = lane & 3;
+        int it = 0;
+        bool ok = true;
+        for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
+            const Tile tl = a.tiles[t / MT];
+            const int mt = t % MT;
+            const int slot = tl.key % a.num_slots;
+            const uint8_t* mat = a.slots + (size_t)slot * a.slot_stride + (GATEUP ? 0 : w13_bytes);
+            const uint8_t* p0 = mat + (size_t)(mt * 8 + 2 * pw) * KB * kBlockBytes;      // panel 2*pw of the tile
+            const uint8_t* p1 = p0 + (size_t)KB * kBlockBytes;
+            uint4 w[2][2];
+            uint32_t sc[2];
+            w[0][0] = ldg_stream128(p0 + lane * 16);
+            w[0][1] = ldg_stream128(p0 + 512 + lane * 16);
+            sc[0] = ldg_stream32(p0 + kCodeBytes + q * 4);
+            w[1][0] = ldg_stream128(p1 + lane * 16);
+            w[1][1] = ldg_stream128(p1 + 512 + lane * 16);
+            sc[1] = ldg_stream32(p1 + kCodeBytes + q * 4);
+            for (int kb = 0; kb < KB; ++kb, ++it) {
+                const int s = it % STAGES;
+                uint4 cur[2][2] = {{w[0][0], w[0][1]}, {w[1][0], w[1][1]}};
+                uint32_t csc[2] = {sc[0], sc[1]};
+                if (kb + 1 < KB) {                                 // next block's codes fly while this one is converted
+                    const uint8_t* n0 = p0 + (size_t)(kb + 1) * kBlockBytes;
+                    const uint8_t* n1 = p1 + (size_t)(kb + 1) * kBlockBytes;
+                    w[0][0] = ldg_stream128(n0 + lane * 16);
+                    w[0][1] = ldg_stream128(n0 + 512 + lane * 16);
+                    sc[0] = ldg_stream32(n0 + kCodeBytes + q * 4);
+                    w[1][0] = ldg_stream128(n1 + lane * 16);
+                    w[1][1] = ldg_stream128(n1 + 512 + lane * 16);
+                    sc[1] = ldg_stream32(n1 + kCodeBytes + q * 4);
+                }
+                ok = mbar_wait(&empty[s], ((it / STAGES) & 1) ^ 1, abort_flag, a.status);
+                ok = __all_sync(0xffffffffu, ok);
+                if (!ok) break;
+                unsigned char* dst = sA + s * A_STAGE_BYTES;
+#pragma unroll
+                for (int pp = 0; pp < 2; ++pp) {
+                    const __half2 sh = *reinterpret_cast<const __half2*>(&csc[pp]);
+                    const __nv_bfloat162 s_lo = __float2bfloat162_rn(__low2float(sh));    // row q
+                    const __nv_bfloat162 s_hi = __float2bfloat162_rn(__high2float(sh));   // row q + 8
+                    const int rg = 2 * (2 * pw + pp);                                     // 8-row group of row q
+#pragma unroll
+                    for (int h = 0; h < 2; ++h) {
+                        const uint32_t words[4] = {cur[pp][h].x, cur[pp][h].y, cur[pp][h].z, cur[pp][h].w};
+#pragma unroll
+                        for (int wi = 0; wi < 4; ++wi) {
+                            const int r = wi & 1, set = wi >> 1;
+                            const int kc = 8 * h + 4 * set + c;                           // 16-byte k-chunk
+                            const uint4 val = dequant_word(words[wi], r ? s_hi : s_lo);
+                            *reinterpret_cast<uint4*>(dst + (rg + r) * SBO + kc * LBO + q * 16) = val;
+                        }
+                    }
+                }
+                fence_proxy_async();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&full[s]);
+            }
+        }
+    } else if (warp >= 12) {
+        // ------------------------------------------------------------------ B producers (gather token rows)
+        const int bw = warp - 12;                                  // k-chunks 4*bw .. 4*bw+3 of every row
+        const int nl = lane & 7, kcl = lane >> 3;
+        int it = 0;
+        bool ok = true;
+        for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
+            const Tile tl = a.tiles[t / MT];
+            const int row0 = offsets[tl.key] + tl.n0;
+            const int n_mma = (tl.nrows + 15) & ~15;
+            const int groups = n_mma / 8;                          // 8-row groups to fill
+            int src_row[BN / 8];                                   // source row of (group g, row nl); -1 = zero fill
+#pragma unroll
+            for (int g = 0; g < BN / 8; ++g) {
+                const int n = 8 * g + nl;
+                src_row[g] = -1;
+                if (n < tl.nrows) src_row[g] = GATEUP ? a.perm[row0 + n] / a.top_k : row0 + n;
+            }
+            for (int kb = 0; kb < KB; ++kb, ++it) {
+                const int s = it % STAGES;
+                ok = mbar_wait(&empty[s], ((it / STAGES) & 1) ^ 1, abort_flag, a.status);
+                ok = __all_sync(0xffffffffu, ok);
+                if (!ok) break;
+                const uint32_t dst = smem_u32(sB + s * B_STAGE_BYTES) + (4 * bw + kcl) * LBO + nl * 16;
+                const __nv_bfloat16* col = x_src + kb * BK + (4 * bw + kcl) * 8;
+#pragma unroll
+                for (int g = 0; g < BN / 8; ++g) {
+                    if (g < groups) {
+                        const bool live = src_row[g] >= 0;           // rows beyond the tile are zero-filled
+                        cp_async16(dst + g * SBO, col + (size_t)(live ? src_row[g] : 0) * K, live ? 16 : 0);
+                    }
+                }
+                cp_async_commit();
+                cp_async_wait<0>();
+                fence_proxy_async();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&full[s]);
+            }
+        }
+        cp_async_wait<0>();
+    }
+
+    // ---------------------------------------------------------------------- teardown (all roles, abort or not)
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    if (warp == 0) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512));
+}
+
+// n-tiles of one wave: every active group is cut into runs of at most BN grouped rows
+__global__ void tile_list_kernel(const int32_t* __restrict__ counts, const int32_t* __restrict__ group_keys,
+                                 const int32_t* __restrict__ wave_start, Tile* __restrict__ tiles,
+                                 int32_t* __restrict__ n_tiles) {
+    if (threadIdx.x != 0) return;
+    int n = 0;
+    for (int g = wave_start[0]; g < wave_start[1]; ++g) {
+        const int key = group_keys[g], cnt = counts[key];
+        const int pieces = (cnt + BN - 1) / BN;
+        const int per = ((cnt + pieces - 1) / pieces + 15) & ~15;   // balanced pieces, multiples of 16 rows
+        for (int n0 = 0; n0 < cnt; n0 += per) tiles[n++] = Tile{key, n0, min(per, cnt - n0), 0};
+    }
+    *n_tiles = n;
+}
+
+}  // namespace
+
+size_t prefill_scratch_bytes(int max_pairs, int num_experts) {
+    return ((size_t)max_pairs / 16 + num_experts + 16) * sizeof(Tile) + 256;
+}
+
+// One wave of the tensor-core path: tile list, gate/up GEMM + SwiGLU, down GEMM x routing weight.
+void launch_prefill_wave(const GemmArgs& g, const int32_t* wave_start, void* scratch, int* status,
+                         const __nv_bfloat16* hidden, __nv_bfloat16* act, const float* topk_w, float* y, int which,
+                         cudaStream_t st) {
+    int32_t* n_tiles = reinterpret_cast<int32_t*>(scratch);
+    Tile* tiles = reinterpret_cast<Tile*>(reinterpret_cast<unsigned char*>(scratch) + 256);
+    PrefillArgs a{};
+    a.slots = g.slots;
+    a.slot_stride = g.slot_stride;
+    a.perm = g.perm;
+    a.tiles = tiles;
+    a.n_tiles = n_tiles;
+    a.num_slots = g.num_slots;
+    a.top_k = g.top_k;
+    a.H = g.H;
+    a.I = g.I;
+    a.status = status;
+    const size_t smem = (size_t)STAGES * (A_STAGE_BYTES + B_STAGE_BYTES) + 256;
+    static bool attr_done = false;
+    if (!attr_done) {
+        cudaFuncSetAttribute(prefill_gemm_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        cudaFuncSetAttribute(prefill_gemm_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        attr_done = true;
+    }
+    int dev = 0, sms = 148;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    if (which & 1) {
+        tile_list_kernel<<<1, 32, 0, st>>>(g.counts, g.group_keys, wave_start, tiles, n_tiles);
+        prefill_gemm_kernel<true><<<sms, NUM_THREADS, smem, st>>>(a, hidden, act, nullptr, g.offsets, nullptr);
+        count_launch(2);
+    }
+    if (which & 2) {
+        if (!(which & 1)) {
+            tile_list_kernel<<<1, 32, 0, st>>>(g.counts, g.group_keys, wave_start, tiles, n_tiles);
+            count_launch();
+        }
+        prefill_gemm_kernel<false><<<sms, NUM_THREADS, smem, st>>>(a, act, nullptr, topk_w, g.offsets, y);
+        count_launch();
+    }
+}
+
+}  // namespace exmoe

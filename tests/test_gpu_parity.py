@@ -243,6 +243,51 @@ def test_group_size_sweep_single_expert(B, M):
     cache.close()
 
 
+# ------------------------------------------------------------------------------------ tensor-core path
+@pytest.mark.parametrize("T,alpha", [(130, 0.0), (200, 1.0), (513, 0.5)])
+def test_prefill_path_mid_shape(B, mid_layer, T, alpha):
+    """T*k > 512 routes through the tcgen05/TMEM kernels: ragged groups, several n-tiles, all tokens checked."""
+    ora, bank = mid_layer
+    s = synth.MID
+    hidden, ids, p = helpers.routed_inputs(s, T, seed=600 + T, alpha=alpha)
+    y, ref = ora.forward(hidden, ids, p)
+    cache = B.Cache(s, [bank], s.num_experts, max_tokens=600)
+    out = cache.forward(0, hidden.cuda(), ids.cuda(), p.cuda())
+    helpers.check_output(out, y, ref, f"T={T}")
+    assert cache.status() == 0
+    cache2 = B.Cache(s, [bank], 6, max_tokens=600, wave_cap=3)       # multi-wave with misses, same kernels
+    sc = ocache.SlotCache(s.num_experts, 6, 3, bytes_per_expert=cache2.bytes_per_expert)
+    out2 = cache2.forward(0, hidden.cuda(), ids.cuda(), p.cuda())
+    compare_plan(cache2, sc, ids)
+    assert torch.equal(out2.view(torch.int16), out.view(torch.int16))
+    assert cache2.status() == 0
+    cache.close()
+    cache2.close()
+
+
+@pytest.mark.parametrize("alpha", [0.0, 1.0])
+def test_config4_prefill_olmoe_sampled(B, olmoe_layer, alpha):
+    """Config 4: 2048 tokens x top-8 = 16384 rows over 64 experts (uniform and Zipf-skewed), 64 slots.
+    The plan is compared in full; the output on sampled tokens the oracle computes one by one."""
+    ora, bank = olmoe_layer
+    s = synth.OLMOE
+    T = 2048
+    hidden, ids, p = helpers.routed_inputs(s, T, seed=4000, alpha=alpha)
+    cache = B.Cache(s, [bank], 64, max_tokens=T)
+    sc = ocache.SlotCache(64, 64, 0, bytes_per_expert=cache.bytes_per_expert)
+    out = cache.forward(0, hidden.cuda(), ids.cuda(), p.cuda())
+    plan = compare_plan(cache, sc, ids)
+    rows = np.bincount(ids.numpy().reshape(-1), minlength=64)
+    assert rows.sum() == 16384 and (rows.max() > 1500 if alpha else rows.max() < 400)
+    sample = [0, 1, 777, 1023, 1024, 2047] + list(range(300, 306))
+    y, ref = ora.forward(hidden[sample], ids[sample], p[sample])
+    helpers.check_output(out[sample], y, ref, f"alpha={alpha}")
+    assert cache.status() == 0
+    again = cache.forward(0, hidden.cuda(), ids.cuda(), p.cuda())      # deterministic
+    assert torch.equal(again.view(torch.int16), out.view(torch.int16))
+    cache.close()
+
+
 # ------------------------------------------------------------------------------------ edge cases
 def test_edge_cases(B, tiny_layer):
     ora, bank = tiny_layer
