@@ -332,7 +332,8 @@ def main():
         flops = 2.0 * T * shape.top_k * 2 * shape.d_ff * shape.d_model          # gate/up GEMM of one step
         achieved = flops / (kinds["gate_up"]["us_per_launch"] * 1e-6) / 1e12
         roof = {"bound": "tensor", "achieved": achieved, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
-                "frac": achieved / peaks["bf16_tflops"], "traffic": None, "kernel": "gate_up", "peak_source": peaks["source"]}
+                "frac": achieved / peaks["bf16_tflops"], "traffic": None, "kernel": "gate_up (prefill_gemm_kernel<true>, tcgen05)", "flops_per_launch": flops,
+                "peak_source": peaks["source"] + " cuBLAS bf16, burst"}
     else:
         gu_bytes = active * w13_bytes                                            # packed gate/up codes + scales
         achieved = gu_bytes / (kinds["gate_up"]["us_per_launch"] * 1e-6) / 1e9
@@ -340,6 +341,7 @@ def main():
                 "frac": achieved / peaks["hbm_gbs"], "traffic": None, "kernel": "gate_up (decode_gemm_kernel)",
                 "bytes_per_launch": gu_bytes, "peak_source": peaks["source"] + " copy rate, burst"}
     step_gbs = active * bpe / (ms * 1e-3 / K) / 1e9
+    step_tflops = 2.0 * T * shape.top_k * 3 * shape.d_ff * shape.d_model / (ms * 1e-3 / K) / 1e12
 
     # ---- end to end: host buffers in, host buffer out, copies inside the timed region
     n_e2e = min(K, 300)
@@ -350,7 +352,7 @@ def main():
     d_h, d_i, d_w, d_o = torch.empty_like(hs[0]), torch.empty_like(ids[0]), torch.empty_like(ws[0]), torch.empty_like(hs[0])
 
     def e2e_step(i):
-        j = i % 8
+        j = i % len(h_h)
         with torch.cuda.stream(stream):
             d_h.copy_(h_h[j], non_blocking=True)
             d_i.copy_(h_i[j], non_blocking=True)
@@ -392,6 +394,7 @@ def main():
                            if L > 1 else "single layer bank (%.0f MB packed) vs 126 MB L2" % (64 * bpe / 1e6),
                            "timing": "CUDA graph replay of all steps" if identity else "host-driven loop (one plan read-back per step)",
                            "active_experts_per_step": active, "packed_gb_per_s_whole_step": step_gbs,
+                           "tflops_whole_step": step_tflops,
                            "kernel_us": kinds, "parallelism": "replicas only (no collective)", "status": status, **extra},
                 "roofline": roof, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": int(launches), "clocks": clocks}
         print(json.dumps(line), flush=True)

@@ -63,6 +63,8 @@ struct exmoe_cache {
     bool last_pair;
     int32_t* saved_ids;                       // ids of the last pairwise call (plan materialised on request)
     void* tc_scratch;                         // tile list of the tensor-core path
+    __nv_bfloat16* xg;                        // [max_pairs, H] hidden rows in plan order (tensor-core path only)
+    PrefillMaps tc_maps;                      // TMA descriptors of xg and act
     int32_t* h_plan;                          // pinned staging of the plan
     cudaStream_t copy_stream;
     cudaEvent_t ev_plan;
@@ -130,6 +132,7 @@ static void carve_workspace(exmoe_cache* c, uint8_t* ws, size_t* total) {
     c->arrive = k.take<int>(c->arrive_words);
     c->saved_ids = k.take<int32_t>(kPairMaxPairs);
     c->tc_scratch = k.take<uint8_t>(prefill_scratch_bytes(c->max_pairs, E));
+    c->xg = c->max_pairs > kSmallMaxPairs ? k.take<__nv_bfloat16>((size_t)c->max_pairs * s.d_model) : nullptr;
     *total = k.off;
 }
 
@@ -269,6 +272,7 @@ int exmoe_cache_create(exmoe_cache** out, const exmoe_shape* shape, int num_laye
     ok = ok && cudaMemset(c->plan.header, 0, c->plan_d2h_bytes) == cudaSuccess;
     ok = ok && cudaMemset(c->arrive, 0, c->arrive_words * 4) == cudaSuccess;
     for (int l = 0; l < num_layers && ok; ++l) ok = reset_layer(c, l) == EXMOE_OK;
+    if (ok && c->xg) ok = prefill_setup(&c->tc_maps, c->xg, c->act, c->max_pairs, c->shape.d_model, c->shape.d_ff) == EXMOE_OK;
     if (ok && c->C == c->shape.num_experts) {            // full residency: preload, slot = expert id
         for (int l = 0; l < num_layers && ok; ++l)
             ok = cudaMemcpy(c->slot_mem + (size_t)l * c->C * c->bpe, c->bank[l], (size_t)c->C * c->bpe,
@@ -336,6 +340,11 @@ int exmoe_moe_forward(exmoe_cache* c, int layer, const void* hidden, const int32
 
     const bool pairwise = small && P <= kPairMaxPairs && n_waves == 1;
     c->last_pair = pairwise;
+    if (!small && (!c->prof_only || c->prof_only == PROF_GATEUP)) {
+        ProfScope ps(c, PROF_PLAN, st);                  // hidden rows in plan order, once for all waves
+        launch_gather_rows((const __nv_bfloat16*)hidden, c->plan.perm, c->plan.offsets + c->n_keys, P, k, s.d_model,
+                           c->xg, st);
+    }
     if (small && n_waves == 0)                           // no valid id at all: the output is zero
         cudaMemsetAsync(out, 0, (size_t)T * s.d_model * 2, st);
     int mi = 0;
@@ -392,13 +401,13 @@ int exmoe_moe_forward(exmoe_cache* c, int layer, const void* hidden, const int32
             // many rows per expert: dense contraction on the tensor cores (tcgen05 / TMEM)
             if (!c->prof_only || c->prof_only == PROF_GATEUP) {
                 ProfScope ps(c, PROF_GATEUP, st);
-                launch_prefill_wave(a, a.wave_start, c->tc_scratch, c->d_status, (const __nv_bfloat16*)hidden, c->act,
-                                    topk_weights, c->y, 1, st);
+                launch_prefill_wave(a, a.wave_start, c->tc_scratch, c->d_status, &c->tc_maps, c->act, topk_weights, c->y, 1,
+                                    st);
             }
             if (!c->prof_only || c->prof_only == PROF_DOWN) {
                 ProfScope ps(c, PROF_DOWN, st);
-                launch_prefill_wave(a, a.wave_start, c->tc_scratch, c->d_status, (const __nv_bfloat16*)hidden, c->act,
-                                    topk_weights, c->y, 2, st);
+                launch_prefill_wave(a, a.wave_start, c->tc_scratch, c->d_status, &c->tc_maps, c->act, topk_weights, c->y, 2,
+                                    st);
             }
         }
         if (!identity) {

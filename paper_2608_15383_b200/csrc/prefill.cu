@@ -13,15 +13,24 @@
 //   warps 4-7     epilogue: tcgen05.ld the accumulator (warp w reads TMEM lanes 32(w%4)..), SwiGLU
 //                 -> BF16 activations, or routing weight -> fp32 pair buffer; two accumulators
 //                 (2 x 256 columns) let the epilogue of tile i overlap the MMAs of tile i+1.
-//   warps 8-11    A producers: stream packed int4 (128-bit loads, one block ahead in registers),
-//                 dequantise to BF16 (shift/lop3 -> 128+u, subtract 136, multiply by the group
-//                 scale) and store the canonical no-swizzle K-major core-matrix layout.
-//   warps 12-15   B producers: gather the tile's token rows with 16-byte cp.async into the same
-//                 canonical layout, two stages in flight.
+//   warp 1        B producer: one thread issues two TMA tile loads (cp.async.bulk.tensor.2d, 128-byte
+//                 swizzle, 256 rows x 64 columns each) per stage from the grouped activation matrix;
+//                 completion is counted in bytes on the stage's full barrier.  No multicast.
+//   warps 8-15    A producers, one 16-row panel each: stream packed int4 (128-bit loads, two blocks
+//                 ahead in registers), dequantise to BF16 (shift/lop3 -> 128+u, subtract 136,
+//                 multiply by the group scale) and store the canonical no-swizzle K-major
+//                 core-matrix layout (k-chunk stride padded to 160 bytes: conflict-free stores).
 // Producers -> MMA through full[stage] mbarriers (generic-proxy writes are fenced with
 // fence.proxy.async before the arrive), MMA -> producers through tcgen05.commit on empty[stage].
+// The gate/up GEMM reads its tokens from a grouped copy of the hidden states (rows in plan order),
+// written once per call by gather_rows_kernel, so that both GEMMs load B with plain tiled TMA.
 // Every wait is bounded: on expiry the CTA raises EXMOE_ERR_TIMEOUT, all roles drain, TMEM is freed.
+#include <cuda.h>
+
 #include "common.cuh"
+#ifdef EXMOE_PREFILL_PROF
+#include <cstdio>
+#endif
 
 namespace exmoe {
 
@@ -31,10 +40,15 @@ constexpr int BM = 128;            // weight rows per tile
 constexpr int BN = 256;            // max grouped rows (tokens) per tile
 constexpr int BK = 128;            // K per stage = one packed block / one scale group
 constexpr int STAGES = 2;
-constexpr int A_STAGE_BYTES = BM * BK * 2;     // 32 KB
-constexpr int B_STAGE_BYTES = BN * BK * 2;     // 64 KB
-constexpr int SBO = 16 * 128;      // bytes between 8-row groups (16 k-chunks of one 8-row group are contiguous)
-constexpr int LBO = 128;           // bytes between the two 16-byte k-chunks of one K16 step
+// A (dequantised weights): no swizzle; core matrix = 8 rows x 16 B; k-chunks 160 B apart (128 + 32 pad, so that
+// the 8 lanes of a quarter warp, 2 rows x 4 k-chunks, hit 8 different 16-byte bank groups), row groups 2560 B apart
+constexpr int A_LBO = 160;
+constexpr int A_SBO = 16 * A_LBO;
+constexpr int A_STAGE_BYTES = 16 * A_SBO;      // 40 KB
+// B (tokens): TMA 128-byte swizzle; two halves of 64 columns, each 256 rows x 128 B; 8-row atoms of 1024 B
+constexpr int B_HALF_BYTES = BN * 128;         // 32 KB
+constexpr int B_STAGE_BYTES = 2 * B_HALF_BYTES;
+constexpr int B_SBO = 1024;
 constexpr int NUM_THREADS = 512;
 constexpr long long kWaitBudget = 2000000000ll;   // clock64 ticks (~1 s) before a wait gives up
 
@@ -58,6 +72,18 @@ __device__ __forceinline__ bool mbar_try(uint64_t* bar, uint32_t parity) {
         : "memory");
     return ok != 0;
 }
+#ifdef EXMOE_PREFILL_PROF
+#define PROF_DECL long long prof_t0 = clock64(), prof_wait = 0
+#define PROF_WAIT_BEGIN long long prof_w0 = clock64()
+#define PROF_WAIT_END prof_wait += clock64() - prof_w0
+#define PROF_REPORT(name) if (blockIdx.x == 7 && lane == 0) printf("%s warp %d: total %lld wait %lld\n", name, warp, clock64() - prof_t0, prof_wait)
+#else
+#define PROF_DECL
+#define PROF_WAIT_BEGIN
+#define PROF_WAIT_END
+#define PROF_REPORT(name)
+#endif
+
 // bounded wait; returns false when the CTA is aborting (and raises the abort on expiry)
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag, int* status) {
     if (mbar_try(bar, parity)) return true;
@@ -98,14 +124,32 @@ __device__ __forceinline__ void tc_ld32(uint32_t taddr, uint32_t (&r)[32]) {
 }
 __device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
-// shared-memory matrix descriptor: no swizzle, K-major, version 1 (sm_100)
-__device__ __forceinline__ uint64_t make_desc(uint32_t saddr) {
+// shared-memory matrix descriptors, K-major, version 1 (sm_100)
+__device__ __forceinline__ uint64_t make_desc_a(uint32_t saddr) {            // no swizzle
     uint64_t d = 0;
     d |= (uint64_t)((saddr >> 4) & 0x3fff);
-    d |= (uint64_t)((LBO >> 4) & 0x3fff) << 16;
-    d |= (uint64_t)((SBO >> 4) & 0x3fff) << 32;
+    d |= (uint64_t)((A_LBO >> 4) & 0x3fff) << 16;
+    d |= (uint64_t)((A_SBO >> 4) & 0x3fff) << 32;
     d |= (uint64_t)1 << 46;
     return d;
+}
+__device__ __forceinline__ uint64_t make_desc_b(uint32_t saddr) {            // 128-byte swizzle
+    uint64_t d = 0;
+    d |= (uint64_t)((saddr >> 4) & 0x3fff);
+    d |= (uint64_t)1 << 16;                                                  // leading offset unused with swizzle
+    d |= (uint64_t)((B_SBO >> 4) & 0x3fff) << 32;
+    d |= (uint64_t)1 << 46;
+    d |= (uint64_t)2 << 61;
+    return d;
+}
+__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint64_t* bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+        ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(smem_u32(bar))
+        : "memory");
 }
 // instruction descriptor: D fp32, A/B BF16, both K-major, M = 128, N = n
 __device__ __forceinline__ uint32_t make_idesc(int n) {
@@ -158,12 +202,13 @@ struct PrefillArgs {
 
 template <bool GATEUP>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
-prefill_gemm_kernel(PrefillArgs a, const __nv_bfloat16* __restrict__ x_src, __nv_bfloat16* __restrict__ act_out,
+prefill_gemm_kernel(PrefillArgs a, const __grid_constant__ CUtensorMap tmap_b, __nv_bfloat16* __restrict__ act_out,
                     const float* __restrict__ topk_w, const int32_t* __restrict__ offsets, float* __restrict__ y_out) {
-    extern __shared__ __align__(1024) unsigned char smem[];
-    unsigned char* sA = smem;                                     // [STAGES][32 KB]
-    unsigned char* sB = smem + STAGES * A_STAGE_BYTES;            // [STAGES][64 KB]
-    uint64_t* bars = reinterpret_cast<uint64_t*>(sB + STAGES * B_STAGE_BYTES);
+    extern __shared__ unsigned char smem_raw[];
+    unsigned char* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);   // swizzled tiles need 1 KB alignment
+    unsigned char* sB = smem;                                     // [STAGES][64 KB]
+    unsigned char* sA = smem + STAGES * B_STAGE_BYTES;            // [STAGES][40 KB]
+    uint64_t* bars = reinterpret_cast<uint64_t*>(sA + STAGES * A_STAGE_BYTES);
     uint64_t* full = bars;              // [STAGES]  producers -> MMA (8 warp arrivals)
     uint64_t* empty = bars + 2;         // [STAGES]  MMA -> producers (tcgen05.commit)
     uint64_t* acc_full = bars + 4;      // [2]       MMA -> epilogue
@@ -180,7 +225,7 @@ prefill_gemm_kernel(PrefillArgs a, const __nv_bfloat16* __restrict__ x_src, __nv
 
     if (tid == 0) {
         for (int s = 0; s < STAGES; ++s) {
-            mbar_init(&full[s], 8);
+            mbar_init(&full[s], 9);           // 8 A-producer warps + the TMA thread's expect_tx arrive
             mbar_init(&empty[s], 1);
         }
         for (int b = 0; b < 2; ++b) {
@@ -205,29 +250,38 @@ prefill_gemm_kernel(PrefillArgs a, const __nv_bfloat16* __restrict__ x_src, __nv
         int it = 0;                                                // running k-block counter (stage/phase)
         int tcount = 0;
         bool ok = true;
+        PROF_DECL;
         for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x, ++tcount) {
             const Tile tl = a.tiles[t / MT];
             const int n_mma = (tl.nrows + 15) & ~15;
             const uint32_t idesc = make_idesc(n_mma);
             const int buf = tcount & 1;
+            PROF_WAIT_BEGIN;
             ok = mbar_wait(&acc_empty[buf], ((tcount >> 1) & 1) ^ 1, abort_flag, a.status);
+            PROF_WAIT_END;
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
             tc_fence_after();
             const uint32_t d_tmem = tmem_base + buf * BN;
             for (int kb = 0; kb < KB; ++kb, ++it) {
                 const int s = it % STAGES;
-                ok = mbar_wait(&full[s], (it / STAGES) & 1, abort_flag, a.status);
+                {
+                    PROF_WAIT_BEGIN;
+                    ok = mbar_wait(&full[s], (it / STAGES) & 1, abort_flag, a.status);
+                    PROF_WAIT_END;
+                }
                 ok = __all_sync(0xffffffffu, ok);
                 if (!ok) break;
                 tc_fence_after();
                 if (lane == 0) {
-                    const uint64_t da = make_desc(smem_u32(sA + s * A_STAGE_BYTES));
-                    const uint64_t db = make_desc(smem_u32(sB + s * B_STAGE_BYTES));
+                    const uint64_t da = make_desc_a(smem_u32(sA + s * A_STAGE_BYTES));
+                    const uint64_t db = make_desc_b(smem_u32(sB + s * B_STAGE_BYTES));
 #pragma unroll
-                    for (int j = 0; j < BK / 16; ++j)              // K16 step j: two 16-byte k-chunks = 256 bytes on
-                        tc_mma(d_tmem, da + (uint64_t)(j * 2 * LBO >> 4), db + (uint64_t)(j * 2 * LBO >> 4), idesc,
-                               (kb | j) ? 1u : 0u);
+                    for (int j = 0; j < BK / 16; ++j) {            // K16 step j: A two k-chunks on, B 32 bytes on in its half
+                        const uint64_t aj = da + (uint64_t)(j * 2 * A_LBO >> 4);
+                        const uint64_t bj = db + (uint64_t)(((j >> 2) * B_HALF_BYTES + (j & 3) * 32) >> 4);
+                        tc_mma(d_tmem, aj, bj, idesc, (kb | j) ? 1u : 0u);
+                    }
                     tc_commit(&empty[s]);                          // stage reusable once these MMAs have read it
                 }
                 __syncwarp();
@@ -235,16 +289,20 @@ prefill_gemm_kernel(PrefillArgs a, const __nv_bfloat16* __restrict__ x_src, __nv
             if (ok && lane == 0) tc_commit(&acc_full[buf]);        // accumulator complete
             __syncwarp();
         }
+        PROF_REPORT("mma");
     } else if (warp >= 4 && warp < 8) {
         // ------------------------------------------------------------------ epilogue
         const int e = warp & 3;                                    // TMEM lane quarter
         int tcount = 0;
         bool ok = true;
+        PROF_DECL;
         for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x, ++tcount) {
             const Tile tl = a.tiles[t / MT];
             const int mt = t % MT;
             const int buf = tcount & 1;
+            PROF_WAIT_BEGIN;
             ok = mbar_wait(&acc_full[buf], (tcount >> 1) & 1, abort_flag, a.status);
+            PROF_WAIT_END;
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
             tc_fence_after();
@@ -266,17 +324,21 @@ prefill_gemm_kernel(PrefillArgs a, const __nv_bfloat16* __restrict__ x_src, __nv
                         const float u = __uint_as_float((lane < 16) ? recv : v[j + 16]);
                         const int n = c0 + col;
                         if (n < tl.nrows)
-                            act_out[(size_t)(row0 + n) * a.I + interm] = __float2bfloat16_rn(g / (1.f + __expf(-g)) * u);
+                            act_out[(size_t)(row0 + n) * a.I + interm] = __float2bfloat16_rn(__fdividef(g, 1.f + __expf(-g)) * u);
                     }
                 } else {
                     const int h = mt * BM + 32 * e + lane;
+                    int my_pair = 0;                               // lane j holds pair and weight of column c0 + j
+                    float my_w = 0.f;
+                    if (c0 + lane < tl.nrows) {
+                        my_pair = a.perm[row0 + c0 + lane];
+                        my_w = topk_w[my_pair];
+                    }
 #pragma unroll
                     for (int j = 0; j < 32; ++j) {
-                        const int n = c0 + j;
-                        if (n < tl.nrows) {
-                            const int pair = a.perm[row0 + n];
-                            y_out[(size_t)pair * a.H + h] = topk_w[pair] * __uint_as_float(v[j]);
-                        }
+                        const int pair = __shfl_sync(0xffffffffu, my_pair, j);
+                        const float wj = __shfl_sync(0xffffffffu, my_w, j);
+                        if (c0 + j < tl.nrows) y_out[(size_t)pair * a.H + h] = wj * __uint_as_float(v[j]);
                     }
                 }
             }
@@ -284,108 +346,102 @@ prefill_gemm_kernel(PrefillArgs a, const __nv_bfloat16* __restrict__ x_src, __nv
             __syncwarp();
             if (lane == 0) mbar_arrive(&acc_empty[buf]);
         }
-    } else if (warp >= 8 && warp < 12) {
-        // ------------------------------------------------------------------ A producers (dequantise)
-        const int pw = warp - 8;                                   // handles panels 2*pw, 2*pw+1 of the tile
+        PROF_REPORT("epilogue");
+    } else if (warp == 1) {
+        // ------------------------------------------------------------------ B producer (TMA, one thread issues)
+        int it = 0;
+        bool ok = true;
+        PROF_DECL;
+        for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
+            const Tile tl = a.tiles[t / MT];
+            const int row0 = offsets[tl.key] + tl.n0;
+            for (int kb = 0; kb < KB; ++kb, ++it) {
+                const int s = it % STAGES;
+                {
+                    PROF_WAIT_BEGIN;
+                    ok = mbar_wait(&empty[s], ((it / STAGES) & 1) ^ 1, abort_flag, a.status);
+                    PROF_WAIT_END;
+                }
+                ok = __all_sync(0xffffffffu, ok);
+                if (!ok) break;
+                if (lane == 0) {
+                    const uint32_t dst = smem_u32(sB + s * B_STAGE_BYTES);
+                    mbar_expect_tx(&full[s], B_STAGE_BYTES);
+                    tma_load_2d(dst, &tmap_b, kb * BK, row0, &full[s]);                   // columns kb*128 .. +63
+                    tma_load_2d(dst + B_HALF_BYTES, &tmap_b, kb * BK + 64, row0, &full[s]);
+                }
+                __syncwarp();
+            }
+        }
+        PROF_REPORT("B producer");
+    } else if (warp >= 8) {
+        // ------------------------------------------------------------------ A producers (dequantise), one panel each
+        const int pw = warp - 8;                                   // panel of the tile = 8-row groups 2*pw, 2*pw+1
         const int q = lane >> 2, c = lane & 3;
         int it = 0;
         bool ok = true;
+        PROF_DECL;
         for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
             const Tile tl = a.tiles[t / MT];
             const int mt = t % MT;
             const int slot = tl.key % a.num_slots;
             const uint8_t* mat = a.slots + (size_t)slot * a.slot_stride + (GATEUP ? 0 : w13_bytes);
-            const uint8_t* p0 = mat + (size_t)(mt * 8 + 2 * pw) * KB * kBlockBytes;      // panel 2*pw of the tile
-            const uint8_t* p1 = p0 + (size_t)KB * kBlockBytes;
-            uint4 w[2][2];
-            uint32_t sc[2];
-            w[0][0] = ldg_stream128(p0 + lane * 16);
-            w[0][1] = ldg_stream128(p0 + 512 + lane * 16);
-            sc[0] = ldg_stream32(p0 + kCodeBytes + q * 4);
-            w[1][0] = ldg_stream128(p1 + lane * 16);
-            w[1][1] = ldg_stream128(p1 + 512 + lane * 16);
-            sc[1] = ldg_stream32(p1 + kCodeBytes + q * 4);
-            for (int kb = 0; kb < KB; ++kb, ++it) {
-                const int s = it % STAGES;
-                uint4 cur[2][2] = {{w[0][0], w[0][1]}, {w[1][0], w[1][1]}};
-                uint32_t csc[2] = {sc[0], sc[1]};
-                if (kb + 1 < KB) {                                 // next block's codes fly while this one is converted
-                    const uint8_t* n0 = p0 + (size_t)(kb + 1) * kBlockBytes;
-                    const uint8_t* n1 = p1 + (size_t)(kb + 1) * kBlockBytes;
-                    w[0][0] = ldg_stream128(n0 + lane * 16);
-                    w[0][1] = ldg_stream128(n0 + 512 + lane * 16);
-                    sc[0] = ldg_stream32(n0 + kCodeBytes + q * 4);
-                    w[1][0] = ldg_stream128(n1 + lane * 16);
-                    w[1][1] = ldg_stream128(n1 + 512 + lane * 16);
-                    sc[1] = ldg_stream32(n1 + kCodeBytes + q * 4);
-                }
-                ok = mbar_wait(&empty[s], ((it / STAGES) & 1) ^ 1, abort_flag, a.status);
-                ok = __all_sync(0xffffffffu, ok);
-                if (!ok) break;
-                unsigned char* dst = sA + s * A_STAGE_BYTES;
+            const uint8_t* pn = mat + (size_t)(mt * 8 + pw) * KB * kBlockBytes;
+            constexpr int PF = 3;                                  // blocks in flight per lane (this one + 2 ahead)
+            uint4 w[PF][2];
+            uint32_t sc[PF];
 #pragma unroll
-                for (int pp = 0; pp < 2; ++pp) {
-                    const __half2 sh = *reinterpret_cast<const __half2*>(&csc[pp]);
+            for (int i = 0; i < PF - 1; ++i)
+                if (i < KB) {
+                    const uint8_t* blk = pn + (size_t)i * kBlockBytes;
+                    w[i][0] = ldg_stream128(blk + lane * 16);
+                    w[i][1] = ldg_stream128(blk + 512 + lane * 16);
+                    sc[i] = ldg_stream32(blk + kCodeBytes + q * 4);
+                }
+            for (int kb0 = 0; kb0 < KB; kb0 += PF) {
+#pragma unroll
+                for (int u = 0; u < PF; ++u) {
+                    const int kb = kb0 + u;
+                    if (kb >= KB) break;
+                    const int s = it % STAGES;
+                    constexpr int nx_off = PF - 1;
+                    if (kb + nx_off < KB) {                        // keep two blocks of codes in flight
+                        const uint8_t* blk = pn + (size_t)(kb + nx_off) * kBlockBytes;
+                        w[(u + nx_off) % PF][0] = ldg_stream128(blk + lane * 16);
+                        w[(u + nx_off) % PF][1] = ldg_stream128(blk + 512 + lane * 16);
+                        sc[(u + nx_off) % PF] = ldg_stream32(blk + kCodeBytes + q * 4);
+                    }
+                    {
+                        PROF_WAIT_BEGIN;
+                        ok = mbar_wait(&empty[s], ((it / STAGES) & 1) ^ 1, abort_flag, a.status);
+                        PROF_WAIT_END;
+                    }
+                    ok = __all_sync(0xffffffffu, ok);
+                    if (!ok) break;
+                    unsigned char* dst = sA + s * A_STAGE_BYTES;
+                    const __half2 sh = *reinterpret_cast<const __half2*>(&sc[u]);
                     const __nv_bfloat162 s_lo = __float2bfloat162_rn(__low2float(sh));    // row q
                     const __nv_bfloat162 s_hi = __float2bfloat162_rn(__high2float(sh));   // row q + 8
-                    const int rg = 2 * (2 * pw + pp);                                     // 8-row group of row q
 #pragma unroll
                     for (int h = 0; h < 2; ++h) {
-                        const uint32_t words[4] = {cur[pp][h].x, cur[pp][h].y, cur[pp][h].z, cur[pp][h].w};
+                        const uint32_t words[4] = {w[u][h].x, w[u][h].y, w[u][h].z, w[u][h].w};
 #pragma unroll
                         for (int wi = 0; wi < 4; ++wi) {
                             const int r = wi & 1, set = wi >> 1;
                             const int kc = 8 * h + 4 * set + c;                           // 16-byte k-chunk
                             const uint4 val = dequant_word(words[wi], r ? s_hi : s_lo);
-                            *reinterpret_cast<uint4*>(dst + (rg + r) * SBO + kc * LBO + q * 16) = val;
+                            *reinterpret_cast<uint4*>(dst + (2 * pw + r) * A_SBO + kc * A_LBO + q * 16) = val;
                         }
                     }
+                    fence_proxy_async();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(&full[s]);
+                    ++it;
                 }
-                fence_proxy_async();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(&full[s]);
-            }
-        }
-    } else if (warp >= 12) {
-        // ------------------------------------------------------------------ B producers (gather token rows)
-        const int bw = warp - 12;                                  // k-chunks 4*bw .. 4*bw+3 of every row
-        const int nl = lane & 7, kcl = lane >> 3;
-        int it = 0;
-        bool ok = true;
-        for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
-            const Tile tl = a.tiles[t / MT];
-            const int row0 = offsets[tl.key] + tl.n0;
-            const int n_mma = (tl.nrows + 15) & ~15;
-            const int groups = n_mma / 8;                          // 8-row groups to fill
-            int src_row[BN / 8];                                   // source row of (group g, row nl); -1 = zero fill
-#pragma unroll
-            for (int g = 0; g < BN / 8; ++g) {
-                const int n = 8 * g + nl;
-                src_row[g] = -1;
-                if (n < tl.nrows) src_row[g] = GATEUP ? a.perm[row0 + n] / a.top_k : row0 + n;
-            }
-            for (int kb = 0; kb < KB; ++kb, ++it) {
-                const int s = it % STAGES;
-                ok = mbar_wait(&empty[s], ((it / STAGES) & 1) ^ 1, abort_flag, a.status);
-                ok = __all_sync(0xffffffffu, ok);
                 if (!ok) break;
-                const uint32_t dst = smem_u32(sB + s * B_STAGE_BYTES) + (4 * bw + kcl) * LBO + nl * 16;
-                const __nv_bfloat16* col = x_src + kb * BK + (4 * bw + kcl) * 8;
-#pragma unroll
-                for (int g = 0; g < BN / 8; ++g) {
-                    if (g < groups) {
-                        const bool live = src_row[g] >= 0;           // rows beyond the tile are zero-filled
-                        cp_async16(dst + g * SBO, col + (size_t)(live ? src_row[g] : 0) * K, live ? 16 : 0);
-                    }
-                }
-                cp_async_commit();
-                cp_async_wait<0>();
-                fence_proxy_async();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(&full[s]);
             }
         }
-        cp_async_wait<0>();
+        PROF_REPORT("A producer");
     }
 
     // ---------------------------------------------------------------------- teardown (all roles, abort or not)
@@ -393,6 +449,17 @@ prefill_gemm_kernel(PrefillArgs a, const __nv_bfloat16* __restrict__ x_src, __nv
     __syncthreads();
     tc_fence_after();
     if (warp == 0) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512));
+}
+
+// grouped copy of the hidden states: row r of the plan order = hidden row of token perm[r] / k
+__global__ void __launch_bounds__(256)
+gather_rows_kernel(const __nv_bfloat16* __restrict__ hidden, const int32_t* __restrict__ perm,
+                   const int32_t* __restrict__ n_valid, int top_k, int H, __nv_bfloat16* __restrict__ xg) {
+    const int r = blockIdx.x;
+    if (r >= *n_valid) return;
+    const uint4* src = reinterpret_cast<const uint4*>(hidden + (size_t)(perm[r] / top_k) * H);
+    uint4* dst = reinterpret_cast<uint4*>(xg + (size_t)r * H);
+    for (int i = threadIdx.x; i < H / 8; i += 256) dst[i] = src[i];
 }
 
 // n-tiles of one wave: every active group is cut into runs of at most BN grouped rows
@@ -416,10 +483,45 @@ size_t prefill_scratch_bytes(int max_pairs, int num_experts) {
     return ((size_t)max_pairs / 16 + num_experts + 16) * sizeof(Tile) + 256;
 }
 
+static_assert(sizeof(CUtensorMap) == 128, "PrefillMaps mirrors two CUtensorMap objects");
+
+// 2-D row-major BF16 matrix [rows, cols] -> tensor map with a 64-column x 256-row box, 128-byte swizzle
+static int encode_map(CUtensorMap* out, const void* base, int rows, int cols) {
+    typedef CUresult (*EncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                 const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                 CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+    static EncodeFn fn = nullptr;
+    if (!fn) {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult qr;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qr) != cudaSuccess || !p) return EXMOE_ERR_CUDA;
+        fn = reinterpret_cast<EncodeFn>(p);
+    }
+    const cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+    const cuuint64_t strides[1] = {(cuuint64_t)cols * 2};
+    const cuuint32_t box[2] = {64, (cuuint32_t)BN};
+    const cuuint32_t estr[2] = {1, 1};
+    const CUresult rc = fn(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+                           CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return rc == CUDA_SUCCESS ? EXMOE_OK : EXMOE_ERR_CUDA;
+}
+
+int prefill_setup(PrefillMaps* maps, const __nv_bfloat16* xg, const __nv_bfloat16* act, int max_pairs, int H, int I) {
+    int rc = encode_map(reinterpret_cast<CUtensorMap*>(maps->x), xg, max_pairs, H);
+    if (rc) return rc;
+    return encode_map(reinterpret_cast<CUtensorMap*>(maps->act), act, max_pairs, I);
+}
+
+void launch_gather_rows(const __nv_bfloat16* hidden, const int32_t* perm, const int32_t* n_valid, int n_pairs, int top_k,
+                        int H, __nv_bfloat16* xg, cudaStream_t st) {
+    gather_rows_kernel<<<n_pairs, 256, 0, st>>>(hidden, perm, n_valid, top_k, H, xg);
+    count_launch();
+}
+
 // One wave of the tensor-core path: tile list, gate/up GEMM + SwiGLU, down GEMM x routing weight.
-void launch_prefill_wave(const GemmArgs& g, const int32_t* wave_start, void* scratch, int* status,
-                         const __nv_bfloat16* hidden, __nv_bfloat16* act, const float* topk_w, float* y, int which,
-                         cudaStream_t st) {
+void launch_prefill_wave(const GemmArgs& g, const int32_t* wave_start, void* scratch, int* status, const PrefillMaps* maps,
+                         __nv_bfloat16* act, const float* topk_w, float* y, int which, cudaStream_t st) {
     int32_t* n_tiles = reinterpret_cast<int32_t*>(scratch);
     Tile* tiles = reinterpret_cast<Tile*>(reinterpret_cast<unsigned char*>(scratch) + 256);
     PrefillArgs a{};
@@ -433,7 +535,7 @@ void launch_prefill_wave(const GemmArgs& g, const int32_t* wave_start, void* scr
     a.H = g.H;
     a.I = g.I;
     a.status = status;
-    const size_t smem = (size_t)STAGES * (A_STAGE_BYTES + B_STAGE_BYTES) + 256;
+    const size_t smem = (size_t)STAGES * (A_STAGE_BYTES + B_STAGE_BYTES) + 256 + 1024;
     static bool attr_done = false;
     if (!attr_done) {
         cudaFuncSetAttribute(prefill_gemm_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
@@ -443,9 +545,11 @@ void launch_prefill_wave(const GemmArgs& g, const int32_t* wave_start, void* scr
     int dev = 0, sms = 148;
     cudaGetDevice(&dev);
     cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    const CUtensorMap* mx = reinterpret_cast<const CUtensorMap*>(maps->x);
+    const CUtensorMap* ma = reinterpret_cast<const CUtensorMap*>(maps->act);
     if (which & 1) {
         tile_list_kernel<<<1, 32, 0, st>>>(g.counts, g.group_keys, wave_start, tiles, n_tiles);
-        prefill_gemm_kernel<true><<<sms, NUM_THREADS, smem, st>>>(a, hidden, act, nullptr, g.offsets, nullptr);
+        prefill_gemm_kernel<true><<<sms, NUM_THREADS, smem, st>>>(a, *mx, act, nullptr, g.offsets, nullptr);
         count_launch(2);
     }
     if (which & 2) {
@@ -453,7 +557,7 @@ void launch_prefill_wave(const GemmArgs& g, const int32_t* wave_start, void* scr
             tile_list_kernel<<<1, 32, 0, st>>>(g.counts, g.group_keys, wave_start, tiles, n_tiles);
             count_launch();
         }
-        prefill_gemm_kernel<false><<<sms, NUM_THREADS, smem, st>>>(a, act, nullptr, topk_w, g.offsets, y);
+        prefill_gemm_kernel<false><<<sms, NUM_THREADS, smem, st>>>(a, *ma, nullptr, topk_w, g.offsets, y);
         count_launch();
     }
 }
