@@ -309,7 +309,9 @@ int exmoe_moe_forward(exmoe_cache* c, int layer, const void* hidden, const int32
             return EXMOE_ERR_CUDA;
         if (cudaEventRecord(c->ev_plan, st) != cudaSuccess) return EXMOE_ERR_CUDA;
     }
-    if (!small) {
+    // timing runs that launch one kernel kind reuse the plan, grouped rows and tile list of the previous full call
+    const bool build_plan = (c->prof_only == 0);
+    if (!small && build_plan) {
         ProfScope ps(c, PROF_PLAN, st);
         launch_group(s, C, c->n_keys, c->max_waves, identity, topk_ids, P, c->plan, c->d_status, st);
     }
@@ -340,7 +342,7 @@ int exmoe_moe_forward(exmoe_cache* c, int layer, const void* hidden, const int32
 
     const bool pairwise = small && P <= kPairMaxPairs && n_waves == 1;
     c->last_pair = pairwise;
-    if (!small && (!c->prof_only || c->prof_only == PROF_GATEUP)) {
+    if (!small && build_plan) {
         ProfScope ps(c, PROF_PLAN, st);                  // hidden rows in plan order, once for all waves
         launch_gather_rows((const __nv_bfloat16*)hidden, c->plan.perm, c->plan.offsets + c->n_keys, P, k, s.d_model,
                            c->xg, st);
@@ -399,6 +401,7 @@ int exmoe_moe_forward(exmoe_cache* c, int layer, const void* hidden, const int32
             }
         } else {
             // many rows per expert: dense contraction on the tensor cores (tcgen05 / TMEM)
+            if (build_plan) launch_prefill_wave(a, a.wave_start, c->tc_scratch, c->d_status, &c->tc_maps, c->act, topk_weights, c->y, 4, st);
             if (!c->prof_only || c->prof_only == PROF_GATEUP) {
                 ProfScope ps(c, PROF_GATEUP, st);
                 launch_prefill_wave(a, a.wave_start, c->tc_scratch, c->d_status, &c->tc_maps, c->act, topk_weights, c->y, 1,

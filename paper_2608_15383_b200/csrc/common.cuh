@@ -100,7 +100,7 @@ struct alignas(64) PrefillMaps { unsigned char x[128], act[128]; };   // two CUt
 int prefill_setup(PrefillMaps* maps, const __nv_bfloat16* xg, const __nv_bfloat16* act, int max_pairs, int H, int I);
 void launch_gather_rows(const __nv_bfloat16* hidden, const int32_t* perm, const int32_t* n_valid, int n_pairs, int top_k,
                         int H, __nv_bfloat16* xg, cudaStream_t st);
-// which: bit 0 = gate/up GEMM + SwiGLU, bit 1 = down GEMM x routing weight
+// which: bit 0 = gate/up GEMM + SwiGLU, bit 1 = down GEMM x routing weight, bit 2 = (re)build the wave's tile list
 void launch_prefill_wave(const GemmArgs& g, const int32_t* wave_start, void* scratch, int* status, const PrefillMaps* maps,
                          __nv_bfloat16* act, const float* topk_w, float* y, int which, cudaStream_t st);
 void launch_combine(const float* y, const int32_t* ids, int E, int T, int k, int H, __nv_bfloat16* out,

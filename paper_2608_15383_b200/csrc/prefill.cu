@@ -10,14 +10,15 @@
 // A persistent CTA (one per SM, 16 warps) is specialised by warp:
 //   warp 0        allocates TMEM, then one elected thread issues tcgen05.mma (8 x K16 per 128-wide
 //                 block) and tcgen05.commit to the stage-empty / accumulator-full mbarriers.
-//   warps 4-7     epilogue: tcgen05.ld the accumulator (warp w reads TMEM lanes 32(w%4)..), SwiGLU
-//                 -> BF16 activations, or routing weight -> fp32 pair buffer; two accumulators
-//                 (2 x 256 columns) let the epilogue of tile i overlap the MMAs of tile i+1.
+//   warps 4-7,    epilogue (two groups, even / odd 32-column chunks): tcgen05.ld the accumulator (warp w
+//   16-19         reads TMEM lanes 32(w%4)..), SwiGLU -> BF16 activations, or routing weight -> fp32
+//                 pair buffer; two accumulators (2 x 256 columns) let the epilogue of tile i overlap
+//                 the MMAs of tile i+1.
 //   warp 1        B producer: one thread issues two TMA tile loads (cp.async.bulk.tensor.2d, 128-byte
 //                 swizzle, 256 rows x 64 columns each) per stage from the grouped activation matrix;
 //                 completion is counted in bytes on the stage's full barrier.  No multicast.
-//   warps 8-15    A producers, one 16-row panel each: stream packed int4 (128-bit loads, two blocks
-//                 ahead in registers), dequantise to BF16 (shift/lop3 -> 128+u, subtract 136,
+//   warps 8-15,   A producers, one 16-row panel and one 64-wide k-half each: stream packed int4 (128-bit
+//   20-27         loads, two blocks ahead in registers), dequantise to BF16 (shift/lop3 -> 128+u, subtract 136,
 //                 multiply by the group scale) and store the canonical no-swizzle K-major
 //                 core-matrix layout (k-chunk stride padded to 160 bytes: conflict-free stores).
 // Producers -> MMA through full[stage] mbarriers (generic-proxy writes are fenced with
@@ -49,7 +50,7 @@ constexpr int A_STAGE_BYTES = 16 * A_SBO;      // 40 KB
 constexpr int B_HALF_BYTES = BN * 128;         // 32 KB
 constexpr int B_STAGE_BYTES = 2 * B_HALF_BYTES;
 constexpr int B_SBO = 1024;
-constexpr int NUM_THREADS = 512;
+constexpr int NUM_THREADS = 896;   // 28 warps: MMA, TMA, 2 idle, 4 + 4 epilogue, 8 + 8 dequant
 constexpr long long kWaitBudget = 2000000000ll;   // clock64 ticks (~1 s) before a wait gives up
 
 struct Tile { int key, n0, nrows, pad; };
@@ -225,12 +226,12 @@ prefill_gemm_kernel(PrefillArgs a, const __grid_constant__ CUtensorMap tmap_b, _
 
     if (tid == 0) {
         for (int s = 0; s < STAGES; ++s) {
-            mbar_init(&full[s], 9);           // 8 A-producer warps + the TMA thread's expect_tx arrive
+            mbar_init(&full[s], 17);          // 16 A-producer warps + the TMA thread's expect_tx arrive
             mbar_init(&empty[s], 1);
         }
         for (int b = 0; b < 2; ++b) {
             mbar_init(&acc_full[b], 1);
-            mbar_init(&acc_empty[b], 4);
+            mbar_init(&acc_empty[b], 8);
         }
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -290,9 +291,10 @@ prefill_gemm_kernel(PrefillArgs a, const __grid_constant__ CUtensorMap tmap_b, _
             __syncwarp();
         }
         PROF_REPORT("mma");
-    } else if (warp >= 4 && warp < 8) {
+    } else if ((warp >= 4 && warp < 8) || (warp >= 16 && warp < 20)) {
         // ------------------------------------------------------------------ epilogue
         const int e = warp & 3;                                    // TMEM lane quarter
+        const int odd = warp >= 16 ? 32 : 0;                       // second group takes the odd 32-column chunks
         int tcount = 0;
         bool ok = true;
         PROF_DECL;
@@ -308,7 +310,7 @@ prefill_gemm_kernel(PrefillArgs a, const __grid_constant__ CUtensorMap tmap_b, _
             tc_fence_after();
             const int row0 = offsets[tl.key] + tl.n0;
             const uint32_t taddr = tmem_base + buf * BN + ((uint32_t)(32 * e) << 16);
-            for (int c0 = 0; c0 < tl.nrows; c0 += 32) {
+            for (int c0 = odd; c0 < tl.nrows; c0 += 64) {
                 uint32_t v[32];
                 tc_ld32(taddr + c0, v);
                 tc_wait_ld();
@@ -374,9 +376,10 @@ prefill_gemm_kernel(PrefillArgs a, const __grid_constant__ CUtensorMap tmap_b, _
             }
         }
         PROF_REPORT("B producer");
-    } else if (warp >= 8) {
-        // ------------------------------------------------------------------ A producers (dequantise), one panel each
-        const int pw = warp - 8;                                   // panel of the tile = 8-row groups 2*pw, 2*pw+1
+    } else if (warp >= 8 && !(warp >= 16 && warp < 20)) {
+        // ------------------------------------------------------------------ A producers (dequantise)
+        const int pw = warp & 7;                                   // panel of the tile = 8-row groups 2*pw, 2*pw+1
+        const int hh = warp >= 20 ? 1 : 0;                         // 64-wide k-half of every block
         const int q = lane >> 2, c = lane & 3;
         int it = 0;
         bool ok = true;
@@ -388,14 +391,13 @@ prefill_gemm_kernel(PrefillArgs a, const __grid_constant__ CUtensorMap tmap_b, _
             const uint8_t* mat = a.slots + (size_t)slot * a.slot_stride + (GATEUP ? 0 : w13_bytes);
             const uint8_t* pn = mat + (size_t)(mt * 8 + pw) * KB * kBlockBytes;
             constexpr int PF = 3;                                  // blocks in flight per lane (this one + 2 ahead)
-            uint4 w[PF][2];
+            uint4 w[PF];
             uint32_t sc[PF];
 #pragma unroll
             for (int i = 0; i < PF - 1; ++i)
                 if (i < KB) {
                     const uint8_t* blk = pn + (size_t)i * kBlockBytes;
-                    w[i][0] = ldg_stream128(blk + lane * 16);
-                    w[i][1] = ldg_stream128(blk + 512 + lane * 16);
+                    w[i] = ldg_stream128(blk + hh * 512 + lane * 16);
                     sc[i] = ldg_stream32(blk + kCodeBytes + q * 4);
                 }
             for (int kb0 = 0; kb0 < KB; kb0 += PF) {
@@ -407,8 +409,7 @@ prefill_gemm_kernel(PrefillArgs a, const __grid_constant__ CUtensorMap tmap_b, _
                     constexpr int nx_off = PF - 1;
                     if (kb + nx_off < KB) {                        // keep two blocks of codes in flight
                         const uint8_t* blk = pn + (size_t)(kb + nx_off) * kBlockBytes;
-                        w[(u + nx_off) % PF][0] = ldg_stream128(blk + lane * 16);
-                        w[(u + nx_off) % PF][1] = ldg_stream128(blk + 512 + lane * 16);
+                        w[(u + nx_off) % PF] = ldg_stream128(blk + hh * 512 + lane * 16);
                         sc[(u + nx_off) % PF] = ldg_stream32(blk + kCodeBytes + q * 4);
                     }
                     {
@@ -422,16 +423,13 @@ prefill_gemm_kernel(PrefillArgs a, const __grid_constant__ CUtensorMap tmap_b, _
                     const __half2 sh = *reinterpret_cast<const __half2*>(&sc[u]);
                     const __nv_bfloat162 s_lo = __float2bfloat162_rn(__low2float(sh));    // row q
                     const __nv_bfloat162 s_hi = __float2bfloat162_rn(__high2float(sh));   // row q + 8
+                    const uint32_t words[4] = {w[u].x, w[u].y, w[u].z, w[u].w};
 #pragma unroll
-                    for (int h = 0; h < 2; ++h) {
-                        const uint32_t words[4] = {w[u][h].x, w[u][h].y, w[u][h].z, w[u][h].w};
-#pragma unroll
-                        for (int wi = 0; wi < 4; ++wi) {
-                            const int r = wi & 1, set = wi >> 1;
-                            const int kc = 8 * h + 4 * set + c;                           // 16-byte k-chunk
-                            const uint4 val = dequant_word(words[wi], r ? s_hi : s_lo);
-                            *reinterpret_cast<uint4*>(dst + (2 * pw + r) * A_SBO + kc * A_LBO + q * 16) = val;
-                        }
+                    for (int wi = 0; wi < 4; ++wi) {
+                        const int r = wi & 1, set = wi >> 1;
+                        const int kc = 8 * hh + 4 * set + c;                              // 16-byte k-chunk
+                        const uint4 val = dequant_word(words[wi], r ? s_hi : s_lo);
+                        *reinterpret_cast<uint4*>(dst + (2 * pw + r) * A_SBO + kc * A_LBO + q * 16) = val;
                     }
                     fence_proxy_async();
                     __syncwarp();
@@ -462,19 +460,47 @@ gather_rows_kernel(const __nv_bfloat16* __restrict__ hidden, const int32_t* __re
     for (int i = threadIdx.x; i < H / 8; i += 256) dst[i] = src[i];
 }
 
-// n-tiles of one wave: every active group is cut into runs of at most BN grouped rows
-__global__ void tile_list_kernel(const int32_t* __restrict__ counts, const int32_t* __restrict__ group_keys,
-                                 const int32_t* __restrict__ wave_start, Tile* __restrict__ tiles,
-                                 int32_t* __restrict__ n_tiles) {
-    if (threadIdx.x != 0) return;
-    int n = 0;
-    for (int g = wave_start[0]; g < wave_start[1]; ++g) {
-        const int key = group_keys[g], cnt = counts[key];
-        const int pieces = (cnt + BN - 1) / BN;
-        const int per = ((cnt + pieces - 1) / pieces + 15) & ~15;   // balanced pieces, multiples of 16 rows
-        for (int n0 = 0; n0 < cnt; n0 += per) tiles[n++] = Tile{key, n0, min(per, cnt - n0), 0};
+// n-tiles of one wave: every active group is cut into balanced runs of at most BN grouped rows (multiples of 16).
+// One CTA; thread g handles group g, an exclusive scan of the piece counts places its tiles.
+__global__ void __launch_bounds__(1024)
+tile_list_kernel(const int32_t* __restrict__ counts, const int32_t* __restrict__ group_keys,
+                 const int32_t* __restrict__ wave_start, Tile* __restrict__ tiles, int32_t* __restrict__ n_tiles) {
+    __shared__ int s_warp[32];
+    __shared__ int s_running;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int g0 = wave_start[0], ng = wave_start[1] - g0;
+    if (tid == 0) s_running = 0;
+    __syncthreads();
+    for (int base = 0; base < ng; base += 1024) {
+        const int g = base + tid;
+        int key = 0, cnt = 0, pieces = 0, per = 0;
+        if (g < ng) {
+            key = group_keys[g0 + g];
+            cnt = counts[key];
+            pieces = (cnt + BN - 1) / BN;
+            per = ((cnt + pieces - 1) / pieces + 15) & ~15;
+            pieces = (cnt + per - 1) / per;
+        }
+        int incl = pieces;
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) {
+            const int o = __shfl_up_sync(0xffffffffu, incl, d);
+            if (lane >= d) incl += o;
+        }
+        if (lane == 31) s_warp[warp] = incl;
+        __syncthreads();
+        int wbase = 0, total = 0;
+        for (int w = 0; w < 32; ++w) {
+            if (w < warp) wbase += s_warp[w];
+            total += s_warp[w];
+        }
+        int pos = s_running + wbase + incl - pieces;
+        for (int n0 = 0; n0 < cnt; n0 += per) tiles[pos++] = Tile{key, n0, min(per, cnt - n0), 0};
+        __syncthreads();
+        if (tid == 0) s_running += total;
+        __syncthreads();
     }
-    *n_tiles = n;
+    if (tid == 0) *n_tiles = s_running;
 }
 
 }  // namespace
@@ -547,16 +573,15 @@ void launch_prefill_wave(const GemmArgs& g, const int32_t* wave_start, void* scr
     cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
     const CUtensorMap* mx = reinterpret_cast<const CUtensorMap*>(maps->x);
     const CUtensorMap* ma = reinterpret_cast<const CUtensorMap*>(maps->act);
+    if (which & 4) {
+        tile_list_kernel<<<1, 1024, 0, st>>>(g.counts, g.group_keys, wave_start, tiles, n_tiles);
+        count_launch();
+    }
     if (which & 1) {
-        tile_list_kernel<<<1, 32, 0, st>>>(g.counts, g.group_keys, wave_start, tiles, n_tiles);
         prefill_gemm_kernel<true><<<sms, NUM_THREADS, smem, st>>>(a, *mx, act, nullptr, g.offsets, nullptr);
-        count_launch(2);
+        count_launch();
     }
     if (which & 2) {
-        if (!(which & 1)) {
-            tile_list_kernel<<<1, 32, 0, st>>>(g.counts, g.group_keys, wave_start, tiles, n_tiles);
-            count_launch();
-        }
         prefill_gemm_kernel<false><<<sms, NUM_THREADS, smem, st>>>(a, *ma, nullptr, topk_w, g.offsets, y);
         count_launch();
     }
