@@ -19,7 +19,7 @@
 //                 completion is counted in bytes on the stage's full barrier.  No multicast.
 //   warps 8-15,   A producers, one 16-row panel and one 64-wide k-half each: stream packed int4 (128-bit
 //   20-27         loads, two blocks ahead in registers), dequantise to BF16 (shift/lop3 -> 128+u, subtract 136,
-//                 multiply by the group scale) and store the canonical no-swizzle K-major
+//                 multiply by the exactly split group scale: one rounding) and store the canonical no-swizzle K-major
 //                 core-matrix layout (k-chunk stride padded to 160 bytes: conflict-free stores).
 // Producers -> MMA through full[stage] mbarriers (generic-proxy writes are fenced with
 // fence.proxy.async before the arrive), MMA -> producers through tcgen05.commit on empty[stage].
@@ -175,8 +175,17 @@ __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commi
 template <int N>
 __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
 
-// eight codes of one word -> eight BF16 weights (q * s), K order, as one 16-byte value
-__device__ __forceinline__ uint4 dequant_word(uint32_t w, __nv_bfloat162 scale2) {
+// The FP16 group scale s is split exactly into two BF16 numbers, s = hi + lo (hi = bf16(s), lo = s - hi has at most
+// four significant bits).  For a code q in [-8, 7]: q*lo is exact in BF16 and fma(q, hi, q*lo) rounds the exact
+// product q*s once, so the staged weight is the correctly rounded BF16 of the dequantised value s*q.
+struct ScaleSplit { __nv_bfloat162 hi, lo; };
+__device__ __forceinline__ ScaleSplit split_scale(float s) {
+    const __nv_bfloat16 hi = __float2bfloat16_rn(s);
+    const __nv_bfloat16 lo = __float2bfloat16_rn(s - __bfloat162float(hi));
+    return ScaleSplit{__nv_bfloat162(hi, hi), __nv_bfloat162(lo, lo)};
+}
+// eight codes of one word -> eight BF16 weights bf16(q * s), K order, as one 16-byte value
+__device__ __forceinline__ uint4 dequant_word(uint32_t w, const ScaleSplit& sc) {
     uint32_t bias = 0x43084308u;                                   // BF16 136 twice
     const __nv_bfloat162 b2 = *reinterpret_cast<__nv_bfloat162*>(&bias);
     uint32_t out[4];
@@ -184,9 +193,9 @@ __device__ __forceinline__ uint4 dequant_word(uint32_t w, __nv_bfloat162 scale2)
     for (int s = 0; s < 4; ++s) {
         uint32_t v;
         asm("lop3.b32 %0, %1, 0x000f000f, 0x43004300, 0xea;" : "=r"(v) : "r"(w >> (4 * s)));   // (128+u, 128+u')
-        __nv_bfloat162 q2 = __hsub2(*reinterpret_cast<__nv_bfloat162*>(&v), b2);               // exact small integers
-        q2 = __hmul2(q2, scale2);                                                               // one rounding to BF16
-        out[s] = *reinterpret_cast<uint32_t*>(&q2);
+        const __nv_bfloat162 q2 = __hsub2(*reinterpret_cast<__nv_bfloat162*>(&v), b2);         // exact small integers
+        const __nv_bfloat162 r2 = __hfma2(q2, sc.hi, __hmul2(q2, sc.lo));                       // one rounding of q*s
+        out[s] = *reinterpret_cast<const uint32_t*>(&r2);
     }
     return make_uint4(out[0], out[1], out[2], out[3]);
 }
@@ -421,8 +430,8 @@ prefill_gemm_kernel(PrefillArgs a, const __grid_constant__ CUtensorMap tmap_b, _
                     if (!ok) break;
                     unsigned char* dst = sA + s * A_STAGE_BYTES;
                     const __half2 sh = *reinterpret_cast<const __half2*>(&sc[u]);
-                    const __nv_bfloat162 s_lo = __float2bfloat162_rn(__low2float(sh));    // row q
-                    const __nv_bfloat162 s_hi = __float2bfloat162_rn(__high2float(sh));   // row q + 8
+                    const ScaleSplit s_lo = split_scale(__low2float(sh));                 // row q
+                    const ScaleSplit s_hi = split_scale(__high2float(sh));                // row q + 8
                     const uint32_t words[4] = {w[u].x, w[u].y, w[u].z, w[u].w};
 #pragma unroll
                     for (int wi = 0; wi < 4; ++wi) {
