@@ -21,6 +21,14 @@
 //     to finish a (token, column tile) sums the k pair rows in order j = 0..k-1 (no spin wait).
 //   otherwise: the grouping kernels' global plan is used and a separate combine kernel follows.
 #include "common.cuh"
+#ifdef EXMOE_DECODE_PROF
+#include <cstdio>
+#define DPROF_T(i) long long dprof_##i = clock64()
+#define DPROF_PRINT(name, ...) if ((blockIdx.x == 5 || blockIdx.x == 100) && threadIdx.x == 64) printf(name " blk %d: " __VA_ARGS__)
+#else
+#define DPROF_T(i)
+#define DPROF_PRINT(name, ...)
+#endif
 
 namespace exmoe {
 
@@ -36,6 +44,17 @@ __device__ __forceinline__ uint4 ldg_stream128(const void* p) {
 __device__ __forceinline__ uint32_t ldg_stream32(const void* p) {
     uint32_t v;
     asm volatile("ld.global.nc.L1::no_allocate.u32 %0, [%1];" : "=r"(v) : "l"(p));
+    return v;
+}
+// loads that must be ISSUED where they are written (volatile asm: the compiler may not sink them to their use)
+__device__ __forceinline__ uint4 ldg_early128(const void* p) {
+    uint4 v;
+    asm volatile("ld.global.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+    return v;
+}
+__device__ __forceinline__ float ldg_early_f32(const void* p) {
+    float v;
+    asm volatile("ld.global.f32 %0, [%1];" : "=f"(v) : "l"(p));
     return v;
 }
 __device__ __forceinline__ void mma_m16n8k16(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
@@ -483,7 +502,7 @@ token_down_kernel(GemmArgs a, SmallArgs sa, const __nv_bfloat16* __restrict__ ac
         int id = -1;
         if (j < k) id = sa.ids[pair];
         const bool valid = (j < k) && id >= 0 && id < sa.E;
-        const float rw = valid ? topk_w[pair] : 0.f;   // requested early: it is needed only in the epilogue
+        const float rw = valid ? ldg_early_f32(topk_w + pair) : 0.f;   // requested early: needed only in the epilogue
         float result[2] = {0.f, 0.f};
         float total[2] = {0.f, 0.f};
         for (int b0 = 0; b0 < KB; b0 += NBT) {
@@ -576,6 +595,7 @@ __global__ void __launch_bounds__(256, 2)
 pair_gateup_kernel(GemmArgs a, SmallArgs sa, const __nv_bfloat16* __restrict__ hidden,
                    __nv_bfloat16* __restrict__ act_out, int KS) {
     extern __shared__ __align__(16) unsigned char smem[];
+    DPROF_T(0);
     grid_launch_dependents();
     const int K = a.H, KB = K / kGroup, PP = 8 / KS;
     const int tiles = a.I / (kPanelRows * PP);
@@ -590,7 +610,7 @@ pair_gateup_kernel(GemmArgs a, SmallArgs sa, const __nv_bfloat16* __restrict__ h
     // The hidden row does not depend on the ids: request it first so that it is not queued behind the weights.
     const __nv_bfloat16* xrow = hidden + (size_t)(p / a.top_k) * K;
     uint4 xpre = make_uint4(0, 0, 0, 0);
-    if (tid < K / 8) xpre = *reinterpret_cast<const uint4*>(xrow + tid * 8);
+    if (tid < K / 8) xpre = ldg_early128(xrow + tid * 8);
     const int id = sa.ids[p];
     if (blockIdx.x == 0 && tid < sa.n_pairs) {         // keep the ids so the plan can be materialised on request
         const int v = sa.ids[tid];
@@ -612,6 +632,7 @@ pair_gateup_kernel(GemmArgs a, SmallArgs sa, const __nv_bfloat16* __restrict__ h
             wreg[m][b][1] = ldg_stream128(blk + 512 + lane * 16);
             sreg[m][b] = ldg_stream32(blk + kCodeBytes + q * 4);
         }
+    DPROF_T(1);
     // stage the token's hidden row; adj[kb] = -136 * (sum of the row over block kb)
     const int total = K / 8;
     for (int base = warp * 32; base < total; base += 256) {
@@ -627,6 +648,11 @@ pair_gateup_kernel(GemmArgs a, SmallArgs sa, const __nv_bfloat16* __restrict__ h
         if (ck < total && (ck & 15) == 0) adj[ck >> 4] = -136.f * sx;
     }
     __syncthreads();
+    DPROF_T(2);
+#ifdef EXMOE_DECODE_PROF
+    long long dprof_first = 0;
+    { volatile uint32_t touch = wreg[0][0][0].x; (void)touch; dprof_first = clock64(); }
+#endif
 
     float tot[2][4];
 #pragma unroll
@@ -664,6 +690,7 @@ pair_gateup_kernel(GemmArgs a, SmallArgs sa, const __nv_bfloat16* __restrict__ h
             tot[m][2] = fmaf(s_hi, acc[m][2] + cr, tot[m][2]);
         }
     }
+    DPROF_T(3);
     if (ks > 0 && c == 0) {
         red[(((ks - 1) * PP + pp) * 2 + 0) * 16 + q] = tot[0][0];
         red[(((ks - 1) * PP + pp) * 2 + 0) * 16 + q + 8] = tot[0][2];
@@ -684,6 +711,10 @@ pair_gateup_kernel(GemmArgs a, SmallArgs sa, const __nv_bfloat16* __restrict__ h
             act_out[(size_t)p * a.I + panel * kPanelRows + q + 4 * i] = __float2bfloat16_rn(g / (1.f + __expf(-g)) * u);
         }
     }
+#ifdef EXMOE_DECODE_PROF
+    DPROF_PRINT("gateup", "ids+issue %lld stage %lld firstdata %lld compute %lld end %lld (tot %f)\n", blockIdx.x, dprof_1 - dprof_0,
+                dprof_2 - dprof_1, dprof_first - dprof_2, dprof_3 - dprof_first, clock64() - dprof_3, tot[0][0]);
+#endif
 }
 
 template <int NB>
@@ -699,6 +730,108 @@ void launch_pair_gateup(const GemmArgs& a, const SmallArgs& sa, const __nv_bfloa
     }
     kern<<<sa.n_pairs * tiles, 256, smem, st>>>(a, sa, hidden, act, KS);
     count_launch();
+}
+
+// Lean variant of token_down_kernel for k * (K-split ranges) <= 32 warps: warp = (expert j, K range r), NBW blocks in
+// registers, no loops around the arithmetic.  Partial sums are added per expert in range order, multiplied by the
+// routing weight and added over the experts in order, i.e. exactly the grouped kernel's order.
+template <int NBW>
+__global__ void __launch_bounds__(1024, 1)
+token_down_split_kernel(GemmArgs a, SmallArgs sa, const __nv_bfloat16* __restrict__ act,
+                        const float* __restrict__ topk_w, int ranges) {
+    extern __shared__ __align__(16) unsigned char smem[];
+    const int K = a.I, KB = K / kGroup, k = a.top_k;
+    const int x_stride = K * 2 + 64;
+    unsigned char* xs = smem;                                              // [k][x_stride]
+    float* part = reinterpret_cast<float*>(smem + (size_t)k * x_stride);  // [k][ranges][16]
+    float* adj = part + k * ranges * 16;                                   // [KB][k]
+    int* s_valid = reinterpret_cast<int*>(adj + KB * k);                   // [k]
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int q = lane >> 2, c = lane & 3;
+    const int panels = a.H / kPanelRows;
+    const int t = blockIdx.x / panels, panel = blockIdx.x % panels;
+    const int j = warp / ranges, r = warp % ranges;
+    const int pair = t * k + j;
+    const int id = sa.ids[pair];
+    const bool valid = id >= 0 && id < sa.E;
+    float rw = 0.f;
+    uint4 wreg[NBW][2];
+    uint32_t sreg[NBW];
+    if (valid) {
+        const int slot = sa.slot_of ? sa.slot_of[id] : id;
+        const uint8_t* mat = a.slots + (size_t)slot * a.slot_stride + matrix_bytes(2 * a.I, a.H) +
+                             ((size_t)panel * KB + r * NBW) * kBlockBytes;
+#pragma unroll
+        for (int b = 0; b < NBW; ++b) {
+            const uint8_t* blk = mat + (size_t)b * kBlockBytes;
+            wreg[b][0] = ldg_stream128(blk + lane * 16);
+            wreg[b][1] = ldg_stream128(blk + 512 + lane * 16);
+            sreg[b] = ldg_stream32(blk + kCodeBytes + q * 4);
+        }
+        if (r == 0) rw = topk_w[pair];
+    }
+    grid_dependency_wait();                                                // activations of the gate/up kernel
+    {
+        const int chunks_per_row = K / 8, total = k * chunks_per_row;
+        const int nthreads = blockDim.x;
+        for (int base = warp * 32; base < total; base += nthreads) {
+            const int idx = base + lane;
+            const int n = idx / chunks_per_row, ck = idx % chunks_per_row;
+            uint4 v = make_uint4(0, 0, 0, 0);
+            if (idx < total) {
+                v = *reinterpret_cast<const uint4*>(act + (size_t)(t * k + n) * K + ck * 8);
+                *reinterpret_cast<uint4*>(xs + (size_t)n * x_stride + ck * 16) = v;
+            }
+            float sx = sum8_bf16(v);
+#pragma unroll
+            for (int m = 8; m >= 1; m >>= 1) sx += __shfl_xor_sync(0xffffffffu, sx, m);
+            if (idx < total && (ck & 15) == 0) adj[(ck >> 4) * k + n] = -136.f * sx;
+        }
+    }
+    __syncthreads();
+    float total0 = 0.f, total1 = 0.f;
+    if (valid) {
+#pragma unroll
+        for (int b = 0; b < NBW; ++b) {
+            float acc[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+            for (int h = 0; h < 2; ++h)
+#pragma unroll
+                for (int set = 0; set < 2; ++set) {
+                    const int k0 = (r * NBW + b) * kGroup + 64 * h + 32 * set + 8 * c;
+                    uint4 xb = make_uint4(0, 0, 0, 0);
+                    if (q == 0) xb = *reinterpret_cast<const uint4*>(xs + (size_t)j * x_stride + k0 * 2);
+                    const uint32_t wq = set ? wreg[b][h].z : wreg[b][h].x;
+                    const uint32_t wq8 = set ? wreg[b][h].w : wreg[b][h].y;
+                    mma_m16n8k16(acc, code_pair(wq, 0), code_pair(wq8, 0), code_pair(wq, 4), code_pair(wq8, 4), xb.x, xb.y);
+                    mma_m16n8k16(acc, code_pair(wq, 8), code_pair(wq8, 8), code_pair(wq, 12), code_pair(wq8, 12), xb.z, xb.w);
+                }
+            const __half2 sc = *reinterpret_cast<const __half2*>(&sreg[b]);
+            const float cr = adj[(r * NBW + b) * k + j];
+            total0 = fmaf(__low2float(sc), acc[0] + cr, total0);
+            total1 = fmaf(__high2float(sc), acc[2] + cr, total1);
+        }
+    }
+    if (c == 0) {
+        part[(j * ranges + r) * 16 + q] = total0;
+        part[(j * ranges + r) * 16 + q + 8] = total1;
+    }
+    __shared__ float s_rw[32];
+    if (r == 0 && lane == 0) {
+        s_valid[j] = valid ? 1 : 0;
+        s_rw[j] = rw;
+    }
+    __syncthreads();
+    if (tid < 16) {
+        float sum = 0.f;
+        for (int jj = 0; jj < k; ++jj) {
+            if (!s_valid[jj]) continue;
+            float res = part[(jj * ranges) * 16 + tid];
+            for (int rr = 1; rr < ranges; ++rr) res += part[(jj * ranges + rr) * 16 + tid];
+            sum += s_rw[jj] * res;
+        }
+        sa.out[(size_t)t * a.H + panel * kPanelRows + tid] = __float2bfloat16_rn(sum);
+    }
 }
 
 // K split over KS warps (KS in {1,2,4,8}, 8/KS panels per CTA) and register depth NB; aims at
@@ -847,6 +980,31 @@ void launch_token_down(const GemmArgs& a, const SmallArgs& sa, const __nv_bfloat
     count_launch();
 }
 
+template <int NBW>
+void launch_token_down_split(const GemmArgs& a, const SmallArgs& sa, const __nv_bfloat16* act, const float* w, int T,
+                             int ranges, cudaStream_t st) {
+    auto kern = token_down_split_kernel<NBW>;
+    const int k = a.top_k, KB = a.I / kGroup;
+    const size_t smem = (size_t)k * (a.I * 2 + 64) + (size_t)k * ranges * 16 * 4 + (size_t)(KB * k + 4) * 4 + (size_t)k * 4;
+    static bool attr_done = false;
+    if (!attr_done) {
+        cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+        attr_done = true;
+    }
+    cudaLaunchConfig_t lc{};
+    lc.gridDim = dim3(T * (a.H / kPanelRows));
+    lc.blockDim = dim3(32 * k * ranges);
+    lc.dynamicSmemBytes = smem;
+    lc.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    lc.attrs = attr;
+    lc.numAttrs = 1;
+    cudaLaunchKernelEx(&lc, kern, a, sa, act, w, ranges);
+    count_launch();
+}
+
 // One wave of the SMALL path: gate/up kernel, then the down kernel with the fused combine.
 void launch_small_wave(const GemmArgs& a, const SmallWave& w, cudaStream_t st, bool gateup, bool down) {
     SmallArgs sa{};
@@ -876,7 +1034,12 @@ void launch_small_wave(const GemmArgs& a, const SmallWave& w, cudaStream_t st, b
             const int KB = a.I / kGroup;
             const int bpwg = pick_cfg(a.I, a.H).bpw;    // the grouped kernel's K-split range, replayed for rounding
             const int T = w.n_pairs / a.top_k;
-            if (KB % 8 == 0) launch_token_down<8>(a, sa, w.act, w.topk_w, T, bpwg, st);
+            const int ranges = KB / bpwg;
+            if (false && a.top_k * ranges <= 32 && KB % bpwg == 0 && (bpwg == 4 || bpwg == 2 || bpwg == 1) && a.top_k <= 32) {
+                if (bpwg == 4) launch_token_down_split<4>(a, sa, w.act, w.topk_w, T, ranges, st);
+                else if (bpwg == 2) launch_token_down_split<2>(a, sa, w.act, w.topk_w, T, ranges, st);
+                else launch_token_down_split<1>(a, sa, w.act, w.topk_w, T, ranges, st);
+            } else if (KB % 8 == 0) launch_token_down<8>(a, sa, w.act, w.topk_w, T, bpwg, st);
             else if (KB % 4 == 0) launch_token_down<4>(a, sa, w.act, w.topk_w, T, bpwg, st);
             else if (KB % 2 == 0) launch_token_down<2>(a, sa, w.act, w.topk_w, T, bpwg, st);
             else launch_token_down<1>(a, sa, w.act, w.topk_w, T, bpwg, st);

@@ -78,3 +78,28 @@ def route(hidden, w_router, top_k, bias=None):
     order = torch.sort(-p, dim=-1, stable=True).indices[:, :top_k]     # ties -> lower id
     w = torch.gather(p, 1, order)
     return order.to(torch.int32).contiguous(), w.contiguous()
+
+
+class SyntheticStack:
+    """Stand-in for a 16-layer sparse model around the MoE layers (config 5): per layer a BF16 router
+    (Eq. 1 with an optional Zipf bias), and between layers the dense parts abstracted to
+    h <- bf16(h + moe_out + N(0, 0.1)).  Only input generation: the MoE layer itself is `layer_fn`."""
+
+    def __init__(self, shape: Shape, num_layers, seed, alpha=1.0, device="cpu"):
+        self.shape, self.L, self.device = shape, int(num_layers), device
+        self.routers = [router_weights(shape, seed + 17 * l, device=device) for l in range(self.L)]
+        self.bias = [zipf_bias(shape.num_experts, alpha, seed + 1000 + l).to(device) if alpha else None
+                     for l in range(self.L)]
+        self.gen = _gen(seed + 5, device)
+
+    def step(self, layer_fn, hidden, record=None):
+        """layer_fn(layer, hidden, ids, weights) -> moe output.  Returns the hidden state after all layers."""
+        h = hidden
+        for l in range(self.L):
+            ids, w = route(h, self.routers[l], self.shape.top_k, self.bias[l])
+            out = layer_fn(l, h, ids, w)
+            if record is not None:
+                record.append((l, h, ids, w, out))
+            noise = torch.randn(h.shape, generator=self.gen, device=h.device, dtype=torch.float32) * 0.1
+            h = (h.float() + out.float() + noise).to(torch.bfloat16)
+        return h

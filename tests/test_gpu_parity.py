@@ -288,6 +288,32 @@ def test_config4_prefill_olmoe_sampled(B, olmoe_layer, alpha):
     cache.close()
 
 
+def test_config5_stack_teacher_forced(B):
+    """Config 5 in small: a 4-layer stack with per-layer routers and the identity-plus-noise residual, slots < experts.
+    The stack runs free on the GPU; every layer is then checked on its own (the oracle gets the GPU's layer input
+    and routing), because near-ties in the router would let two free-running stacks pick different experts."""
+    s = synth.MID
+    L = 4
+    layers = [helpers.make_layer(s, seed=900 + l) for l in range(L)]
+    cache = B.Cache(s, [bank for _, bank in layers], 6, max_tokens=16)
+    models = [ocache.SlotCache(s.num_experts, 6, 0, bytes_per_expert=cache.bytes_per_expert) for _ in range(L)]
+    stack = synth.SyntheticStack(s, L, seed=31, alpha=1.0, device="cuda")
+    h = synth.hidden_states(s, 5, seed=3).cuda()
+    for step in range(3):
+        rec = []
+        h = stack.step(lambda l, x, ids, w: cache.forward(l, x, ids, w).clone(), h, record=rec)
+        for (l, x, ids, w, out) in rec:
+            y, ref = layers[l][0].forward(x.cpu(), ids.cpu(), w.cpu())
+            helpers.check_output(out, y, ref, f"step {step} layer {l}")
+            models[l].resolve(ids.cpu().numpy())
+    for l in range(L):
+        st = cache.stats(l)
+        assert (st["hits"], st["misses"], st["waves"]) == (models[l].stats.hits, models[l].stats.misses, models[l].stats.waves)
+        assert st["h2d_bytes"] == st["misses"] * cache.bytes_per_expert
+    assert cache.status() == 0
+    cache.close()
+
+
 # ------------------------------------------------------------------------------------ edge cases
 def test_edge_cases(B, tiny_layer):
     ora, bank = tiny_layer
