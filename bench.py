@@ -235,7 +235,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=50)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="decode", choices=sorted(WORKLOADS) + ["stack"])
-    ap.add_argument("--alpha", type=float, default=1.0, help="Zipf skew of the stack workload's routers")
+    ap.add_argument("--alpha", type=float, default=0.5, help="Zipf skew of the stack workload's routers")
+    ap.add_argument("--tokens", type=int, default=0, help="override the workload's tokens per step")
     ap.add_argument("--cpu-budget", type=float, default=15.0, help="seconds of CPU oracle work for cpu_baseline")
     ap.add_argument("--layers", type=int, default=0, help="layer banks to rotate over (0 = the workload's default)")
     args = ap.parse_args()
@@ -275,6 +276,8 @@ def main():
         return
     T, C, L, alpha, desc = WORKLOADS[args.workload]
     L = args.layers or L
+    if args.tokens:
+        T, desc = args.tokens, desc + " [tokens per step overridden: %d]" % args.tokens
     shape = synth.OLMOE
     K, W = args.steps, max(args.warmup, 3)
     peaks = load_peaks()

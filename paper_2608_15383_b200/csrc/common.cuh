@@ -77,7 +77,10 @@ struct SmallWave {
     int32_t* saved_ids;         // [kPairMaxPairs]
 };
 constexpr int kPairMaxPairs = 32;
-constexpr int kSmallMaxPairs = 512;
+#ifndef EXMOE_SMALL_MAX_PAIRS
+#define EXMOE_SMALL_MAX_PAIRS 40
+#endif
+constexpr int kSmallMaxPairs = EXMOE_SMALL_MAX_PAIRS;
 constexpr int kSmallMaxSlots = 1024;
 
 // launch accounting (exmoe_launch_count)

@@ -13,7 +13,7 @@
 // K-split partials are reduced through shared memory in a fixed order.
 //
 // Two flavours share the body:
-//   SMALL (T*k <= 512): a decode step is launch-latency bound, so the chain of dependent global
+//   SMALL (T*k <= kSmallMaxPairs = 40): a decode step is launch-latency bound, so the chain of dependent global
 //     loads is cut to two levels: every CTA rebuilds the wave's token grouping (histogram, prefix
 //     sum, stable permutation) in shared memory straight from topk_ids; CTA 0 also publishes it.
 //     The down kernel is launched with programmatic dependent launch: it prefetches its weights
@@ -168,7 +168,7 @@ __device__ __forceinline__ void build_small_plan(const SmallArgs& sa, int C, Sma
 enum { MODE_PLAN = 0, MODE_SMALL = 1, MODE_PAIR = 2 };
 
 // MODE_PLAN  : groups come from the grouping kernels' global plan
-// MODE_SMALL : every CTA rebuilds the wave's grouping in shared memory (T*k <= 512)
+// MODE_SMALL : every CTA rebuilds the wave's grouping in shared memory (T*k <= kSmallMaxPairs)
 // MODE_PAIR  : one item per token-expert pair, no grouping at all (T*k <= 32, gate/up only)
 #ifndef EXMOE_MINB_NB2
 #define EXMOE_MINB_NB2 1
