@@ -98,6 +98,21 @@ class ClockSampler:
         return out
 
 
+def max_over_ranks(x, world, device="cpu"):
+    """Slowest rank's value (device time of the timed region): the job is as fast as its slowest replica."""
+    if world <= 1:
+        return float(x)
+    import torch.distributed as dist
+    t = torch.tensor([float(x)], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_tokens_per_s(world, steps, tokens_per_step, ms_max):
+    """Replicas only (no collective on the data path): every rank runs the same workload on its own GPU."""
+    return world * steps * tokens_per_step / (ms_max * 1e-3)
+
+
 def make_inputs(shape, T, n_sets, alpha, seed0, device):
     """n_sets independent (hidden, ids, weights) batches, generated on the device, routed by Eq. 1."""
     wr = synth.router_weights(shape, seed0 + 1, device=device)
@@ -181,7 +196,8 @@ def run_reference(args, rank, world):
     line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": 1e3 * dt / max(args.steps, 1), "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-            "config": {"workload": desc, "note": "CPU oracle on a bounded sample: first min(T,8) tokens of each step"},
+            "config": {"workload": desc, "note": "CPU oracle on a bounded sample: first min(T,8) tokens of each step",
+                       "steps_requested": args.steps_requested},
             "cpu_baseline": {"value": value, "unit": UNIT, "cores": leg["cores"] if leg else 1, "kind": "oracle",
                              "sample": f"{args.steps} steps x {min(T, 8)} tokens"},
             "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
@@ -246,6 +262,7 @@ def main():
     world = int(os.environ.get("WORLD_SIZE", "1"))
 
     if args.impl == "reference":
+        args.steps_requested = args.steps
         if args.steps > 50:
             args.steps = 50
         args.warmup = min(args.warmup, 3)
@@ -344,10 +361,8 @@ def main():
     clocks = sampler.stop()
     if world > 1:
         dist.barrier()
-        t = torch.tensor([ms], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = float(t.item())
-    value = world * K * T / (ms * 1e-3)
+    ms = max_over_ranks(ms, world, dev)
+    value = whole_job_tokens_per_s(world, K, T, ms)
 
     # ---- per-kernel times (roofline of the dominant kernel): the same steps with ONLY one kernel kind
     # launched, timed with CUDA events on the launching stream (graph replay when fully resident)
@@ -424,10 +439,7 @@ def main():
     for i in range(n_e2e):
         e2e_step(i)
     dt = time.perf_counter() - t0
-    if world > 1:
-        t = torch.tensor([dt], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        dt = float(t.item())
+    dt = max_over_ranks(dt, world, dev)
     h2d = h_h[0].numel() * 2 + h_i[0].numel() * 4 + h_w[0].numel() * 4
     e2e = {"value": world * n_e2e * T / dt, "unit": UNIT, "h2d_bytes_per_step": int(h2d),
            "d2h_bytes_per_step": int(h_out.numel() * 2), "steps": n_e2e}
@@ -438,6 +450,34 @@ def main():
         st = cache.stats(0)
         extra = {"hit_rate": st["hits"] / max(st["lookups"], 1), "h2d_expert_bytes_per_token":
                  st["h2d_bytes"] / max(st["forwards"] * T, 1), "waves_per_step": st["waves"] / max(st["forwards"], 1)}
+        # the H2D link is the roofline of this workload: copy-stream busy time and rate vs a plain pinned copy
+        n_c = min(K, 100)
+        cache.profile_enable(True)
+        b0 = cache.stats(0)["h2d_bytes"]
+        c0, c1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        with torch.cuda.stream(stream):
+            c0.record(stream)
+            for i in range(W, W + n_c):
+                step(i, outs[i & 1])
+            c1.record(stream)
+        stream.synchronize()
+        copy_ms, n_waves_copied = cache.profile_read(4)
+        wall_ms = c0.elapsed_time(c1)
+        moved = cache.stats(0)["h2d_bytes"] - b0
+        cache.profile_enable(False)
+        big = banks[0][:32]                                  # 104 MB of the pinned bank
+        dst = torch.empty_like(big, device=dev)
+        p0, p1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        dst.copy_(big, non_blocking=True)
+        torch.cuda.synchronize()
+        p0.record()
+        dst.copy_(big, non_blocking=True)
+        p1.record()
+        torch.cuda.synchronize()
+        extra.update({"h2d_gb_per_s_during_copies": moved / max(copy_ms, 1e-9) / 1e6,
+                      "copy_stream_busy_fraction": copy_ms / wall_ms,
+                      "pinned_copy_ceiling_gb_per_s": big.numel() / p0.elapsed_time(p1) / 1e6,
+                      "h2d_bytes_per_step": moved / n_c})
 
     if rank == 0:
         cpu = oracle_leg(shape, T, w_cpu, hs, ids, ws, args.cpu_budget)

@@ -247,7 +247,7 @@ class Cache:
         _check(lib().exmoe_profile_enable(self.handle, int(bool(on)) | (int(only) << 4)), "exmoe_profile_enable")
 
     def profile_read(self, kind):
-        """(total event ms, bracketed launches) of kind 0 plan, 1 gate/up, 2 down, 3 combine."""
+        """(total event ms, bracketed launches) of kind 0 plan, 1 gate/up, 2 down, 3 combine, 4 miss copies."""
         ms, n = ctypes.c_double(), c_uint64()
         _check(lib().exmoe_profile_read(self.handle, int(kind), byref(ms), byref(n)), "exmoe_profile_read")
         return ms.value, int(n.value)

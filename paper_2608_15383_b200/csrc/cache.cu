@@ -77,29 +77,29 @@ struct exmoe_cache {
     int last_T;
     bool prof_on;                             // per-kernel CUDA-event timing (exmoe_profile_*)
     int prof_only;                            // 0 = all kernels; 1..3 = launch only that kind (timing runs)
-    std::vector<cudaEvent_t> prof_ev[4];      // begin/end pairs per kernel kind
-    size_t prof_used[4];
+    std::vector<cudaEvent_t> prof_ev[5];      // begin/end pairs per kernel kind (4 = miss copies, copy stream)
+    size_t prof_used[5];
 };
 
-enum { PROF_PLAN = 0, PROF_GATEUP = 1, PROF_DOWN = 2, PROF_COMBINE = 3 };
+enum { PROF_PLAN = 0, PROF_GATEUP = 1, PROF_DOWN = 2, PROF_COMBINE = 3, PROF_COPY = 4 };
 
 // Brackets one launch (or launch group) with a pair of events on its own stream when profiling is on.
+static void prof_mark(exmoe_cache* c, int kind, cudaStream_t st) {
+    if (!c->prof_on) return;
+    std::vector<cudaEvent_t>& v = c->prof_ev[kind];
+    if (c->prof_used[kind] == v.size()) {
+        cudaEvent_t e;
+        if (cudaEventCreate(&e) != cudaSuccess) return;
+        v.push_back(e);
+    }
+    cudaEventRecord(v[c->prof_used[kind]++], st);
+}
 struct ProfScope {
     exmoe_cache* c;
     int kind;
     cudaStream_t st;
-    ProfScope(exmoe_cache* c_, int kind_, cudaStream_t st_) : c(c_), kind(kind_), st(st_) { mark(); }
-    ~ProfScope() { mark(); }
-    void mark() {
-        if (!c->prof_on) return;
-        std::vector<cudaEvent_t>& v = c->prof_ev[kind];
-        if (c->prof_used[kind] == v.size()) {
-            cudaEvent_t e;
-            if (cudaEventCreate(&e) != cudaSuccess) return;
-            v.push_back(e);
-        }
-        cudaEventRecord(v[c->prof_used[kind]++], st);
-    }
+    ProfScope(exmoe_cache* c_, int kind_, cudaStream_t st_) : c(c_), kind(kind_), st(st_) { prof_mark(c, kind, st); }
+    ~ProfScope() { prof_mark(c, kind, st); }
 };
 
 static void carve_workspace(exmoe_cache* c, uint8_t* ws, size_t* total) {
@@ -354,6 +354,8 @@ int exmoe_moe_forward(exmoe_cache* c, int layer, const void* hidden, const int32
         int groups = identity ? (E < P ? E : P) : 0;
         if (!identity) {
             bool copied = false;
+            const bool wave_has_miss = mi < n_miss && h_miss[3 * mi + 2] == w;
+            if (wave_has_miss) prof_mark(c, PROF_COPY, c->copy_stream);       // begin of the wave's copies
             for (; mi < n_miss && h_miss[3 * mi + 2] == w; ++mi) {
                 const int e = h_miss[3 * mi], v = h_miss[3 * mi + 1];
                 const uint64_t last = c->slot_last_seq[layer][v];
@@ -363,6 +365,7 @@ int exmoe_moe_forward(exmoe_cache* c, int layer, const void* hidden, const int32
                     return EXMOE_ERR_CUDA;
                 copied = true;
             }
+            if (copied) prof_mark(c, PROF_COPY, c->copy_stream);              // end of the wave's copies
             if (copied) {
                 cudaEvent_t ev = c->ev_copy[(++c->copy_seq) % kEventRing];
                 cudaEventRecord(ev, c->copy_stream);
@@ -521,12 +524,12 @@ int exmoe_profile_enable(exmoe_cache* c, int on) {
     if (cudaDeviceSynchronize() != cudaSuccess) return EXMOE_ERR_CUDA;
     c->prof_on = (on & 1) != 0;
     c->prof_only = (on >> 4) & 3;
-    for (int k = 0; k < 4; ++k) c->prof_used[k] = 0;
+    for (int k = 0; k < 5; ++k) c->prof_used[k] = 0;
     return EXMOE_OK;
 }
 
 int exmoe_profile_read(exmoe_cache* c, int kind, double* total_ms, uint64_t* launches) {
-    if (!c || kind < 0 || kind > 3 || !total_ms || !launches) return EXMOE_ERR_ARG;
+    if (!c || kind < 0 || kind > 4 || !total_ms || !launches) return EXMOE_ERR_ARG;
     if (cudaDeviceSynchronize() != cudaSuccess) return EXMOE_ERR_CUDA;
     double sum = 0.0;
     const size_t n = c->prof_used[kind] / 2;
@@ -544,7 +547,7 @@ int exmoe_profile_read(exmoe_cache* c, int kind, double* total_ms, uint64_t* lau
 int exmoe_cache_destroy(exmoe_cache* c) {
     if (!c) return EXMOE_ERR_ARG;
     cudaDeviceSynchronize();
-    for (int k = 0; k < 4; ++k)
+    for (int k = 0; k < 5; ++k)
         for (cudaEvent_t e : c->prof_ev[k]) cudaEventDestroy(e);
     if (c->h_plan) cudaFreeHost(c->h_plan);
     if (c->copy_stream) cudaStreamDestroy(c->copy_stream);
