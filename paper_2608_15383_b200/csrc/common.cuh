@@ -97,6 +97,12 @@ void launch_decode_gateup(const GemmArgs& a, const __nv_bfloat16* hidden, __nv_b
                           int max_groups, cudaStream_t st);
 void launch_decode_down(const GemmArgs& a, const __nv_bfloat16* act, const float* topk_w, float* y, int max_rows,
                         int max_groups, cudaStream_t st);
+bool launch_lean_wave(const GemmArgs& a, const __nv_bfloat16* hidden, __nv_bfloat16* act, const float* topk_w, float* y,
+                      int max_rows, int max_groups, bool gateup, bool down, cudaStream_t st);
+#ifndef EXMOE_LEAN_MAX_PAIRS
+#define EXMOE_LEAN_MAX_PAIRS 192
+#endif
+constexpr int kLeanMaxPairs = EXMOE_LEAN_MAX_PAIRS;   // above: tensor-core path
 void launch_small_wave(const GemmArgs& a, const SmallWave& w, cudaStream_t st, bool gateup, bool down);
 size_t prefill_scratch_bytes(int max_pairs, int num_experts);
 struct alignas(64) PrefillMaps { unsigned char x[128], act[128]; };   // two CUtensorMap objects (grouped hidden, activations)
