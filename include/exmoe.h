@@ -160,6 +160,14 @@ int exmoe_debug_last_plan(exmoe_cache* cache, int layer, int32_t* n_active, int3
 /* Copy one slot's bytes back to the host (test hook for the miss-copy path; synchronises). */
 int exmoe_debug_read_slot(exmoe_cache* cache, int layer, int slot, void* host_out);
 
+/* Failure-detection self-test (no paper counterpart).  Every device-side wait in this library is bounded: when
+ * its budget of clock ticks runs out the waiting code raises the sticky status EXMOE_ERR_TIMEOUT, the CTA's
+ * roles leave their loops, tensor memory is released and the kernel returns, so the context stays usable.
+ * This hook runs a one-warp kernel that waits, with a budget of `budget_cycles` SM clock ticks (1..4e9), on a
+ * barrier that nothing completes.  *gave_up gets bit 0 = the wait returned "expired", bit 1 = the abort flag was
+ * raised; exmoe_status() then reports EXMOE_ERR_TIMEOUT.  Synchronous. */
+int exmoe_debug_wait_timeout(exmoe_cache* cache, long long budget_cycles, int* gave_up);
+
 int exmoe_cache_stats(exmoe_cache* cache, int layer, exmoe_stats* out);   /* synchronises */
 int exmoe_cache_reset(exmoe_cache* cache, int layer);                     /* empty cache, zero counters */
 int exmoe_status(exmoe_cache* cache);   /* synchronises; returns and clears the sticky device status */

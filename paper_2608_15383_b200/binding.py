@@ -51,6 +51,7 @@ _SIGNATURES = {
     "exmoe_cache_get_state": (c_int, [c_void_p, c_int, c_void_p, c_void_p, c_void_p, c_void_p]),
     "exmoe_debug_last_plan": (c_int, [c_void_p, c_int] + [c_void_p] * 9),
     "exmoe_debug_read_slot": (c_int, [c_void_p, c_int, c_int, c_void_p]),
+    "exmoe_debug_wait_timeout": (c_int, [c_void_p, ctypes.c_longlong, POINTER(c_int)]),
     "exmoe_cache_stats": (c_int, [c_void_p, c_int, POINTER(exmoe_stats)]),
     "exmoe_cache_reset": (c_int, [c_void_p, c_int]),
     "exmoe_status": (c_int, [c_void_p]),
@@ -230,6 +231,12 @@ class Cache:
         out = torch.empty(self.bytes_per_expert, dtype=torch.uint8)
         _check(lib().exmoe_debug_read_slot(self.handle, layer, slot, out.data_ptr()), "exmoe_debug_read_slot")
         return out.numpy()
+
+    def wait_timeout_selftest(self, budget_cycles=2_000_000):
+        """Run the bounded-wait self-test kernel; returns the flag word (3 = gave up and raised the abort flag)."""
+        v = c_int()
+        _check(lib().exmoe_debug_wait_timeout(self.handle, int(budget_cycles), byref(v)), "exmoe_debug_wait_timeout")
+        return v.value
 
     def stats(self, layer):
         s = exmoe_stats()

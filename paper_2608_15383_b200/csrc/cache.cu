@@ -560,6 +560,15 @@ int exmoe_profile_read(exmoe_cache* c, int kind, double* total_ms, uint64_t* lau
     return EXMOE_OK;
 }
 
+int exmoe_debug_wait_timeout(exmoe_cache* c, long long budget_cycles, int* gave_up) {
+    if (!c || !gave_up || budget_cycles <= 0 || budget_cycles > 4000000000ll) return EXMOE_ERR_ARG;
+    if (cudaDeviceSynchronize() != cudaSuccess) return EXMOE_ERR_CUDA;
+    int* d_result = c->d_status + 8;                       // spare word of the status block
+    launch_wait_selftest(c->d_status, budget_cycles, d_result, nullptr);
+    if (cudaDeviceSynchronize() != cudaSuccess) return EXMOE_ERR_CUDA;
+    return cudaMemcpy(gave_up, d_result, 4, cudaMemcpyDeviceToHost) == cudaSuccess ? EXMOE_OK : EXMOE_ERR_CUDA;
+}
+
 int exmoe_cache_destroy(exmoe_cache* c) {
     if (!c) return EXMOE_ERR_ARG;
     cudaDeviceSynchronize();

@@ -107,6 +107,7 @@ void launch_small_wave(const GemmArgs& a, const SmallWave& w, cudaStream_t st, b
 size_t prefill_scratch_bytes(int max_pairs, int num_experts);
 struct alignas(64) PrefillMaps { unsigned char x[128], act[128]; };   // two CUtensorMap objects (grouped hidden, activations)
 int prefill_setup(PrefillMaps* maps, const __nv_bfloat16* xg, const __nv_bfloat16* act, int max_pairs, int H, int I);
+void launch_wait_selftest(int* status, long long budget_cycles, int* result, cudaStream_t st);
 void launch_gather_rows(const __nv_bfloat16* hidden, const int32_t* perm, const int32_t* n_valid, int n_pairs, int top_k,
                         int H, __nv_bfloat16* xg, cudaStream_t st);
 // which: bit 0 = gate/up GEMM + SwiGLU, bit 1 = down GEMM x routing weight, bit 2 = (re)build the wave's tile list

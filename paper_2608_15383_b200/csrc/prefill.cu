@@ -86,12 +86,13 @@ __device__ __forceinline__ bool mbar_try(uint64_t* bar, uint32_t parity) {
 #endif
 
 // bounded wait; returns false when the CTA is aborting (and raises the abort on expiry)
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag, int* status) {
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag, int* status,
+                                          long long budget = kWaitBudget) {
     if (mbar_try(bar, parity)) return true;
     const long long t0 = clock64();
     while (!mbar_try(bar, parity)) {
         if (*abort_flag) return false;
-        if (clock64() - t0 > kWaitBudget) {
+        if (clock64() - t0 > budget) {
             *abort_flag = 1;
             atomicExch(status, EXMOE_ERR_TIMEOUT);
             return false;
@@ -458,6 +459,22 @@ prefill_gemm_kernel(PrefillArgs a, const __grid_constant__ CUtensorMap tmap_b, _
     if (warp == 0) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512));
 }
 
+// Self-test of the bounded wait: one warp waits on an mbarrier that nothing will ever complete, with a short
+// budget; the wait must give up, raise the abort flag and the status word, and the kernel must return normally.
+__global__ void wait_timeout_selftest_kernel(int* status, long long budget, int* result) {
+    __shared__ uint64_t bar;
+    __shared__ int abort_word;
+    if (threadIdx.x == 0) {
+        mbar_init(&bar, 1);
+        abort_word = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+    const bool ok = mbar_wait(&bar, 0, &abort_word, status, budget);     // phase 0 never completes
+    __syncthreads();
+    if (threadIdx.x == 0) *result = (ok ? 0 : 1) | (abort_word ? 2 : 0);
+}
+
 // grouped copy of the hidden states: row r of the plan order = hidden row of token perm[r] / k
 __global__ void __launch_bounds__(256)
 gather_rows_kernel(const __nv_bfloat16* __restrict__ hidden, const int32_t* __restrict__ perm,
@@ -546,6 +563,11 @@ int prefill_setup(PrefillMaps* maps, const __nv_bfloat16* xg, const __nv_bfloat1
     int rc = encode_map(reinterpret_cast<CUtensorMap*>(maps->x), xg, max_pairs, H);
     if (rc) return rc;
     return encode_map(reinterpret_cast<CUtensorMap*>(maps->act), act, max_pairs, I);
+}
+
+void launch_wait_selftest(int* status, long long budget_cycles, int* result, cudaStream_t st) {
+    wait_timeout_selftest_kernel<<<1, 32, 0, st>>>(status, budget_cycles, result);
+    count_launch();
 }
 
 void launch_gather_rows(const __nv_bfloat16* hidden, const int32_t* perm, const int32_t* n_valid, int n_pairs, int top_k,

@@ -349,6 +349,49 @@ def test_edge_cases(B, tiny_layer):
     cache.close()
 
 
+def test_bounded_wait_expires_and_reports(B, tiny_layer):
+    """Failure detection without a fault: a wait that can never succeed runs out of its (short) budget, the kernel
+    returns, the sticky status says EXMOE_ERR_TIMEOUT and the context keeps working."""
+    ora, bank = tiny_layer
+    s = synth.TINY
+    cache = B.Cache(s, [bank], 8, max_tokens=16)
+    assert cache.status() == 0
+    assert cache.wait_timeout_selftest(budget_cycles=2_000_000) == 3          # ~1 ms at 1.9 GHz
+    assert cache.status() == B.EXMOE_ERR_TIMEOUT
+    assert cache.status() == 0
+    hidden, ids, p = helpers.routed_inputs(s, 4, seed=12)
+    y, ref = ora.forward(hidden, ids, p)
+    helpers.check_output(cache.forward(0, hidden.cuda(), ids.cuda(), p.cuda()), y, ref, "after timeout")
+    cache.close()
+
+
+def test_graph_replay_matches_oracle(B, olmoe_layer):
+    """The launch configuration bench.py times: fully resident decode steps captured in a CUDA graph and replayed."""
+    ora, bank = olmoe_layer
+    s = synth.OLMOE
+    cache = B.Cache(s, [bank], 64, max_tokens=4)
+    inputs = [tuple(x.cuda() for x in helpers.routed_inputs(s, 1, seed=8100 + i)) for i in range(6)]
+    outs = [torch.empty_like(inputs[0][0]) for _ in inputs]
+    stream = torch.cuda.Stream()
+    with torch.cuda.stream(stream):
+        cache.forward(0, *inputs[0], out=outs[0], stream=stream)            # first call outside capture
+    stream.synchronize()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g, stream=stream):
+        for (h, i, w), o in zip(inputs, outs):
+            cache.forward(0, h, i, w, out=o, stream=stream)
+    for o in outs:
+        o.zero_()
+    with torch.cuda.stream(stream):
+        g.replay()
+    stream.synchronize()
+    for idx in (0, 3, 5):
+        h, i, w = inputs[idx]
+        y, ref = ora.forward(h.cpu(), i.cpu(), w.cpu())
+        helpers.check_output(outs[idx], y, ref, f"graph step {idx}")
+    cache.close()
+
+
 def test_create_rejects_bad_arguments(B, tiny_layer):
     ora, bank = tiny_layer
     s = synth.TINY
