@@ -127,6 +127,17 @@ static void carve_workspace(exmoe_cache* c, uint8_t* ws, size_t* total) {
     c->plan.group_keys = k.take<int32_t>(c->n_keys);
     c->plan.wave_start = k.take<int32_t>(c->max_waves + 1);
     c->plan.perm = k.take<int32_t>(c->max_pairs);
+    {
+        const size_t chunks = ((size_t)c->max_pairs + 511) / 512;
+        const size_t need = (size_t)c->n_keys * chunks, cap = (size_t)1 << 20;
+        // reserve min(need, cap): monotone in the key space, so the size query (largest key space) bounds every create
+        const size_t reserve = c->max_pairs <= 1024 ? 0 : (need < cap ? need : cap);
+        int32_t* tab = reserve ? k.take<int32_t>(reserve) : nullptr;
+        const bool usable = reserve && need <= cap;                       // larger key spaces keep the per-key scheme
+        c->plan.chunk_table = usable ? tab : nullptr;
+        c->plan.chunk_table_words = usable ? need : 0;
+        c->plan.chunk_done = k.take<int32_t>(64);
+    }
     c->act = k.take<__nv_bfloat16>((size_t)c->max_pairs * s.d_ff);
     c->y = k.take<float>((size_t)c->max_pairs * s.d_model);
     c->arrive_words = (size_t)(kSmallMaxPairs / s.top_k + 1) * (s.d_model / kPanelRows);
@@ -277,6 +288,7 @@ int exmoe_cache_create(exmoe_cache** out, const exmoe_shape* shape, int num_laye
     ok = ok && cudaMemset(c->d_status, 0, 256) == cudaSuccess;
     ok = ok && cudaMemset(c->plan.header, 0, c->plan_d2h_bytes) == cudaSuccess;
     ok = ok && cudaMemset(c->arrive, 0, c->arrive_words * 4) == cudaSuccess;
+    ok = ok && cudaMemset(c->plan.chunk_done, 0, 256) == cudaSuccess;
     for (int l = 0; l < num_layers && ok; ++l) ok = reset_layer(c, l) == EXMOE_OK;
     if (ok && c->xg) ok = prefill_setup(&c->tc_maps, c->xg, c->act, c->max_pairs, c->shape.d_model, c->shape.d_ff) == EXMOE_OK;
     if (ok && c->C == c->shape.num_experts) {            // full residency: preload, slot = expert id

@@ -35,6 +35,9 @@ struct PlanPtrs {
     int32_t* group_keys;    // [n_keys] active keys, ascending
     int32_t* wave_start;    // [max_waves + 1] index into group_keys
     int32_t* perm;          // [max_pairs]
+    int32_t* chunk_table;   // [n_keys][chunks] scratch of the chunked grouping (may be null)
+    size_t chunk_table_words;
+    int32_t* chunk_done;    // arrival counter of the chunked grouping (zero between calls)
 };
 
 struct LayerState {         // Section 3.3 state of one layer, device memory

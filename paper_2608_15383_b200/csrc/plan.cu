@@ -306,6 +306,102 @@ group_scatter_kernel(const int32_t* __restrict__ ids, int n_pairs, int E, int C,
     }
 }
 
+
+// Large problems, second scheme (used when the scratch fits): the pairs are cut into chunks of 512.
+//   kernel 1: one CTA per chunk histograms its pairs in shared memory and publishes count[key][chunk]; the last CTA
+//             to finish (arrival counter, no spin) turns the table into absolute bases: offsets[key] from the
+//             scan over keys, then the exclusive scan over the chunks of each key.
+//   kernel 2: one CTA per chunk places its pairs: rank inside the warp from match_any, warps take their turn in
+//             order to advance a shared-memory cursor per key, so equal keys keep ascending pair order (stable).
+constexpr int kChunk = 512;
+
+__global__ void __launch_bounds__(kChunk)
+group_chunk_count_kernel(const int32_t* __restrict__ ids, int n_pairs, int E, int C, int n_keys, int max_waves,
+                         bool identity, PlanPtrs plan, int32_t* __restrict__ table, int32_t* __restrict__ done,
+                         int* __restrict__ status) {
+    extern __shared__ __align__(16) int s_hist[];          // [n_keys] (+ [n_keys + 1] scratch offsets for the last CTA)
+    __shared__ int s_last, s_bad;
+    const int tid = threadIdx.x, chunk = blockIdx.x, n_chunks = gridDim.x;
+    if (tid == 0) s_bad = 0;
+    for (int i = tid; i < n_keys; i += kChunk) s_hist[i] = 0;
+    __syncthreads();
+    const int p = chunk * kChunk + tid;
+    if (p < n_pairs) {
+        const int key = pair_key(ids[p], E, C, identity, plan.wave_of, plan.slot_of);
+        if (key >= 0) atomicAdd(&s_hist[key], 1);
+        else s_bad = 1;
+    }
+    __syncthreads();
+    for (int i = tid; i < n_keys; i += kChunk) table[(size_t)i * n_chunks + chunk] = s_hist[i];
+    if (tid == 0 && s_bad) {
+        plan.header[HDR_BAD_ID] = 1;
+        atomicExch(status, EXMOE_ERR_BAD_EXPERT_ID);
+    }
+    __threadfence();
+    __syncthreads();
+    if (tid == 0) s_last = (atomicAdd(done, 1) == n_chunks - 1);
+    __syncthreads();
+    if (!s_last) return;
+    __threadfence();
+    if (tid == 0) *done = 0;                               // ready for the next call
+    // totals per key -> plan.counts (one warp per key, lanes over chunks); warp 0 then scans the keys
+    const int lane = tid & 31, warp = tid >> 5;
+    for (int i = warp; i < n_keys; i += kChunk / 32) {
+        int tot = 0;
+        for (int c = lane; c < n_chunks; c += 32) tot += __ldcg(&table[(size_t)i * n_chunks + c]);
+#pragma unroll
+        for (int m = 16; m >= 1; m >>= 1) tot += __shfl_xor_sync(0xffffffffu, tot, m);
+        if (lane == 0) {
+            plan.counts[i] = tot;
+            s_hist[i] = tot;
+        }
+    }
+    __syncthreads();
+    int* s_off = s_hist + n_keys;
+    if (tid < 32) scan_keys_warp0(s_hist, n_keys, C, max_waves, plan, s_off, identity, 0);
+    __syncthreads();
+    for (int i = warp; i < n_keys; i += kChunk / 32) {     // absolute base of every (key, chunk): exclusive scan over chunks
+        int running = s_off[i];
+        for (int c0 = 0; c0 < n_chunks; c0 += 32) {
+            const int c = c0 + lane;
+            const int v = c < n_chunks ? __ldcg(&table[(size_t)i * n_chunks + c]) : 0;
+            int incl = v;
+#pragma unroll
+            for (int d = 1; d < 32; d <<= 1) {
+                const int o = __shfl_up_sync(0xffffffffu, incl, d);
+                if (lane >= d) incl += o;
+            }
+            if (c < n_chunks) table[(size_t)i * n_chunks + c] = running + incl - v;
+            running += __shfl_sync(0xffffffffu, incl, 31);
+        }
+    }
+}
+
+__global__ void __launch_bounds__(kChunk)
+group_chunk_scatter_kernel(const int32_t* __restrict__ ids, int n_pairs, int E, int C, int n_keys, bool identity,
+                           PlanPtrs plan, const int32_t* __restrict__ table) {
+    extern __shared__ __align__(16) int s_cur[];           // [n_keys] pairs of this chunk already placed, per key
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, chunk = blockIdx.x, n_chunks = gridDim.x;
+    for (int i = tid; i < n_keys; i += kChunk) s_cur[i] = 0;
+    const int p = chunk * kChunk + tid;
+    int key = -1;
+    if (p < n_pairs) key = pair_key(ids[p], E, C, identity, plan.wave_of, plan.slot_of);
+    const unsigned same = __match_any_sync(0xffffffffu, key);
+    const int rank = __popc(same & ((1u << lane) - 1u));
+    const bool leader = key >= 0 && rank == 0;
+    __syncthreads();
+    int base = 0;
+    for (int w = 0; w < kChunk / 32; ++w) {                // warps in order: ascending pair index
+        if (warp == w && leader) {
+            base = s_cur[key];
+            s_cur[key] = base + __popc(same);
+        }
+        __syncthreads();
+    }
+    base = __shfl_sync(0xffffffffu, base, __ffs(same) - 1);
+    if (key >= 0) plan.perm[table[(size_t)key * n_chunks + chunk] + base + rank] = p;
+}
+
 void launch_group(const exmoe_shape& s, int C, int n_keys, int max_waves, bool identity, const int32_t* ids,
                   int n_pairs, PlanPtrs plan, int* d_status, cudaStream_t st) {
     const int E = s.num_experts;
@@ -313,6 +409,16 @@ void launch_group(const exmoe_shape& s, int C, int n_keys, int max_waves, bool i
         const size_t smem = (size_t)(2 * n_keys + 1 + n_pairs) * 4;
         group_small_kernel<<<1, 256, smem, st>>>(ids, n_pairs, E, C, n_keys, max_waves, identity, plan, d_status);
         count_launch();
+        return;
+    }
+    const int n_chunks = (n_pairs + kChunk - 1) / kChunk;
+    if (plan.chunk_table && (size_t)n_keys * n_chunks <= plan.chunk_table_words && n_keys <= 5000) {
+        if (identity) cudaMemsetAsync(plan.header + HDR_BAD_ID, 0, 4, st);
+        group_chunk_count_kernel<<<n_chunks, kChunk, (size_t)(2 * n_keys + 1) * 4, st>>>(
+            ids, n_pairs, E, C, n_keys, max_waves, identity, plan, plan.chunk_table, plan.chunk_done, d_status);
+        group_chunk_scatter_kernel<<<n_chunks, kChunk, (size_t)n_keys * 4, st>>>(ids, n_pairs, E, C, n_keys, identity, plan,
+                                                                               plan.chunk_table);
+        count_launch(2);
         return;
     }
     // counts doubles as the histogram; it is rewritten with the same values by CTA 0's scan
