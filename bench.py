@@ -216,17 +216,36 @@ def run_stack_sweep(args, dev, binding):
             torch.cuda.reset_peak_memory_stats(dev)
             cache = binding.Cache(shape, banks, C, max_tokens=64, device=dev)
             stack = synth.SyntheticStack(shape, L, seed=5100, alpha=args.alpha, device=dev)
-            h = synth.hidden_states(shape, T, 5200, device=dev)
+            # every step decodes fresh tokens: a new seeded hidden state enters layer 0 (as an embedding would)
+            pool = [synth.hidden_states(shape, T, 5200 + i, device=dev) for i in range(16)]
             fwd = lambda l, x, ids, w: cache.forward(l, x, ids, w)
             warm, timed = (args.warmup or 16), (args.steps if args.steps < 1000 else 64)
-            for _ in range(warm):
-                h = stack.step(fwd, h)
+            for i in range(warm):
+                h = stack.step(fwd, pool[i % 16])
             torch.cuda.synchronize()
+            graph = None
+            if C == shape.num_experts:                    # fully resident: no host sync inside, the step is graph-capturable
+                noise = stack.draw_noise(T)
+                h_in = pool[0].clone()
+                side = torch.cuda.Stream(device=dev)
+                fwd_s = lambda l, x, ids, w: cache.forward(l, x, ids, w, stream=side)
+                with torch.cuda.stream(side):
+                    stack.step(fwd_s, h_in, noise=noise)
+                side.synchronize()
+                graph = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(graph, stream=side):
+                    h = stack.step(fwd_s, h_in, noise=noise)
+                graph.replay()
+                torch.cuda.synchronize()
             st0 = [cache.stats(l) for l in range(L)]
             e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
             e0.record()
-            for _ in range(timed):
-                h = stack.step(fwd, h)
+            for i in range(timed):
+                if graph is not None:
+                    h_in.copy_(pool[(warm + i) % 16])
+                    graph.replay()
+                else:
+                    h = stack.step(fwd, pool[(warm + i) % 16])
             e1.record()
             torch.cuda.synchronize()
             ms = e0.elapsed_time(e1) / timed
@@ -236,8 +255,9 @@ def run_stack_sweep(args, dev, binding):
                          "h2d_bytes_per_token": d("h2d_bytes") / (timed * T),
                          "hit_rate": (d("hits") / d("lookups")) if d("lookups") else None,
                          "waves_per_layer_call": (d("waves") / d("forwards")) if d("forwards") else 1.0,
-                         "peak_reserved_gib": torch.cuda.max_memory_reserved(dev) / 2 ** 30})
-            assert cache.status() == 0
+                         "peak_reserved_gib": torch.cuda.max_memory_reserved(dev) / 2 ** 30,
+                         "timing": "CUDA graph of the 16-layer step" if graph is not None else "host-driven"})
+            assert cache.status() == 0 and bool(torch.isfinite(h.float()).all())
             cache.close()
             del cache
             print(json.dumps(rows[-1]), file=sys.stderr, flush=True)

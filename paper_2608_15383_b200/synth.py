@@ -92,14 +92,21 @@ class SyntheticStack:
                      for l in range(self.L)]
         self.gen = _gen(seed + 5, device)
 
-    def step(self, layer_fn, hidden, record=None):
-        """layer_fn(layer, hidden, ids, weights) -> moe output.  Returns the hidden state after all layers."""
+    def draw_noise(self, T):
+        """One N(0, 0.1) residual per layer, for callers that need fixed tensors (CUDA-graph capture)."""
+        return [torch.randn((T, self.shape.d_model), generator=self.gen, device=self.device, dtype=torch.float32) * 0.1
+                for _ in range(self.L)]
+
+    def step(self, layer_fn, hidden, record=None, noise=None):
+        """layer_fn(layer, hidden, ids, weights) -> moe output.  Returns the hidden state after all layers.
+        `noise`: per-layer residual tensors to use instead of drawing fresh ones."""
         h = hidden
         for l in range(self.L):
             ids, w = route(h, self.routers[l], self.shape.top_k, self.bias[l])
             out = layer_fn(l, h, ids, w)
             if record is not None:
                 record.append((l, h, ids, w, out))
-            noise = torch.randn(h.shape, generator=self.gen, device=h.device, dtype=torch.float32) * 0.1
-            h = (h.float() + out.float() + noise).to(torch.bfloat16)
+            eps = noise[l] if noise is not None else \
+                torch.randn(h.shape, generator=self.gen, device=h.device, dtype=torch.float32) * 0.1
+            h = (h.float() + out.float() + eps).to(torch.bfloat16)
         return h
