@@ -412,13 +412,18 @@ int exmoe_moe_forward(exmoe_cache* c, int layer, const void* hidden, const int32
             sw.max_groups = groups;
             sw.pairwise = pairwise;
             sw.saved_ids = c->saved_ids;
-            if (!c->prof_only || c->prof_only == PROF_GATEUP) {
-                ProfScope ps(c, PROF_GATEUP, st);
-                launch_small_wave(a, sw, st, true, false);
-            }
-            if (!c->prof_only || c->prof_only == PROF_DOWN) {
-                ProfScope ps(c, PROF_DOWN, st);
-                launch_small_wave(a, sw, st, false, true);
+            sw.grid_bar = reinterpret_cast<unsigned*>(c->plan.chunk_done + 16);   // zeroed at create, self-resetting
+            if (pairwise && !c->prof_only && !c->prof_on) {
+                launch_small_wave(a, sw, st, true, true);                // may fuse both GEMMs into one launch
+            } else {
+                if (!c->prof_only || c->prof_only == PROF_GATEUP) {
+                    ProfScope ps(c, PROF_GATEUP, st);
+                    launch_small_wave(a, sw, st, true, false);
+                }
+                if (!c->prof_only || c->prof_only == PROF_DOWN) {
+                    ProfScope ps(c, PROF_DOWN, st);
+                    launch_small_wave(a, sw, st, false, true);
+                }
             }
         } else if (P <= kLeanMaxPairs && c->lean_ok) {
             // a few rows per expert: lean register-dequant kernels on the global plan, pair buffer + combine

@@ -78,6 +78,7 @@ struct SmallWave {
     int max_rows, max_groups;
     bool pairwise;              // T*k <= kPairMaxPairs and a single wave: per-pair gate/up, by-token down
     int32_t* saved_ids;         // [kPairMaxPairs]
+    unsigned* grid_bar;         // [2] arrival count and generation of the fused kernel's grid barrier (zero-initialised)
 };
 constexpr int kPairMaxPairs = 32;
 #ifndef EXMOE_SMALL_MAX_PAIRS
