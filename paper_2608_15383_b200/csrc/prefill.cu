@@ -90,12 +90,15 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volati
                                           long long budget = kWaitBudget) {
     if (mbar_try(bar, parity)) return true;
     const long long t0 = clock64();
+    unsigned polls = 0;
     while (!mbar_try(bar, parity)) {
-        if (*abort_flag) return false;
-        if (clock64() - t0 > budget) {
-            *abort_flag = 1;
-            atomicExch(status, EXMOE_ERR_TIMEOUT);
-            return false;
+        if ((++polls & 15u) == 0) {                    // the bookkeeping of the bound is amortised over 16 polls
+            if (*abort_flag) return false;
+            if (clock64() - t0 > budget) {
+                *abort_flag = 1;
+                atomicExch(status, EXMOE_ERR_TIMEOUT);
+                return false;
+            }
         }
     }
     return true;
