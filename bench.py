@@ -451,6 +451,35 @@ def main():
             h_out.copy_(d_o, non_blocking=True)
         stream.synchronize()
 
+    e2e_mode = "per-step launches"
+    if identity and T <= 64:
+        # serving-loop form: per layer one CUDA graph of [3 H2D copies, forward, D2H copy] on fixed pinned staging
+        # buffers; a step writes its inputs into the staging buffers, replays the graph and waits for the result
+        s_h, s_i, s_w = (torch.empty_like(x).pin_memory() for x in (h_h[0], h_i[0], h_w[0]))
+        graphs = []
+        with torch.cuda.stream(stream):
+            cache.forward(0, d_h, d_i, d_w, out=d_o, stream=stream)
+        stream.synchronize()
+        for l in range(L):
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g, stream=stream):
+                d_h.copy_(s_h, non_blocking=True)
+                d_i.copy_(s_i, non_blocking=True)
+                d_w.copy_(s_w, non_blocking=True)
+                cache.forward(l, d_h, d_i, d_w, out=d_o, stream=stream)
+                h_out.copy_(d_o, non_blocking=True)
+            graphs.append(g)
+
+        def e2e_step(i):                                   # noqa: F811  (replaces the launch-per-call form)
+            j = i % len(h_h)
+            s_h.copy_(h_h[j])
+            s_i.copy_(h_i[j])
+            s_w.copy_(h_w[j])
+            with torch.cuda.stream(stream):
+                graphs[i % L].replay()
+            stream.synchronize()
+        e2e_mode = "one CUDA graph per step (H2D copies, forward, D2H copy)"
+
     for i in range(3):
         e2e_step(i)
     if world > 1:
@@ -462,7 +491,7 @@ def main():
     dt = max_over_ranks(dt, world, dev)
     h2d = h_h[0].numel() * 2 + h_i[0].numel() * 4 + h_w[0].numel() * 4
     e2e = {"value": world * n_e2e * T / dt, "unit": UNIT, "h2d_bytes_per_step": int(h2d),
-           "d2h_bytes_per_step": int(h_out.numel() * 2), "steps": n_e2e}
+           "d2h_bytes_per_step": int(h_out.numel() * 2), "steps": n_e2e, "mode": e2e_mode}
 
     status = cache.status()
     extra = {}
