@@ -39,6 +39,9 @@ WORKLOADS = {
     "offload": (16, 16, 1, 1.0, "config3: T=16, 16 slots over a 64-expert pinned host bank, Zipf(1.1) routing"),
     "prefill": (2048, 64, 1, 0.0, "config4: OLMoE-shaped prefill, T=2048, 64 slots resident, uniform routing"),
 }
+# DRAM bytes (read + write) per launch of the dominant kernel, from the committed ncu captures under profiles/
+# (decode: profiles/decode_t1_c64_pair_kernels_ncu_full.md; prefill: profiles/prefill_t2048_c64_tcgen05_ncu_full.md)
+NCU_TRAFFIC_BYTES = {"decode": 17.33e6, "prefill": 214.68e6 + 12.51e6}
 METRIC = "moe_layer_tokens_per_s"
 UNIT = "tokens/s"
 
@@ -422,13 +425,18 @@ def main():
         flops = 2.0 * T * shape.top_k * 2 * shape.d_ff * shape.d_model          # gate/up GEMM of one step
         achieved = flops / (kinds["gate_up"]["us_per_launch"] * 1e-6) / 1e12
         roof = {"bound": "tensor", "achieved": achieved, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
-                "frac": achieved / peaks["bf16_tflops"], "traffic": None, "kernel": "gate_up (prefill_gemm_kernel<true>, tcgen05)", "flops_per_launch": flops,
+                "frac": achieved / peaks["bf16_tflops"],
+                "traffic": NCU_TRAFFIC_BYTES.get(args.workload) if not args.tokens else None,
+                "traffic_unit": "bytes per launch (ncu dram read + write)", "kernel": "gate_up (prefill_gemm_kernel<true>, tcgen05)", "flops_per_launch": flops,
                 "peak_source": peaks["source"] + " cuBLAS bf16, burst"}
     else:
         gu_bytes = active * w13_bytes                                            # packed gate/up codes + scales
         achieved = gu_bytes / (kinds["gate_up"]["us_per_launch"] * 1e-6) / 1e9
         roof = {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                "frac": achieved / peaks["hbm_gbs"], "traffic": None, "kernel": "gate_up (decode_gemm_kernel)",
+                "frac": achieved / peaks["hbm_gbs"],
+                "traffic": NCU_TRAFFIC_BYTES.get(args.workload) if not args.tokens else None,
+                "traffic_unit": "bytes per launch (ncu dram read + write)",
+                "kernel": "gate_up (pair_gateup_kernel)" if T * shape.top_k <= 32 else "gate_up",
                 "bytes_per_launch": gu_bytes, "peak_source": peaks["source"] + " copy rate, burst"}
     step_gbs = active * bpe / (ms * 1e-3 / K) / 1e9
     step_tflops = 2.0 * T * shape.top_k * 3 * shape.d_ff * shape.d_model / (ms * 1e-3 / K) / 1e12
