@@ -412,7 +412,6 @@ int exmoe_moe_forward(exmoe_cache* c, int layer, const void* hidden, const int32
             sw.max_groups = groups;
             sw.pairwise = pairwise;
             sw.saved_ids = c->saved_ids;
-            sw.grid_bar = reinterpret_cast<unsigned*>(c->plan.chunk_done + 16);   // zeroed at create, self-resetting
             if (pairwise && !c->prof_only && !c->prof_on) {
                 launch_small_wave(a, sw, st, true, true);                // may fuse both GEMMs into one launch
             } else {

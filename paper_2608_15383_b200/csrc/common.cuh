@@ -78,7 +78,6 @@ struct SmallWave {
     int max_rows, max_groups;
     bool pairwise;              // T*k <= kPairMaxPairs and a single wave: per-pair gate/up, by-token down
     int32_t* saved_ids;         // [kPairMaxPairs]
-    unsigned* grid_bar;         // [2] arrival count and generation of the fused kernel's grid barrier (zero-initialised)
 };
 constexpr int kPairMaxPairs = 32;
 #ifndef EXMOE_SMALL_MAX_PAIRS
@@ -97,10 +96,6 @@ void launch_resolve(const exmoe_shape& s, int C, int Cw, size_t bytes_per_expert
                     LayerState state, PlanPtrs plan, int* d_status, cudaStream_t st);
 void launch_group(const exmoe_shape& s, int C, int n_keys, int max_waves, bool identity, const int32_t* ids,
                   int n_pairs, PlanPtrs plan, int* d_status, cudaStream_t st);
-void launch_decode_gateup(const GemmArgs& a, const __nv_bfloat16* hidden, __nv_bfloat16* act, int max_rows,
-                          int max_groups, cudaStream_t st);
-void launch_decode_down(const GemmArgs& a, const __nv_bfloat16* act, const float* topk_w, float* y, int max_rows,
-                        int max_groups, cudaStream_t st);
 bool launch_lean_wave(const GemmArgs& a, const __nv_bfloat16* hidden, __nv_bfloat16* act, const float* topk_w, float* y,
                       int max_rows, int max_groups, bool gateup, bool down, cudaStream_t st);
 #ifndef EXMOE_LEAN_MAX_PAIRS

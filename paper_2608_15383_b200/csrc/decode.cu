@@ -157,9 +157,8 @@ __device__ __forceinline__ void build_small_plan(const SmallArgs& sa, int C, Sma
 
 // NB  = 128-wide blocks held in registers per warp and matrix
 // NCH = 8-row activation chunks per pass (rows per pass = 8*NCH)
-enum { MODE_PLAN = 0, MODE_SMALL = 1, MODE_PAIR = 2 };
+enum { MODE_SMALL = 1, MODE_PAIR = 2 };
 
-// MODE_PLAN  : groups come from the grouping kernels' global plan
 // MODE_SMALL : every CTA rebuilds the wave's grouping in shared memory (T*k <= kSmallMaxPairs)
 // MODE_PAIR  : one item per token-expert pair, no grouping at all (T*k <= 32, gate/up only)
 #ifndef EXMOE_MINB_NB2
@@ -197,7 +196,7 @@ decode_gemm_kernel(GemmArgs a, SmallArgs sa, const __nv_bfloat16* __restrict__ x
     constexpr bool SMALL = (MODE == MODE_SMALL);
     constexpr bool PAIR = (MODE == MODE_PAIR);
     SmallPlan sp{};
-    int g0 = 0, n_items;
+    int n_items;
     if (PAIR) {
         grid_launch_dependents();
         n_items = sa.n_pairs * tiles;
@@ -206,7 +205,7 @@ decode_gemm_kernel(GemmArgs a, SmallArgs sa, const __nv_bfloat16* __restrict__ x
             sa.saved_ids[tid] = id;
             if (id < 0 || id >= sa.E) atomicExch(sa.status, EXMOE_ERR_BAD_EXPERT_ID);
         }
-    } else if (SMALL) {
+    } else {
         if (GATEUP) grid_launch_dependents();          // let the down kernel start prefetching its weights
         sp.cnt = plan_mem;
         sp.off = sp.cnt + C;
@@ -232,9 +231,6 @@ decode_gemm_kernel(GemmArgs a, SmallArgs sa, const __nv_bfloat16* __restrict__ x
                 if (s_scalars[2]) atomicExch(sa.status, EXMOE_ERR_BAD_EXPERT_ID);
             }
         }
-    } else {
-        g0 = a.wave_start[0];
-        n_items = (a.wave_start[1] - g0) * tiles;
     }
 
     bool waited = false;
@@ -248,16 +244,11 @@ decode_gemm_kernel(GemmArgs a, SmallArgs sa, const __nv_bfloat16* __restrict__ x
             slot = sa.slot_of ? sa.slot_of[id] : id;
             m_rows = 1;
             row0 = p;
-        } else if (SMALL) {
+        } else {
             slot = sp.gkeys[item / tiles];
             m_rows = sp.cnt[slot];
             lrow0 = sp.off[slot];
             row0 = sp.row_base + lrow0;
-        } else {
-            const int key = a.group_keys[g0 + item / tiles];
-            slot = key % C;
-            m_rows = a.counts[key];
-            row0 = a.offsets[key];
         }
         const uint8_t* wbase = a.slots + (size_t)slot * a.slot_stride + (GATEUP ? 0 : w13_bytes);
         const int panel = tile * PP + pp;              // panel (pair) index inside the matrix
@@ -309,7 +300,7 @@ decode_gemm_kernel(GemmArgs a, SmallArgs sa, const __nv_bfloat16* __restrict__ x
                         if (idx < total) {
                             size_t src_row;
                             if (PAIR) src_row = (size_t)(row0 / a.top_k);
-                            else if (GATEUP) src_row = (size_t)((SMALL ? sp.perm[lrow0 + pass0 + n] : a.perm[row0 + pass0 + n]) / a.top_k);
+                            else if (GATEUP) src_row = (size_t)(sp.perm[lrow0 + pass0 + n] / a.top_k);
                             else src_row = (size_t)(row0 + pass0 + n);
                             v = *reinterpret_cast<const uint4*>(x_src + src_row * K + ck * 8);
                             *reinterpret_cast<uint4*>(xs + (size_t)n * x_stride + ck * 16) = v;
@@ -411,7 +402,7 @@ decode_gemm_kernel(GemmArgs a, SmallArgs sa, const __nv_bfloat16* __restrict__ x
                             const float act = g / (1.f + __expf(-g)) * u;
                             act_out[(size_t)(row0 + n) * a.I + orow] = __float2bfloat16_rn(act);
                         } else {
-                            const int pair = SMALL ? sp.perm[lrow0 + n] : a.perm[row0 + n];
+                            const int pair = sp.perm[lrow0 + n];
                             y_out[(size_t)pair * a.H + orow] = topk_w[pair] * tot[0][ch][i];
                         }
                     }
@@ -711,174 +702,6 @@ pair_gateup_kernel(GemmArgs a, SmallArgs sa, const __nv_bfloat16* __restrict__ h
     pair_gateup_item<NB>(a, sa, hidden, act_out, KS, blockIdx.x, smem);
 }
 
-// ------------------------------------------------------------------------------------------------
-// Whole tiny-batch layer in ONE cooperative launch (T*k <= 32, one wave, k <= 8, d_ff <= 1024):
-// phase A = pair_gateup_item over (pair, tile) items, then each CTA requests the packed down-projection
-// weights of its first phase-B item, then a grid-wide barrier (bounded spin on a generation word; the
-// cooperative launch guarantees that every CTA is resident), then phase B = the by-token down projection
-// with the fixed-order combine.  The down weights stream while the barrier is being crossed, and the
-// second kernel launch with its ramp and drain disappears.
-// ------------------------------------------------------------------------------------------------
-__device__ __forceinline__ bool grid_barrier(unsigned* bar, unsigned nblocks, int* status) {
-    __shared__ int s_ok;
-    __syncthreads();
-    if (threadIdx.x == 0) {
-        volatile unsigned* gen = bar + 1;
-        const unsigned my_gen = *gen;                  // read before arriving: nobody can bump it until all arrived
-        int ok = 1;
-        __threadfence();
-        if (atomicAdd(bar, 1u) == nblocks - 1) {
-            bar[0] = 0;
-            __threadfence();
-            atomicAdd(bar + 1, 1u);
-        } else {
-            const long long t0 = clock64();
-            while (*gen == my_gen) {
-                if (clock64() - t0 > 2000000000ll) {   // ~1 s: give up, report, let the kernel finish
-                    atomicExch(status, EXMOE_ERR_TIMEOUT);
-                    ok = 0;
-                    break;
-                }
-            }
-        }
-        __threadfence();
-        s_ok = ok;
-    }
-    __syncthreads();
-    return s_ok != 0;
-}
-
-template <int NBT>
-struct DownRegs {
-    uint4 w[NBT][2];
-    uint32_t s[NBT];
-    float rw;
-    bool valid;
-};
-
-template <int NBT>
-__device__ __forceinline__ void token_down_request(const GemmArgs& a, const SmallArgs& sa, const float* topk_w, int item,
-                                                   DownRegs<NBT>& r) {
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, q = lane >> 2;
-    const int k = a.top_k, KB = a.I / kGroup, panels = a.H / kPanelRows;
-    const int t = item / panels, panel = item % panels;
-    r.valid = false;
-    r.rw = 0.f;
-    if (warp >= k) return;
-    const int pair = t * k + warp;
-    const int id = sa.ids[pair];
-    r.valid = id >= 0 && id < sa.E;
-    if (!r.valid) return;
-    r.rw = ldg_early_f32(topk_w + pair);
-    const int slot = sa.slot_of ? sa.slot_of[id] : id;
-    const uint8_t* mat = a.slots + (size_t)slot * a.slot_stride + matrix_bytes(2 * a.I, a.H) + (size_t)panel * KB * kBlockBytes;
-#pragma unroll
-    for (int b = 0; b < NBT; ++b) {
-        const uint8_t* blk = mat + (size_t)b * kBlockBytes;
-        r.w[b][0] = ldg_stream128(blk + lane * 16);
-        r.w[b][1] = ldg_stream128(blk + 512 + lane * 16);
-        r.s[b] = ldg_stream32(blk + kCodeBytes + q * 4);
-    }
-}
-
-template <int NBT>
-__device__ __forceinline__ void token_down_finish(const GemmArgs& a, const SmallArgs& sa, const __nv_bfloat16* act, int bpwg,
-                                                  int item, DownRegs<NBT>& r, unsigned char* smem) {
-    const int K = a.I, k = a.top_k;
-    const int x_stride = K * 2 + 64;
-    unsigned char* xs = smem;                                          // [k][x_stride]
-    float* ys = reinterpret_cast<float*>(smem + (size_t)k * x_stride); // [k][16]
-    int* s_valid = reinterpret_cast<int*>(ys + k * 16);                // [k]
-    float* adj = reinterpret_cast<float*>(s_valid + k);                // [KB][k]
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int q = lane >> 2, c = lane & 3;
-    const int panels = a.H / kPanelRows;
-    const int t = item / panels, panel = item % panels;
-    const int j = warp;
-    __syncthreads();                                                   // earlier users of the shared memory are done
-    const int chunks_per_row = K / 8, total = k * chunks_per_row;
-    for (int base = warp * 32; base < total; base += 256) {
-        const int idx = base + lane;
-        const int n = idx / chunks_per_row, ck = idx % chunks_per_row;
-        uint4 v = make_uint4(0, 0, 0, 0);
-        if (idx < total) {
-            v = __ldcg(reinterpret_cast<const uint4*>(act + (size_t)(t * k + n) * K + ck * 8));   // written by other CTAs
-            *reinterpret_cast<uint4*>(xs + (size_t)n * x_stride + ck * 16) = v;
-        }
-        float sx = sum8_bf16(v);
-#pragma unroll
-        for (int m = 8; m >= 1; m >>= 1) sx += __shfl_xor_sync(0xffffffffu, sx, m);
-        if (idx < total && (ck & 15) == 0) adj[(ck >> 4) * k + n] = -136.f * sx;
-    }
-    __syncthreads();
-    float result[2] = {0.f, 0.f}, tot[2] = {0.f, 0.f};
-    if (r.valid) {
-#pragma unroll
-        for (int b = 0; b < NBT; ++b) {
-            float acc[4] = {0.f, 0.f, 0.f, 0.f};
-#pragma unroll
-            for (int h = 0; h < 2; ++h)
-#pragma unroll
-                for (int set = 0; set < 2; ++set) {
-                    const int k0 = b * kGroup + 64 * h + 32 * set + 8 * c;
-                    uint4 xb = make_uint4(0, 0, 0, 0);
-                    if (q == 0) xb = *reinterpret_cast<const uint4*>(xs + (size_t)j * x_stride + k0 * 2);
-                    const uint32_t wq = set ? r.w[b][h].z : r.w[b][h].x;
-                    const uint32_t wq8 = set ? r.w[b][h].w : r.w[b][h].y;
-                    mma_m16n8k16(acc, code_pair(wq, 0), code_pair(wq8, 0), code_pair(wq, 4), code_pair(wq8, 4), xb.x, xb.y);
-                    mma_m16n8k16(acc, code_pair(wq, 8), code_pair(wq8, 8), code_pair(wq, 12), code_pair(wq8, 12), xb.z, xb.w);
-                }
-            const __half2 sc = *reinterpret_cast<const __half2*>(&r.s[b]);
-            const float cr = adj[b * k + j];
-            tot[0] = fmaf(__low2float(sc), acc[0] + cr, tot[0]);
-            tot[1] = fmaf(__high2float(sc), acc[2] + cr, tot[1]);
-            if ((b + 1) % bpwg == 0) {                                 // end of one K-split range of the grouped kernel
-                const bool first = (b + 1 == bpwg);
-                result[0] = first ? tot[0] : result[0] + tot[0];
-                result[1] = first ? tot[1] : result[1] + tot[1];
-                tot[0] = tot[1] = 0.f;
-            }
-        }
-    }
-    if (j < k) {
-        if (lane == 0) s_valid[j] = r.valid ? 1 : 0;
-        if (c == 0) {
-            ys[j * 16 + q] = r.rw * result[0];
-            ys[j * 16 + q + 8] = r.rw * result[1];
-        }
-    }
-    __syncthreads();
-    if (tid < 16) {
-        float sum = 0.f;
-        for (int jj = 0; jj < k; ++jj)
-            if (s_valid[jj]) sum += ys[jj * 16 + tid];
-        sa.out[(size_t)t * a.H + panel * kPanelRows + tid] = __float2bfloat16_rn(sum);
-    }
-}
-
-template <int NB, int NBT>
-__global__ void __launch_bounds__(256, 2)
-decode_fused_kernel(GemmArgs a, SmallArgs sa, const __nv_bfloat16* __restrict__ hidden, __nv_bfloat16* __restrict__ act,
-                    const float* __restrict__ topk_w, int KS, int bpwg, unsigned* bar) {
-    extern __shared__ __align__(16) unsigned char smem[];
-    const int tiles = a.I / (kPanelRows * (8 / KS));
-    const int items_a = sa.n_pairs * tiles;
-    const int items_b = (sa.n_pairs / a.top_k) * (a.H / kPanelRows);
-    if (blockIdx.x == 0) keep_pair_ids(sa);
-    for (int item = blockIdx.x; item < items_a; item += gridDim.x) {
-        __syncthreads();                                               // shared memory of the previous item is free
-        pair_gateup_item<NB>(a, sa, hidden, act, KS, item, smem);
-    }
-    DownRegs<NBT> regs;
-    const bool has_b = (int)blockIdx.x < items_b;
-    if (has_b) token_down_request<NBT>(a, sa, topk_w, blockIdx.x, regs);   // weights fly while the barrier is crossed
-    grid_barrier(bar, gridDim.x, sa.status);
-    for (int item = blockIdx.x; item < items_b; item += gridDim.x) {
-        if (item != (int)blockIdx.x) token_down_request<NBT>(a, sa, topk_w, item, regs);
-        token_down_finish<NBT>(a, sa, act, bpwg, item, regs, smem);
-    }
-}
-
 template <int NB>
 void launch_pair_gateup(const GemmArgs& a, const SmallArgs& sa, const __nv_bfloat16* hidden, __nv_bfloat16* act, int KS,
                         cudaStream_t st) {
@@ -892,108 +715,6 @@ void launch_pair_gateup(const GemmArgs& a, const SmallArgs& sa, const __nv_bfloa
     }
     kern<<<sa.n_pairs * tiles, 256, smem, st>>>(a, sa, hidden, act, KS);
     count_launch();
-}
-
-// Lean variant of token_down_kernel for k * (K-split ranges) <= 32 warps: warp = (expert j, K range r), NBW blocks in
-// registers, no loops around the arithmetic.  Partial sums are added per expert in range order, multiplied by the
-// routing weight and added over the experts in order, i.e. exactly the grouped kernel's order.
-template <int NBW>
-__global__ void __launch_bounds__(1024, 1)
-token_down_split_kernel(GemmArgs a, SmallArgs sa, const __nv_bfloat16* __restrict__ act,
-                        const float* __restrict__ topk_w, int ranges) {
-    extern __shared__ __align__(16) unsigned char smem[];
-    const int K = a.I, KB = K / kGroup, k = a.top_k;
-    const int x_stride = K * 2 + 64;
-    unsigned char* xs = smem;                                              // [k][x_stride]
-    float* part = reinterpret_cast<float*>(smem + (size_t)k * x_stride);  // [k][ranges][16]
-    float* adj = part + k * ranges * 16;                                   // [KB][k]
-    int* s_valid = reinterpret_cast<int*>(adj + KB * k);                   // [k]
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int q = lane >> 2, c = lane & 3;
-    const int panels = a.H / kPanelRows;
-    const int t = blockIdx.x / panels, panel = blockIdx.x % panels;
-    const int j = warp / ranges, r = warp % ranges;
-    const int pair = t * k + j;
-    const int id = sa.ids[pair];
-    const bool valid = id >= 0 && id < sa.E;
-    float rw = 0.f;
-    uint4 wreg[NBW][2];
-    uint32_t sreg[NBW];
-    if (valid) {
-        const int slot = sa.slot_of ? sa.slot_of[id] : id;
-        const uint8_t* mat = a.slots + (size_t)slot * a.slot_stride + matrix_bytes(2 * a.I, a.H) +
-                             ((size_t)panel * KB + r * NBW) * kBlockBytes;
-#pragma unroll
-        for (int b = 0; b < NBW; ++b) {
-            const uint8_t* blk = mat + (size_t)b * kBlockBytes;
-            wreg[b][0] = ldg_stream128(blk + lane * 16);
-            wreg[b][1] = ldg_stream128(blk + 512 + lane * 16);
-            sreg[b] = ldg_stream32(blk + kCodeBytes + q * 4);
-        }
-        if (r == 0) rw = topk_w[pair];
-    }
-    grid_dependency_wait();                                                // activations of the gate/up kernel
-    {
-        const int chunks_per_row = K / 8, total = k * chunks_per_row;
-        const int nthreads = blockDim.x;
-        for (int base = warp * 32; base < total; base += nthreads) {
-            const int idx = base + lane;
-            const int n = idx / chunks_per_row, ck = idx % chunks_per_row;
-            uint4 v = make_uint4(0, 0, 0, 0);
-            if (idx < total) {
-                v = *reinterpret_cast<const uint4*>(act + (size_t)(t * k + n) * K + ck * 8);
-                *reinterpret_cast<uint4*>(xs + (size_t)n * x_stride + ck * 16) = v;
-            }
-            float sx = sum8_bf16(v);
-#pragma unroll
-            for (int m = 8; m >= 1; m >>= 1) sx += __shfl_xor_sync(0xffffffffu, sx, m);
-            if (idx < total && (ck & 15) == 0) adj[(ck >> 4) * k + n] = -136.f * sx;
-        }
-    }
-    __syncthreads();
-    float total0 = 0.f, total1 = 0.f;
-    if (valid) {
-#pragma unroll
-        for (int b = 0; b < NBW; ++b) {
-            float acc[4] = {0.f, 0.f, 0.f, 0.f};
-#pragma unroll
-            for (int h = 0; h < 2; ++h)
-#pragma unroll
-                for (int set = 0; set < 2; ++set) {
-                    const int k0 = (r * NBW + b) * kGroup + 64 * h + 32 * set + 8 * c;
-                    uint4 xb = make_uint4(0, 0, 0, 0);
-                    if (q == 0) xb = *reinterpret_cast<const uint4*>(xs + (size_t)j * x_stride + k0 * 2);
-                    const uint32_t wq = set ? wreg[b][h].z : wreg[b][h].x;
-                    const uint32_t wq8 = set ? wreg[b][h].w : wreg[b][h].y;
-                    mma_m16n8k16(acc, code_pair(wq, 0), code_pair(wq8, 0), code_pair(wq, 4), code_pair(wq8, 4), xb.x, xb.y);
-                    mma_m16n8k16(acc, code_pair(wq, 8), code_pair(wq8, 8), code_pair(wq, 12), code_pair(wq8, 12), xb.z, xb.w);
-                }
-            const __half2 sc = *reinterpret_cast<const __half2*>(&sreg[b]);
-            const float cr = adj[(r * NBW + b) * k + j];
-            total0 = fmaf(__low2float(sc), acc[0] + cr, total0);
-            total1 = fmaf(__high2float(sc), acc[2] + cr, total1);
-        }
-    }
-    if (c == 0) {
-        part[(j * ranges + r) * 16 + q] = total0;
-        part[(j * ranges + r) * 16 + q + 8] = total1;
-    }
-    __shared__ float s_rw[32];
-    if (r == 0 && lane == 0) {
-        s_valid[j] = valid ? 1 : 0;
-        s_rw[j] = rw;
-    }
-    __syncthreads();
-    if (tid < 16) {
-        float sum = 0.f;
-        for (int jj = 0; jj < k; ++jj) {
-            if (!s_valid[jj]) continue;
-            float res = part[(jj * ranges) * 16 + tid];
-            for (int rr = 1; rr < ranges; ++rr) res += part[(jj * ranges + rr) * 16 + tid];
-            sum += s_rw[jj] * res;
-        }
-        sa.out[(size_t)t * a.H + panel * kPanelRows + tid] = __float2bfloat16_rn(sum);
-    }
 }
 
 // Lean grouped kernel for the middle regime (a few to a few dozen rows per expert; 40 < T*k <= kLeanMaxPairs):
@@ -1268,14 +989,6 @@ combine_kernel(const float* __restrict__ y, const int32_t* __restrict__ ids, int
 
 }  // namespace
 
-void launch_decode_gateup(const GemmArgs& a, const __nv_bfloat16* hidden, __nv_bfloat16* act, int max_rows,
-                          int max_groups, cudaStream_t st) {
-    launch_decode<true, MODE_PLAN>(a, SmallArgs{}, hidden, act, nullptr, nullptr, max_rows, max_groups, st);
-}
-void launch_decode_down(const GemmArgs& a, const __nv_bfloat16* act, const float* topk_w, float* y, int max_rows,
-                        int max_groups, cudaStream_t st) {
-    launch_decode<false, MODE_PLAN>(a, SmallArgs{}, act, nullptr, topk_w, y, max_rows, max_groups, st);
-}
 // Middle regime: lean register-dequant kernels on the global plan.  Returns false when the shape needs the generic body.
 bool launch_lean_wave(const GemmArgs& a, const __nv_bfloat16* hidden, __nv_bfloat16* act, const float* topk_w, float* y,
                       int max_rows, int max_groups, bool gateup, bool down, cudaStream_t st) {
@@ -1338,72 +1051,6 @@ void launch_token_down(const GemmArgs& a, const SmallArgs& sa, const __nv_bfloat
     count_launch();
 }
 
-template <int NBW>
-void launch_token_down_split(const GemmArgs& a, const SmallArgs& sa, const __nv_bfloat16* act, const float* w, int T,
-                             int ranges, cudaStream_t st) {
-    auto kern = token_down_split_kernel<NBW>;
-    const int k = a.top_k, KB = a.I / kGroup;
-    const size_t smem = (size_t)k * (a.I * 2 + 64) + (size_t)k * ranges * 16 * 4 + (size_t)(KB * k + 4) * 4 + (size_t)k * 4;
-    static bool attr_done = false;
-    if (!attr_done) {
-        cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
-        attr_done = true;
-    }
-    cudaLaunchConfig_t lc{};
-    lc.gridDim = dim3(T * (a.H / kPanelRows));
-    lc.blockDim = dim3(32 * k * ranges);
-    lc.dynamicSmemBytes = smem;
-    lc.stream = st;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = 1;
-    lc.attrs = attr;
-    lc.numAttrs = 1;
-    cudaLaunchKernelEx(&lc, kern, a, sa, act, w, ranges);
-    count_launch();
-}
-
-template <int NB, int NBT>
-bool launch_decode_fused(const GemmArgs& a, const SmallArgs& sa, const __nv_bfloat16* hidden, __nv_bfloat16* act,
-                         const float* w, int KS, int bpwg, unsigned* bar, cudaStream_t st) {
-    auto kern = decode_fused_kernel<NB, NBT>;
-    const int PP = 8 / KS, tiles = a.I / (kPanelRows * PP), k = a.top_k;
-    const size_t smem_a = (size_t)a.H * 2 + 64 + (size_t)(KS - 1) * PP * 2 * 128 * 4 + (size_t)(a.H / kGroup) * 4;
-    const size_t smem_b = (size_t)k * (a.I * 2 + 64) + (size_t)k * 17 * 4 + (size_t)(a.I / kGroup) * k * 4;
-    const size_t smem = smem_a > smem_b ? smem_a : smem_b;
-    static int capacity = -1;                          // co-resident CTAs of this instantiation on this device
-    static size_t capacity_smem = 0;
-    if (capacity < 0 || capacity_smem != smem) {
-        cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 100 * 1024);
-        int dev = 0, sms = 0, per_sm = 0;
-        cudaGetDevice(&dev);
-        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, 256, smem) != cudaSuccess) per_sm = 0;
-        capacity = per_sm * sms;
-        capacity_smem = smem;
-    }
-    if (capacity <= 0) return false;
-    const int items_a = sa.n_pairs * tiles, items_b = (sa.n_pairs / k) * (a.H / kPanelRows);
-    int grid = items_a > items_b ? items_a : items_b;
-    if (grid > capacity) grid = capacity;
-    cudaLaunchConfig_t lc{};
-    lc.gridDim = dim3(grid);
-    lc.blockDim = dim3(256);
-    lc.dynamicSmemBytes = smem;
-    lc.stream = st;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeCooperative;       // every CTA resident: the grid barrier cannot starve
-    attr[0].val.cooperative = 1;
-    lc.attrs = attr;
-    lc.numAttrs = 1;
-    if (cudaLaunchKernelEx(&lc, kern, a, sa, hidden, act, w, KS, bpwg, bar) != cudaSuccess) {
-        cudaGetLastError();
-        return false;
-    }
-    count_launch();
-    return true;
-}
-
 // One wave of the SMALL path: gate/up kernel, then the down kernel with the fused combine.
 void launch_small_wave(const GemmArgs& a, const SmallWave& w, cudaStream_t st, bool gateup, bool down) {
     SmallArgs sa{};
@@ -1421,27 +1068,6 @@ void launch_small_wave(const GemmArgs& a, const SmallWave& w, cudaStream_t st, b
     sa.arrive = w.arrive;
     sa.out = w.out;
     sa.saved_ids = w.saved_ids;
-#ifdef EXMOE_FUSED_DECODE
-    // Measured on B200 (config 2): 17.0 us per step fused against 12.4 us for the two kernels with programmatic
-    // dependent launch (the cooperative launch and the grid-wide barrier cost more than the second launch), so the
-    // fused kernel is compiled in only on request (-DEXMOE_FUSED_DECODE).
-    if (w.pairwise && gateup && down && w.grid_bar && a.top_k <= 8) {
-        // whole layer in one cooperative launch when the shape fits the register budgets
-        const DecodeCfg cfg = pick_cfg(a.H, a.I);
-        const int KBd = a.I / kGroup, bpwg = pick_cfg(a.I, a.H).bpw;
-        bool done = false;
-#define EXMOE_FUSED(NBv, NBTv) done = launch_decode_fused<NBv, NBTv>(a, sa, w.hidden, w.act, w.topk_w, cfg.KS, bpwg, w.grid_bar, st)
-        if (KBd % bpwg == 0) {
-            if (cfg.bpw == 4 && KBd == 8) EXMOE_FUSED(4, 8);
-            else if (cfg.bpw == 4 && KBd == 4) EXMOE_FUSED(4, 4);
-            else if (cfg.bpw == 4 && KBd == 2) EXMOE_FUSED(4, 2);
-            else if (cfg.bpw == 2 && KBd == 1) EXMOE_FUSED(2, 1);
-            else if (cfg.bpw == 2 && KBd == 2) EXMOE_FUSED(2, 2);
-        }
-#undef EXMOE_FUSED
-        if (done) return;
-    }
-#endif
     if (w.pairwise) {                                   // T*k <= 32, one wave: no grouping, by-token down + combine
         if (gateup) {
             const DecodeCfg cfg = pick_cfg(a.H, a.I);
@@ -1454,12 +1080,7 @@ void launch_small_wave(const GemmArgs& a, const SmallWave& w, cudaStream_t st, b
             const int KB = a.I / kGroup;
             const int bpwg = pick_cfg(a.I, a.H).bpw;    // the grouped kernel's K-split range, replayed for rounding
             const int T = w.n_pairs / a.top_k;
-            const int ranges = KB / bpwg;
-            if (false && a.top_k * ranges <= 32 && KB % bpwg == 0 && (bpwg == 4 || bpwg == 2 || bpwg == 1) && a.top_k <= 32) {
-                if (bpwg == 4) launch_token_down_split<4>(a, sa, w.act, w.topk_w, T, ranges, st);
-                else if (bpwg == 2) launch_token_down_split<2>(a, sa, w.act, w.topk_w, T, ranges, st);
-                else launch_token_down_split<1>(a, sa, w.act, w.topk_w, T, ranges, st);
-            } else if (KB % 8 == 0) launch_token_down<8>(a, sa, w.act, w.topk_w, T, bpwg, st);
+            if (KB % 8 == 0) launch_token_down<8>(a, sa, w.act, w.topk_w, T, bpwg, st);
             else if (KB % 4 == 0) launch_token_down<4>(a, sa, w.act, w.topk_w, T, bpwg, st);
             else if (KB % 2 == 0) launch_token_down<2>(a, sa, w.act, w.topk_w, T, bpwg, st);
             else launch_token_down<1>(a, sa, w.act, w.topk_w, T, bpwg, st);

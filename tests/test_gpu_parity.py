@@ -181,6 +181,29 @@ def test_mid_shape_ragged_groups(B, mid_layer, T):
     cache2.close()
 
 
+@pytest.mark.parametrize("T", [1, 7, 16, 30, 90, 300])
+def test_odd_block_counts(B, T):
+    """d_model = 3 * 128 and d_ff = 5 * 128: block counts that are not powers of two take the generic kernel
+    bodies (no K split, one block per step) on every path; 3 experts per token, ragged groups."""
+    s = synth.Shape(d_model=384, d_ff=640, num_experts=8, top_k=3)
+    if not hasattr(test_odd_block_counts, "layer"):
+        test_odd_block_counts.layer = helpers.make_layer(s, seed=123)
+    ora, bank = test_odd_block_counts.layer
+    hidden, ids, p = helpers.routed_inputs(s, T, seed=4100 + T, alpha=1.0)
+    y, ref = ora.forward(hidden, ids, p)
+    cache = B.Cache(s, [bank], s.num_experts, max_tokens=300)
+    out = cache.forward(0, hidden.cuda(), ids.cuda(), p.cuda())
+    helpers.check_output(out, y, ref, f"T={T}")
+    cache2 = B.Cache(s, [bank], 4, max_tokens=300, wave_cap=3)          # several waves, misses
+    sc = ocache.SlotCache(s.num_experts, 4, 3, bytes_per_expert=cache2.bytes_per_expert)
+    out2 = cache2.forward(0, hidden.cuda(), ids.cuda(), p.cuda())
+    compare_plan(cache2, sc, ids)
+    helpers.check_output(out2, y, ref, f"T={T} offloaded")
+    assert cache.status() == 0 and cache2.status() == 0
+    cache.close()
+    cache2.close()
+
+
 def test_config2_decode_olmoe(B, olmoe_layer):
     """Config 2: OLMoE shape, 1 token per step, 64 slots, fresh hidden state per step."""
     ora, bank = olmoe_layer
