@@ -436,7 +436,8 @@ def main():
                 "frac": achieved / peaks["hbm_gbs"],
                 "traffic": NCU_TRAFFIC_BYTES.get(args.workload) if not args.tokens else None,
                 "traffic_unit": "bytes per launch (ncu dram read + write)",
-                "kernel": "gate_up (pair_gateup_kernel)" if T * shape.top_k <= 32 else "gate_up",
+                "kernel": "gate_up (pair_gateup_kernel)" if T * shape.top_k <= 24 else
+                "gate_up (stream_gemm_kernel<1,true,1>)" if T * shape.top_k <= 448 else "gate_up",
                 "bytes_per_launch": gu_bytes, "peak_source": peaks["source"] + " copy rate, burst"}
     step_gbs = active * bpe / (ms * 1e-3 / K) / 1e9
     step_tflops = 2.0 * T * shape.top_k * 3 * shape.d_ff * shape.d_model / (ms * 1e-3 / K) / 1e12

@@ -130,7 +130,11 @@ int exmoe_moe_forward(exmoe_cache* cache, int layer, const void* hidden_bf16, co
  *
  *   experts_dev  : dev, num_experts packed experts back to back (expert e at e * bytes_per_expert), i.e. a
  *                  fully resident layer exactly as exmoe_pack wrote it (slot = expert id, one wave).
- *   hidden_bf16, topk_ids, topk_weights, out_bf16 : as for exmoe_moe_forward.  Same kernels, same result.
+ *   hidden_bf16, topk_ids, topk_weights, out_bf16 : as for exmoe_moe_forward.  These are the kernels
+ *                  exmoe_moe_forward runs for T * top_k <= 24 on a fully resident layer, and there the two
+ *                  entry points return the same bits; for 24 < T * top_k <= 32 exmoe_moe_forward switches to
+ *                  its streaming kernels, which split K differently, and the two agree within the output
+ *                  tolerance (a few BF16 roundings), not bit for bit.
  *
  * Limits (fixed by the size of the scratch): T * top_k <= 32 and d_ff <= 4096; anything larger is refused
  * with EXMOE_ERR_SHAPE before any work is queued.  T = 0 is a no-op.

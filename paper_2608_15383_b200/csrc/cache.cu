@@ -62,7 +62,7 @@ struct exmoe_cache {
     bool last_small;
     bool last_pair;
     int32_t* saved_ids;                       // ids of the last pairwise call (plan materialised on request)
-    bool lean_ok;                             // the shape fits the lean middle-regime kernels
+    bool stream_ok;                           // the shape fits the streaming middle-regime kernels
     void* tc_scratch;                         // tile list of the tensor-core path
     __nv_bfloat16* xg;                        // [max_pairs, H] hidden rows in plan order (tensor-core path only)
     PrefillMaps tc_maps;                      // TMA descriptors of xg and act
@@ -273,11 +273,7 @@ int exmoe_cache_create(exmoe_cache** out, const exmoe_shape* shape, int num_laye
     c->slot_last_seq.assign(num_layers, std::vector<uint64_t>(num_slots, 0));
     c->last_layer = -1;
     c->last_T = 0;
-    {
-        const int kbg = c->shape.d_model / kGroup, kbd = c->shape.d_ff / kGroup;
-        auto pow2_le8 = [](int v) { return v == 1 || v == 2 || v == 4 || v == 8 || v == 16 || v == 32; };
-        c->lean_ok = pow2_le8(kbg) && pow2_le8(kbd);      // K splits into 1/2/4 blocks per warp
-    }
+    c->stream_ok = stream_supported(c->shape.d_model, c->shape.d_ff);
     bool ok = cudaMallocHost(&c->h_plan, c->plan_d2h_bytes) == cudaSuccess;
     ok = ok && cudaStreamCreateWithFlags(&c->copy_stream, cudaStreamNonBlocking) == cudaSuccess;
     ok = ok && cudaEventCreateWithFlags(&c->ev_plan, cudaEventDisableTiming) == cudaSuccess;
@@ -360,7 +356,8 @@ int exmoe_moe_forward(exmoe_cache* c, int layer, const void* hidden, const int32
 
     const bool pairwise = small && P <= kPairMaxPairs && n_waves == 1;
     c->last_pair = pairwise;
-    if (!small && build_plan && !(P <= kLeanMaxPairs && c->lean_ok)) {
+    const bool use_stream = !small && c->stream_ok && P <= kStreamMaxPairs;
+    if (!small && build_plan && !use_stream) {
         ProfScope ps(c, PROF_PLAN, st);                  // hidden rows in plan order, once for all waves
         launch_gather_rows((const __nv_bfloat16*)hidden, c->plan.perm, c->plan.offsets + c->n_keys, P, k, s.d_model,
                            c->xg, st);
@@ -424,15 +421,16 @@ int exmoe_moe_forward(exmoe_cache* c, int layer, const void* hidden, const int32
                     launch_small_wave(a, sw, st, false, true);
                 }
             }
-        } else if (P <= kLeanMaxPairs && c->lean_ok) {
-            // a few rows per expert: lean register-dequant kernels on the global plan, pair buffer + combine
-            if (!c->prof_only || c->prof_only == PROF_GATEUP) {
-                ProfScope ps(c, PROF_GATEUP, st);
-                launch_lean_wave(a, (const __nv_bfloat16*)hidden, c->act, topk_weights, c->y, T, groups, true, false, st);
-            }
-            if (!c->prof_only || c->prof_only == PROF_DOWN) {
-                ProfScope ps(c, PROF_DOWN, st);
-                launch_lean_wave(a, (const __nv_bfloat16*)hidden, c->act, topk_weights, c->y, T, groups, false, true, st);
+        } else if (use_stream) {
+            // a few to a few dozen rows per expert: bulk-copy weight ring + register dequantisation, pair buffer + combine
+            if (!c->prof_only) {
+                ProfScope ps(c, PROF_GATEUP, st);    // both kernels: the down kernel is a programmatic dependent
+                launch_stream_wave(a, (const __nv_bfloat16*)hidden, c->act, topk_weights, c->y, c->d_status, groups, true, true,
+                                   st);
+            } else if (c->prof_only == PROF_GATEUP || c->prof_only == PROF_DOWN) {
+                ProfScope ps(c, c->prof_only, st);
+                launch_stream_wave(a, (const __nv_bfloat16*)hidden, c->act, topk_weights, c->y, c->d_status, groups,
+                                   c->prof_only == PROF_GATEUP, c->prof_only == PROF_DOWN, st);
             }
         } else {
             // many rows per expert: dense contraction on the tensor cores (tcgen05 / TMEM)

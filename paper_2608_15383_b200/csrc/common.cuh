@@ -81,7 +81,7 @@ struct SmallWave {
 };
 constexpr int kPairMaxPairs = 32;
 #ifndef EXMOE_SMALL_MAX_PAIRS
-#define EXMOE_SMALL_MAX_PAIRS 40
+#define EXMOE_SMALL_MAX_PAIRS 24
 #endif
 constexpr int kSmallMaxPairs = EXMOE_SMALL_MAX_PAIRS;
 constexpr int kSmallMaxSlots = 1024;
@@ -96,12 +96,14 @@ void launch_resolve(const exmoe_shape& s, int C, int Cw, size_t bytes_per_expert
                     LayerState state, PlanPtrs plan, int* d_status, cudaStream_t st);
 void launch_group(const exmoe_shape& s, int C, int n_keys, int max_waves, bool identity, const int32_t* ids,
                   int n_pairs, PlanPtrs plan, int* d_status, cudaStream_t st);
-bool launch_lean_wave(const GemmArgs& a, const __nv_bfloat16* hidden, __nv_bfloat16* act, const float* topk_w, float* y,
-                      int max_rows, int max_groups, bool gateup, bool down, cudaStream_t st);
-#ifndef EXMOE_LEAN_MAX_PAIRS
-#define EXMOE_LEAN_MAX_PAIRS 192
+// Streaming kernels (bulk-copy weight ring in shared memory) for kSmallMaxPairs < T*k <= kStreamMaxPairs.
+#ifndef EXMOE_STREAM_MAX_PAIRS
+#define EXMOE_STREAM_MAX_PAIRS 448
 #endif
-constexpr int kLeanMaxPairs = EXMOE_LEAN_MAX_PAIRS;   // above: tensor-core path
+constexpr int kStreamMaxPairs = EXMOE_STREAM_MAX_PAIRS;   // above: tensor-core path
+bool stream_supported(int H, int I);
+bool launch_stream_wave(const GemmArgs& a, const __nv_bfloat16* hidden, __nv_bfloat16* act, const float* topk_w, float* y,
+                        int* status, int max_groups, bool gateup, bool down, cudaStream_t st);
 void launch_small_wave(const GemmArgs& a, const SmallWave& w, cudaStream_t st, bool gateup, bool down);
 size_t prefill_scratch_bytes(int max_pairs, int num_experts);
 struct alignas(64) PrefillMaps { unsigned char x[128], act[128]; };   // two CUtensorMap objects (grouped hidden, activations)

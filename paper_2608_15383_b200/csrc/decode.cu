@@ -13,14 +13,17 @@
 // K-split partials are reduced through shared memory in a fixed order.
 //
 // Two flavours share the body:
-//   SMALL (T*k <= kSmallMaxPairs = 40): a decode step is launch-latency bound, so the chain of dependent global
+//   SMALL (T*k <= kSmallMaxPairs): a decode step is launch-latency bound, so the chain of dependent global
 //     loads is cut to two levels: every CTA rebuilds the wave's token grouping (histogram, prefix
 //     sum, stable permutation) in shared memory straight from topk_ids; CTA 0 also publishes it.
 //     The down kernel is launched with programmatic dependent launch: it prefetches its weights
 //     while the gate/up kernel still runs, and it folds the fixed-order combine in: the last CTA
 //     to finish a (token, column tile) sums the k pair rows in order j = 0..k-1 (no spin wait).
-//   otherwise: the grouping kernels' global plan is used and a separate combine kernel follows.
+//   PAIR (T*k <= kPairMaxPairs, one wave): no grouping at all; see pair_gateup_kernel / token_down_kernel.
+// Larger batches run on the streaming kernels (stream.cu) or the tensor-core kernels (prefill.cu) with the
+// grouping kernels' global plan and the separate combine kernel defined here.
 #include "common.cuh"
+#include "frag.cuh"
 
 namespace exmoe {
 
@@ -49,30 +52,6 @@ __device__ __forceinline__ float ldg_early_f32(const void* p) {
     asm volatile("ld.global.f32 %0, [%1];" : "=f"(v) : "l"(p));
     return v;
 }
-__device__ __forceinline__ void mma_m16n8k16(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
-                                             uint32_t b0, uint32_t b1) {
-    asm("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
-        : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
-        : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
-}
-// two offset-binary nibbles (bits s..s+3 of each 16-bit half) -> bf16x2 of 128 + u = 136 + q:
-// 0x4300 | u is that BF16 value exactly (one shift and one lop3 per pair of codes).
-__device__ __forceinline__ uint32_t code_pair(uint32_t w, int s) {
-    uint32_t r;
-    asm("lop3.b32 %0, %1, 0x000f000f, 0x43004300, 0xea;" : "=r"(r) : "r"(w >> s));   // (a & b) | c
-    return r;
-}
-// sum of the 8 BF16 values of a 16-byte chunk, in binary32
-__device__ __forceinline__ float sum8_bf16(const uint4& v) {
-    const uint32_t r[4] = {v.x, v.y, v.z, v.w};
-    float s = 0.f;
-#pragma unroll
-    for (int i = 0; i < 4; ++i) s += __uint_as_float(r[i] << 16) + __uint_as_float(r[i] & 0xffff0000u);
-    return s;
-}
-__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
-__device__ __forceinline__ void grid_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
-
 // Shared-memory plan of ONE wave, rebuilt by every CTA of the SMALL kernels.
 struct SmallPlan {
     int* cnt;     // [C] pairs per slot in this wave
@@ -717,175 +696,6 @@ void launch_pair_gateup(const GemmArgs& a, const SmallArgs& sa, const __nv_bfloa
     count_launch();
 }
 
-// Lean grouped kernel for the middle regime (a few to a few dozen rows per expert; 40 < T*k <= kLeanMaxPairs):
-// one CTA per (active group, tile), straight-line arithmetic, weights loaded once into registers and reused for
-// every 8*NCH-row pass over the group's rows.  Groups come from the grouping kernel's global plan; the down
-// kernel writes the fp32 pair buffer and combine_kernel adds the pairs in fixed order.  Same arithmetic and
-// summation order as the other register-dequant kernels.
-template <int NB, int NCH, bool GATEUP>
-__global__ void __launch_bounds__(256, 2)
-lean_group_kernel(GemmArgs a, const __nv_bfloat16* __restrict__ x_src, __nv_bfloat16* __restrict__ act_out,
-                  const float* __restrict__ topk_w, float* __restrict__ y_out, int KS) {
-    constexpr int NM = GATEUP ? 2 : 1;
-    extern __shared__ __align__(16) unsigned char smem[];
-    const int K = GATEUP ? a.H : a.I, NR = GATEUP ? a.I : a.H;
-    const int KB = K / kGroup, PP = 8 / KS;
-    const int tiles = NR / (kPanelRows * PP);
-    const int g0 = a.wave_start[0], n_groups = a.wave_start[1] - g0;
-    if ((int)blockIdx.x >= n_groups * tiles) return;
-    const int x_stride = K * 2 + 64;
-    unsigned char* xs = smem;                                                    // [8*NCH][x_stride]
-    float* red = reinterpret_cast<float*>(smem + (size_t)8 * NCH * x_stride);    // [KS-1][PP][NM][NCH][32][4]
-    float* adj = red + (size_t)(KS - 1) * PP * NM * NCH * 128;                   // [KB][8*NCH]
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int q = lane >> 2, c = lane & 3;
-    const int ks = warp % KS, pp = warp / KS;
-    const int key = a.group_keys[g0 + blockIdx.x / tiles], tile = blockIdx.x % tiles;
-    const int slot = key % a.num_slots;
-    const int m_rows = a.counts[key], row0 = a.offsets[key];
-    const int panel = tile * PP + pp;
-    const uint8_t* wbase = a.slots + (size_t)slot * a.slot_stride + (GATEUP ? 0 : matrix_bytes(2 * a.I, a.H));
-    uint4 wreg[NM][NB][2];
-    uint32_t sreg[NM][NB];
-#pragma unroll
-    for (int m = 0; m < NM; ++m)
-#pragma unroll
-        for (int b = 0; b < NB; ++b) {
-            const uint8_t* blk = wbase + ((size_t)(GATEUP ? 2 * panel + m : panel) * KB + ks * NB + b) * kBlockBytes;
-            wreg[m][b][0] = ldg_stream128(blk + lane * 16);
-            wreg[m][b][1] = ldg_stream128(blk + 512 + lane * 16);
-            sreg[m][b] = ldg_stream32(blk + kCodeBytes + q * 4);
-        }
-    for (int pass0 = 0; pass0 < m_rows; pass0 += 8 * NCH) {
-        const int rows_here = min(8 * NCH, m_rows - pass0);
-        __syncthreads();                                                         // previous pass is done with xs / red
-        const int chunks_per_row = K / 8, total = rows_here * chunks_per_row;
-        for (int base = warp * 32; base < total; base += 256) {
-            const int idx = base + lane;
-            const int n = idx / chunks_per_row, ck = idx % chunks_per_row;
-            uint4 v = make_uint4(0, 0, 0, 0);
-            if (idx < total) {
-                const size_t src_row = GATEUP ? (size_t)(a.perm[row0 + pass0 + n] / a.top_k) : (size_t)(row0 + pass0 + n);
-                v = *reinterpret_cast<const uint4*>(x_src + src_row * K + ck * 8);
-                *reinterpret_cast<uint4*>(xs + (size_t)n * x_stride + ck * 16) = v;
-            }
-            float sx = sum8_bf16(v);
-#pragma unroll
-            for (int m = 8; m >= 1; m >>= 1) sx += __shfl_xor_sync(0xffffffffu, sx, m);
-            if (idx < total && (ck & 15) == 0) adj[(ck >> 4) * (8 * NCH) + n] = -136.f * sx;
-        }
-        __syncthreads();
-        float tot[NM][NCH][4];
-#pragma unroll
-        for (int m = 0; m < NM; ++m)
-#pragma unroll
-            for (int ch = 0; ch < NCH; ++ch)
-#pragma unroll
-                for (int i = 0; i < 4; ++i) tot[m][ch][i] = 0.f;
-#pragma unroll
-        for (int b = 0; b < NB; ++b) {
-            float acc[NM][NCH][4];
-#pragma unroll
-            for (int m = 0; m < NM; ++m)
-#pragma unroll
-                for (int ch = 0; ch < NCH; ++ch)
-#pragma unroll
-                    for (int i = 0; i < 4; ++i) acc[m][ch][i] = 0.f;
-#pragma unroll
-            for (int h = 0; h < 2; ++h)
-#pragma unroll
-                for (int set = 0; set < 2; ++set) {
-                    const int k0 = (ks * NB + b) * kGroup + 64 * h + 32 * set + 8 * c;
-                    uint4 xb[NCH];
-#pragma unroll
-                    for (int ch = 0; ch < NCH; ++ch) {
-                        xb[ch] = make_uint4(0, 0, 0, 0);
-                        if (8 * ch + q < rows_here) xb[ch] = *reinterpret_cast<const uint4*>(xs + (size_t)(8 * ch + q) * x_stride + k0 * 2);
-                    }
-#pragma unroll
-                    for (int m = 0; m < NM; ++m) {
-                        const uint32_t wq = set ? wreg[m][b][h].z : wreg[m][b][h].x;
-                        const uint32_t wq8 = set ? wreg[m][b][h].w : wreg[m][b][h].y;
-                        uint32_t a0 = code_pair(wq, 0), a1 = code_pair(wq8, 0), a2 = code_pair(wq, 4), a3 = code_pair(wq8, 4);
-#pragma unroll
-                        for (int ch = 0; ch < NCH; ++ch) mma_m16n8k16(acc[m][ch], a0, a1, a2, a3, xb[ch].x, xb[ch].y);
-                        a0 = code_pair(wq, 8), a1 = code_pair(wq8, 8), a2 = code_pair(wq, 12), a3 = code_pair(wq8, 12);
-#pragma unroll
-                        for (int ch = 0; ch < NCH; ++ch) mma_m16n8k16(acc[m][ch], a0, a1, a2, a3, xb[ch].z, xb[ch].w);
-                    }
-                }
-            float2 cr[NCH];
-#pragma unroll
-            for (int ch = 0; ch < NCH; ++ch)
-                cr[ch] = *reinterpret_cast<const float2*>(adj + (size_t)(ks * NB + b) * (8 * NCH) + 8 * ch + 2 * c);
-#pragma unroll
-            for (int m = 0; m < NM; ++m) {
-                const __half2 sc = *reinterpret_cast<const __half2*>(&sreg[m][b]);
-                const float s_lo = __low2float(sc), s_hi = __high2float(sc);
-#pragma unroll
-                for (int ch = 0; ch < NCH; ++ch) {
-                    tot[m][ch][0] = fmaf(s_lo, acc[m][ch][0] + cr[ch].x, tot[m][ch][0]);
-                    tot[m][ch][1] = fmaf(s_lo, acc[m][ch][1] + cr[ch].y, tot[m][ch][1]);
-                    tot[m][ch][2] = fmaf(s_hi, acc[m][ch][2] + cr[ch].x, tot[m][ch][2]);
-                    tot[m][ch][3] = fmaf(s_hi, acc[m][ch][3] + cr[ch].y, tot[m][ch][3]);
-                }
-            }
-        }
-        if (ks > 0) {
-#pragma unroll
-            for (int m = 0; m < NM; ++m)
-#pragma unroll
-                for (int ch = 0; ch < NCH; ++ch)
-                    *reinterpret_cast<float4*>(red + ((((size_t)(ks - 1) * PP + pp) * NM + m) * NCH + ch) * 128 + lane * 4) =
-                        make_float4(tot[m][ch][0], tot[m][ch][1], tot[m][ch][2], tot[m][ch][3]);
-        }
-        __syncthreads();
-        if (ks == 0) {
-            for (int s = 1; s < KS; ++s)
-#pragma unroll
-                for (int m = 0; m < NM; ++m)
-#pragma unroll
-                    for (int ch = 0; ch < NCH; ++ch) {
-                        const float4 v = *reinterpret_cast<const float4*>(
-                            red + ((((size_t)(s - 1) * PP + pp) * NM + m) * NCH + ch) * 128 + lane * 4);
-                        tot[m][ch][0] += v.x; tot[m][ch][1] += v.y; tot[m][ch][2] += v.z; tot[m][ch][3] += v.w;
-                    }
-#pragma unroll
-            for (int ch = 0; ch < NCH; ++ch)
-#pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                    const int n = pass0 + 8 * ch + 2 * c + (i & 1);
-                    if (n >= m_rows) continue;
-                    const int orow = panel * kPanelRows + q + 8 * (i >> 1);
-                    if (GATEUP) {
-                        const float g = tot[0][ch][i], u = tot[NM - 1][ch][i];
-                        act_out[(size_t)(row0 + n) * a.I + orow] = __float2bfloat16_rn(g / (1.f + __expf(-g)) * u);
-                    } else {
-                        const int pair = a.perm[row0 + n];
-                        y_out[(size_t)pair * a.H + orow] = topk_w[pair] * tot[0][ch][i];
-                    }
-                }
-        }
-    }
-}
-
-template <int NB, int NCH, bool GATEUP>
-void launch_lean_cfg(const GemmArgs& a, const __nv_bfloat16* x, __nv_bfloat16* act, const float* w, float* y, int KS,
-                     int max_groups, cudaStream_t st) {
-    constexpr int NM = GATEUP ? 2 : 1;
-    const int K = GATEUP ? a.H : a.I, NR = GATEUP ? a.I : a.H;
-    const int PP = 8 / KS, tiles = NR / (kPanelRows * PP);
-    const size_t smem = (size_t)8 * NCH * (K * 2 + 64) + (size_t)(KS - 1) * PP * NM * NCH * 128 * 4 + (size_t)(K / kGroup) * 8 * NCH * 4;
-    auto kern = lean_group_kernel<NB, NCH, GATEUP>;
-    static bool attr_done = false;
-    if (!attr_done) {
-        cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 110 * 1024);
-        attr_done = true;
-    }
-    kern<<<max_groups * tiles, 256, smem, st>>>(a, x, act, w, y, KS);
-    count_launch();
-}
-
 // K split over KS warps (KS in {1,2,4,8}, 8/KS panels per CTA) and register depth NB; aims at
 // four blocks per warp so that all of a warp's weights are in flight at once.
 struct DecodeCfg { int NB, KS, bpw; };
@@ -988,33 +798,6 @@ combine_kernel(const float* __restrict__ y, const int32_t* __restrict__ ids, int
 }
 
 }  // namespace
-
-// Middle regime: lean register-dequant kernels on the global plan.  Returns false when the shape needs the generic body.
-bool launch_lean_wave(const GemmArgs& a, const __nv_bfloat16* hidden, __nv_bfloat16* act, const float* topk_w, float* y,
-                      int max_rows, int max_groups, bool gateup, bool down, cudaStream_t st) {
-    DecodeCfg cg = pick_cfg(a.H, a.I);
-    const DecodeCfg cd = pick_cfg(a.I, a.H);
-    const int kbg = a.H / kGroup;
-    if (kbg % 8 == 0 && kbg / 8 <= 2) cg = {kbg / 8, 8, kbg / 8};   // gate/up holds two matrices: fewer blocks per warp keep it in registers
-    if (cg.bpw != 4 && cg.bpw != 2 && cg.bpw != 1) return false;
-    if (cd.bpw != 4 && cd.bpw != 2 && cd.bpw != 1) return false;
-    const int nch = max_rows <= 8 ? 1 : 2;
-#define EXMOE_LEAN(NBv, GU, cfg, xin)                                                                            \
-    if (nch == 1) launch_lean_cfg<NBv, 1, GU>(a, xin, act, topk_w, y, cfg.KS, max_groups, st);                   \
-    else launch_lean_cfg<NBv, 2, GU>(a, xin, act, topk_w, y, cfg.KS, max_groups, st);
-    if (gateup) {
-        if (cg.bpw == 4) { EXMOE_LEAN(4, true, cg, hidden) }
-        else if (cg.bpw == 2) { EXMOE_LEAN(2, true, cg, hidden) }
-        else { EXMOE_LEAN(1, true, cg, hidden) }
-    }
-    if (down) {
-        if (cd.bpw == 4) { EXMOE_LEAN(4, false, cd, act) }
-        else if (cd.bpw == 2) { EXMOE_LEAN(2, false, cd, act) }
-        else { EXMOE_LEAN(1, false, cd, act) }
-    }
-#undef EXMOE_LEAN
-    return true;
-}
 
 void launch_combine(const float* y, const int32_t* ids, int E, int T, int k, int H, __nv_bfloat16* out,
                     cudaStream_t st) {

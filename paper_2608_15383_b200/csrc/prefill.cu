@@ -172,12 +172,6 @@ __device__ __forceinline__ uint32_t ldg_stream32(const void* p) {
     asm volatile("ld.global.nc.L1::no_allocate.u32 %0, [%1];" : "=r"(v) : "l"(p));
     return v;
 }
-__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src, int src_bytes) {
-    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(src_bytes) : "memory");
-}
-__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
-template <int N>
-__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
 
 // The FP16 group scale s is split exactly into two BF16 numbers, s = hi + lo (hi = bf16(s), lo = s - hi has at most
 // four significant bits).  For a code q in [-8, 7]: q*lo is exact in BF16 and fma(q, hi, q*lo) rounds the exact

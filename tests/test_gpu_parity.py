@@ -181,7 +181,7 @@ def test_mid_shape_ragged_groups(B, mid_layer, T):
     cache2.close()
 
 
-@pytest.mark.parametrize("T", [1, 7, 16, 30, 90, 300])
+@pytest.mark.parametrize("T", [1, 7, 16, 30, 90, 400])
 def test_odd_block_counts(B, T):
     """d_model = 3 * 128 and d_ff = 5 * 128: block counts that are not powers of two take the generic kernel
     bodies (no K split, one block per step) on every path; 3 experts per token, ragged groups."""
@@ -191,10 +191,10 @@ def test_odd_block_counts(B, T):
     ora, bank = test_odd_block_counts.layer
     hidden, ids, p = helpers.routed_inputs(s, T, seed=4100 + T, alpha=1.0)
     y, ref = ora.forward(hidden, ids, p)
-    cache = B.Cache(s, [bank], s.num_experts, max_tokens=300)
+    cache = B.Cache(s, [bank], s.num_experts, max_tokens=400)
     out = cache.forward(0, hidden.cuda(), ids.cuda(), p.cuda())
     helpers.check_output(out, y, ref, f"T={T}")
-    cache2 = B.Cache(s, [bank], 4, max_tokens=300, wave_cap=3)          # several waves, misses
+    cache2 = B.Cache(s, [bank], 4, max_tokens=400, wave_cap=3)          # several waves, misses
     sc = ocache.SlotCache(s.num_experts, 4, 3, bytes_per_expert=cache2.bytes_per_expert)
     out2 = cache2.forward(0, hidden.cuda(), ids.cuda(), p.cuda())
     compare_plan(cache2, sc, ids)

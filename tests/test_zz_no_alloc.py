@@ -3,8 +3,9 @@
 The entry point serves callers that cannot allocate device memory when they need the layer (a serving loop
 whose memory was handed to a pool at start-up, a plug-in under a framework that owns the allocator, code that
 must avoid the device-wide synchronisation of cudaMalloc/cudaFree): its scratch is a fixed `__device__` array
-inside the library.  It runs the same kernels as the cache-based entry point, so the outputs must agree; the
-test also holds both to the oracle-derived tolerance used everywhere else.  Two calls in a row check that the
+inside the library.  Up to 24 token-expert pairs it runs the same kernels as the cache-based entry point, so the
+outputs must agree bit for bit; above that the cache-based entry point takes its streaming kernels and the two
+agree within the oracle-derived tolerance used everywhere else, which the test holds both to in every case.  Two calls in a row check that the
 contents the shared scratch keeps from the first call do not leak into the second.
 Collected last (file name) so that a run stopping at the first failure has already run every other test.
 """
@@ -35,7 +36,7 @@ def close(a, b):
     assert np.linalg.norm(err) <= helpers.REL_FRO * max(np.linalg.norm(b), 1e-30)
 
 
-@pytest.mark.parametrize("shape,T", [(synth.TINY, 3), (synth.OLMOE, 1), (synth.OLMOE, 4)])
+@pytest.mark.parametrize("shape,T", [(synth.TINY, 3), (synth.OLMOE, 1), (synth.OLMOE, 3), (synth.OLMOE, 4)])
 def test_static_forward_matches_cache_forward_twice(B, shape, T):
     ora, bank = helpers.make_layer(shape, seed=4242)
     experts = bank.cuda()                                  # fully resident layer: expert e at e * bytes_per_expert
@@ -51,7 +52,8 @@ def test_static_forward_matches_cache_forward_twice(B, shape, T):
         got = B.exmoe_moe_forward_static(shape, experts, h, i, w, out)
         torch.cuda.synchronize()
         close(got, ref)
-        assert torch.equal(got.view(torch.int16), ref.view(torch.int16))      # same kernels, same order: same bits
+        if T * shape.top_k <= 24:                          # same kernels, same order: same bits
+            assert torch.equal(got.view(torch.int16), ref.view(torch.int16))
         if shape is synth.TINY or call == 0:
             y, o = ora.forward(hidden, ids, p)
             helpers.check_output(got, y, o, f"static T={T} call={call}")
