@@ -184,7 +184,7 @@ stream_gemm_kernel(const StreamArgs p) {
     constexpr int NM = GATEUP ? 2 : 1;                                // matrices per tile
     constexpr int MS = NM / NMW;                                      // warps a panel's matrices are split over
     constexpr int R = 8 * NCH;
-    constexpr int CHN = (NMW * NCH >= 4) ? 1 : (NMW * NCH == 2 ? 2 : 4);   // accumulator chains per (matrix, chunk): 4 in all
+    constexpr int CHN = (NMW * NCH >= 2) ? 1 : 2;                          // accumulator chains per (matrix, chunk): two independent MMA chains per warp at least
     extern __shared__ __align__(128) unsigned char smem[];
     const GemmArgs& a = p.a;
     const int K = GATEUP ? a.H : a.I, NR = GATEUP ? a.I : a.H;
@@ -401,6 +401,12 @@ stream_gemm_kernel(const StreamArgs p) {
                     for (int m = 8; m >= 1; m >>= 1) sx += __shfl_xor_sync(0xffffffffu, sx, m);
                     if (idx < total && (ck & 15) == 0) adjb[(ck >> 4) * R + nn] = -136.f * sx;
                 }
+                // rows beyond the group's last are zeroed once per staging (both consumer groups write the same zeros:
+                // each reads them only after its own barrier below; no copy targets these rows until every warp
+                // has released the buffer), so the fragment loads of the MMA loop need no row predicate
+                for (int idx = total + cw * 32 + lane; idx < R * chunks_per_row; idx += kGroupThreads)
+                        *reinterpret_cast<uint4*>(const_cast<unsigned char*>(xbuf) + (size_t)(idx / chunks_per_row) * p.x_stride +
+                                                  (idx % chunks_per_row) * 16) = make_uint4(0, 0, 0, 0);
                 group_sync(grp);
             }
             SPROF(long long c1 = clock64(); t_x += c1 - c0;)
@@ -453,9 +459,7 @@ stream_gemm_kernel(const StreamArgs p) {
                         uint4 xv[NCH];
 #pragma unroll
                         for (int ch = 0; ch < NCH; ++ch) {
-                            xv[ch] = make_uint4(0, 0, 0, 0);
-                            if (8 * ch + q < rows_here)
-                                xv[ch] = *reinterpret_cast<const uint4*>(xbuf + (size_t)(8 * ch + q) * p.x_stride + k0 * 2);
+                            xv[ch] = *reinterpret_cast<const uint4*>(xbuf + (size_t)(8 * ch + q) * p.x_stride + k0 * 2);
                         }
 #pragma unroll
                         for (int m = 0; m < NMW; ++m) {
