@@ -781,6 +781,7 @@ combine_kernel(const float* __restrict__ y, const int32_t* __restrict__ ids, int
                __nv_bfloat16* __restrict__ out) {
     const int per_row = H / 4;
     const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    grid_dependency_wait();                            // launched as a programmatic dependent of the down kernel
     if (idx >= (long long)T * per_row) return;
     const int t = (int)(idx / per_row), h4 = (int)(idx % per_row);
     float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -802,7 +803,19 @@ combine_kernel(const float* __restrict__ y, const int32_t* __restrict__ ids, int
 void launch_combine(const float* y, const int32_t* ids, int E, int T, int k, int H, __nv_bfloat16* out,
                     cudaStream_t st) {
     const long long n = (long long)T * (H / 4);
-    combine_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(y, ids, E, T, k, H, out);
+    cudaLaunchConfig_t lc{};
+    lc.gridDim = dim3((unsigned)((n + 255) / 256));
+    lc.blockDim = dim3(256);
+    lc.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    lc.attrs = attr;
+    lc.numAttrs = 1;
+#ifdef EXMOE_DISABLE_PDL
+    lc.numAttrs = 0;
+#endif
+    cudaLaunchKernelEx(&lc, combine_kernel, y, ids, E, T, k, H, out);
     count_launch();
 }
 

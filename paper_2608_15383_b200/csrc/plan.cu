@@ -211,6 +211,9 @@ group_small_kernel(const int32_t* __restrict__ ids, int n_pairs, int E, int C, i
     int* s_key = s_off + n_keys + 1;       // [n_pairs]
     __shared__ int s_bad;
     const int tid = threadIdx.x;
+    // a kernel launched behind this one as a programmatic dependent may be placed now; it waits for this grid's
+    // completion before it reads the plan
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     if (tid == 0) s_bad = 0;
     for (int i = tid; i < n_keys; i += blockDim.x) s_cnt[i] = 0;
     __syncthreads();

@@ -216,6 +216,12 @@ stream_gemm_kernel(const StreamArgs p) {
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
+#ifndef EXMOE_STREAM_NO_ENTRY_PDL
+    // The gate/up kernel is itself launched as a programmatic dependent (of the grouping kernel when that runs
+    // just before it): its CTAs are placed and their barriers initialised while the plan is still being
+    // written; the plan is read only after this wait.
+    if (GATEUP) grid_dependency_wait();
+#endif
     if (warp == 0) {
         // This CTA's share of the wave's units, and the plan entries of the groups it touches (usually one or
         // two).  The plan entries of up to 32 * kScanChunks active groups are fetched in one go and kept in
@@ -295,7 +301,8 @@ stream_gemm_kernel(const StreamArgs p) {
         }
     }
     __syncthreads();
-    if (GATEUP) grid_launch_dependents();              // the down kernel may start filling its weight ring
+    grid_launch_dependents();                          // gate/up: the down kernel may start filling its weight ring; down: the
+                                                       // combine kernel may be placed (it waits for this grid before it reads)
     const int u0 = s_range[0], u1 = s_range[1];
     const size_t mat_off = GATEUP ? 0 : matrix_bytes(2 * a.I, a.H);
     Cursor cur{0, 0, 0};
@@ -636,7 +643,12 @@ bool stream_supported(int H, int I) {
 bool launch_stream_wave(const GemmArgs& a, const __nv_bfloat16* hidden, __nv_bfloat16* act, const float* topk_w, float* y,
                         int* status, int max_groups, bool gateup, bool down, cudaStream_t st) {
     bool ok = true;
-    if (gateup) ok = launch_stream_cfg<1, true>(a, hidden, act, topk_w, y, status, max_groups, false, st);
+#ifndef EXMOE_STREAM_NO_ENTRY_PDL
+    const bool entry_dependent = true;
+#else
+    const bool entry_dependent = false;
+#endif
+    if (gateup) ok = launch_stream_cfg<1, true>(a, hidden, act, topk_w, y, status, max_groups, entry_dependent, st);
     // a programmatic dependent only when the gate/up kernel of the same wave was launched just before it
     if (down && ok) ok = launch_stream_cfg<1, false>(a, act, act, topk_w, y, status, max_groups, gateup, st);
     return ok;
