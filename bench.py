@@ -40,8 +40,9 @@ WORKLOADS = {
     "prefill": (2048, 64, 1, 0.0, "config4: OLMoE-shaped prefill, T=2048, 64 slots resident, uniform routing"),
 }
 # DRAM bytes (read + write) per launch of the dominant kernel, from the committed ncu captures under profiles/
-# (decode: profiles/decode_t1_c64_pair_kernels_ncu_full.md; prefill: profiles/prefill_t2048_c64_tcgen05_ncu_full.md)
-NCU_TRAFFIC_BYTES = {"decode": 17.33e6, "prefill": 214.68e6 + 12.51e6}
+# (decode: profiles/decode_t1_c64_pair_kernels_ncu_full.md; decode16: profiles/decode16_t16_c64_stream_kernels_ncu_full.md;
+# prefill: profiles/prefill_t2048_c64_tcgen05_ncu_full.md)
+NCU_TRAFFIC_BYTES = {"decode": 17.33e6, "decode16": 62.83e6 + 0.87e6, "prefill": 214.68e6 + 12.51e6}
 METRIC = "moe_layer_tokens_per_s"
 UNIT = "tokens/s"
 
