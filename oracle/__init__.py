@@ -14,6 +14,7 @@ Modules (each function cites the passage of the paper it follows):
   moe.py     Sparse block output, per token over its selected experts (Eq. 2).
   cache.py   Slot cache: global-expert -> slot map, LRU, waves, expert map with
              sentinel, token grouping (Sections 3.3 and 3.4).
+  router.py  Router logits, softmax over all experts, top-k with ties to the lower id (Eq. 1).
 
 Pins (tests/test_oracle_*.py, run without a GPU) hold every function to
 something other than itself: closed forms, invariants, brute force on tiny
