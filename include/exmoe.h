@@ -117,6 +117,17 @@ int exmoe_cache_create(exmoe_cache** out, const exmoe_shape* shape, int num_laye
 int exmoe_moe_forward(exmoe_cache* cache, int layer, const void* hidden_bf16, const int32_t* topk_ids,
                       const float* topk_weights, int T, void* out_bf16, void* stream);
 
+/* Router of one sparse block (Eq. 1; Sec. 3.4 "router weights are ... not renormalized"): logits z_t = W_r h_t in
+ * binary32 (BF16 products, fixed summation order), plus `bias` if given, softmax over all E experts, the k
+ * largest, equal values ordered by ascending expert id.  Writes exmoe_moe_forward's inputs on the device.
+ *   hidden_bf16  : dev, BF16 [T, H], 16-byte aligned     router_bf16 : dev, BF16 [E, H], 16-byte aligned
+ *   bias         : dev, float32 [E], or NULL
+ *   topk_ids     : dev, int32 [T, k], descending probability     topk_weights : dev, float32 [T, k]
+ * Uses shape->d_model (a multiple of 8), num_experts (<= 4096) and top_k; asynchronous on `stream`;
+ * allocates nothing; T = 0 is a no-op.  EXMOE_ERR_SHAPE / EXMOE_ERR_ARG before any work is queued. */
+int exmoe_route(const exmoe_shape* shape, const void* hidden_bf16, const void* router_bf16, const float* bias,
+                int T, int32_t* topk_ids, float* topk_weights, void* stream);
+
 /* Tiny-batch forward that allocates nothing and needs no cache object (the paper has no counterpart: this
  * is a service for one kind of caller, not a step of the method).
  *

@@ -48,6 +48,7 @@ _SIGNATURES = {
                                    c_void_p, c_int, c_int]),
     "exmoe_moe_forward": (c_int, [c_void_p, c_int, c_void_p, c_void_p, c_void_p, c_int, c_void_p, c_void_p]),
     "exmoe_moe_forward_static": (c_int, [POINTER(exmoe_shape), c_void_p, c_void_p, c_void_p, c_void_p, c_int, c_void_p, c_void_p]),
+    "exmoe_route": (c_int, [POINTER(exmoe_shape), c_void_p, c_void_p, c_void_p, c_int, c_void_p, c_void_p, c_void_p]),
     "exmoe_cache_get_state": (c_int, [c_void_p, c_int, c_void_p, c_void_p, c_void_p, c_void_p]),
     "exmoe_debug_last_plan": (c_int, [c_void_p, c_int] + [c_void_p] * 9),
     "exmoe_debug_read_slot": (c_int, [c_void_p, c_int, c_int, c_void_p]),
@@ -143,6 +144,22 @@ def exmoe_moe_forward_static(shape, experts_dev, hidden, topk_ids, topk_weights,
                                         _dev(out, torch.bfloat16, "out"), _stream_ptr(stream))
     _check(rc, "exmoe_moe_forward_static")
     return out
+
+
+def exmoe_route(shape, hidden, w_router, bias=None, topk_ids=None, topk_weights=None, stream=None):
+    """Eq. 1 on the device: logits, softmax over all experts, top-k.  Returns (ids int32 [T, k], weights fp32 [T, k])."""
+    T = int(hidden.shape[0])
+    if topk_ids is None:
+        topk_ids = torch.empty((T, shape.top_k), dtype=torch.int32, device=hidden.device)
+    if topk_weights is None:
+        topk_weights = torch.empty((T, shape.top_k), dtype=torch.float32, device=hidden.device)
+    rc = lib().exmoe_route(byref(_shape(shape)), _dev(hidden, torch.bfloat16, "hidden"),
+                           _dev(w_router, torch.bfloat16, "w_router"),
+                           _dev(bias, torch.float32, "bias") if bias is not None else None, T,
+                           _dev(topk_ids, torch.int32, "topk_ids"), _dev(topk_weights, torch.float32, "topk_weights"),
+                           _stream_ptr(stream))
+    _check(rc, "exmoe_route")
+    return topk_ids, topk_weights
 
 
 def exmoe_launch_count():
