@@ -29,6 +29,7 @@
 #include <cuda.h>
 
 #include "common.cuh"
+#include "mbar.cuh"
 #ifdef EXMOE_PREFILL_PROF
 #include <cstdio>
 #endif
@@ -51,28 +52,9 @@ constexpr int B_HALF_BYTES = BN * 128;         // 32 KB
 constexpr int B_STAGE_BYTES = 2 * B_HALF_BYTES;
 constexpr int B_SBO = 1024;
 constexpr int NUM_THREADS = 896;   // 28 warps: MMA, TMA, 2 idle, 4 + 4 epilogue, 8 + 8 dequant
-constexpr long long kWaitBudget = 2000000000ll;   // clock64 ticks (~1 s) before a wait gives up
 
 struct Tile { int key, n0, nrows, pad; };
 
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-__device__ __forceinline__ void mbar_init(uint64_t* bar, int count) {
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
-}
-__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
-}
-__device__ __forceinline__ bool mbar_try(uint64_t* bar, uint32_t parity) {
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok)
-        : "r"(smem_u32(bar)), "r"(parity)
-        : "memory");
-    return ok != 0;
-}
 #ifdef EXMOE_PREFILL_PROF
 #define PROF_DECL long long prof_t0 = clock64(), prof_wait = 0
 #define PROF_WAIT_BEGIN long long prof_w0 = clock64()
@@ -85,24 +67,6 @@ __device__ __forceinline__ bool mbar_try(uint64_t* bar, uint32_t parity) {
 #define PROF_REPORT(name)
 #endif
 
-// bounded wait; returns false when the CTA is aborting (and raises the abort on expiry)
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag, int* status,
-                                          long long budget = kWaitBudget) {
-    if (mbar_try(bar, parity)) return true;
-    const long long t0 = clock64();
-    unsigned polls = 0;
-    while (!mbar_try(bar, parity)) {
-        if ((++polls & 15u) == 0) {                    // the bookkeeping of the bound is amortised over 16 polls
-            if (*abort_flag) return false;
-            if (clock64() - t0 > budget) {
-                *abort_flag = 1;
-                atomicExch(status, EXMOE_ERR_TIMEOUT);
-                return false;
-            }
-        }
-    }
-    return true;
-}
 __device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
@@ -146,9 +110,6 @@ __device__ __forceinline__ uint64_t make_desc_b(uint32_t saddr) {            // 
     d |= (uint64_t)1 << 46;
     d |= (uint64_t)2 << 61;
     return d;
-}
-__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
 }
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint64_t* bar) {
     asm volatile(

@@ -23,6 +23,7 @@
 // loops and the producers wait (bounded) for their copies in flight before the CTA exits.
 #include "common.cuh"
 #include "frag.cuh"
+#include "mbar.cuh"
 #ifdef EXMOE_STREAM_PROF
 #include <cstdio>
 #define SPROF(...) __VA_ARGS__
@@ -40,49 +41,10 @@ constexpr int kGroups = 2;                           // consumer groups, alterna
 constexpr int kConsumerWarps = kGroups * kGroupWarps;
 constexpr int kStreamThreads = 32 * (kConsumerWarps + 2);
 constexpr int kMaxStages = 8;
-constexpr long long kWaitBudget = 2000000000ll;      // clock64 ticks (~1 s) before a wait gives up
 constexpr size_t kSmemLimit = 227 * 1024;
 constexpr int kScanChunks = 4;                       // chunks of 32 groups whose plan entries the scan keeps in registers
 constexpr int kMetaGroups = 64;                      // most groups one CTA's share of the units can touch (see stream_geometry)
 
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-__device__ __forceinline__ void mbar_init(uint64_t* bar, int count) {
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
-}
-__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
-}
-__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ bool mbar_try(uint64_t* bar, uint32_t parity) {
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok)
-        : "r"(smem_u32(bar)), "r"(parity)
-        : "memory");
-    return ok != 0;
-}
-// bounded wait; returns false when the CTA is aborting (and raises the abort on expiry)
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag, int* status) {
-    if (mbar_try(bar, parity)) return true;
-    const long long t0 = clock64();
-    unsigned polls = 0;
-    while (!mbar_try(bar, parity)) {
-        if ((++polls & 15u) == 0) {
-            if (*abort_flag) return false;
-            if (clock64() - t0 > kWaitBudget) {
-                *abort_flag = 1;
-                atomicExch(status, EXMOE_ERR_TIMEOUT);
-                return false;
-            }
-        }
-    }
-    return true;
-}
 // one lane waits, the whole warp learns the outcome (the producers' control flow stays warp-uniform)
 __device__ __forceinline__ bool warp_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag, int* status) {
     int ok = 1;

@@ -388,12 +388,15 @@ def test_bounded_wait_expires_and_reports(B, tiny_layer):
     cache.close()
 
 
-def test_graph_replay_matches_oracle(B, olmoe_layer):
-    """The launch configuration bench.py times: fully resident decode steps captured in a CUDA graph and replayed."""
+@pytest.mark.parametrize("T", [1, 8])
+def test_graph_replay_matches_oracle(B, olmoe_layer, T):
+    """The launch configuration bench.py times: fully resident decode steps captured in a CUDA graph and replayed
+    (T = 1: pairwise kernels; T = 8: grouping + streaming kernels + combine, chained by programmatic dependent
+    launches inside the graph)."""
     ora, bank = olmoe_layer
     s = synth.OLMOE
-    cache = B.Cache(s, [bank], 64, max_tokens=4)
-    inputs = [tuple(x.cuda() for x in helpers.routed_inputs(s, 1, seed=8100 + i)) for i in range(6)]
+    cache = B.Cache(s, [bank], 64, max_tokens=8)
+    inputs = [tuple(x.cuda() for x in helpers.routed_inputs(s, T, seed=8100 + i, alpha=1.0)) for i in range(6)]
     outs = [torch.empty_like(inputs[0][0]) for _ in inputs]
     stream = torch.cuda.Stream()
     with torch.cuda.stream(stream):
