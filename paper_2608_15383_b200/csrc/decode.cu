@@ -24,6 +24,7 @@
 // grouping kernels' global plan and the separate combine kernel defined here.
 #include "common.cuh"
 #include "frag.cuh"
+#include "mbar.cuh"
 
 namespace exmoe {
 
@@ -681,6 +682,142 @@ pair_gateup_kernel(GemmArgs a, SmallArgs sa, const __nv_bfloat16* __restrict__ h
     pair_gateup_item<NB>(a, sa, hidden, act_out, KS, blockIdx.x, smem);
 }
 
+// ------------------------------------------------------------------------------------------------
+// Bulk-copy variant of the by-token down kernel, used for two or more tokens.  Each expert warp brings its
+// panel (one contiguous range of the packed image) into SHARED MEMORY with one cp.async.bulk, completion counted
+// in bytes on an mbarrier, instead of into registers: the CTA is light in registers, all of its weight bytes are
+// requested in its first instructions (before the dependency on the gate/up kernel), and the MMA loop reads
+// them back in lane order.  Measured (OLMoE shape): T=2 19.3 us per step against 22.2 us with the register
+// kernel, T=3 27.0 against 31.4; at T=1 the register kernel overlaps the gate/up kernel better (12.9 against
+// 13.9 us) and stays.  A bulk-copy gate/up kernel (two-stage ring, one CTA per SM) measured slower at every
+// size (T=1: 15.0 us per step) and was dropped.  Arithmetic and summation order are those of
+// token_down_kernel (same bits).
+// ------------------------------------------------------------------------------------------------
+__device__ __forceinline__ void bulk_load_g2s(void* dst, const void* src, uint32_t bytes, uint64_t* bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(smem_u32(dst)), "l"(src), "r"(bytes), "r"(smem_u32(bar))
+                 : "memory");
+}
+// after a failed wait: give copies that may still be in flight a bounded time to land before the CTA ends
+__device__ __forceinline__ void drain_bar(uint64_t* bar, uint32_t parity) {
+    const long long t0 = clock64();
+    while (!mbar_try(bar, parity) && clock64() - t0 < kWaitBudget) {}
+}
+
+template <int NBT>
+__global__ void __launch_bounds__(256, 1)
+token_down_bulk_kernel(GemmArgs a, SmallArgs sa, const __nv_bfloat16* __restrict__ act, const float* __restrict__ topk_w,
+                       int bpwg) {
+    extern __shared__ __align__(128) unsigned char smem[];
+    const int K = a.I, KB = K / kGroup, k = a.top_k;                     // k <= 8: one warp per selected expert
+    const uint32_t panel_bytes = (uint32_t)KB * kBlockBytes;
+    const int x_stride = K * 2 + 64;
+    unsigned char* wst = smem;                                           // [k][panel_bytes]
+    unsigned char* xs = smem + (size_t)k * panel_bytes;                  // [k][x_stride]
+    float* ys = reinterpret_cast<float*>(xs + (size_t)k * x_stride);     // [k][16]
+    int* s_valid = reinterpret_cast<int*>(ys + k * 16);                  // [k]
+    float* adj = reinterpret_cast<float*>(s_valid + 8);                  // [KB][k]
+    uint64_t* bar = reinterpret_cast<uint64_t*>(adj + (((size_t)KB * k + 3) & ~(size_t)3));
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(bar + 1);
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int q = lane >> 2, c = lane & 3;
+    const int panels = a.H / kPanelRows;
+    const int t = blockIdx.x / panels, panel = blockIdx.x % panels;
+    if (tid == 0) {
+        mbar_init(bar, k);                                               // one arrival per expert warp
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+    const int j = warp;
+    const int pair = t * k + j;
+    int id = -1;
+    if (j < k) id = sa.ids[pair];
+    const bool valid = (j < k) && id >= 0 && id < sa.E;
+    const float rw = valid ? ldg_early_f32(topk_w + pair) : 0.f;
+    if (j < k && lane == 0) {                                            // the expert's panel: one contiguous range
+        if (valid) {
+            const int slot = sa.slot_of ? sa.slot_of[id] : id;
+            const uint8_t* src = a.slots + (size_t)slot * a.slot_stride + matrix_bytes(2 * a.I, a.H) + (size_t)panel * panel_bytes;
+            mbar_expect_tx(bar, panel_bytes);
+            bulk_load_g2s(wst + (size_t)j * panel_bytes, src, panel_bytes, bar);
+        } else {
+            mbar_arrive(bar);
+        }
+    }
+    grid_dependency_wait();                                              // the gate/up kernel's activations are complete and visible
+    {
+        const int chunks_per_row = K / 8, total = k * chunks_per_row;
+        for (int base = warp * 32; base < total; base += 256) {
+            const int idx = base + lane;
+            const int n = idx / chunks_per_row, ck = idx % chunks_per_row;
+            uint4 v = make_uint4(0, 0, 0, 0);
+            if (idx < total) {
+                v = *reinterpret_cast<const uint4*>(act + (size_t)(t * k + n) * K + ck * 8);
+                *reinterpret_cast<uint4*>(xs + (size_t)n * x_stride + ck * 16) = v;
+            }
+            float sx = sum8_bf16(v);
+#pragma unroll
+            for (int m = 8; m >= 1; m >>= 1) sx += __shfl_xor_sync(0xffffffffu, sx, m);
+            if (idx < total && (ck & 15) == 0) adj[(ck >> 4) * k + n] = -136.f * sx;
+        }
+    }
+    __syncthreads();
+    const bool ok = mbar_wait(bar, 0, abort_flag, sa.status);
+    float result[2] = {0.f, 0.f}, total2[2] = {0.f, 0.f};
+    if (valid) {
+        const unsigned char* mine = wst + (size_t)j * panel_bytes;
+        for (int b0 = 0; b0 < KB; b0 += NBT) {
+#pragma unroll
+            for (int b = 0; b < NBT; ++b) {
+                const unsigned char* blk = mine + (size_t)(b0 + b) * kBlockBytes;
+                const uint4 w0 = *reinterpret_cast<const uint4*>(blk + lane * 16);
+                const uint4 w1 = *reinterpret_cast<const uint4*>(blk + 512 + lane * 16);
+                const uint32_t sv = *reinterpret_cast<const uint32_t*>(blk + kCodeBytes + q * 4);
+                float acc[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+                for (int h = 0; h < 2; ++h)
+#pragma unroll
+                    for (int set = 0; set < 2; ++set) {
+                        const int k0 = (b0 + b) * kGroup + 64 * h + 32 * set + 8 * c;
+                        uint4 xb = make_uint4(0, 0, 0, 0);
+                        if (q == 0) xb = *reinterpret_cast<const uint4*>(xs + (size_t)j * x_stride + k0 * 2);
+                        const uint4& wh = h ? w1 : w0;
+                        const uint32_t wq = set ? wh.z : wh.x;
+                        const uint32_t wq8 = set ? wh.w : wh.y;
+                        mma_m16n8k16(acc, code_pair(wq, 0), code_pair(wq8, 0), code_pair(wq, 4), code_pair(wq8, 4), xb.x, xb.y);
+                        mma_m16n8k16(acc, code_pair(wq, 8), code_pair(wq8, 8), code_pair(wq, 12), code_pair(wq8, 12), xb.z, xb.w);
+                    }
+                const __half2 sc = *reinterpret_cast<const __half2*>(&sv);
+                const float cr = adj[(b0 + b) * k + j];
+                total2[0] = fmaf(__low2float(sc), acc[0] + cr, total2[0]);
+                total2[1] = fmaf(__high2float(sc), acc[2] + cr, total2[1]);
+                if ((b0 + b + 1) % bpwg == 0) {                          // end of one K-split range of the grouped kernel
+                    const bool first = (b0 + b + 1 == bpwg);
+                    result[0] = first ? total2[0] : result[0] + total2[0];
+                    result[1] = first ? total2[1] : result[1] + total2[1];
+                    total2[0] = total2[1] = 0.f;
+                }
+            }
+        }
+    }
+    if (j < k) {
+        if (lane == 0) s_valid[j] = valid ? 1 : 0;
+        if (c == 0) {
+            ys[j * 16 + q] = rw * result[0];
+            ys[j * 16 + q + 8] = rw * result[1];
+        }
+    }
+    __syncthreads();
+    if (tid < 16 && ok) {
+        float sum = 0.f;
+        for (int jj = 0; jj < k; ++jj)
+            if (s_valid[jj]) sum += ys[jj * 16 + tid];
+        sa.out[(size_t)t * a.H + panel * kPanelRows + tid] = __float2bfloat16_rn(sum);
+    }
+    if (!ok && tid == 0) drain_bar(bar, 0);
+}
+
 template <int NB>
 void launch_pair_gateup(const GemmArgs& a, const SmallArgs& sa, const __nv_bfloat16* hidden, __nv_bfloat16* act, int KS,
                         cudaStream_t st) {
@@ -847,6 +984,39 @@ void launch_token_down(const GemmArgs& a, const SmallArgs& sa, const __nv_bfloat
     count_launch();
 }
 
+// false when the shape does not fit the kernel's shared-memory budget (the caller then takes the register variant)
+template <int NBT>
+bool launch_token_down_bulk(const GemmArgs& a, const SmallArgs& sa, const __nv_bfloat16* act, const float* w, int T, int bpwg,
+                            cudaStream_t st) {
+    const int K = a.I, KB = K / kGroup, k = a.top_k;
+    if (k > 8) return false;
+    const size_t smem = (size_t)k * KB * kBlockBytes + (size_t)k * (K * 2 + 64) + (size_t)k * 16 * 4 + 32 +
+                        (((size_t)KB * k + 3) & ~(size_t)3) * 4 + 64;
+    if (smem > 100 * 1024) return false;
+    auto kern = token_down_bulk_kernel<NBT>;
+    static bool attr_done = false;
+    if (!attr_done) {
+        cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 100 * 1024);
+        attr_done = true;
+    }
+    cudaLaunchConfig_t lc{};
+    lc.gridDim = dim3(T * (a.H / kPanelRows));
+    lc.blockDim = dim3(256);
+    lc.dynamicSmemBytes = smem;
+    lc.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    lc.attrs = attr;
+    lc.numAttrs = 1;
+#ifdef EXMOE_DISABLE_PDL
+    lc.numAttrs = 0;
+#endif
+    cudaLaunchKernelEx(&lc, kern, a, sa, act, w, bpwg);
+    count_launch();
+    return true;
+}
+
 // One wave of the SMALL path: gate/up kernel, then the down kernel with the fused combine.
 void launch_small_wave(const GemmArgs& a, const SmallWave& w, cudaStream_t st, bool gateup, bool down) {
     SmallArgs sa{};
@@ -876,7 +1046,17 @@ void launch_small_wave(const GemmArgs& a, const SmallWave& w, cudaStream_t st, b
             const int KB = a.I / kGroup;
             const int bpwg = pick_cfg(a.I, a.H).bpw;    // the grouped kernel's K-split range, replayed for rounding
             const int T = w.n_pairs / a.top_k;
-            if (KB % 8 == 0) launch_token_down<8>(a, sa, w.act, w.topk_w, T, bpwg, st);
+            bool done = false;
+#ifndef EXMOE_NO_BULK_DECODE
+            if (T >= 2) {                               // one token: the register kernel overlaps the gate/up kernel better
+                if (KB % 8 == 0) done = launch_token_down_bulk<8>(a, sa, w.act, w.topk_w, T, bpwg, st);
+                else if (KB % 4 == 0) done = launch_token_down_bulk<4>(a, sa, w.act, w.topk_w, T, bpwg, st);
+                else if (KB % 2 == 0) done = launch_token_down_bulk<2>(a, sa, w.act, w.topk_w, T, bpwg, st);
+                else done = launch_token_down_bulk<1>(a, sa, w.act, w.topk_w, T, bpwg, st);
+            }
+#endif
+            if (done) {}
+            else if (KB % 8 == 0) launch_token_down<8>(a, sa, w.act, w.topk_w, T, bpwg, st);
             else if (KB % 4 == 0) launch_token_down<4>(a, sa, w.act, w.topk_w, T, bpwg, st);
             else if (KB % 2 == 0) launch_token_down<2>(a, sa, w.act, w.topk_w, T, bpwg, st);
             else launch_token_down<1>(a, sa, w.act, w.topk_w, T, bpwg, st);
