@@ -204,6 +204,29 @@ def test_odd_block_counts(B, T):
     cache2.close()
 
 
+@pytest.mark.parametrize("T", [7, 100, 300])
+def test_many_experts_small_dims(B, T):
+    """256 experts of 128 x 128: more active groups than the streaming kernel's scan keeps in registers, one tile per
+    group, several groups per CTA; fully resident and with 64 slots (several waves)."""
+    s = synth.Shape(d_model=128, d_ff=128, num_experts=256, top_k=4)
+    if not hasattr(test_many_experts_small_dims, "layer"):
+        test_many_experts_small_dims.layer = helpers.make_layer(s, seed=321)
+    ora, bank = test_many_experts_small_dims.layer
+    hidden, ids, p = helpers.routed_inputs(s, T, seed=5200 + T, alpha=0.3)
+    y, ref = ora.forward(hidden, ids, p)
+    cache = B.Cache(s, [bank], s.num_experts, max_tokens=300)
+    out = cache.forward(0, hidden.cuda(), ids.cuda(), p.cuda())
+    helpers.check_output(out, y, ref, f"T={T}")
+    cache2 = B.Cache(s, [bank], 64, max_tokens=300, wave_cap=48)
+    sc = ocache.SlotCache(s.num_experts, 64, 48, bytes_per_expert=cache2.bytes_per_expert)
+    out2 = cache2.forward(0, hidden.cuda(), ids.cuda(), p.cuda())
+    compare_plan(cache2, sc, ids)
+    assert torch.equal(out2.view(torch.int16), out.view(torch.int16))
+    assert cache.status() == 0 and cache2.status() == 0
+    cache.close()
+    cache2.close()
+
+
 def test_config2_decode_olmoe(B, olmoe_layer):
     """Config 2: OLMoE shape, 1 token per step, 64 slots, fresh hidden state per step."""
     ora, bank = olmoe_layer
