@@ -106,14 +106,21 @@ bool launch_stream_wave(const GemmArgs& a, const __nv_bfloat16* hidden, __nv_bfl
                         int* status, int max_groups, bool gateup, bool down, cudaStream_t st);
 void launch_small_wave(const GemmArgs& a, const SmallWave& w, cudaStream_t st, bool gateup, bool down);
 size_t prefill_scratch_bytes(int max_pairs, int num_experts);
-struct alignas(64) PrefillMaps { unsigned char x[128], act[128]; };   // two CUtensorMap objects (grouped hidden, activations)
+// CUtensorMap objects of the grouped hidden rows and of the activations: 256-row boxes for the large-N kernel shape,
+// 64-row boxes for the small-N shape
+struct alignas(64) PrefillMaps { unsigned char x[128], act[128], x_small[128], act_small[128]; };
 int prefill_setup(PrefillMaps* maps, const __nv_bfloat16* xg, const __nv_bfloat16* act, int max_pairs, int H, int I);
 void launch_wait_selftest(int* status, long long budget_cycles, int* result, cudaStream_t st);
 void launch_gather_rows(const __nv_bfloat16* hidden, const int32_t* perm, const int32_t* n_valid, int n_pairs, int top_k,
                         int H, __nv_bfloat16* xg, cudaStream_t st);
 // which: bit 0 = gate/up GEMM + SwiGLU, bit 1 = down GEMM x routing weight, bit 2 = (re)build the wave's tile list
+// small_n: the 64-row, four-stage kernel shape (a few dozen rows per expert) instead of the 256-row, two-stage one
 void launch_prefill_wave(const GemmArgs& g, const int32_t* wave_start, void* scratch, int* status, const PrefillMaps* maps,
-                         __nv_bfloat16* act, const float* topk_w, float* y, int which, cudaStream_t st);
+                         __nv_bfloat16* act, const float* topk_w, float* y, int which, bool small_n, cudaStream_t st);
+#ifndef EXMOE_PREFILL_SMALL_N_MAX_PAIRS
+#define EXMOE_PREFILL_SMALL_N_MAX_PAIRS 1024
+#endif
+constexpr int kPrefillSmallNMaxPairs = EXMOE_PREFILL_SMALL_N_MAX_PAIRS;
 void launch_combine(const float* y, const int32_t* ids, int E, int T, int k, int H, __nv_bfloat16* out,
                     cudaStream_t st);
 

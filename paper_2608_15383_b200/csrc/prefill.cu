@@ -39,17 +39,15 @@ namespace exmoe {
 namespace {
 
 constexpr int BM = 128;            // weight rows per tile
-constexpr int BN = 256;            // max grouped rows (tokens) per tile
+constexpr int BN = 256;            // max grouped rows (tokens) per tile of the large-N kernel shape
+constexpr int BN_SMALL = 64;       // ... and of the small-N shape (a few dozen rows per expert: four stages fit)
 constexpr int BK = 128;            // K per stage = one packed block / one scale group
-constexpr int STAGES = 2;
 // A (dequantised weights): no swizzle; core matrix = 8 rows x 16 B; k-chunks 160 B apart (128 + 32 pad, so that
 // the 8 lanes of a quarter warp, 2 rows x 4 k-chunks, hit 8 different 16-byte bank groups), row groups 2560 B apart
 constexpr int A_LBO = 160;
 constexpr int A_SBO = 16 * A_LBO;
 constexpr int A_STAGE_BYTES = 16 * A_SBO;      // 40 KB
 // B (tokens): TMA 128-byte swizzle; two halves of 64 columns, each 256 rows x 128 B; 8-row atoms of 1024 B
-constexpr int B_HALF_BYTES = BN * 128;         // 32 KB
-constexpr int B_STAGE_BYTES = 2 * B_HALF_BYTES;
 constexpr int B_SBO = 1024;
 constexpr int NUM_THREADS = 896;   // 28 warps: MMA, TMA, 2 idle, 4 + 4 epilogue, 8 + 8 dequant
 
@@ -169,20 +167,26 @@ struct PrefillArgs {
     int* status;
 };
 
-template <bool GATEUP>
+// BN_T = token rows per tile (256 or 64), STAGES = ring depth (2 or 4).  The round trip of one stage (MMAs
+// complete -> commit -> dequantisation warps refill -> MMA issuer wakes) is about 2000 cycles whatever the tile
+// holds, so with few rows per expert (tiny MMAs) the ring depth sets the rate: the small-N shape spends the
+// shared memory it saves on the token tile on two more stages.
+template <bool GATEUP, int BN_T, int STAGES>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 prefill_gemm_kernel(PrefillArgs a, const __grid_constant__ CUtensorMap tmap_b, __nv_bfloat16* __restrict__ act_out,
                     const float* __restrict__ topk_w, const int32_t* __restrict__ offsets, float* __restrict__ y_out) {
     extern __shared__ unsigned char smem_raw[];
     unsigned char* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);   // swizzled tiles need 1 KB alignment
-    unsigned char* sB = smem;                                     // [STAGES][64 KB]
+    constexpr int B_HALF_BYTES = BN_T * 128;                      // BN_T rows x 64 columns
+    constexpr int B_STAGE_BYTES = 2 * B_HALF_BYTES;
+    unsigned char* sB = smem;                                     // [STAGES][B_STAGE_BYTES]
     unsigned char* sA = smem + STAGES * B_STAGE_BYTES;            // [STAGES][40 KB]
     uint64_t* bars = reinterpret_cast<uint64_t*>(sA + STAGES * A_STAGE_BYTES);
-    uint64_t* full = bars;              // [STAGES]  producers -> MMA (8 warp arrivals)
-    uint64_t* empty = bars + 2;         // [STAGES]  MMA -> producers (tcgen05.commit)
-    uint64_t* acc_full = bars + 4;      // [2]       MMA -> epilogue
-    uint64_t* acc_empty = bars + 6;     // [2]       epilogue -> MMA (4 warp arrivals)
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 8);
+    uint64_t* full = bars;                          // [STAGES]  producers -> MMA
+    uint64_t* empty = bars + STAGES;                // [STAGES]  MMA -> producers (tcgen05.commit)
+    uint64_t* acc_full = bars + 2 * STAGES;         // [2]       MMA -> epilogue
+    uint64_t* acc_empty = bars + 2 * STAGES + 2;    // [2]       epilogue -> MMA (8 warp arrivals)
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * STAGES + 4);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -231,7 +235,7 @@ prefill_gemm_kernel(PrefillArgs a, const __grid_constant__ CUtensorMap tmap_b, _
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
             tc_fence_after();
-            const uint32_t d_tmem = tmem_base + buf * BN;
+            const uint32_t d_tmem = tmem_base + buf * BN_T;
             for (int kb = 0; kb < KB; ++kb, ++it) {
                 const int s = it % STAGES;
                 {
@@ -277,7 +281,7 @@ prefill_gemm_kernel(PrefillArgs a, const __grid_constant__ CUtensorMap tmap_b, _
             if (!ok) break;
             tc_fence_after();
             const int row0 = offsets[tl.key] + tl.n0;
-            const uint32_t taddr = tmem_base + buf * BN + ((uint32_t)(32 * e) << 16);
+            const uint32_t taddr = tmem_base + buf * BN_T + ((uint32_t)(32 * e) << 16);
             for (int c0 = odd; c0 < tl.nrows; c0 += 64) {
                 uint32_t v[32];
                 tc_ld32(taddr + c0, v);
@@ -444,11 +448,11 @@ gather_rows_kernel(const __nv_bfloat16* __restrict__ hidden, const int32_t* __re
     for (int i = threadIdx.x; i < H / 8; i += 256) dst[i] = src[i];
 }
 
-// n-tiles of one wave: every active group is cut into balanced runs of at most BN grouped rows (multiples of 16).
+// n-tiles of one wave: every active group is cut into balanced runs of at most `bn` grouped rows (multiples of 16).
 // One CTA; thread g handles group g, an exclusive scan of the piece counts places its tiles.
 __global__ void __launch_bounds__(1024)
 tile_list_kernel(const int32_t* __restrict__ counts, const int32_t* __restrict__ group_keys,
-                 const int32_t* __restrict__ wave_start, Tile* __restrict__ tiles, int32_t* __restrict__ n_tiles) {
+                 const int32_t* __restrict__ wave_start, Tile* __restrict__ tiles, int32_t* __restrict__ n_tiles, int bn) {
     __shared__ int s_warp[32];
     __shared__ int s_running;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -461,7 +465,7 @@ tile_list_kernel(const int32_t* __restrict__ counts, const int32_t* __restrict__
         if (g < ng) {
             key = group_keys[g0 + g];
             cnt = counts[key];
-            pieces = (cnt + BN - 1) / BN;
+            pieces = (cnt + bn - 1) / bn;
             per = ((cnt + pieces - 1) / pieces + 15) & ~15;
             pieces = (cnt + per - 1) / per;
         }
@@ -493,10 +497,10 @@ size_t prefill_scratch_bytes(int max_pairs, int num_experts) {
     return ((size_t)max_pairs / 16 + num_experts + 16) * sizeof(Tile) + 256;
 }
 
-static_assert(sizeof(CUtensorMap) == 128, "PrefillMaps mirrors two CUtensorMap objects");
+static_assert(sizeof(CUtensorMap) == 128, "PrefillMaps mirrors CUtensorMap objects");
 
-// 2-D row-major BF16 matrix [rows, cols] -> tensor map with a 64-column x 256-row box, 128-byte swizzle
-static int encode_map(CUtensorMap* out, const void* base, int rows, int cols) {
+// 2-D row-major BF16 matrix [rows, cols] -> tensor map with a 64-column x `box_rows`-row box, 128-byte swizzle
+static int encode_map(CUtensorMap* out, const void* base, int rows, int cols, int box_rows) {
     typedef CUresult (*EncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
@@ -509,7 +513,7 @@ static int encode_map(CUtensorMap* out, const void* base, int rows, int cols) {
     }
     const cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
     const cuuint64_t strides[1] = {(cuuint64_t)cols * 2};
-    const cuuint32_t box[2] = {64, (cuuint32_t)BN};
+    const cuuint32_t box[2] = {64, (cuuint32_t)box_rows};
     const cuuint32_t estr[2] = {1, 1};
     const CUresult rc = fn(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
                            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
@@ -518,9 +522,11 @@ static int encode_map(CUtensorMap* out, const void* base, int rows, int cols) {
 }
 
 int prefill_setup(PrefillMaps* maps, const __nv_bfloat16* xg, const __nv_bfloat16* act, int max_pairs, int H, int I) {
-    int rc = encode_map(reinterpret_cast<CUtensorMap*>(maps->x), xg, max_pairs, H);
-    if (rc) return rc;
-    return encode_map(reinterpret_cast<CUtensorMap*>(maps->act), act, max_pairs, I);
+    int rc = encode_map(reinterpret_cast<CUtensorMap*>(maps->x), xg, max_pairs, H, BN);
+    if (!rc) rc = encode_map(reinterpret_cast<CUtensorMap*>(maps->act), act, max_pairs, I, BN);
+    if (!rc) rc = encode_map(reinterpret_cast<CUtensorMap*>(maps->x_small), xg, max_pairs, H, BN_SMALL);
+    if (!rc) rc = encode_map(reinterpret_cast<CUtensorMap*>(maps->act_small), act, max_pairs, I, BN_SMALL);
+    return rc;
 }
 
 void launch_wait_selftest(int* status, long long budget_cycles, int* result, cudaStream_t st) {
@@ -536,7 +542,7 @@ void launch_gather_rows(const __nv_bfloat16* hidden, const int32_t* perm, const 
 
 // One wave of the tensor-core path: tile list, gate/up GEMM + SwiGLU, down GEMM x routing weight.
 void launch_prefill_wave(const GemmArgs& g, const int32_t* wave_start, void* scratch, int* status, const PrefillMaps* maps,
-                         __nv_bfloat16* act, const float* topk_w, float* y, int which, cudaStream_t st) {
+                         __nv_bfloat16* act, const float* topk_w, float* y, int which, bool small_n, cudaStream_t st) {
     int32_t* n_tiles = reinterpret_cast<int32_t*>(scratch);
     Tile* tiles = reinterpret_cast<Tile*>(reinterpret_cast<unsigned char*>(scratch) + 256);
     PrefillArgs a{};
@@ -550,28 +556,38 @@ void launch_prefill_wave(const GemmArgs& g, const int32_t* wave_start, void* scr
     a.H = g.H;
     a.I = g.I;
     a.status = status;
-    const size_t smem = (size_t)STAGES * (A_STAGE_BYTES + B_STAGE_BYTES) + 256 + 1024;
+    constexpr int kStagesLarge = 2, kStagesSmall = 4;
+    const size_t smem_large = (size_t)kStagesLarge * (A_STAGE_BYTES + 2 * BN * 128) + 256 + 1024;
+    const size_t smem_small = (size_t)kStagesSmall * (A_STAGE_BYTES + 2 * BN_SMALL * 128) + 256 + 1024;
     static bool attr_done = false;
     if (!attr_done) {
-        cudaFuncSetAttribute(prefill_gemm_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        cudaFuncSetAttribute(prefill_gemm_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        cudaFuncSetAttribute(prefill_gemm_kernel<true, BN, kStagesLarge>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_large);
+        cudaFuncSetAttribute(prefill_gemm_kernel<false, BN, kStagesLarge>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_large);
+        cudaFuncSetAttribute(prefill_gemm_kernel<true, BN_SMALL, kStagesSmall>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_small);
+        cudaFuncSetAttribute(prefill_gemm_kernel<false, BN_SMALL, kStagesSmall>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_small);
         attr_done = true;
     }
     int dev = 0, sms = 148;
     cudaGetDevice(&dev);
     cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-    const CUtensorMap* mx = reinterpret_cast<const CUtensorMap*>(maps->x);
-    const CUtensorMap* ma = reinterpret_cast<const CUtensorMap*>(maps->act);
+    const CUtensorMap* mx = reinterpret_cast<const CUtensorMap*>(small_n ? maps->x_small : maps->x);
+    const CUtensorMap* ma = reinterpret_cast<const CUtensorMap*>(small_n ? maps->act_small : maps->act);
     if (which & 4) {
-        tile_list_kernel<<<1, 1024, 0, st>>>(g.counts, g.group_keys, wave_start, tiles, n_tiles);
+        tile_list_kernel<<<1, 1024, 0, st>>>(g.counts, g.group_keys, wave_start, tiles, n_tiles, small_n ? BN_SMALL : BN);
         count_launch();
     }
     if (which & 1) {
-        prefill_gemm_kernel<true><<<sms, NUM_THREADS, smem, st>>>(a, *mx, act, nullptr, g.offsets, nullptr);
+        if (small_n)
+            prefill_gemm_kernel<true, BN_SMALL, kStagesSmall><<<sms, NUM_THREADS, smem_small, st>>>(a, *mx, act, nullptr, g.offsets, nullptr);
+        else
+            prefill_gemm_kernel<true, BN, kStagesLarge><<<sms, NUM_THREADS, smem_large, st>>>(a, *mx, act, nullptr, g.offsets, nullptr);
         count_launch();
     }
     if (which & 2) {
-        prefill_gemm_kernel<false><<<sms, NUM_THREADS, smem, st>>>(a, *ma, nullptr, topk_w, g.offsets, y);
+        if (small_n)
+            prefill_gemm_kernel<false, BN_SMALL, kStagesSmall><<<sms, NUM_THREADS, smem_small, st>>>(a, *ma, nullptr, topk_w, g.offsets, y);
+        else
+            prefill_gemm_kernel<false, BN, kStagesLarge><<<sms, NUM_THREADS, smem_large, st>>>(a, *ma, nullptr, topk_w, g.offsets, y);
         count_launch();
     }
 }
