@@ -141,14 +141,8 @@ enum { MODE_SMALL = 1, MODE_PAIR = 2 };
 
 // MODE_SMALL : every CTA rebuilds the wave's grouping in shared memory (T*k <= kSmallMaxPairs)
 // MODE_PAIR  : one item per token-expert pair, no grouping at all (T*k <= 32, gate/up only)
-#ifndef EXMOE_MINB_NB2
-#define EXMOE_MINB_NB2 1
-#endif
-#ifndef EXMOE_MINB_NB4
-#define EXMOE_MINB_NB4 1
-#endif
 template <int NB, int NCH, bool GATEUP, int MODE>
-__global__ void __launch_bounds__(256, (NCH == 1 && NB == 2) ? EXMOE_MINB_NB2 : (NCH == 1 && NB == 4) ? EXMOE_MINB_NB4 : 1)
+__global__ void __launch_bounds__(256, 1)
 decode_gemm_kernel(GemmArgs a, SmallArgs sa, const __nv_bfloat16* __restrict__ x_src,
                    __nv_bfloat16* __restrict__ act_out, const float* __restrict__ topk_w, float* __restrict__ y_out,
                    int KS, int blocks_per_warp) {
@@ -891,13 +885,7 @@ template <bool GATEUP, int MODE>
 void launch_decode(const GemmArgs& a, const SmallArgs& sa, const __nv_bfloat16* x, __nv_bfloat16* act, const float* w,
                    float* y, int max_rows, int max_groups, cudaStream_t st) {
     const int K = GATEUP ? a.H : a.I, NR = GATEUP ? a.I : a.H;
-    DecodeCfg cfg = pick_cfg(K, NR);
-#ifdef EXMOE_PAIR_KS
-    if (MODE == MODE_PAIR && (K / kGroup) % EXMOE_PAIR_KS == 0) {
-        const int bpw = K / kGroup / EXMOE_PAIR_KS;
-        cfg = {(bpw % 4 == 0) ? 4 : (bpw % 2 == 0) ? 2 : 1, EXMOE_PAIR_KS, bpw};
-    }
-#endif
+    const DecodeCfg cfg = pick_cfg(K, NR);
     // rows per pass: one 8-row chunk covers decode; more chunks amortise the dequantisation
     int nch = max_rows <= 8 ? 1 : (max_rows <= 16 ? 2 : 4);
     while (nch > 1 && (size_t)8 * nch * (K * 2 + 64) > 150 * 1024) nch >>= 1;
