@@ -201,7 +201,7 @@ __device__ __forceinline__ void scan_keys_warp0(const int32_t* cnt, int n_keys, 
     }
 }
 
-// Small problems (decode): one CTA does histogram, scan and the stable permutation.
+// Small problems (up to 1024 pairs): one CTA does histogram, scan and the stable permutation.
 __global__ void __launch_bounds__(256)
 group_small_kernel(const int32_t* __restrict__ ids, int n_pairs, int E, int C, int n_keys, int max_waves,
                    bool identity, PlanPtrs plan, int* __restrict__ status) {
@@ -232,12 +232,25 @@ group_small_kernel(const int32_t* __restrict__ ids, int n_pairs, int E, int C, i
         plan.header[HDR_BAD_ID] = 0;
     }
     __syncthreads();
-    for (int p = tid; p < n_pairs; p += blockDim.x) {
-        const int key = s_key[p];
-        if (key < 0) continue;
-        int r = 0;
-        for (int j = 0; j < p; ++j) r += (s_key[j] == key);
-        plan.perm[s_off[key] + r] = p;
+    // Stable placement, 256 pairs at a time in pair order: inside a warp equal keys are ranked by lane
+    // (match_any), the warps of a chunk advance the per-key cursors (s_off, consumed here) one after the other.
+    const int lane = tid & 31, warp = tid >> 5;
+    for (int base = 0; base < n_pairs; base += 256) {
+        const int p = base + tid;
+        const int key = (p < n_pairs) ? s_key[p] : -1;
+        const unsigned same = __match_any_sync(0xffffffffu, key);
+        const int leader = __ffs(same) - 1;
+        const int rank = __popc(same & ((1u << lane) - 1u));
+        int pos0 = 0;
+        for (int w = 0; w < 8; ++w) {
+            if (warp == w && key >= 0 && lane == leader) {
+                pos0 = s_off[key];
+                s_off[key] = pos0 + __popc(same);
+            }
+            __syncthreads();
+        }
+        pos0 = __shfl_sync(0xffffffffu, pos0, leader);
+        if (key >= 0) plan.perm[pos0 + rank] = p;
     }
 }
 
@@ -317,6 +330,9 @@ group_scatter_kernel(const int32_t* __restrict__ ids, int n_pairs, int E, int C,
 //   kernel 2: one CTA per chunk places its pairs: rank inside the warp from match_any, warps take their turn in
 //             order to advance a shared-memory cursor per key, so equal keys keep ascending pair order (stable).
 constexpr int kChunk = 512;
+#ifndef EXMOE_GROUP_SMALL_MAX
+#define EXMOE_GROUP_SMALL_MAX 2048
+#endif
 
 __global__ void __launch_bounds__(kChunk)
 group_chunk_count_kernel(const int32_t* __restrict__ ids, int n_pairs, int E, int C, int n_keys, int max_waves,
@@ -408,8 +424,13 @@ group_chunk_scatter_kernel(const int32_t* __restrict__ ids, int n_pairs, int E, 
 void launch_group(const exmoe_shape& s, int C, int n_keys, int max_waves, bool identity, const int32_t* ids,
                   int n_pairs, PlanPtrs plan, int* d_status, cudaStream_t st) {
     const int E = s.num_experts;
-    if (n_pairs <= 1024 && n_keys <= 4096) {
+    if (n_pairs <= EXMOE_GROUP_SMALL_MAX && n_keys <= 4096) {
         const size_t smem = (size_t)(2 * n_keys + 1 + n_pairs) * 4;
+        static bool attr_done = false;
+        if (!attr_done) {
+            cudaFuncSetAttribute(group_small_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 64 * 1024);
+            attr_done = true;
+        }
         group_small_kernel<<<1, 256, smem, st>>>(ids, n_pairs, E, C, n_keys, max_waves, identity, plan, d_status);
         count_launch();
         return;
