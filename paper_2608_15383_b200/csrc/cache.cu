@@ -354,14 +354,16 @@ int exmoe_moe_forward(exmoe_cache* c, int layer, const void* hidden, const int32
     a.H = s.d_model;
     a.I = s.d_ff;
 
+    bool tiles_fused = false;
     const bool pairwise = small && P <= kPairMaxPairs && n_waves == 1;
     c->last_pair = pairwise;
     const bool use_stream = !small && c->stream_ok && P <= kStreamMaxPairs;
     const bool small_n = P <= kPrefillSmallNMaxPairs;      // tensor-core path: which kernel shape
     if (!small && build_plan && !use_stream) {
         ProfScope ps(c, PROF_PLAN, st);                  // hidden rows in plan order, once for all waves
+        tiles_fused = (n_waves == 1);                    // one wave: its tile list comes out of the same launch
         launch_gather_rows((const __nv_bfloat16*)hidden, c->plan.perm, c->plan.offsets + c->n_keys, P, k, s.d_model,
-                           c->xg, st);
+                           c->xg, tiles_fused ? &a : nullptr, c->plan.wave_start, c->tc_scratch, small_n, st);
     }
     if (small && n_waves == 0)                           // no valid id at all: the output is zero
         cudaMemsetAsync(out, 0, (size_t)T * s.d_model * 2, st);
@@ -435,7 +437,8 @@ int exmoe_moe_forward(exmoe_cache* c, int layer, const void* hidden, const int32
             }
         } else {
             // many rows per expert: dense contraction on the tensor cores (tcgen05 / TMEM)
-            if (build_plan) launch_prefill_wave(a, a.wave_start, c->tc_scratch, c->d_status, &c->tc_maps, c->act, topk_weights, c->y, 4, small_n, st);
+            if (build_plan && !tiles_fused)
+                launch_prefill_wave(a, a.wave_start, c->tc_scratch, c->d_status, &c->tc_maps, c->act, topk_weights, c->y, 4, small_n, st);
             if (!c->prof_only || c->prof_only == PROF_GATEUP) {
                 ProfScope ps(c, PROF_GATEUP, st);
                 launch_prefill_wave(a, a.wave_start, c->tc_scratch, c->d_status, &c->tc_maps, c->act, topk_weights, c->y, 1,

@@ -111,8 +111,10 @@ size_t prefill_scratch_bytes(int max_pairs, int num_experts);
 struct alignas(64) PrefillMaps { unsigned char x[128], act[128], x_small[128], act_small[128]; };
 int prefill_setup(PrefillMaps* maps, const __nv_bfloat16* xg, const __nv_bfloat16* act, int max_pairs, int H, int I);
 void launch_wait_selftest(int* status, long long budget_cycles, int* result, cudaStream_t st);
+// grouped copy of the hidden rows; when `single_wave` is given its CTA 0 also builds that wave's tile list in `scratch`
 void launch_gather_rows(const __nv_bfloat16* hidden, const int32_t* perm, const int32_t* n_valid, int n_pairs, int top_k,
-                        int H, __nv_bfloat16* xg, cudaStream_t st);
+                        int H, __nv_bfloat16* xg, const GemmArgs* single_wave, const int32_t* wave_start, void* scratch,
+                        bool small_n, cudaStream_t st);
 // which: bit 0 = gate/up GEMM + SwiGLU, bit 1 = down GEMM x routing weight, bit 2 = (re)build the wave's tile list
 // small_n: the 64-row, four-stage kernel shape (a few dozen rows per expert) instead of the 256-row, two-stage one
 void launch_prefill_wave(const GemmArgs& g, const int32_t* wave_start, void* scratch, int* status, const PrefillMaps* maps,

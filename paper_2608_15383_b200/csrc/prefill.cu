@@ -437,29 +437,19 @@ __global__ void wait_timeout_selftest_kernel(int* status, long long budget, int*
     if (threadIdx.x == 0) *result = (ok ? 0 : 1) | (abort_word ? 2 : 0);
 }
 
-// grouped copy of the hidden states: row r of the plan order = hidden row of token perm[r] / k
-__global__ void __launch_bounds__(256)
-gather_rows_kernel(const __nv_bfloat16* __restrict__ hidden, const int32_t* __restrict__ perm,
-                   const int32_t* __restrict__ n_valid, int top_k, int H, __nv_bfloat16* __restrict__ xg) {
-    const int r = blockIdx.x;
-    if (r >= *n_valid) return;
-    const uint4* src = reinterpret_cast<const uint4*>(hidden + (size_t)(perm[r] / top_k) * H);
-    uint4* dst = reinterpret_cast<uint4*>(xg + (size_t)r * H);
-    for (int i = threadIdx.x; i < H / 8; i += 256) dst[i] = src[i];
-}
-
 // n-tiles of one wave: every active group is cut into balanced runs of at most `bn` grouped rows (multiples of 16).
-// One CTA; thread g handles group g, an exclusive scan of the piece counts places its tiles.
-__global__ void __launch_bounds__(1024)
-tile_list_kernel(const int32_t* __restrict__ counts, const int32_t* __restrict__ group_keys,
-                 const int32_t* __restrict__ wave_start, Tile* __restrict__ tiles, int32_t* __restrict__ n_tiles, int bn) {
+// Executed by one whole CTA (any multiple of 32 threads up to 1024): thread g handles group g, an exclusive scan of
+// the piece counts places its tiles.
+__device__ void build_tile_list(const int32_t* __restrict__ counts, const int32_t* __restrict__ group_keys,
+                                const int32_t* __restrict__ wave_start, Tile* __restrict__ tiles,
+                                int32_t* __restrict__ n_tiles, int bn) {
     __shared__ int s_warp[32];
     __shared__ int s_running;
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nthr = blockDim.x, nwarp = nthr >> 5;
     const int g0 = wave_start[0], ng = wave_start[1] - g0;
     if (tid == 0) s_running = 0;
     __syncthreads();
-    for (int base = 0; base < ng; base += 1024) {
+    for (int base = 0; base < ng; base += nthr) {
         const int g = base + tid;
         int key = 0, cnt = 0, pieces = 0, per = 0;
         if (g < ng) {
@@ -478,7 +468,7 @@ tile_list_kernel(const int32_t* __restrict__ counts, const int32_t* __restrict__
         if (lane == 31) s_warp[warp] = incl;
         __syncthreads();
         int wbase = 0, total = 0;
-        for (int w = 0; w < 32; ++w) {
+        for (int w = 0; w < nwarp; ++w) {
             if (w < warp) wbase += s_warp[w];
             total += s_warp[w];
         }
@@ -489,6 +479,27 @@ tile_list_kernel(const int32_t* __restrict__ counts, const int32_t* __restrict__
         __syncthreads();
     }
     if (tid == 0) *n_tiles = s_running;
+}
+
+__global__ void __launch_bounds__(1024)
+tile_list_kernel(const int32_t* __restrict__ counts, const int32_t* __restrict__ group_keys,
+                 const int32_t* __restrict__ wave_start, Tile* __restrict__ tiles, int32_t* __restrict__ n_tiles, int bn) {
+    build_tile_list(counts, group_keys, wave_start, tiles, n_tiles, bn);
+}
+
+// grouped copy of the hidden states: row r of the plan order = hidden row of token perm[r] / k
+// CTA 0 also builds the tile list of the call's only wave when `tiles` is given (one launch less).
+__global__ void __launch_bounds__(256)
+gather_rows_kernel(const __nv_bfloat16* __restrict__ hidden, const int32_t* __restrict__ perm,
+                   const int32_t* __restrict__ n_valid, int top_k, int H, __nv_bfloat16* __restrict__ xg,
+                   const int32_t* __restrict__ counts, const int32_t* __restrict__ group_keys,
+                   const int32_t* __restrict__ wave_start, Tile* __restrict__ tiles, int32_t* __restrict__ n_tiles, int bn) {
+    const int r = blockIdx.x;
+    if (r == 0 && tiles) build_tile_list(counts, group_keys, wave_start, tiles, n_tiles, bn);
+    if (r >= *n_valid) return;
+    const uint4* src = reinterpret_cast<const uint4*>(hidden + (size_t)(perm[r] / top_k) * H);
+    uint4* dst = reinterpret_cast<uint4*>(xg + (size_t)r * H);
+    for (int i = threadIdx.x; i < H / 8; i += 256) dst[i] = src[i];
 }
 
 }  // namespace
@@ -535,8 +546,13 @@ void launch_wait_selftest(int* status, long long budget_cycles, int* result, cud
 }
 
 void launch_gather_rows(const __nv_bfloat16* hidden, const int32_t* perm, const int32_t* n_valid, int n_pairs, int top_k,
-                        int H, __nv_bfloat16* xg, cudaStream_t st) {
-    gather_rows_kernel<<<n_pairs, 256, 0, st>>>(hidden, perm, n_valid, top_k, H, xg);
+                        int H, __nv_bfloat16* xg, const GemmArgs* single_wave, const int32_t* wave_start, void* scratch,
+                        bool small_n, cudaStream_t st) {
+    int32_t* n_tiles = reinterpret_cast<int32_t*>(scratch);
+    Tile* tiles = single_wave ? reinterpret_cast<Tile*>(reinterpret_cast<unsigned char*>(scratch) + 256) : nullptr;
+    gather_rows_kernel<<<n_pairs, 256, 0, st>>>(hidden, perm, n_valid, top_k, H, xg, single_wave ? single_wave->counts : nullptr,
+                                                 single_wave ? single_wave->group_keys : nullptr, wave_start, tiles, n_tiles,
+                                                 small_n ? BN_SMALL : BN);
     count_launch();
 }
 
