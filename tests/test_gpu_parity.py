@@ -441,6 +441,34 @@ def test_graph_replay_matches_oracle(B, olmoe_layer, T):
     cache.close()
 
 
+def test_random_sizes_are_invariant_to_slots_and_waves(B, olmoe_layer):
+    """Section 3.4, last sentence, over every kernel path: for random batch sizes and routing skews the output of a
+    16-slot cache and of a 24-slot cache with 10-expert waves equals the fully resident output bit for bit, and a
+    repeated call reproduces it."""
+    _, bank = olmoe_layer
+    s = synth.OLMOE
+    full = B.Cache(s, [bank], 64, max_tokens=300)
+    part = B.Cache(s, [bank], 16, max_tokens=300)
+    half = B.Cache(s, [bank], 24, max_tokens=300, wave_cap=10)
+    rng = np.random.default_rng(7)
+    sizes = [1, 2, 3, 4, 5, 8, 16, 33, 56, 57, 64, 128, 129, 300]
+    for it in range(24):
+        T = int(sizes[it % len(sizes)])
+        alpha = float(rng.choice([0.0, 0.5, 1.0, 2.0]))
+        hidden, ids, p = helpers.routed_inputs(s, T, seed=12000 + it, alpha=alpha)
+        h, i, w = hidden.cuda(), ids.cuda(), p.cuda()
+        a = full.forward(0, h, i, w).clone()
+        b = part.forward(0, h, i, w).clone()
+        c = half.forward(0, h, i, w).clone()
+        a2 = full.forward(0, h, i, w).clone()
+        assert bool(torch.isfinite(a.float()).all()), (T, alpha)
+        for other, what in ((b, "16 slots"), (c, "24 slots, waves of 10"), (a2, "repeat")):
+            assert torch.equal(a.view(torch.int16), other.view(torch.int16)), (T, alpha, what)
+    for c_ in (full, part, half):
+        assert c_.status() == 0
+        c_.close()
+
+
 def test_create_rejects_bad_arguments(B, tiny_layer):
     ora, bank = tiny_layer
     s = synth.TINY
