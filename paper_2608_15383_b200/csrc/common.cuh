@@ -89,6 +89,19 @@ constexpr int kSmallMaxSlots = 1024;
 // launch accounting (exmoe_launch_count)
 void count_launch(int n = 1);
 
+// Raise a kernel's dynamic shared-memory limit once per device (function attributes are per device; the cache of
+// "already done" is the caller's static SmemOnce, one per kernel instantiation).
+struct SmemOnce { unsigned long long mask = 0; };
+template <typename F>
+inline bool allow_smem(F kern, int bytes, SmemOnce& once) {
+    int dev = 0;
+    const bool known = cudaGetDevice(&dev) == cudaSuccess && dev >= 0 && dev < 64;
+    if (known && ((once.mask >> dev) & 1ull)) return true;
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes) != cudaSuccess) return false;
+    if (known) once.mask |= 1ull << dev;
+    return true;
+}
+
 // ---- kernel launchers (defined in the .cu files) ------------------------------------------------
 int launch_pack(const exmoe_shape& s, const void* wg, const void* wu, const void* wd, void* out,
                 int* d_flag, cudaStream_t st);

@@ -818,11 +818,8 @@ void launch_pair_gateup(const GemmArgs& a, const SmallArgs& sa, const __nv_bfloa
     auto kern = pair_gateup_kernel<NB>;
     const int PP = 8 / KS, tiles = a.I / (kPanelRows * PP);
     const size_t smem = (size_t)a.H * 2 + 64 + (size_t)(KS - 1) * PP * 2 * 128 * 4 + (size_t)(a.H / kGroup) * 4;
-    static bool attr_done = false;
-    if (!attr_done) {
-        cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 100 * 1024);
-        attr_done = true;
-    }
+    static SmemOnce smem_once;
+    allow_smem(kern, 100 * 1024, smem_once);
     kern<<<sa.n_pairs * tiles, 256, smem, st>>>(a, sa, hidden, act, KS);
     count_launch();
 }
@@ -857,11 +854,8 @@ void launch_cfg(const GemmArgs& a, const SmallArgs& sa, const __nv_bfloat16* x, 
     constexpr bool SMALL = (MODE == MODE_SMALL);
     if (SMALL) smem += (size_t)(3 * a.num_slots + 1 + 2 * sa.n_pairs) * 4;
     auto kern = decode_gemm_kernel<NB, NCH, GATEUP, MODE>;
-    static bool attr_done = false;                      // per instantiation
-    if (!attr_done) {
-        cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
-        attr_done = true;
-    }
+    static SmemOnce smem_once;                      // per instantiation
+    allow_smem(kern, 200 * 1024, smem_once);
     long long items = (long long)max_groups * tiles;
     const int grid = (int)(items < 148 * 8 ? (items < 1 ? 1 : items) : 148 * 8);
     cudaLaunchConfig_t lc{};
@@ -950,11 +944,8 @@ void launch_token_down(const GemmArgs& a, const SmallArgs& sa, const __nv_bfloat
                        int bpwg, cudaStream_t st) {
     auto kern = token_down_kernel<NBT>;
     const size_t smem = (size_t)a.top_k * (a.I * 2 + 64) + (size_t)a.top_k * 17 * 4 + (size_t)(a.I / kGroup) * a.top_k * 4;
-    static bool attr_done = false;
-    if (!attr_done) {
-        cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
-        attr_done = true;
-    }
+    static SmemOnce smem_once;
+    allow_smem(kern, 200 * 1024, smem_once);
     cudaLaunchConfig_t lc{};
     lc.gridDim = dim3(T * (a.H / kPanelRows));
     lc.blockDim = dim3(256);
@@ -982,11 +973,8 @@ bool launch_token_down_bulk(const GemmArgs& a, const SmallArgs& sa, const __nv_b
                         (((size_t)KB * k + 3) & ~(size_t)3) * 4 + 64;
     if (smem > 100 * 1024) return false;
     auto kern = token_down_bulk_kernel<NBT>;
-    static bool attr_done = false;
-    if (!attr_done) {
-        cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 100 * 1024);
-        attr_done = true;
-    }
+    static SmemOnce smem_once;
+    allow_smem(kern, 100 * 1024, smem_once);
     cudaLaunchConfig_t lc{};
     lc.gridDim = dim3(T * (a.H / kPanelRows));
     lc.blockDim = dim3(256);

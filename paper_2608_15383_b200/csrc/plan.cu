@@ -426,11 +426,8 @@ void launch_group(const exmoe_shape& s, int C, int n_keys, int max_waves, bool i
     const int E = s.num_experts;
     if (n_pairs <= EXMOE_GROUP_SMALL_MAX && n_keys <= 4096) {
         const size_t smem = (size_t)(2 * n_keys + 1 + n_pairs) * 4;
-        static bool attr_done = false;
-        if (!attr_done) {
-            cudaFuncSetAttribute(group_small_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 64 * 1024);
-            attr_done = true;
-        }
+        static SmemOnce smem_once;
+        allow_smem(group_small_kernel, 64 * 1024, smem_once);
         group_small_kernel<<<1, 256, smem, st>>>(ids, n_pairs, E, C, n_keys, max_waves, identity, plan, d_status);
         count_launch();
         return;

@@ -575,14 +575,11 @@ void launch_prefill_wave(const GemmArgs& g, const int32_t* wave_start, void* scr
     constexpr int kStagesLarge = 2, kStagesSmall = 4;
     const size_t smem_large = (size_t)kStagesLarge * (A_STAGE_BYTES + 2 * BN * 128) + 256 + 1024;
     const size_t smem_small = (size_t)kStagesSmall * (A_STAGE_BYTES + 2 * BN_SMALL * 128) + 256 + 1024;
-    static bool attr_done = false;
-    if (!attr_done) {
-        cudaFuncSetAttribute(prefill_gemm_kernel<true, BN, kStagesLarge>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_large);
-        cudaFuncSetAttribute(prefill_gemm_kernel<false, BN, kStagesLarge>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_large);
-        cudaFuncSetAttribute(prefill_gemm_kernel<true, BN_SMALL, kStagesSmall>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_small);
-        cudaFuncSetAttribute(prefill_gemm_kernel<false, BN_SMALL, kStagesSmall>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_small);
-        attr_done = true;
-    }
+    static SmemOnce once[4];
+    allow_smem(prefill_gemm_kernel<true, BN, kStagesLarge>, (int)smem_large, once[0]);
+    allow_smem(prefill_gemm_kernel<false, BN, kStagesLarge>, (int)smem_large, once[1]);
+    allow_smem(prefill_gemm_kernel<true, BN_SMALL, kStagesSmall>, (int)smem_small, once[2]);
+    allow_smem(prefill_gemm_kernel<false, BN_SMALL, kStagesSmall>, (int)smem_small, once[3]);
     int dev = 0, sms = 148;
     cudaGetDevice(&dev);
     cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);

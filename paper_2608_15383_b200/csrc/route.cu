@@ -105,12 +105,8 @@ extern "C" int exmoe_route(const exmoe_shape* shape, const void* hidden_bf16, co
     if ((reinterpret_cast<uintptr_t>(hidden_bf16) | reinterpret_cast<uintptr_t>(router_bf16)) & 15) return EXMOE_ERR_ARG;
     const size_t smem = (size_t)shape->d_model * 2 + (size_t)shape->num_experts * 4;
     if (smem > 200 * 1024) return EXMOE_ERR_SHAPE;
-    static bool attr_done = false;
-    if (!attr_done) {
-        if (cudaFuncSetAttribute(route_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024) != cudaSuccess)
-            return EXMOE_ERR_CUDA;
-        attr_done = true;
-    }
+    static SmemOnce smem_once;
+    if (!allow_smem(route_kernel, 200 * 1024, smem_once)) return EXMOE_ERR_CUDA;
     route_kernel<<<T, kRouteThreads, smem, (cudaStream_t)stream>>>(
         (const __nv_bfloat16*)hidden_bf16, (const __nv_bfloat16*)router_bf16, bias, shape->d_model, shape->num_experts,
         shape->top_k, topk_ids, topk_weights);

@@ -547,18 +547,11 @@ bool launch_stream_cfg(const GemmArgs& a, const __nv_bfloat16* x, __nv_bfloat16*
     if (!stream_geometry(GATEUP ? a.H : a.I, GATEUP ? a.I : a.H, NM, NCH, &g)) return false;
     void (*kern)(const StreamArgs) = stream_gemm_kernel<NCH, GATEUP, 1>;
     if (GATEUP && g.NMW == 2) kern = stream_gemm_kernel<NCH, GATEUP, GATEUP ? 2 : 1>;
-    static bool attr_done[2] = {false, false};
-    if (!attr_done[g.NMW - 1]) {
-        cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemLimit);
-        attr_done[g.NMW - 1] = true;
-    }
-    static int sms = 0;
-    if (!sms) {
-        int dev = 0;
-        if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess ||
-            sms <= 0)
-            sms = 148;
-    }
+    static SmemOnce smem_once[2];
+    allow_smem(kern, (int)kSmemLimit, smem_once[g.NMW - 1]);
+    int sms = 0, dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0)
+        sms = 148;
     StreamArgs p{};
     p.a = a;
     p.x_src = x;
