@@ -36,7 +36,8 @@ WORKLOADS = {
     # name: (tokens per step, slots, layers rotated over, Zipf alpha, description)
     "decode": (1, 64, 16, 0.0, "config2: OLMoE-shaped decode, T=1, 64 slots resident, top-8 of 64, int4 g128"),
     "decode16": (16, 64, 16, 1.0, "OLMoE-shaped batched decode, T=16, 64 slots resident, Zipf(1.1) routing"),
-    "offload": (16, 16, 1, 1.0, "config3: T=16, 16 slots over a 64-expert pinned host bank, Zipf(1.1) routing"),
+    "offload": (16, 16, 1, "cycle", "config3: T=16, 16 slots over a 64-expert pinned host bank, Zipf(1.1) routing bias "
+                "x alpha, alpha cycling over {2, 1, 0.5, 0} in four blocks of steps (1-4 waves per step)"),
     "prefill": (2048, 64, 1, 0.0, "config4: OLMoE-shaped prefill, T=2048, 64 slots resident, uniform routing"),
 }
 # DRAM bytes (read + write) per launch of the dominant kernel, from the committed ncu captures under profiles/
@@ -165,11 +166,15 @@ def whole_job_tokens_per_s(world, steps, tokens_per_step, ms_max):
 
 
 def make_inputs(shape, T, n_sets, alpha, seed0, device):
-    """n_sets independent (hidden, ids, weights) batches, generated on the device, routed by Eq. 1."""
+    """n_sets independent (hidden, ids, weights) batches, generated on the device, routed by Eq. 1.
+    alpha = "cycle": the sets fall into four consecutive blocks with alpha = 2, 1, 0.5, 0 (same rank permutation)."""
     wr = synth.router_weights(shape, seed0 + 1, device=device)
-    bias = synth.zipf_bias(shape.num_experts, alpha, seed0 + 2).to(device) if alpha else None
+    cycle = (2.0, 1.0, 0.5, 0.0)
+    base = synth.zipf_bias(shape.num_experts, 1.0, seed0 + 2).to(device)
     hs, ids, ws = [], [], []
     for i in range(n_sets):
+        al = cycle[min(3, i * 4 // max(n_sets, 1))] if alpha == "cycle" else float(alpha)
+        bias = base * al if al else None
         h = synth.hidden_states(shape, T, seed0 + 10 + i, device=device)
         a, b = synth.route(h, wr, shape.top_k, bias)
         hs.append(h)
@@ -266,7 +271,7 @@ def run_stack_sweep(args, dev, binding):
             torch.cuda.empty_cache()
             torch.cuda.reset_peak_memory_stats(dev)
             cache = binding.Cache(shape, banks, C, max_tokens=64, device=dev)
-            stack = synth.SyntheticStack(shape, L, seed=5100, alpha=args.alpha, device=dev)
+            stack = synth.SyntheticStack(shape, L, seed=5100, alpha=(0.5 if args.alpha is None else args.alpha), device=dev)
             # every step decodes fresh tokens: a new seeded hidden state enters layer 0 (as an embedding would)
             pool = [synth.hidden_states(shape, T, 5200 + i, device=dev) for i in range(16)]
             fwd = lambda l, x, ids, w: cache.forward(l, x, ids, w)
@@ -325,7 +330,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=50)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="decode", choices=sorted(WORKLOADS) + ["stack"])
-    ap.add_argument("--alpha", type=float, default=0.5, help="Zipf skew of the stack workload's routers")
+    ap.add_argument("--alpha", type=float, default=None,
+                    help="Zipf skew: overrides the workload's alpha (stack workload: default 0.5)")
     ap.add_argument("--tokens", type=int, default=0, help="override the workload's tokens per step")
     ap.add_argument("--cpu-budget", type=float, default=15.0, help="seconds of CPU oracle work for cpu_baseline")
     ap.add_argument("--layers", type=int, default=0, help="layer banks to rotate over (0 = the workload's default)")
@@ -369,6 +375,8 @@ def main():
     L = args.layers or L
     if args.tokens:
         T, desc = args.tokens, desc + " [tokens per step overridden: %d]" % args.tokens
+    if args.alpha is not None:
+        alpha, desc = args.alpha, desc + " [routing skew alpha overridden: %g]" % args.alpha
     shape = synth.OLMOE
     K, W = args.steps, max(args.warmup, 3)
     peaks = load_peaks()
@@ -472,7 +480,8 @@ def main():
     cache.profile_enable(False)
     bpe = cache.bytes_per_expert
     w13_bytes = bpe * 2 // 3
-    active = float(np.mean([len(torch.unique(ids[i % n_sets])) for i in range(W, W + n_prof)]))
+    active = float(np.mean([len(torch.unique(ids[i % n_sets])) for i in range(W, W + n_prof)]))      # the steps timed above
+    active_all = float(np.mean([len(torch.unique(ids[i % n_sets])) for i in range(W, W + K, max(K // 200, 1))]))
     if args.workload == "prefill":
         flops = 2.0 * T * shape.top_k * 2 * shape.d_ff * shape.d_model          # gate/up GEMM of one step
         achieved = flops / (kinds["gate_up"]["us_per_launch"] * 1e-6) / 1e12
@@ -491,7 +500,7 @@ def main():
                 "kernel": "gate_up (pair_gateup_kernel)" if T * shape.top_k <= 24 else
                 "gate_up (stream_gemm_kernel<1,true,1>)" if T * shape.top_k <= 448 else "gate_up",
                 "bytes_per_launch": gu_bytes, "peak_source": peaks["source"] + " copy rate, burst"}
-    step_gbs = active * bpe / (ms * 1e-3 / K) / 1e9
+    step_gbs = active_all * bpe / (ms * 1e-3 / K) / 1e9
     step_tflops = 2.0 * T * shape.top_k * 3 * shape.d_ff * shape.d_model / (ms * 1e-3 / K) / 1e12
 
     # ---- end to end: host buffers in, host buffer out, copies inside the timed region
@@ -585,7 +594,8 @@ def main():
         c0, c1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         with torch.cuda.stream(stream):
             c0.record(stream)
-            for i in range(W, W + n_c):
+            for j in range(n_c):                              # steps spread evenly over the timed range (all alpha blocks)
+                i = W + j * max(K // n_c, 1)
                 step(i, outs[i & 1])
             c1.record(stream)
         stream.synchronize()
@@ -616,7 +626,7 @@ def main():
                            "l2": "inputs larger than L2: steps rotate over %d layer banks (%.2f GB packed)" % (L, L * 64 * bpe / 1e9)
                            if L > 1 else "single layer bank (%.0f MB packed) vs 126 MB L2" % (64 * bpe / 1e6),
                            "timing": "CUDA graph replay of all steps" if identity else "host-driven loop (one plan read-back per step)",
-                           "active_experts_per_step": active, "packed_gb_per_s_whole_step": step_gbs,
+                           "active_experts_per_step": active_all, "packed_gb_per_s_whole_step": step_gbs,
                            "tflops_whole_step": step_tflops,
                            "kernel_us": kinds, "parallelism": "replicas only (no collective)", "status": status, **extra},
                 "roofline": roof, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": int(launches), "clocks": clocks}

@@ -27,16 +27,23 @@ def silu(g):
         return g / (1.0 + np.exp(-g))
 
 
-def expert_ffn(x, w_gate, w_up, w_down):
-    """One expert on one token: W_d [ phi(W_g x) (.) W_u x ]  (the bracket of Eq. 2)."""
+def expert_ffn(x, w_gate, w_up, w_down, round_activation=False):
+    """One expert on one token: W_d [ phi(W_g x) (.) W_u x ]  (the bracket of Eq. 2).
+
+    round_activation: round the bracket's left factor a = phi(g) (.) u to BF16 before the down projection.  This is
+    NOT the definition; it is the one rounding every implementation with BF16 activations between the two
+    projections must make, kept as a second mode so that a test can see how much of the distance to the
+    definition that single rounding explains."""
     x = np.asarray(x, dtype=np.float64)
     g = np.asarray(w_gate, dtype=np.float64) @ x
     u = np.asarray(w_up, dtype=np.float64) @ x
     a = silu(g) * u
+    if round_activation:
+        a = round_to_bf16(a)
     return np.asarray(w_down, dtype=np.float64) @ a
 
 
-def moe_layer_forward(hidden, topk_ids, topk_weights, expert_weights, num_experts):
+def moe_layer_forward(hidden, topk_ids, topk_weights, expert_weights, num_experts, round_activation=False):
     """Eq. 2 for every token.
 
     hidden        float [T, H]  (BF16-valued)
@@ -59,6 +66,6 @@ def moe_layer_forward(hidden, topk_ids, topk_weights, expert_weights, num_expert
             if e < 0 or e >= num_experts:
                 continue
             wg, wu, wd = expert_weights(e)
-            acc += topk_weights[t, j] * expert_ffn(hidden[t], wg, wu, wd)
+            acc += topk_weights[t, j] * expert_ffn(hidden[t], wg, wu, wd, round_activation)
         y[t] = acc
     return y, round_to_bf16(y)

@@ -40,9 +40,9 @@ class OracleLayer:
         return olayout.pack_expert(self.wg[e].float().cpu().numpy(), self.wu[e].float().cpu().numpy(),
                                    self.wd[e].float().cpu().numpy())
 
-    def forward(self, hidden, ids, w):
+    def forward(self, hidden, ids, w, round_activation=False):
         return omoe.moe_layer_forward(hidden.float().cpu().numpy(), ids.cpu().numpy(), w.cpu().numpy(),
-                                      self.expert, self.shape.num_experts)
+                                      self.expert, self.shape.num_experts, round_activation=round_activation)
 
 
 def check_output(out_gpu, y_ref, out_ref, what=""):

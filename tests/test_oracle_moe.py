@@ -125,3 +125,21 @@ def test_w4_error_against_unquantised_weights_is_the_quantiser_noise(layer):
     yf, _ = moe.moe_layer_forward(hidden, ids, p, full, SHAPE.num_experts)
     rel = np.linalg.norm(yq - yf) / np.linalg.norm(yf)
     assert 0.02 < rel < 0.5
+
+
+def test_rounding_matched_mode_differs_only_by_the_activation_rounding():
+    """The second oracle mode rounds phi(g)*u to BF16 before the down projection: its distance to the definition is
+    bounded by that rounding (relative 2^-9 per activation), and with an activation that is BF16-exact it is zero."""
+    from oracle import moe as omoe
+    from oracle.bf16 import round_to_bf16
+    rng = np.random.default_rng(11)
+    H, I = 16, 8
+    wg, wu, wd = rng.standard_normal((I, H)), rng.standard_normal((I, H)), rng.standard_normal((H, I))
+    x = round_to_bf16(rng.standard_normal(H))
+    plain = omoe.expert_ffn(x, wg, wu, wd)
+    matched = omoe.expert_ffn(x, wg, wu, wd, round_activation=True)
+    a = omoe.silu(wg @ x) * (wu @ x)
+    bound = np.abs(wd) @ (np.abs(a) * 2.0 ** -9)
+    assert np.all(np.abs(plain - matched) <= bound + 1e-15) and np.any(plain != matched)
+    # gate = 0 rows make a = 0 exactly: both modes agree bit for bit
+    assert np.array_equal(omoe.expert_ffn(x, np.zeros((I, H)), wu, wd), omoe.expert_ffn(x, np.zeros((I, H)), wu, wd, True))
