@@ -6,7 +6,8 @@
 // `PP` 16-row panels (gate/up: panel pairs) of one active expert and splits K over `KS` warps per
 // panel; each warp issues ALL of its 128-bit weight loads up front (NB blocks x 2 halves per
 // matrix: up to 8 KB in flight per warp), stages the group's activation rows in shared memory while
-// they fly, then dequantises in registers (shift + lop3 + one packed subtract per code pair) straight
+// they fly, then dequantises in registers (one shift and one lop3 per code pair; the code bias of 136 is
+// removed after the MMA with a per-block correction formed while the activations are staged) straight
 // into m16n8k16 fragments: the packed layout IS the fragment order, so no shuffle or shared-memory
 // round trip touches the weights.  Per 128-wide group the integer-valued partial sums are scaled
 // in binary32 by the FP16 group scale (post-scaling: codes and activations enter the MMA exactly).
@@ -19,7 +20,8 @@
 //     The down kernel is launched with programmatic dependent launch: it prefetches its weights
 //     while the gate/up kernel still runs, and it folds the fixed-order combine in: the last CTA
 //     to finish a (token, column tile) sums the k pair rows in order j = 0..k-1 (no spin wait).
-//   PAIR (T*k <= kPairMaxPairs, one wave): no grouping at all; see pair_gateup_kernel / token_down_kernel.
+//   PAIR (same sizes, one wave; the allocation-free entry point up to kPairMaxPairs): no grouping at all; see
+//     pair_gateup_kernel, token_down_kernel (one token) and token_down_bulk_kernel (two or more tokens).
 // Larger batches run on the streaming kernels (stream.cu) or the tensor-core kernels (prefill.cu) with the
 // grouping kernels' global plan and the separate combine kernel defined here.
 #include "common.cuh"
