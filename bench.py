@@ -332,6 +332,9 @@ def main():
     ap.add_argument("--workload", default="decode", choices=sorted(WORKLOADS) + ["stack"])
     ap.add_argument("--alpha", type=float, default=None,
                     help="Zipf skew: overrides the workload's alpha (stack workload: default 0.5)")
+    ap.add_argument("--miss-path", default="host", choices=["host", "device"],
+                    help="C < E workloads: host-issued miss copies (default) or the device-initiated fetch kernel")
+    ap.add_argument("--slots", type=int, default=0, help="override the workload's resident slots per layer")
     ap.add_argument("--tokens", type=int, default=0, help="override the workload's tokens per step")
     ap.add_argument("--cpu-budget", type=float, default=15.0, help="seconds of CPU oracle work for cpu_baseline")
     ap.add_argument("--layers", type=int, default=0, help="layer banks to rotate over (0 = the workload's default)")
@@ -375,6 +378,8 @@ def main():
     L = args.layers or L
     if args.tokens:
         T, desc = args.tokens, desc + " [tokens per step overridden: %d]" % args.tokens
+    if args.slots:
+        C, desc = args.slots, desc + " [slots overridden: %d]" % args.slots
     if args.alpha is not None:
         alpha, desc = args.alpha, desc + " [routing skew alpha overridden: %g]" % args.alpha
     shape = synth.OLMOE
@@ -385,11 +390,15 @@ def main():
     seed0 = 2000 + 100000 * rank
     banks, w_cpu = build_banks(shape, L, seed0, dev, keep_layer0=(rank == 0))
     cache = binding.Cache(shape, banks, C, max_tokens=T, device=dev)
+    if args.miss_path == "device":
+        cache.set_miss_path(binding.MISS_DEVICE_FETCH)
+        desc += " [device-initiated miss fetch]"
     n_sets = min(K + W, 1024) if T <= 64 else 4
     hs, ids, ws = make_inputs(shape, T, n_sets, alpha, seed0, dev)
     outs = [torch.empty_like(hs[0]) for _ in range(2)]
     stream = torch.cuda.Stream(device=dev)
     identity = (C == shape.num_experts)
+    graphable = identity or args.miss_path == "device"       # no host wait inside the call: the steps replay from a graph
 
     def step(i, out):
         cache.forward(i % L, hs[i % n_sets], ids[i % n_sets], ws[i % n_sets], out=out, stream=stream)
@@ -402,7 +411,7 @@ def main():
     # ---- device-timed region: CUDA-graph replay when the layer is fully resident (no host sync inside)
     launches0 = binding.exmoe_launch_count()
     graph_w = graph_k = None
-    if identity:
+    if graphable:
         graph_w, graph_k = torch.cuda.CUDAGraph(), torch.cuda.CUDAGraph()
         with torch.cuda.graph(graph_w, stream=stream):
             for i in range(W):
@@ -430,7 +439,7 @@ def main():
     sampler.mark()
     with torch.cuda.stream(stream):
         e0.record(stream)
-        if identity:
+        if graphable:
             graph_k.replay()
         else:
             launches0 = binding.exmoe_launch_count()
@@ -625,7 +634,7 @@ def main():
                 "config": {"workload": desc, "tokens_per_step": T, "slots": C, "layers_rotated": L,
                            "l2": "inputs larger than L2: steps rotate over %d layer banks (%.2f GB packed)" % (L, L * 64 * bpe / 1e9)
                            if L > 1 else "single layer bank (%.0f MB packed) vs 126 MB L2" % (64 * bpe / 1e6),
-                           "timing": "CUDA graph replay of all steps" if identity else "host-driven loop (one plan read-back per step)",
+                           "timing": "CUDA graph replay of all steps" if graphable else "host-driven loop (one plan read-back per step)",
                            "active_experts_per_step": active_all, "packed_gb_per_s_whole_step": step_gbs,
                            "tflops_whole_step": step_tflops,
                            "kernel_us": kinds, "parallelism": "replicas only (no collective)", "status": status, **extra},

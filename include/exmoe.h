@@ -117,6 +117,21 @@ int exmoe_cache_create(exmoe_cache** out, const exmoe_shape* shape, int num_laye
 int exmoe_moe_forward(exmoe_cache* cache, int layer, const void* hidden_bf16, const int32_t* topk_ids,
                       const float* topk_weights, int T, void* out_bf16, void* stream);
 
+/* How the misses of a C < E cache reach their slots (Sec. 3.4 step 3; the paper's runtime issues host copies).
+ *   EXMOE_MISS_HOST_COPIES  (default): as described at exmoe_moe_forward: the host reads the miss plan once per
+ *       call and issues one copy per missed expert on the library's copy stream; copies of a wave overlap the
+ *       kernels of the wave before it.
+ *   EXMOE_MISS_DEVICE_FETCH: the miss list stays on the device; before each wave's GEMM kernels a kernel on the
+ *       caller's stream reads the wave's missed experts straight out of the pinned host bank (through its mapped
+ *       device address, over PCIe) into their slots.  The host waits for nothing and exmoe_moe_forward becomes a
+ *       fixed launch sequence that may be captured in a CUDA graph.  It launches ceil(min(T*k, E) / wave_cap)
+ *       waves whatever the ids turn out to be (a wave without work finds none), and within one call copies do
+ *       not overlap kernels.  Outputs, cache state and statistics are identical in both modes.
+ * Synchronises the device, so the switch is ordered against earlier calls.  EXMOE_ERR_NOT_PINNED if a host
+ * bank has no 16-byte aligned device-visible address; the mode is then unchanged.  No effect when C = E. */
+enum { EXMOE_MISS_HOST_COPIES = 0, EXMOE_MISS_DEVICE_FETCH = 1 };
+int exmoe_cache_set_miss_path(exmoe_cache* cache, int mode);
+
 /* Router of one sparse block (Eq. 1; Sec. 3.4 "router weights are ... not renormalized"): logits z_t = W_r h_t in
  * binary32 (BF16 products, fixed summation order), plus `bias` if given, softmax over all E experts, the k
  * largest, equal values ordered by ascending expert id.  Writes exmoe_moe_forward's inputs on the device.

@@ -55,6 +55,7 @@ _SIGNATURES = {
     "exmoe_debug_wait_timeout": (c_int, [c_void_p, ctypes.c_longlong, POINTER(c_int)]),
     "exmoe_cache_stats": (c_int, [c_void_p, c_int, POINTER(exmoe_stats)]),
     "exmoe_cache_reset": (c_int, [c_void_p, c_int]),
+    "exmoe_cache_set_miss_path": (c_int, [c_void_p, c_int]),
     "exmoe_status": (c_int, [c_void_p]),
     "exmoe_cache_destroy": (c_int, [c_void_p]),
     "exmoe_profile_enable": (c_int, [c_void_p, c_int]),
@@ -179,6 +180,9 @@ def pack_bank(shape, w_gate, w_up, w_down, device="cuda"):
     return bank
 
 
+MISS_HOST_COPIES, MISS_DEVICE_FETCH = 0, 1
+
+
 class Cache:
     """exmoe_cache handle plus the torch buffers it borrows (slot memory, workspace, host banks)."""
 
@@ -259,6 +263,11 @@ class Cache:
         s = exmoe_stats()
         _check(lib().exmoe_cache_stats(self.handle, layer, byref(s)), "exmoe_cache_stats")
         return {k: int(getattr(s, k)) for k, _ in exmoe_stats._fields_}
+
+    # exmoe_cache_set_miss_path
+    def set_miss_path(self, mode):
+        """mode: MISS_HOST_COPIES (default) or MISS_DEVICE_FETCH (no host wait; graph-capturable with C < E)."""
+        _check(lib().exmoe_cache_set_miss_path(self.handle, int(mode)), "exmoe_cache_set_miss_path")
 
     def reset(self, layer):
         _check(lib().exmoe_cache_reset(self.handle, layer), "exmoe_cache_reset")

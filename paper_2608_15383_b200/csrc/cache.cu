@@ -1,6 +1,7 @@
 // Host side of the C ABI: slot caches (Section 3.3), the wave executor (Section 3.4), miss copies on a
 // side stream ordered by events, and the test hooks.  All arithmetic of the path runs in kernels;
 // this file only validates, carves the caller's workspace, launches and orders.
+#include <algorithm>
 #include <atomic>
 #include <cstring>
 #include <new>
@@ -50,6 +51,8 @@ struct exmoe_cache {
     int L, C, Cw, max_tokens, max_pairs, n_keys, max_waves;
     size_t bpe;                               // bytes per packed expert = slot stride
     std::vector<const uint8_t*> bank;
+    std::vector<const uint8_t*> bank_dev;     // device-visible address of each bank (device-initiated miss path)
+    int miss_path;                            // EXMOE_MISS_HOST_COPIES or EXMOE_MISS_DEVICE_FETCH
     uint8_t* slot_mem;
     int* d_status;
     std::vector<LayerState> state;
@@ -311,6 +314,7 @@ int exmoe_moe_forward(exmoe_cache* c, int layer, const void* hidden, const int32
     const exmoe_shape& s = c->shape;
     const int E = s.num_experts, C = c->C, k = s.top_k, P = T * k;
     const bool identity = (C == E);
+    const bool dev_fetch = !identity && c->miss_path == EXMOE_MISS_DEVICE_FETCH;   // no host wait, no host-issued copies
     c->last_layer = layer;
     c->last_T = T;
 
@@ -319,9 +323,11 @@ int exmoe_moe_forward(exmoe_cache* c, int layer, const void* hidden, const int32
     if (!identity) {
         ProfScope ps(c, PROF_PLAN, st);
         launch_resolve(s, C, c->Cw, c->bpe, topk_ids, P, c->state[layer], c->plan, c->d_status, st);
-        if (cudaMemcpyAsync(c->h_plan, c->plan.header, c->plan_d2h_bytes, cudaMemcpyDeviceToHost, st) != cudaSuccess)
-            return EXMOE_ERR_CUDA;
-        if (cudaEventRecord(c->ev_plan, st) != cudaSuccess) return EXMOE_ERR_CUDA;
+        if (!dev_fetch) {
+            if (cudaMemcpyAsync(c->h_plan, c->plan.header, c->plan_d2h_bytes, cudaMemcpyDeviceToHost, st) != cudaSuccess)
+                return EXMOE_ERR_CUDA;
+            if (cudaEventRecord(c->ev_plan, st) != cudaSuccess) return EXMOE_ERR_CUDA;
+        }
     }
     // timing runs that launch one kernel kind reuse the plan, grouped rows and tile list of the previous full call
     const bool build_plan = (c->prof_only == 0);
@@ -333,7 +339,15 @@ int exmoe_moe_forward(exmoe_cache* c, int layer, const void* hidden, const int32
     int n_waves = 1;
     const int32_t *h_wave_of = nullptr, *h_slot_of = nullptr, *h_miss = nullptr;
     int n_miss = 0;
-    if (!identity) {
+    if (dev_fetch) {
+        // The host does not learn the plan.  A call activates at most min(P, E) experts and a wave holds up to
+        // wave_cap of them, so this many waves always suffice; a wave that turns out empty costs its launches only
+        // (every kernel takes its group count from the device plan and finds nothing to do).
+        const int act_max = P < E ? P : E;
+        n_waves = (act_max + c->Cw - 1) / c->Cw;
+        if (n_waves > c->max_waves) n_waves = c->max_waves;
+        if (n_waves < 1) n_waves = 1;
+    } else if (!identity) {
         if (cudaEventSynchronize(c->ev_plan) != cudaSuccess) return EXMOE_ERR_CUDA;   // the one batched id transfer
         n_waves = c->h_plan[HDR_N_WAVES];
         n_miss = c->h_plan[HDR_N_MISSES];
@@ -370,7 +384,12 @@ int exmoe_moe_forward(exmoe_cache* c, int layer, const void* hidden, const int32
     int mi = 0;
     for (int w = 0; w < n_waves; ++w) {
         int groups = identity ? (E < P ? E : P) : 0;
-        if (!identity) {
+        if (dev_fetch) {
+            ProfScope ps(c, PROF_COPY, st);
+            launch_fetch_misses(c->plan, w, c->bank_dev[layer], const_cast<uint8_t*>(a.slots), c->bpe, E, C, st);
+            groups = c->Cw < P ? c->Cw : P;              // upper bound of the wave's groups (sizes the grids only)
+            if (groups > E) groups = E;
+        } else if (!identity) {
             bool copied = false;
             const bool wave_has_miss = mi < n_miss && h_miss[3 * mi + 2] == w;
             if (wave_has_miss) prof_mark(c, PROF_COPY, c->copy_stream);       // begin of the wave's copies
@@ -450,7 +469,7 @@ int exmoe_moe_forward(exmoe_cache* c, int layer, const void* hidden, const int32
                                     small_n, st);
             }
         }
-        if (!identity) {
+        if (!identity && !dev_fetch) {
             ++c->seq;
             cudaEventRecord(c->ev_compute[c->seq % kEventRing], st);                  // completion event of the wave
             for (int e = 0; e < E; ++e)
@@ -462,6 +481,27 @@ int exmoe_moe_forward(exmoe_cache* c, int layer, const void* hidden, const int32
         launch_combine(c->y, topk_ids, E, T, k, s.d_model, (__nv_bfloat16*)out, st);
     }
     return cudaGetLastError() == cudaSuccess ? EXMOE_OK : EXMOE_ERR_CUDA;
+}
+
+int exmoe_cache_set_miss_path(exmoe_cache* c, int mode) {
+    if (!c || (mode != EXMOE_MISS_HOST_COPIES && mode != EXMOE_MISS_DEVICE_FETCH)) return EXMOE_ERR_ARG;
+    if (cudaDeviceSynchronize() != cudaSuccess) return EXMOE_ERR_CUDA;     // no wave of the other mode is in flight
+    if (mode == EXMOE_MISS_DEVICE_FETCH) {
+        std::vector<const uint8_t*> devp;
+        for (int l = 0; l < c->L; ++l) {
+            void* d = nullptr;
+            if (cudaHostGetDevicePointer(&d, const_cast<uint8_t*>(c->bank[l]), 0) != cudaSuccess || !d ||
+                (reinterpret_cast<uintptr_t>(d) & 15)) {
+                cudaGetLastError();
+                return EXMOE_ERR_NOT_PINNED;                                 // not mapped into the device's address space
+            }
+            devp.push_back(static_cast<const uint8_t*>(d));
+        }
+        c->bank_dev = devp;
+    }
+    for (auto& v : c->slot_last_seq) std::fill(v.begin(), v.end(), 0);       // everything earlier has completed
+    c->miss_path = mode;
+    return EXMOE_OK;
 }
 
 int exmoe_cache_get_state(exmoe_cache* c, int layer, int32_t* expert_slot, int32_t* slot_expert, uint64_t* slot_stamp,

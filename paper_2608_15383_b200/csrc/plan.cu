@@ -145,6 +145,72 @@ void launch_resolve(const exmoe_shape& s, int C, int Cw, size_t bytes_per_expert
 }
 
 // ------------------------------------------------------------------------------------------------
+// Device-initiated miss path (Section 3.4 step 3 without the host in the loop): the misses of one wave
+// are fetched by this kernel straight from the pinned host bank, which the GPU reads over PCIe through
+// its mapped address.  The miss list stays on the device, so the host neither waits for the plan nor
+// issues a copy per expert, and the whole layer call is a fixed launch sequence (capturable in a CUDA
+// graph even with C < E).  Stream order is the slot's ready flag: the kernel runs on the compute
+// stream after every earlier reader of the slots it overwrites and before the wave's GEMM kernels.
+//
+// Work split: the wave's missed experts are cut into 32 KiB pieces handed round-robin to the CTAs;
+// a thread has eight 16-byte loads in flight before its first store (256 threads x 8 x 16 B per CTA),
+// which is what keeps the PCIe read pipeline full.
+// ------------------------------------------------------------------------------------------------
+constexpr int kFetchThreads = 256;
+constexpr int kFetchVec = 8;
+constexpr int kFetchPiece = kFetchThreads * kFetchVec * 16;           // 32,768 B
+
+__global__ void __launch_bounds__(kFetchThreads)
+fetch_misses_kernel(const int32_t* __restrict__ header, const int32_t* __restrict__ misses, int wave,
+                    const uint8_t* __restrict__ bank, uint8_t* __restrict__ slots, unsigned long long bpe, int E, int C) {
+    __shared__ int s_lo, s_hi;
+    if (threadIdx.x == 0) {                            // the list is ordered by wave: this wave's entries are one run
+        int n = header[HDR_N_MISSES];
+        n = n < 0 ? 0 : (n > E ? E : n);
+        int lo = 0;
+        while (lo < n && misses[3 * lo + 2] < wave) ++lo;
+        int hi = lo;
+        while (hi < n && misses[3 * hi + 2] == wave) ++hi;
+        s_lo = lo;
+        s_hi = hi;
+    }
+    __syncthreads();
+    const long long per = (long long)((bpe + kFetchPiece - 1) / kFetchPiece);
+    const long long total = (long long)(s_hi - s_lo) * per;
+    for (long long c = blockIdx.x; c < total; c += gridDim.x) {
+        const int m = s_lo + (int)(c / per);
+        const unsigned long long off = (unsigned long long)(c % per) * kFetchPiece;
+        const int e = misses[3 * m], v = misses[3 * m + 1];
+        if (e < 0 || e >= E || v < 0 || v >= C) continue;             // never leave the bank or the slot memory
+        const unsigned long long left = bpe - off;
+        const int n16 = (int)((left < (unsigned long long)kFetchPiece ? left : (unsigned long long)kFetchPiece) / 16);
+        const int4* src = reinterpret_cast<const int4*>(bank + (size_t)e * bpe + off);
+        int4* dst = reinterpret_cast<int4*>(slots + (size_t)v * bpe + off);
+        int4 r[kFetchVec];
+#pragma unroll
+        for (int j = 0; j < kFetchVec; ++j) {
+            const int i = threadIdx.x + kFetchThreads * j;
+            if (i < n16) r[j] = __ldcs(src + i);
+        }
+#pragma unroll
+        for (int j = 0; j < kFetchVec; ++j) {
+            const int i = threadIdx.x + kFetchThreads * j;
+            if (i < n16) __stcg(dst + i, r[j]);
+        }
+    }
+}
+
+void launch_fetch_misses(const PlanPtrs& plan, int wave, const uint8_t* bank_dev, uint8_t* slots, size_t bpe, int E, int C,
+                         cudaStream_t st) {
+    int sms = 0, dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0)
+        sms = 148;
+    fetch_misses_kernel<<<2 * sms, kFetchThreads, 0, st>>>(plan.header, plan.misses, wave, bank_dev, slots,
+                                                         (unsigned long long)bpe, E, C);
+    count_launch();
+}
+
+// ------------------------------------------------------------------------------------------------
 // Grouping.  key(pair p) = wave_of[e]*C + slot_of[e]  (identity mode, C = E: key = e).
 // Pairs with an invalid id are left out.  perm = pair indices ordered by key, ties by ascending p.
 // ------------------------------------------------------------------------------------------------

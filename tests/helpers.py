@@ -76,3 +76,24 @@ def oracle_plan(sc: ocache.SlotCache, ids):
     plan = sc.resolve(ids)
     counts, offsets, perm = ocache.group_pairs(ids, plan, sc.C, sc.max_waves)
     return plan, counts, offsets, perm
+
+
+def compare_plan(cache, sc, ids, layer=0):
+    """Advance the oracle's slot cache by this call and compare plan, grouping, state and counters bit for bit."""
+    plan, counts, offsets, perm = oracle_plan(sc, ids.numpy())
+    got = cache.last_plan(layer, ids.numel())
+    assert got["n_active"] == plan.n_active and got["n_waves"] == plan.n_waves
+    assert np.array_equal(got["wave_of"], plan.wave_of)
+    assert np.array_equal(got["slot_of"], plan.slot_of)
+    assert got["misses"] == plan.misses
+    assert np.array_equal(got["counts"], counts)
+    assert np.array_equal(got["offsets"], offsets)
+    assert np.array_equal(got["perm"], perm)
+    if sc.C < sc.E:
+        es, se, stamp, tick = cache.state(layer)
+        assert np.array_equal(es, sc.expert_slot) and np.array_equal(se, sc.slot_expert)
+        assert np.array_equal(stamp, sc.slot_stamp) and tick == sc.tick
+    st = cache.stats(layer)
+    assert st == {"lookups": sc.stats.lookups, "hits": sc.stats.hits, "misses": sc.stats.misses,
+                  "waves": sc.stats.waves, "h2d_bytes": sc.stats.h2d_bytes, "forwards": sc.stats.forwards}
+    return plan

@@ -81,24 +81,7 @@ def test_pack_special_groups_and_errors(B):
 
 
 # ------------------------------------------------------------------------------------ a1/a2: plan
-def compare_plan(cache, sc, ids, layer=0):
-    plan, counts, offsets, perm = helpers.oracle_plan(sc, ids.numpy())
-    got = cache.last_plan(layer, ids.numel())
-    assert got["n_active"] == plan.n_active and got["n_waves"] == plan.n_waves
-    assert np.array_equal(got["wave_of"], plan.wave_of)
-    assert np.array_equal(got["slot_of"], plan.slot_of)
-    assert got["misses"] == plan.misses
-    assert np.array_equal(got["counts"], counts)
-    assert np.array_equal(got["offsets"], offsets)
-    assert np.array_equal(got["perm"], perm)
-    if sc.C < sc.E:
-        es, se, stamp, tick = cache.state(layer)
-        assert np.array_equal(es, sc.expert_slot) and np.array_equal(se, sc.slot_expert)
-        assert np.array_equal(stamp, sc.slot_stamp) and tick == sc.tick
-    st = cache.stats(layer)
-    assert st == {"lookups": sc.stats.lookups, "hits": sc.stats.hits, "misses": sc.stats.misses,
-                  "waves": sc.stats.waves, "h2d_bytes": sc.stats.h2d_bytes, "forwards": sc.stats.forwards}
-    return plan
+compare_plan = helpers.compare_plan
 
 
 @pytest.mark.parametrize("C,Cw,T,alpha", [(8, 0, 16, 0.0), (2, 0, 5, 0.0), (4, 2, 16, 1.0), (3, 0, 1, 0.0), (5, 3, 40, 0.5)])
