@@ -271,6 +271,9 @@ def run_stack_sweep(args, dev, binding):
             torch.cuda.empty_cache()
             torch.cuda.reset_peak_memory_stats(dev)
             cache = binding.Cache(shape, banks, C, max_tokens=64, device=dev)
+            device_fetch = args.miss_path == "device" and C < shape.num_experts
+            if C < shape.num_experts:
+                cache.set_miss_path(binding.MISS_DEVICE_FETCH if device_fetch else binding.MISS_HOST_COPIES)
             stack = synth.SyntheticStack(shape, L, seed=5100, alpha=(0.5 if args.alpha is None else args.alpha), device=dev)
             # every step decodes fresh tokens: a new seeded hidden state enters layer 0 (as an embedding would)
             pool = [synth.hidden_states(shape, T, 5200 + i, device=dev) for i in range(16)]
@@ -283,8 +286,12 @@ def run_stack_sweep(args, dev, binding):
                 h = stack.step(fwd, pool[i % 16], route_fn=rt)
             torch.cuda.synchronize()
             graph = None
-            if C == shape.num_experts:                    # fully resident: no host sync inside, the step is graph-capturable
-                noise = stack.draw_noise(T)
+            if C == shape.num_experts or device_fetch:    # no host wait inside the layer call: the step is graph-capturable
+                # residual noise of all layers in one tensor the graph reads; redrawn before every replay (two launches),
+                # so that the replayed steps see the same random walk as host-driven ones
+                noise_all = torch.empty((L, T, shape.d_model), device=dev, dtype=torch.float32)
+                noise_all.normal_(generator=stack.gen).mul_(0.1)
+                noise = list(noise_all.unbind(0))
                 h_in = pool[0].clone()
                 side = torch.cuda.Stream(device=dev)
                 fwd_s = lambda l, x, ids, w: cache.forward(l, x, ids, w, stream=side)
@@ -302,6 +309,7 @@ def run_stack_sweep(args, dev, binding):
             for i in range(timed):
                 if graph is not None:
                     h_in.copy_(pool[(warm + i) % 16])
+                    noise_all.normal_(generator=stack.gen).mul_(0.1)
                     graph.replay()
                 else:
                     h = stack.step(fwd, pool[(warm + i) % 16], route_fn=rt)
@@ -315,6 +323,7 @@ def run_stack_sweep(args, dev, binding):
                          "hit_rate": (d("hits") / d("lookups")) if d("lookups") else None,
                          "waves_per_layer_call": (d("waves") / d("forwards")) if d("forwards") else 1.0,
                          "peak_reserved_gib": torch.cuda.max_memory_reserved(dev) / 2 ** 30,
+                         "miss_path": "device fetch" if device_fetch else ("host copies" if C < shape.num_experts else None),
                          "timing": "CUDA graph of the 16-layer step" if graph is not None else "host-driven"})
             assert cache.status() == 0 and bool(torch.isfinite(h.float()).all())
             cache.close()
@@ -332,8 +341,8 @@ def main():
     ap.add_argument("--workload", default="decode", choices=sorted(WORKLOADS) + ["stack"])
     ap.add_argument("--alpha", type=float, default=None,
                     help="Zipf skew: overrides the workload's alpha (stack workload: default 0.5)")
-    ap.add_argument("--miss-path", default="host", choices=["host", "device"],
-                    help="C < E workloads: host-issued miss copies (default) or the device-initiated fetch kernel")
+    ap.add_argument("--miss-path", default="device", choices=["host", "device"],
+                    help="C < E workloads: the device-initiated fetch kernel (the library's default) or host-issued miss copies")
     ap.add_argument("--slots", type=int, default=0, help="override the workload's resident slots per layer")
     ap.add_argument("--tokens", type=int, default=0, help="override the workload's tokens per step")
     ap.add_argument("--cpu-budget", type=float, default=15.0, help="seconds of CPU oracle work for cpu_baseline")
@@ -390,9 +399,9 @@ def main():
     seed0 = 2000 + 100000 * rank
     banks, w_cpu = build_banks(shape, L, seed0, dev, keep_layer0=(rank == 0))
     cache = binding.Cache(shape, banks, C, max_tokens=T, device=dev)
-    if args.miss_path == "device":
-        cache.set_miss_path(binding.MISS_DEVICE_FETCH)
-        desc += " [device-initiated miss fetch]"
+    if C < shape.num_experts:
+        cache.set_miss_path(binding.MISS_DEVICE_FETCH if args.miss_path == "device" else binding.MISS_HOST_COPIES)
+        desc += " [miss path: %s]" % ("device-initiated fetch kernel" if args.miss_path == "device" else "host-issued copies")
     n_sets = min(K + W, 1024) if T <= 64 else 4
     hs, ids, ws = make_inputs(shape, T, n_sets, alpha, seed0, dev)
     outs = [torch.empty_like(hs[0]) for _ in range(2)]
@@ -509,14 +518,22 @@ def main():
                 "kernel": "gate_up (pair_gateup_kernel)" if T * shape.top_k <= 24 else
                 "gate_up (stream_gemm_kernel<1,true,1>)" if T * shape.top_k <= 448 else "gate_up",
                 "bytes_per_launch": gu_bytes, "peak_source": peaks["source"] + " copy rate, burst"}
+    if not identity:
+        roof["note"] = ("C < E: the timed launches include resolution and the waves' miss traffic, so this fraction is not a "
+                        "kernel figure; the workload is bound by the host link: compare config.h2d_gb_per_s_during_copies "
+                        "with config.pinned_copy_ceiling_gb_per_s")
     step_gbs = active_all * bpe / (ms * 1e-3 / K) / 1e9
     step_tflops = 2.0 * T * shape.top_k * 3 * shape.d_ff * shape.d_model / (ms * 1e-3 / K) / 1e12
 
     # ---- end to end: host buffers in, host buffer out, copies inside the timed region
     n_e2e = min(K, 300)
-    h_h = [h.cpu().pin_memory() for h in hs[:8]]
-    h_i = [x.cpu().pin_memory() for x in ids[:8]]
-    h_w = [x.cpu().pin_memory() for x in ws[:8]]
+    # fully resident: eight input sets; with a cache (C < E) the sets are spread over the whole timed range, so that the
+    # end-to-end loop sees the same routing mix (hit rate) as the device-timed one
+    n_host = 8 if identity else min(n_sets, 128)
+    pick = [(j * n_sets) // n_host for j in range(n_host)]
+    h_h = [hs[j].cpu().pin_memory() for j in pick]
+    h_i = [ids[j].cpu().pin_memory() for j in pick]
+    h_w = [ws[j].cpu().pin_memory() for j in pick]
     h_out = torch.empty_like(h_h[0]).pin_memory()
     d_h, d_i, d_w, d_o = torch.empty_like(hs[0]), torch.empty_like(ids[0]), torch.empty_like(ws[0]), torch.empty_like(hs[0])
 
@@ -531,7 +548,7 @@ def main():
         stream.synchronize()
 
     e2e_mode = "per-step launches"
-    if identity and T <= 64:
+    if graphable and T <= 64:
         # serving-loop form: the step's inputs (hidden | ids | weights) sit in ONE pinned staging buffer and go to the
         # device in ONE copy; per layer one CUDA graph of [H2D copy, forward, D2H copy].  A step writes its inputs
         # into the staging buffer, replays the graph and waits for the result.

@@ -111,24 +111,26 @@ int exmoe_cache_create(exmoe_cache** out, const exmoe_shape* shape, int num_laye
  * accumulated in binary32 in the order j = 0..k-1 and rounded once to BF16, so the result does not
  * depend on C, wave_cap or cache history.  T = 0 is a no-op.  An id outside [0, E) contributes
  * nothing and sets the sticky status EXMOE_ERR_BAD_EXPERT_ID (see exmoe_status).
- * C = E: fully asynchronous on `stream`.  C < E: the resolution kernel's miss plan is read back
- * once (the paper's single batched id transfer) and the host waits for it; miss copies run on the
- * library's copy stream, ordered against the compute stream by events, and return before they finish. */
+ * C = E: fully asynchronous on `stream`.  C < E: see exmoe_cache_set_miss_path; with the default
+ * device-initiated miss path the call is fully asynchronous on `stream` as well. */
 int exmoe_moe_forward(exmoe_cache* cache, int layer, const void* hidden_bf16, const int32_t* topk_ids,
                       const float* topk_weights, int T, void* out_bf16, void* stream);
 
 /* How the misses of a C < E cache reach their slots (Sec. 3.4 step 3; the paper's runtime issues host copies).
- *   EXMOE_MISS_HOST_COPIES  (default): as described at exmoe_moe_forward: the host reads the miss plan once per
- *       call and issues one copy per missed expert on the library's copy stream; copies of a wave overlap the
- *       kernels of the wave before it.
- *   EXMOE_MISS_DEVICE_FETCH: the miss list stays on the device; before each wave's GEMM kernels a kernel on the
- *       caller's stream reads the wave's missed experts straight out of the pinned host bank (through its mapped
- *       device address, over PCIe) into their slots.  The host waits for nothing and exmoe_moe_forward becomes a
- *       fixed launch sequence that may be captured in a CUDA graph.  It launches ceil(min(T*k, E) / wave_cap)
- *       waves whatever the ids turn out to be (a wave without work finds none), and within one call copies do
- *       not overlap kernels.  Outputs, cache state and statistics are identical in both modes.
- * Synchronises the device, so the switch is ordered against earlier calls.  EXMOE_ERR_NOT_PINNED if a host
- * bank has no 16-byte aligned device-visible address; the mode is then unchanged.  No effect when C = E. */
+ *   EXMOE_MISS_DEVICE_FETCH (default when every host bank has a 16-byte aligned device-visible address, which
+ *       page-locked memory of cudaHostAlloc / cudaHostRegister has): the miss list stays on the device; before each
+ *       wave's GEMM kernels a kernel on the caller's stream reads the wave's missed experts straight out of the
+ *       pinned host bank (through its mapped address, over PCIe) into their slots.  The host waits for nothing and
+ *       exmoe_moe_forward is a fixed launch sequence that may be captured in a CUDA graph.  It launches
+ *       ceil(min(T*k, E) / wave_cap) waves whatever the ids turn out to be (a wave without work finds none), and
+ *       within one call copies do not overlap kernels.
+ *   EXMOE_MISS_HOST_COPIES: the resolution kernel's miss plan is read back once per call (the paper's single
+ *       batched id transfer) and the host waits for it, then issues one copy per missed expert on the library's
+ *       copy stream, ordered against the compute stream by events; the copies of a wave overlap the kernels of
+ *       the wave before it, and the call returns before they finish.  Not capturable.
+ * Outputs, cache state and statistics are identical in both modes.  The call synchronises the device, so the
+ * switch is ordered against earlier calls.  EXMOE_ERR_NOT_PINNED if device fetch is asked for and a bank has no
+ * such address; the mode is then unchanged.  No effect when C = E. */
 enum { EXMOE_MISS_HOST_COPIES = 0, EXMOE_MISS_DEVICE_FETCH = 1 };
 int exmoe_cache_set_miss_path(exmoe_cache* cache, int mode);
 

@@ -188,6 +188,23 @@ static int reset_layer(exmoe_cache* c, int layer) {
     return EXMOE_OK;
 }
 
+// Device-visible addresses of the host banks (the device-initiated miss path reads them over PCIe); false if a bank
+// is not mapped into the device's address space or its mapped address is not 16-byte aligned.
+static bool map_banks(exmoe_cache* c) {
+    std::vector<const uint8_t*> devp;
+    for (int l = 0; l < c->L; ++l) {
+        void* d = nullptr;
+        if (cudaHostGetDevicePointer(&d, const_cast<uint8_t*>(c->bank[l]), 0) != cudaSuccess || !d ||
+            (reinterpret_cast<uintptr_t>(d) & 15)) {
+            cudaGetLastError();
+            return false;
+        }
+        devp.push_back(static_cast<const uint8_t*>(d));
+    }
+    c->bank_dev = devp;
+    return true;
+}
+
 extern "C" {
 
 const char* exmoe_strerror(int code) {
@@ -277,6 +294,7 @@ int exmoe_cache_create(exmoe_cache** out, const exmoe_shape* shape, int num_laye
     c->last_layer = -1;
     c->last_T = 0;
     c->stream_ok = stream_supported(c->shape.d_model, c->shape.d_ff);
+    c->miss_path = map_banks(c) ? EXMOE_MISS_DEVICE_FETCH : EXMOE_MISS_HOST_COPIES;
     bool ok = cudaMallocHost(&c->h_plan, c->plan_d2h_bytes) == cudaSuccess;
     ok = ok && cudaStreamCreateWithFlags(&c->copy_stream, cudaStreamNonBlocking) == cudaSuccess;
     ok = ok && cudaEventCreateWithFlags(&c->ev_plan, cudaEventDisableTiming) == cudaSuccess;
@@ -486,19 +504,7 @@ int exmoe_moe_forward(exmoe_cache* c, int layer, const void* hidden, const int32
 int exmoe_cache_set_miss_path(exmoe_cache* c, int mode) {
     if (!c || (mode != EXMOE_MISS_HOST_COPIES && mode != EXMOE_MISS_DEVICE_FETCH)) return EXMOE_ERR_ARG;
     if (cudaDeviceSynchronize() != cudaSuccess) return EXMOE_ERR_CUDA;     // no wave of the other mode is in flight
-    if (mode == EXMOE_MISS_DEVICE_FETCH) {
-        std::vector<const uint8_t*> devp;
-        for (int l = 0; l < c->L; ++l) {
-            void* d = nullptr;
-            if (cudaHostGetDevicePointer(&d, const_cast<uint8_t*>(c->bank[l]), 0) != cudaSuccess || !d ||
-                (reinterpret_cast<uintptr_t>(d) & 15)) {
-                cudaGetLastError();
-                return EXMOE_ERR_NOT_PINNED;                                 // not mapped into the device's address space
-            }
-            devp.push_back(static_cast<const uint8_t*>(d));
-        }
-        c->bank_dev = devp;
-    }
+    if (mode == EXMOE_MISS_DEVICE_FETCH && !map_banks(c)) return EXMOE_ERR_NOT_PINNED;
     for (auto& v : c->slot_last_seq) std::fill(v.begin(), v.end(), 0);       // everything earlier has completed
     c->miss_path = mode;
     return EXMOE_OK;

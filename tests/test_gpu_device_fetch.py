@@ -35,8 +35,7 @@ def test_state_slots_and_output_match_oracle_and_resident_run(B, olmoe_layer, C,
     ora, bank = olmoe_layer
     s = synth.OLMOE
     full = B.Cache(s, [bank], 64, max_tokens=300)
-    dev = B.Cache(s, [bank], C, max_tokens=300, wave_cap=Cw)
-    dev.set_miss_path(B.MISS_DEVICE_FETCH)
+    dev = B.Cache(s, [bank], C, max_tokens=300, wave_cap=Cw)            # device-initiated fetch is the default
     sc = ocache.SlotCache(64, C, Cw, bytes_per_expert=dev.bytes_per_expert)
     waves = set()
     # pairwise (1, 2, 3), grouped small with several waves, streaming (16..56), tensor-core small-N and large-N

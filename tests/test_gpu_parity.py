@@ -84,11 +84,13 @@ def test_pack_special_groups_and_errors(B):
 compare_plan = helpers.compare_plan
 
 
+@pytest.mark.parametrize("miss_path", ["device", "host"])
 @pytest.mark.parametrize("C,Cw,T,alpha", [(8, 0, 16, 0.0), (2, 0, 5, 0.0), (4, 2, 16, 1.0), (3, 0, 1, 0.0), (5, 3, 40, 0.5)])
-def test_plan_bit_exact_tiny(B, tiny_layer, C, Cw, T, alpha):
+def test_plan_bit_exact_tiny(B, tiny_layer, C, Cw, T, alpha, miss_path):
     ora, bank = tiny_layer
     s = synth.TINY
     cache = B.Cache(s, [bank], C, max_tokens=64, wave_cap=Cw)
+    cache.set_miss_path(B.MISS_DEVICE_FETCH if miss_path == "device" else B.MISS_HOST_COPIES)
     sc = ocache.SlotCache(s.num_experts, C, Cw, bytes_per_expert=cache.bytes_per_expert)
     for step in range(12):
         hidden, ids, p = helpers.routed_inputs(s, T, seed=100 + step, alpha=alpha)
@@ -101,10 +103,12 @@ def test_plan_bit_exact_tiny(B, tiny_layer, C, Cw, T, alpha):
 @pytest.mark.parametrize("C,Cw,T,alpha", [(16, 0, 16, 1.0), (16, 8, 16, 0.5), (32, 0, 4, 1.0), (8, 0, 1, 0.0),
                                           (64, 0, 16, 1.0), (16, 0, 200, 0.0), (64, 0, 300, 1.0)])
 def test_plan_bit_exact_olmoe(B, olmoe_layer, C, Cw, T, alpha):
-    """Resolution, LRU, waves and grouping on OLMoE geometry, incl. the multi-CTA grouping path (T*k > 1024)."""
+    """Resolution, LRU, waves and grouping on OLMoE geometry, incl. the multi-CTA grouping path (T*k > 1024);
+    host-issued miss copies here, the device-initiated path (the default) has the same test in its own file."""
     ora, bank = olmoe_layer
     s = synth.OLMOE
     cache = B.Cache(s, [bank], C, max_tokens=max(T, 16), wave_cap=Cw)
+    cache.set_miss_path(B.MISS_HOST_COPIES)
     sc = ocache.SlotCache(s.num_experts, C, Cw, bytes_per_expert=cache.bytes_per_expert)
     for step in range(4 if T > 64 else 10):
         hidden, ids, p = helpers.routed_inputs(s, T, seed=300 + step, alpha=alpha)
@@ -113,11 +117,13 @@ def test_plan_bit_exact_olmoe(B, olmoe_layer, C, Cw, T, alpha):
     cache.close()
 
 
-def test_slot_bytes_after_miss_copies(B, olmoe_layer):
+@pytest.mark.parametrize("miss_path", ["device", "host"])
+def test_slot_bytes_after_miss_copies(B, olmoe_layer, miss_path):
     """After misses, every occupied slot holds exactly the host bank's bytes of its expert (Section 3.3)."""
     ora, bank = olmoe_layer
     s = synth.OLMOE
     cache = B.Cache(s, [bank], 16, max_tokens=16)
+    cache.set_miss_path(B.MISS_DEVICE_FETCH if miss_path == "device" else B.MISS_HOST_COPIES)
     for step in range(3):
         hidden, ids, p = helpers.routed_inputs(s, 16, seed=400 + step, alpha=0.5)
         cache.forward(0, hidden.cuda(), ids.cuda(), p.cuda())
@@ -233,6 +239,7 @@ def test_config3_offload_matches_resident(B, olmoe_layer):
     full = B.Cache(s, [bank], 64, max_tokens=16)
     small = B.Cache(s, [bank], 16, max_tokens=16)
     half = B.Cache(s, [bank], 16, max_tokens=16, wave_cap=8)
+    half.set_miss_path(B.MISS_HOST_COPIES)               # `small` takes the default, the device-initiated miss path
     sc = ocache.SlotCache(64, 16, 0, bytes_per_expert=small.bytes_per_expert)
     waves = set()
     for step, alpha in enumerate([2.0, 1.0, 0.5, 0.0, 2.0, 0.0]):
@@ -451,6 +458,7 @@ def test_random_sizes_are_invariant_to_slots_and_waves(B, olmoe_layer):
     full = B.Cache(s, [bank], 64, max_tokens=300)
     part = B.Cache(s, [bank], 16, max_tokens=300)
     half = B.Cache(s, [bank], 24, max_tokens=300, wave_cap=10)
+    part.set_miss_path(B.MISS_HOST_COPIES)               # one cache per miss path (`half`: device-initiated, the default)
     rng = np.random.default_rng(7)
     sizes = [1, 2, 3, 4, 5, 8, 16, 33, 56, 57, 64, 128, 129, 300]
     for it in range(24):
