@@ -507,3 +507,36 @@ def test_multi_layer_caches_are_independent(B, tiny_layer):
     cache.reset(0)
     assert cache.stats(0)["forwards"] == 0 and (cache.state(0)[0] == -1).all()
     cache.close()
+
+
+@pytest.mark.parametrize("T", [1, 5, 40, 160])
+def test_shared_expert_geometry(B, T):
+    """A Qwen-MoE-like block: routed experts with d_ff = 1408 (11 blocks of 128) chosen 4 at a time, plus a shared
+    expert of d_ff = 5632 (44 blocks) that every token uses with weight 1.  The shared expert is a second bank with
+    one expert and top_k = 1; the block output is the sum of the two layer outputs.  Both run on every kernel path
+    (pairwise, grouped small, streaming, tensor-core small-N) as T grows."""
+    routed = synth.Shape(d_model=2048, d_ff=1408, num_experts=12, top_k=4)
+    shared = synth.Shape(d_model=2048, d_ff=5632, num_experts=1, top_k=1)
+    if not hasattr(test_shared_expert_geometry, "layers"):
+        test_shared_expert_geometry.layers = (helpers.make_layer(routed, seed=611), helpers.make_layer(shared, seed=612))
+    (ora_r, bank_r), (ora_s, bank_s) = test_shared_expert_geometry.layers
+    hidden, ids, p = helpers.routed_inputs(routed, T, seed=6100 + T, alpha=0.5)
+    ids_s = torch.zeros((T, 1), dtype=torch.int32)
+    w_s = torch.ones((T, 1), dtype=torch.float32)
+    y_r, ref_r = ora_r.forward(hidden, ids, p)
+    y_s, ref_s = ora_s.forward(hidden, ids_s, w_s)
+    cr = B.Cache(routed, [bank_r], 6, max_tokens=160)                       # half of the routed experts resident
+    cs = B.Cache(shared, [bank_s], 1, max_tokens=160)
+    out_r = cr.forward(0, hidden.cuda(), ids.cuda(), p.cuda()).clone()
+    out_s = cs.forward(0, hidden.cuda(), ids_s.cuda(), w_s.cuda()).clone()
+    helpers.check_output(out_r, y_r, ref_r, f"routed T={T}")
+    helpers.check_output(out_s, y_s, ref_s, f"shared T={T}")
+    block = out_r.float() + out_s.float()                                    # the caller's sum, as for the residual
+    want = ref_r.astype(np.float64) + ref_s.astype(np.float64)
+    err = block.cpu().numpy().astype(np.float64) - want
+    assert np.linalg.norm(err) <= 2 * helpers.REL_FRO * np.linalg.norm(want)
+    full = B.Cache(routed, [bank_r], 12, max_tokens=160)
+    assert torch.equal(full.forward(0, hidden.cuda(), ids.cuda(), p.cuda()).view(torch.int16), out_r.view(torch.int16))
+    for c in (cr, cs, full):
+        assert c.status() == 0
+        c.close()
