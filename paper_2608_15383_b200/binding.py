@@ -180,6 +180,30 @@ def pack_bank(shape, w_gate, w_up, w_down, device="cuda"):
     return bank
 
 
+def padded_dims(d_model, d_ff, group=128):
+    """Section 3.2 asks for dims that are multiples of the group size (other shapes "may require padding"): the
+    next multiples of 128."""
+    up = lambda n: -(-int(n) // group) * group
+    return up(d_model), up(d_ff)
+
+
+def pad_expert_weights(w_gate, w_up, w_down, group=128):
+    """Zero-pad [E, I, H], [E, I, H], [E, H, I] expert tensors to multiples of 128 in both dims.  The padded
+    intermediate channels compute SiLU(0) * 0 = 0 and meet zero columns of W_down; the padded hidden channels meet
+    zero weights: columns [0, H) of the padded layer's output are the layer applied to the unpadded hidden state
+    (quantised in groups that end at the padded length), columns [H, H_pad) are zero.  Pad the hidden state with
+    pad_hidden and slice the output back."""
+    E, I, H = w_gate.shape
+    Hp, Ip = padded_dims(H, I, group)
+    pad = torch.nn.functional.pad
+    return (pad(w_gate, (0, Hp - H, 0, Ip - I)).contiguous(), pad(w_up, (0, Hp - H, 0, Ip - I)).contiguous(),
+            pad(w_down, (0, Ip - I, 0, Hp - H)).contiguous())
+
+
+def pad_hidden(hidden, d_model_padded):
+    return torch.nn.functional.pad(hidden, (0, d_model_padded - hidden.shape[-1])).contiguous()
+
+
 MISS_HOST_COPIES, MISS_DEVICE_FETCH = 0, 1
 
 

@@ -28,6 +28,8 @@ resolve_kernel(const int32_t* __restrict__ ids, int n_pairs, int E, int C, int C
     __shared__ int s_bad;
 
     const int tid = threadIdx.x;
+    // the miss-fetch kernel of the first wave may be placed now; it reads the plan only after this grid has completed
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     if (tid == 0) s_bad = 0;
     for (int e = tid; e < E; e += blockDim.x) {
         s_flag[e] = 0;
@@ -164,6 +166,7 @@ __global__ void __launch_bounds__(kFetchThreads)
 fetch_misses_kernel(const int32_t* __restrict__ header, const int32_t* __restrict__ misses, int wave,
                     const uint8_t* __restrict__ bank, uint8_t* __restrict__ slots, unsigned long long bpe, int E, int C) {
     __shared__ int s_lo, s_hi;
+    asm volatile("griddepcontrol.wait;" ::: "memory");  // launched as a programmatic dependent of the resolution kernel (wave 0)
     if (threadIdx.x == 0) {                            // the list is ordered by wave: this wave's entries are one run
         int n = header[HDR_N_MISSES];
         n = n < 0 ? 0 : (n > E ? E : n);
@@ -205,8 +208,20 @@ void launch_fetch_misses(const PlanPtrs& plan, int wave, const uint8_t* bank_dev
     int sms = 0, dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0)
         sms = 148;
-    fetch_misses_kernel<<<2 * sms, kFetchThreads, 0, st>>>(plan.header, plan.misses, wave, bank_dev, slots,
-                                                         (unsigned long long)bpe, E, C);
+    cudaLaunchConfig_t lc{};
+    lc.gridDim = dim3(2 * sms);
+    lc.blockDim = dim3(kFetchThreads);
+    lc.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    lc.attrs = attr;
+    lc.numAttrs = (wave == 0) ? 1 : 0;                 // wave 0 directly follows the resolution kernel
+#ifdef EXMOE_DISABLE_PDL
+    lc.numAttrs = 0;
+#endif
+    cudaLaunchKernelEx(&lc, fetch_misses_kernel, (const int32_t*)plan.header, (const int32_t*)plan.misses, wave, bank_dev, slots,
+                       (unsigned long long)bpe, E, C);
     count_launch();
 }
 

@@ -540,3 +540,45 @@ def test_shared_expert_geometry(B, T):
     for c in (cr, cs, full):
         assert c.status() == 0
         c.close()
+
+
+def test_padding_of_dims_that_are_not_multiples_of_128(B):
+    """Section 3.2: other shapes "may require padding".  d_model = 200, d_ff = 300 padded with zeros to 256 / 384:
+    the padded layer matches the oracle on the padded weights, its extra output columns are exactly zero, and the
+    first 200 columns agree, up to int4 quantisation noise, with the unquantised layer (Eq. 2) on the unpadded weights."""
+    raw = synth.Shape(d_model=200, d_ff=300, num_experts=4, top_k=2)
+    g = torch.Generator().manual_seed(99)
+    wg = (torch.randn((4, 300, 200), generator=g) * 0.05).bfloat16()
+    wu = (torch.randn((4, 300, 200), generator=g) * 0.05).bfloat16()
+    wd = (torch.randn((4, 200, 300), generator=g) * 0.05).bfloat16()
+    Hp, Ip = B.padded_dims(200, 300)
+    assert (Hp, Ip) == (256, 384)
+    pg, pu, pd = B.pad_expert_weights(wg, wu, wd)
+    assert pg.shape == (4, 384, 256) and pd.shape == (4, 256, 384)
+    assert torch.equal(pg[:, :300, :200], wg) and float(pg[:, 300:, :].abs().max()) == 0 and float(pd[:, 200:, :].abs().max()) == 0
+    s = synth.Shape(d_model=Hp, d_ff=Ip, num_experts=4, top_k=2)
+    ora = helpers.OracleLayer(s, pg, pu, pd)
+    bank = B.pack_bank(s, pg, pu, pd)
+    T = 9
+    hidden = torch.randn((T, 200), generator=g).bfloat16()
+    ids = torch.stack([torch.randperm(4, generator=g)[:2] for _ in range(T)]).int()
+    p = torch.rand((T, 2), generator=g).float()
+    hp = B.pad_hidden(hidden, Hp)
+    cache = B.Cache(s, [bank], 4, max_tokens=16)
+    out = cache.forward(0, hp.cuda(), ids.cuda(), p.cuda())
+    y, ref = ora.forward(hp, ids, p)
+    helpers.check_output(out, y, ref, "padded")
+    assert float(out[:, 200:].float().abs().max()) == 0.0
+    # the unpadded, unquantised layer in fp64: Eq. 2 on the original tensors
+    x = hidden.double().numpy()
+    want = np.zeros((T, 200))
+    for t in range(T):
+        for j in range(2):
+            e = int(ids[t, j])
+            a, b = wg[e].double().numpy() @ x[t], wu[e].double().numpy() @ x[t]
+            want[t] += float(p[t, j]) * (wd[e].double().numpy() @ (a / (1 + np.exp(-a)) * b))
+    got = out[:, :200].float().cpu().numpy().astype(np.float64)
+    # int4 group quantisation noise of three matrices is ~0.2 of the signal; a misplaced column or slice gives ~1.4
+    assert np.linalg.norm(got - want) <= 0.35 * np.linalg.norm(want)
+    assert cache.status() == 0
+    cache.close()
