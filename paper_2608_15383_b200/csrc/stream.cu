@@ -248,7 +248,7 @@ stream_gemm_kernel(const StreamArgs p) {
             const unsigned ballot = __ballot_sync(0xffffffffu, overlap);
             if (overlap) {
                 const int idx = found + __popc(ballot & ((1u << lane) - 1u));
-                if (idx < kMetaGroups) meta_w[idx] = make_int4(key, rows, row0, ustart);
+                if (idx < kMetaGroups) meta_w[idx] = make_int4(key % a.num_slots, rows, row0, ustart);   // .x = slot of the group
             }
             found += __popc(ballot);
             run += __shfl_sync(0xffffffffu, incl, 31);
@@ -276,19 +276,24 @@ stream_gemm_kernel(const StreamArgs p) {
 
     if (warp == kConsumerWarps) {
         // ---------------------------------------------------------------- weight producer
-        int n = 0;
+        // ring position and phase are carried along: no division in any per-unit path of this kernel (a runtime
+        // integer division costs some 25 instructions, several of them on the quarter-rate conversion pipe)
+        int n = 0, s = 0;
+        uint32_t ph = 1;                               // parity of the stage's previous phase
         for (int u = u0; u < u1; ++u, ++n) {
-            const int s = n % S;
-            if (n >= S && !warp_wait(&w_empty[s], ((n / S) - 1) & 1, abort_flag, p.status)) break;
+            if (n >= S && !warp_wait(&w_empty[s], ph, abort_flag, p.status)) break;
             const int4 gm = meta[cur.gi];
             if (lane == 0) {
-                const int slot = gm.x % a.num_slots;
-                const uint8_t* src = a.slots + (size_t)slot * a.slot_stride + mat_off + (size_t)cur.tile * p.stage_bytes;
+                const uint8_t* src = a.slots + (size_t)gm.x * a.slot_stride + mat_off + (size_t)cur.tile * p.stage_bytes;
                 mbar_expect_tx(&w_full[s], p.stage_bytes);
                 bulk_load(wst + (size_t)s * p.stage_bytes, src, p.stage_bytes, &w_full[s]);
             }
             __syncwarp();
             cur.advance(tiles, (gm.y + R - 1) / R);
+            if (++s == S) {
+                s = 0;
+                ph ^= 1u;
+            }
         }
         if (*abort_flag && lane == 0) {                // copies in flight land before the shared memory is given up
             for (int j = (n > S ? n - S : 0); j < n; ++j) {
@@ -299,12 +304,12 @@ stream_gemm_kernel(const StreamArgs p) {
     } else if (warp == kConsumerWarps + 1) {
         // ---------------------------------------------------------------- activation producer
         if (!GATEUP) grid_dependency_wait();           // the gate/up kernel's activations are complete and visible
-        int n = 0;
+        int n = 0, b = 0;
+        uint32_t ph = 1;
         for (int u = u0; u < u1; ++u) {
             const int4 gm = meta[cur.gi];
             if (u == u0 || cur.tile == 0) {            // first unit of a (group, pass): stage its rows
-                const int b = n % NX;
-                if (n >= NX && !warp_wait(&x_empty[b], ((n / NX) - 1) & 1, abort_flag, p.status)) break;
+                if (n >= NX && !warp_wait(&x_empty[b], ph, abort_flag, p.status)) break;
                 const int pass0 = cur.pass * R;
                 const int rows_here = min(R, gm.y - pass0);
                 if (lane == 0) mbar_expect_tx(&x_full[b], (uint32_t)rows_here * K * 2);
@@ -316,6 +321,10 @@ stream_gemm_kernel(const StreamArgs p) {
                 }
                 __syncwarp();
                 ++n;
+                if (++b == NX) {
+                    b = 0;
+                    ph ^= 1u;
+                }
             }
             cur.advance(tiles, (gm.y + R - 1) / R);
         }
@@ -334,7 +343,9 @@ stream_gemm_kernel(const StreamArgs p) {
         // partials of one unit: [pp][matrix][ks][ch][i][lane], one buffer per group and unit parity
         const int part_words = kGroupWarps * NMW * NCH * 128;
         float* adjg = adj + (size_t)grp * NX * KB * R;
-        int xk = 0, mine_cnt = 0;
+        int mine_cnt = 0;
+        int s = -1, xb = -1;                           // weight stage and row buffer of the current unit
+        uint32_t w_ph = 1, x_ph = 1;                   // their barrier parities (flipped when the index wraps to 0)
         // Both groups walk ALL units in order and observe every phase of every full barrier, also for units and
         // rows the other group computes on, and release each stage only then: a parity wait is only valid for a
         // waiter that is at most one phase behind.
@@ -350,36 +361,42 @@ stream_gemm_kernel(const StreamArgs p) {
             const bool fresh = (u == u0 || tile == 0);
             const bool x_done = (u + 1 == u1 || tile == tiles - 1);
             cur.advance(tiles, (m_rows + R - 1) / R);
-            if (fresh) ++xk;
-            const int xb = (xk - 1) % NX;
+            if (fresh && ++xb == NX) xb = 0;
+            if (fresh && xb == 0) x_ph ^= 1u;
             const int rows_here = min(R, m_rows - pass0);
-            const int s = n % S;
+            if (++s == S) s = 0;
+            if (s == 0) w_ph ^= 1u;
             const unsigned char* xbuf = xs + (size_t)xb * R * p.x_stride;
             float* adjb = adjg + (size_t)xb * KB * R;
             if (fresh) {                               // new rows: each group forms its own copy of the corrections
-                if (!mbar_wait(&x_full[xb], ((xk - 1) / NX) & 1, abort_flag, p.status)) ok = false;
-                // adj[kb][n] = -136 * sum of the row's activations over block kb (removes the code bias after the MMA)
-                const int chunks_per_row = K / 8, total = rows_here * chunks_per_row;
-                for (int base = cw * 32; base < total; base += kGroupThreads) {
-                    const int idx = base + lane;
-                    const int nn = idx / chunks_per_row, ck = idx % chunks_per_row;
-                    uint4 v = make_uint4(0, 0, 0, 0);
-                    if (idx < total) v = *reinterpret_cast<const uint4*>(xbuf + (size_t)nn * p.x_stride + ck * 16);
-                    float sx = sum8_bf16(v);
+                if (!mbar_wait(&x_full[xb], x_ph, abort_flag, p.status)) ok = false;
+                // adj[kb][n] = -136 * sum of the row's activations over block kb (removes the code bias after the MMA);
+                // a block is 16 chunks of 8 values: the 16 lanes of a half-warp hold one block of one row
+                const int chunks_per_row = K >> 3;
+                for (int nn = 0; nn < rows_here; ++nn) {
+                    const unsigned char* xrow = xbuf + (size_t)nn * p.x_stride;
+                    for (int base = cw * 32; base < chunks_per_row; base += kGroupThreads) {
+                        const int ck = base + lane;
+                        uint4 v = make_uint4(0, 0, 0, 0);
+                        if (ck < chunks_per_row) v = *reinterpret_cast<const uint4*>(xrow + ck * 16);
+                        float sx = sum8_bf16(v);
 #pragma unroll
-                    for (int m = 8; m >= 1; m >>= 1) sx += __shfl_xor_sync(0xffffffffu, sx, m);
-                    if (idx < total && (ck & 15) == 0) adjb[(ck >> 4) * R + nn] = -136.f * sx;
+                        for (int m = 8; m >= 1; m >>= 1) sx += __shfl_xor_sync(0xffffffffu, sx, m);
+                        if (ck < chunks_per_row && (ck & 15) == 0) adjb[(ck >> 4) * R + nn] = -136.f * sx;
+                    }
                 }
                 // rows beyond the group's last are zeroed once per staging (both consumer groups write the same zeros:
                 // each reads them only after its own barrier below; no copy targets these rows until every warp
                 // has released the buffer), so the fragment loads of the MMA loop need no row predicate
-                for (int idx = total + cw * 32 + lane; idx < R * chunks_per_row; idx += kGroupThreads)
-                        *reinterpret_cast<uint4*>(const_cast<unsigned char*>(xbuf) + (size_t)(idx / chunks_per_row) * p.x_stride +
-                                                  (idx % chunks_per_row) * 16) = make_uint4(0, 0, 0, 0);
+                for (int nn = rows_here; nn < R; ++nn) {
+                    unsigned char* xrow = const_cast<unsigned char*>(xbuf) + (size_t)nn * p.x_stride;
+                    for (int ck = cw * 32 + lane; ck < chunks_per_row; ck += kGroupThreads)
+                        *reinterpret_cast<uint4*>(xrow + ck * 16) = make_uint4(0, 0, 0, 0);
+                }
                 group_sync(grp);
             }
             SPROF(long long c1 = clock64(); t_x += c1 - c0;)
-            if (!mbar_wait(&w_full[s], (n / S) & 1, abort_flag, p.status)) ok = false;
+            if (!mbar_wait(&w_full[s], w_ph, abort_flag, p.status)) ok = false;
             SPROF(long long c2 = clock64(); t_w += c2 - c1;)
             if ((n & 1) != grp) {                      // the other group's unit: nothing of this warp reads it
                 if (lane == 0) {
