@@ -516,7 +516,7 @@ def main():
                 "traffic": NCU_TRAFFIC_BYTES.get(args.workload) if not args.tokens else None,
                 "traffic_unit": "bytes per launch (ncu dram read + write)",
                 "kernel": "gate_up (pair_gateup_kernel)" if T * shape.top_k <= 24 else
-                "gate_up (stream_gemm_kernel<1,true,1>)" if T * shape.top_k <= 448 else "gate_up",
+                "gate_up (stream_gemm_kernel<1,true,1>)" if T * shape.top_k <= 512 else "gate_up",
                 "bytes_per_launch": gu_bytes, "peak_source": peaks["source"] + " copy rate, burst"}
     if not identity:
         roof["note"] = ("C < E: the timed launches include resolution and the waves' miss traffic, so this fraction is not a "

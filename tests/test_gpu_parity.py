@@ -434,7 +434,7 @@ def test_graph_replay_matches_oracle(B, olmoe_layer, T):
 @pytest.mark.parametrize("T", [1, 3, 8, 33, 100])
 def test_rounding_matched_oracle_mode_is_nearly_bit_exact(B, mid_layer, T):
     """Against the oracle's second mode (SwiGLU output rounded to BF16 before the down projection, the one rounding
-    the BF16 activation buffer forces) the register-dequantisation paths (T*k <= 448: codes and activations enter the
+    the BF16 activation buffer forces) the register-dequantisation paths (T*k <= 512: codes and activations enter the
     MMA exactly, scales are applied in binary32) agree almost bit for bit: what is left is binary32 summation order
     meeting a BF16 rounding boundary."""
     ora, bank = mid_layer
