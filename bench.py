@@ -281,9 +281,41 @@ def run_stack_sweep(args, dev, binding):
             bias32 = [None if b is None else b.float().contiguous() for b in stack.bias]
             # the library's fused router (Eq. 1) on the current stream instead of the harness's torch router
             rt = lambda l, x: binding.exmoe_route(shape, x, stack.routers[l], bias32[l])
+            # next-layer prefetch policy: layer l+1's router applied to layer l's input, on a side stream; layer l+1's
+            # forward waits for that prefetch (an event), layer l's kernels run beside it
+            # (only while the guessed set fits the layer's slots: a larger prefetch would evict its own first wave)
+            use_pf = args.prefetch and device_fetch and T * shape.top_k <= C
+            pf_side = torch.cuda.Stream(device=dev) if use_pf else None
+            pf_done = {}
+
+            def make_hooks(main_stream):
+                if not use_pf:
+                    return None, (lambda l, x, ids, w: cache.forward(l, x, ids, w, stream=main_stream))
+
+                def look(l_next, x):
+                    ready = torch.cuda.Event()
+                    ready.record(main_stream)
+                    pf_side.wait_event(ready)
+                    x.record_stream(pf_side)                       # the side stream reads the layer input after this call returns
+                    with torch.cuda.stream(pf_side):
+                        guess, _ = binding.exmoe_route(shape, x, stack.routers[l_next], bias32[l_next], stream=pf_side)
+                        cache.prefetch(l_next, guess, stream=pf_side)
+                        ev = torch.cuda.Event()
+                        ev.record(pf_side)
+                    pf_done[l_next] = ev
+
+                def fwd_pf(l, x, ids, w):
+                    ev = pf_done.pop(l, None)
+                    if ev is not None:
+                        main_stream.wait_event(ev)
+                    return cache.forward(l, x, ids, w, stream=main_stream)
+                return look, fwd_pf
             warm, timed = (args.warmup or 16), (args.steps if args.steps < 1000 else 64)
+            look0, fwd0 = make_hooks(torch.cuda.current_stream())
+            if use_pf:
+                fwd = fwd0
             for i in range(warm):
-                h = stack.step(fwd, pool[i % 16], route_fn=rt)
+                h = stack.step(fwd, pool[i % 16], route_fn=rt, lookahead_fn=look0)
             torch.cuda.synchronize()
             graph = None
             if C == shape.num_experts or device_fetch:    # no host wait inside the layer call: the step is graph-capturable
@@ -294,13 +326,14 @@ def run_stack_sweep(args, dev, binding):
                 noise = list(noise_all.unbind(0))
                 h_in = pool[0].clone()
                 side = torch.cuda.Stream(device=dev)
-                fwd_s = lambda l, x, ids, w: cache.forward(l, x, ids, w, stream=side)
+                look_s, fwd_s = make_hooks(side)
                 with torch.cuda.stream(side):
-                    stack.step(fwd_s, h_in, noise=noise, route_fn=rt)
+                    stack.step(fwd_s, h_in, noise=noise, route_fn=rt, lookahead_fn=look_s)
                 side.synchronize()
+                torch.cuda.synchronize()
                 graph = torch.cuda.CUDAGraph()
                 with torch.cuda.graph(graph, stream=side):
-                    h = stack.step(fwd_s, h_in, noise=noise, route_fn=rt)
+                    h = stack.step(fwd_s, h_in, noise=noise, route_fn=rt, lookahead_fn=look_s)
                 graph.replay()
                 torch.cuda.synchronize()
             st0 = [cache.stats(l) for l in range(L)]
@@ -312,7 +345,7 @@ def run_stack_sweep(args, dev, binding):
                     noise_all.normal_(generator=stack.gen).mul_(0.1)
                     graph.replay()
                 else:
-                    h = stack.step(fwd, pool[(warm + i) % 16], route_fn=rt)
+                    h = stack.step(fwd, pool[(warm + i) % 16], route_fn=rt, lookahead_fn=look0)
             e1.record()
             torch.cuda.synchronize()
             ms = e0.elapsed_time(e1) / timed
@@ -323,6 +356,7 @@ def run_stack_sweep(args, dev, binding):
                          "hit_rate": (d("hits") / d("lookups")) if d("lookups") else None,
                          "waves_per_layer_call": (d("waves") / d("forwards")) if d("forwards") else 1.0,
                          "peak_reserved_gib": torch.cuda.max_memory_reserved(dev) / 2 ** 30,
+                         "prefetch": bool(use_pf),
                          "miss_path": "device fetch" if device_fetch else ("host copies" if C < shape.num_experts else None),
                          "timing": "CUDA graph of the 16-layer step" if graph is not None else "host-driven"})
             assert cache.status() == 0 and bool(torch.isfinite(h.float()).all())
@@ -343,6 +377,9 @@ def main():
                     help="Zipf skew: overrides the workload's alpha (stack workload: default 0.5)")
     ap.add_argument("--miss-path", default="device", choices=["host", "device"],
                     help="C < E workloads: the device-initiated fetch kernel (the library's default) or host-issued miss copies")
+    ap.add_argument("--prefetch", action="store_true",
+                    help="stack workload, C < E: guess layer l+1's experts by routing layer l's input with layer l+1's "
+                         "router and prefetch them on a side stream while layer l runs (exmoe_cache_prefetch)")
     ap.add_argument("--slots", type=int, default=0, help="override the workload's resident slots per layer")
     ap.add_argument("--tokens", type=int, default=0, help="override the workload's tokens per step")
     ap.add_argument("--cpu-budget", type=float, default=15.0, help="seconds of CPU oracle work for cpu_baseline")

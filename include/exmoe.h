@@ -134,6 +134,19 @@ int exmoe_moe_forward(exmoe_cache* cache, int layer, const void* hidden_bf16, co
 enum { EXMOE_MISS_HOST_COPIES = 0, EXMOE_MISS_DEVICE_FETCH = 1 };
 int exmoe_cache_set_miss_path(exmoe_cache* cache, int mode);
 
+/* Prefetch (the paper cites prefetching as related work and leaves it out; Sec. 3.3's slot map is what it acts on).
+ * Treats `expert_ids` (dev, int32 [n_ids], any order, repeats allowed, n_ids <= max_tokens * top_k) as the ids of a
+ * layer call without tokens: the slot map, LRU stamps, waves and counters of `layer` advance exactly as in
+ * Sec. 3.3 / 3.4 steps 1-3 for those ids (hits are stamped, misses evict the least recently used unprotected slots
+ * and are fetched from the host bank), and nothing is computed.  A later exmoe_moe_forward that selects these
+ * experts then finds them resident.  Outputs never depend on the cache state, so a wrong guess costs transfer time
+ * and slots, not correctness.  Asynchronous on `stream`; uses its own resolution buffers, so it may run beside an
+ * exmoe_moe_forward of ANOTHER layer on another stream; calls on the same layer (prefetch or forward) must be
+ * ordered by the caller (same stream, or events).  Needs the device-initiated miss path (EXMOE_ERR_STATE
+ * otherwise); no-op when C = E or n_ids = 0.  An id outside [0, E) is ignored and sets the sticky status
+ * EXMOE_ERR_BAD_EXPERT_ID. */
+int exmoe_cache_prefetch(exmoe_cache* cache, int layer, const int32_t* expert_ids, int n_ids, void* stream);
+
 /* Router of one sparse block (Eq. 1; Sec. 3.4 "router weights are ... not renormalized"): logits z_t = W_r h_t in
  * binary32 (BF16 products, fixed summation order), plus `bias` if given, softmax over all E experts, the k
  * largest, equal values ordered by ascending expert id.  Writes exmoe_moe_forward's inputs on the device.

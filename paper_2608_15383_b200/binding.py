@@ -56,6 +56,7 @@ _SIGNATURES = {
     "exmoe_cache_stats": (c_int, [c_void_p, c_int, POINTER(exmoe_stats)]),
     "exmoe_cache_reset": (c_int, [c_void_p, c_int]),
     "exmoe_cache_set_miss_path": (c_int, [c_void_p, c_int]),
+    "exmoe_cache_prefetch": (c_int, [c_void_p, c_int, c_void_p, c_int, c_void_p]),
     "exmoe_status": (c_int, [c_void_p]),
     "exmoe_cache_destroy": (c_int, [c_void_p]),
     "exmoe_profile_enable": (c_int, [c_void_p, c_int]),
@@ -292,6 +293,11 @@ class Cache:
     def set_miss_path(self, mode):
         """mode: MISS_HOST_COPIES (default) or MISS_DEVICE_FETCH (no host wait; graph-capturable with C < E)."""
         _check(lib().exmoe_cache_set_miss_path(self.handle, int(mode)), "exmoe_cache_set_miss_path")
+
+    # exmoe_cache_prefetch
+    def prefetch(self, layer, expert_ids, stream=None):
+        _check(lib().exmoe_cache_prefetch(self.handle, int(layer), _dev(expert_ids, torch.int32, "expert_ids"),
+                                          int(expert_ids.numel()), _stream_ptr(stream)), "exmoe_cache_prefetch")
 
     def reset(self, layer):
         _check(lib().exmoe_cache_reset(self.handle, layer), "exmoe_cache_reset")

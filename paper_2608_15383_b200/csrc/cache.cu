@@ -57,6 +57,7 @@ struct exmoe_cache {
     int* d_status;
     std::vector<LayerState> state;
     PlanPtrs plan;
+    PlanPtrs plan_pf;                         // resolution results of exmoe_cache_prefetch (its own copy: may overlap a forward)
     size_t plan_d2h_bytes;                    // header | wave_of | slot_of | misses, contiguous
     __nv_bfloat16* act;                       // [max_pairs, I] SwiGLU output, grouped row order
     float* y;                                 // [max_pairs, H] weighted expert outputs, pair order
@@ -125,6 +126,12 @@ static void carve_workspace(exmoe_cache* c, uint8_t* ws, size_t* total) {
     c->plan.slot_of = p ? p + HDR_WORDS + E : nullptr;
     c->plan.misses = p ? p + HDR_WORDS + 2 * E : nullptr;
     c->plan_d2h_bytes = (HDR_WORDS + 5 * (size_t)E) * 4;
+    int32_t* pf = k.take<int32_t>(HDR_WORDS + 5 * (size_t)E);
+    c->plan_pf = PlanPtrs{};
+    c->plan_pf.header = pf;
+    c->plan_pf.wave_of = pf ? pf + HDR_WORDS : nullptr;
+    c->plan_pf.slot_of = pf ? pf + HDR_WORDS + E : nullptr;
+    c->plan_pf.misses = pf ? pf + HDR_WORDS + 2 * E : nullptr;
     c->plan.counts = k.take<int32_t>(c->n_keys);
     c->plan.offsets = k.take<int32_t>(c->n_keys + 1);
     c->plan.group_keys = k.take<int32_t>(c->n_keys);
@@ -304,6 +311,7 @@ int exmoe_cache_create(exmoe_cache** out, const exmoe_shape* shape, int num_laye
     }
     ok = ok && cudaMemset(c->d_status, 0, 256) == cudaSuccess;
     ok = ok && cudaMemset(c->plan.header, 0, c->plan_d2h_bytes) == cudaSuccess;
+    ok = ok && cudaMemset(c->plan_pf.header, 0, c->plan_d2h_bytes) == cudaSuccess;
     ok = ok && cudaMemset(c->arrive, 0, c->arrive_words * 4) == cudaSuccess;
     ok = ok && cudaMemset(c->plan.chunk_done, 0, 256) == cudaSuccess;
     for (int l = 0; l < num_layers && ok; ++l) ok = reset_layer(c, l) == EXMOE_OK;
@@ -508,6 +516,23 @@ int exmoe_cache_set_miss_path(exmoe_cache* c, int mode) {
     for (auto& v : c->slot_last_seq) std::fill(v.begin(), v.end(), 0);       // everything earlier has completed
     c->miss_path = mode;
     return EXMOE_OK;
+}
+
+int exmoe_cache_prefetch(exmoe_cache* c, int layer, const int32_t* expert_ids, int n_ids, void* stream) {
+    if (!c || layer < 0 || layer >= c->L || n_ids < 0 || n_ids > c->max_pairs) return EXMOE_ERR_ARG;
+    if (n_ids == 0 || c->C == c->shape.num_experts) return EXMOE_OK;          // nothing to bring in
+    if (!expert_ids) return EXMOE_ERR_ARG;
+    if (c->miss_path != EXMOE_MISS_DEVICE_FETCH) return EXMOE_ERR_STATE;
+    cudaStream_t st = (cudaStream_t)stream;
+    const int E = c->shape.num_experts;
+    launch_resolve(c->shape, c->C, c->Cw, c->bpe, expert_ids, n_ids, c->state[layer], c->plan_pf, c->d_status, st);
+    const int act_max = n_ids < E ? n_ids : E;
+    int n_waves = (act_max + c->Cw - 1) / c->Cw;
+    if (n_waves > c->max_waves) n_waves = c->max_waves;
+    for (int w = 0; w < n_waves; ++w)
+        launch_fetch_misses(c->plan_pf, w, c->bank_dev[layer], c->slot_mem + (size_t)layer * c->C * c->bpe, c->bpe, E, c->C, st,
+                            /*small_grid=*/true);
+    return cudaGetLastError() == cudaSuccess ? EXMOE_OK : EXMOE_ERR_CUDA;
 }
 
 int exmoe_cache_get_state(exmoe_cache* c, int layer, int32_t* expert_slot, int32_t* slot_expert, uint64_t* slot_stamp,

@@ -109,7 +109,7 @@ void launch_resolve(const exmoe_shape& s, int C, int Cw, size_t bytes_per_expert
                     LayerState state, PlanPtrs plan, int* d_status, cudaStream_t st);
 // Device-initiated miss path: one kernel copies wave `wave`'s missed experts from the mapped host bank into their slots.
 void launch_fetch_misses(const PlanPtrs& plan, int wave, const uint8_t* bank_dev, uint8_t* slots, size_t bpe, int E, int C,
-                         cudaStream_t st);
+                         cudaStream_t st, bool small_grid = false);
 void launch_group(const exmoe_shape& s, int C, int n_keys, int max_waves, bool identity, const int32_t* ids,
                   int n_pairs, PlanPtrs plan, int* d_status, cudaStream_t st);
 // Streaming kernels (bulk-copy weight ring in shared memory) for kSmallMaxPairs < T*k <= kStreamMaxPairs.

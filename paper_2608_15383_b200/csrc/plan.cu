@@ -204,12 +204,14 @@ fetch_misses_kernel(const int32_t* __restrict__ header, const int32_t* __restric
 }
 
 void launch_fetch_misses(const PlanPtrs& plan, int wave, const uint8_t* bank_dev, uint8_t* slots, size_t bpe, int E, int C,
-                         cudaStream_t st) {
+                         cudaStream_t st, bool small_grid) {
     int sms = 0, dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0)
         sms = 148;
     cudaLaunchConfig_t lc{};
-    lc.gridDim = dim3(2 * sms);
+    // a prefetch runs beside another layer's GEMM kernels: 32 CTAs (1 MB of loads in flight) keep the host link
+    // busy and leave the SMs to them
+    lc.gridDim = dim3(small_grid ? 32 : 2 * sms);
     lc.blockDim = dim3(kFetchThreads);
     lc.stream = st;
     cudaLaunchAttribute attr[1];

@@ -97,17 +97,21 @@ class SyntheticStack:
         return [torch.randn((T, self.shape.d_model), generator=self.gen, device=self.device, dtype=torch.float32) * 0.1
                 for _ in range(self.L)]
 
-    def step(self, layer_fn, hidden, record=None, noise=None, route_fn=None):
+    def step(self, layer_fn, hidden, record=None, noise=None, route_fn=None, lookahead_fn=None):
         """layer_fn(layer, hidden, ids, weights) -> moe output.  Returns the hidden state after all layers.
         `noise`: per-layer residual tensors to use instead of drawing fresh ones.
         `route_fn(layer, hidden) -> (ids, weights)`: a router to use instead of this module's `route` (it gets
-        this stack's `routers[layer]` and `bias[layer]` from the caller)."""
+        this stack's `routers[layer]` and `bias[layer]` from the caller).
+        `lookahead_fn(next_layer, hidden)`: called before layer l runs, with layer l's input and l + 1 (a prefetch
+        policy can guess layer l + 1's experts from it); its result is ignored."""
         h = hidden
         for l in range(self.L):
             if route_fn is not None:
                 ids, w = route_fn(l, h)
             else:
                 ids, w = route(h, self.routers[l], self.shape.top_k, self.bias[l])
+            if lookahead_fn is not None and l + 1 < self.L:
+                lookahead_fn(l + 1, h)
             out = layer_fn(l, h, ids, w)
             if record is not None:
                 record.append((l, h, ids, w, out))

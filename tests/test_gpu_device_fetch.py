@@ -118,3 +118,80 @@ def test_offloaded_layer_replays_from_a_cuda_graph(B, olmoe_layer, T):
     helpers.check_output(outs[3], y, ref, "graph, offloaded")
     assert cache.status() == 0
     cache.close(); full.close()
+
+
+def check_state(cache, sc, layer=0):
+    es, se, stamp, tick = cache.state(layer)
+    assert np.array_equal(es, sc.expert_slot) and np.array_equal(se, sc.slot_expert)
+    assert np.array_equal(stamp, sc.slot_stamp) and tick == sc.tick
+    st = cache.stats(layer)
+    assert st == {"lookups": sc.stats.lookups, "hits": sc.stats.hits, "misses": sc.stats.misses,
+                  "waves": sc.stats.waves, "h2d_bytes": sc.stats.h2d_bytes, "forwards": sc.stats.forwards}
+
+
+def test_prefetch_is_a_layer_call_without_tokens(B, olmoe_layer):
+    """exmoe_cache_prefetch advances slot map, LRU stamps and counters exactly as the oracle's resolution of the same
+    ids (Section 3.3 / 3.4 steps 1-3), leaves the slots holding the bank's bytes, and a forward that selects the
+    prefetched experts then misses nothing and still equals the resident run bit for bit."""
+    _, bank = olmoe_layer
+    s = synth.OLMOE
+    cache = B.Cache(s, [bank], 16, max_tokens=16)
+    full = B.Cache(s, [bank], 64, max_tokens=16)
+    sc = ocache.SlotCache(64, 16, 0, bytes_per_expert=cache.bytes_per_expert)
+    rng = np.random.default_rng(5)
+    for step in range(8):
+        T = (1, 2, 16, 1)[step % 4]
+        hidden, ids, p = helpers.routed_inputs(s, T, seed=24000 + step, alpha=0.5)
+        if step % 2 == 0:
+            guess = ids.reshape(-1).clone()                       # a perfect guess (repeats and all)
+        else:
+            guess = torch.from_numpy(rng.integers(0, 64, size=11).astype(np.int32))   # an unrelated one
+        cache.prefetch(0, guess.cuda())
+        sc.resolve(guess.numpy())
+        check_state(cache, sc)
+        before = cache.stats(0)["misses"]
+        a = full.forward(0, hidden.cuda(), ids.cuda(), p.cuda()).clone()
+        b = cache.forward(0, hidden.cuda(), ids.cuda(), p.cuda()).clone()
+        helpers.compare_plan(cache, sc, ids)
+        assert torch.equal(a.view(torch.int16), b.view(torch.int16)), step
+        if step % 2 == 0 and len(set(guess.tolist())) <= 16:
+            assert cache.stats(0)["misses"] == before             # everything selected was already there
+    _, slot_expert, _, _ = cache.state(0)
+    for slot in (0, 9, 15):
+        assert np.array_equal(cache.read_slot(0, slot), bank[int(slot_expert[slot])].numpy())
+    cache.prefetch(0, torch.tensor([3, 99, -1], dtype=torch.int32).cuda())            # invalid ids are ignored, and reported
+    assert cache.status() == B.EXMOE_ERR_BAD_EXPERT_ID
+    cache.set_miss_path(B.MISS_HOST_COPIES)
+    with pytest.raises(B.ExmoeError) as ei:
+        cache.prefetch(0, torch.tensor([1], dtype=torch.int32).cuda())
+    assert ei.value.code == B.EXMOE_ERR_STATE
+    full.prefetch(0, torch.tensor([1], dtype=torch.int32).cuda())                     # C = E: no-op
+    cache.close(); full.close()
+
+
+def test_prefetch_of_the_next_layer_overlaps_a_forward(B):
+    """Two layers, two streams: while layer 0 computes on the main stream, layer 1's experts are prefetched on a side
+    stream (own resolution buffers); layer 1's forward, ordered after the prefetch by an event, finds them resident."""
+    s = synth.MID
+    layers = [helpers.make_layer(s, seed=70 + l) for l in range(2)]
+    cache = B.Cache(s, [b for _, b in layers], 6, max_tokens=32)
+    full = B.Cache(s, [b for _, b in layers], s.num_experts, max_tokens=32)
+    main, side = torch.cuda.Stream(), torch.cuda.Stream()
+    for step in range(6):
+        ins = [tuple(x.cuda() for x in helpers.routed_inputs(s, 20, seed=25000 + 10 * step + l, alpha=0.5)) for l in range(2)]
+        want = [full.forward(l, *ins[l]).clone() for l in range(2)]
+        torch.cuda.synchronize()
+        guess = ins[1][1].reshape(-1)[:6].contiguous()            # six of layer 1's ids: they fit the six slots
+        done = torch.cuda.Event()
+        with torch.cuda.stream(side):
+            cache.prefetch(1, guess, stream=side)
+            done.record(side)
+        with torch.cuda.stream(main):
+            out0 = cache.forward(0, *ins[0], stream=main).clone()
+            main.wait_event(done)
+            out1 = cache.forward(1, *ins[1], stream=main).clone()
+        torch.cuda.synchronize()
+        assert torch.equal(out0.view(torch.int16), want[0].view(torch.int16)), step
+        assert torch.equal(out1.view(torch.int16), want[1].view(torch.int16)), step
+    assert cache.status() == 0
+    cache.close(); full.close()
