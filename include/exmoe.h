@@ -220,8 +220,8 @@ int exmoe_cache_destroy(exmoe_cache* cache);
 
 /* Measurement hooks (the paper has no counterpart).  While enabled, every exmoe_moe_forward brackets
  * its kernels with CUDA events on the caller's stream, per kind: 0 = resolution + grouping,
- * 1 = gate/up GEMM + SwiGLU, 2 = down GEMM, 3 = combine, 4 = a wave's miss copies (on the library's copy
- * stream).  exmoe_profile_read synchronises and returns
+ * 1 = gate/up GEMM + SwiGLU, 2 = down GEMM, 3 = combine, 4 = a wave's miss traffic (the fetch kernel on the
+ * caller's stream, or the host-issued copies on the library's copy stream).  exmoe_profile_read synchronises and returns
  * the summed event time and the number of bracketed launches of one kind since the last enable.
  * Not for use during stream capture.
  * `on` bit 0 switches the event bracketing; bits 4-5, if non-zero, make later forwards launch ONLY
