@@ -437,6 +437,12 @@ decode_gemm_kernel(GemmArgs a, SmallArgs sa, const __nv_bfloat16* __restrict__ x
 // Launched as a programmatic dependent of the gate/up kernel: weights are prefetched before the
 // dependency wait.  `KSg`/`bpwg` replay the grouped kernel's K-split order so that both paths round
 // identically.
+// Placement matters at one token: with its 139 registers a CTA of this kernel does not fit beside a gate/up CTA
+// that is still running, so it starts on SMs the gate/up kernel has left.  Two variants that did fit (a 128-register
+// cap; a prologue without integer divisions, which the compiler allocated in 128 registers) started their weight
+// loads on the 40 SMs holding a single gate/up CTA, delayed the kernel they then wait for, and measured 14.2 and
+// 13.9 us per step against 12.65; forcing the separation with a 220 KB shared-memory request instead cost a
+// carve-out change per launch (13.7 us).  Re-time the whole step, not the kernel alone, after touching this kernel.
 template <int NBT>
 __global__ void __launch_bounds__(256)
 token_down_kernel(GemmArgs a, SmallArgs sa, const __nv_bfloat16* __restrict__ act, const float* __restrict__ topk_w,
@@ -552,20 +558,20 @@ token_down_kernel(GemmArgs a, SmallArgs sa, const __nv_bfloat16* __restrict__ ac
 template <int NB>
 __device__ __forceinline__ void pair_gateup_item(const GemmArgs& a, const SmallArgs& sa,
                                                  const __nv_bfloat16* __restrict__ hidden,
-                                                 __nv_bfloat16* __restrict__ act_out, int KS, int item,
-                                                 unsigned char* smem) {
-    const int K = a.H, KB = K / kGroup, PP = 8 / KS;
-    const int tiles = a.I / (kPanelRows * PP);
+                                                 __nv_bfloat16* __restrict__ act_out, int ks_log2, int p, int token,
+                                                 int tile, unsigned char* smem) {
+    // No integer division anywhere before the first loads are issued (a runtime division is a dependent chain of
+    // some 25 instructions): the K split is a power of two, pair and tile come from the grid's coordinates.
+    const int K = a.H, KB = K / kGroup, KS = 1 << ks_log2, PP = 8 >> ks_log2;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int q = lane >> 2, c = lane & 3;
-    const int ks = warp % KS, pp = warp / KS;
-    const int p = item / tiles, tile = item % tiles;
+    const int ks = warp & (KS - 1), pp = warp >> ks_log2;
     unsigned char* xs = smem;                                            // one activation row
     float* red = reinterpret_cast<float*>(smem + K * 2 + 64);            // [KS-1][PP][2][32][4]
     float* adj = red + (size_t)(KS - 1) * PP * 2 * 128;                  // [KB]
 
     // The hidden row does not depend on the ids: request it first so that it is not queued behind the weights.
-    const __nv_bfloat16* xrow = hidden + (size_t)(p / a.top_k) * K;
+    const __nv_bfloat16* xrow = hidden + (size_t)token * K;
     uint4 xpre = make_uint4(0, 0, 0, 0);
     if (tid < K / 8) xpre = ldg_early128(xrow + tid * 8);
     const int id = sa.ids[p];
@@ -671,11 +677,13 @@ __device__ __forceinline__ void keep_pair_ids(const SmallArgs& sa) {
 template <int NB>
 __global__ void __launch_bounds__(256, 2)
 pair_gateup_kernel(GemmArgs a, SmallArgs sa, const __nv_bfloat16* __restrict__ hidden,
-                   __nv_bfloat16* __restrict__ act_out, int KS) {
+                   __nv_bfloat16* __restrict__ act_out, int ks_log2) {
+    // grid = (tiles of the intermediate dimension, selected expert j, token t): pair p = t * k + j
     extern __shared__ __align__(16) unsigned char smem[];
     grid_launch_dependents();
-    if (blockIdx.x == 0) keep_pair_ids(sa);
-    pair_gateup_item<NB>(a, sa, hidden, act_out, KS, blockIdx.x, smem);
+    if ((blockIdx.x | blockIdx.y | blockIdx.z) == 0) keep_pair_ids(sa);
+    pair_gateup_item<NB>(a, sa, hidden, act_out, ks_log2, (int)(blockIdx.z * a.top_k + blockIdx.y), (int)blockIdx.z,
+                         (int)blockIdx.x, smem);
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -717,8 +725,7 @@ token_down_bulk_kernel(GemmArgs a, SmallArgs sa, const __nv_bfloat16* __restrict
     volatile int* abort_flag = reinterpret_cast<volatile int*>(bar + 1);
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int q = lane >> 2, c = lane & 3;
-    const int panels = a.H / kPanelRows;
-    const int t = blockIdx.x / panels, panel = blockIdx.x % panels;
+    const int t = blockIdx.y, panel = blockIdx.x;                        // grid = (16-row panels of the output, tokens)
     if (tid == 0) {
         mbar_init(bar, k);                                               // one arrival per expert warp
         *abort_flag = 0;
@@ -744,9 +751,17 @@ token_down_bulk_kernel(GemmArgs a, SmallArgs sa, const __nv_bfloat16* __restrict
     grid_dependency_wait();                                              // the gate/up kernel's activations are complete and visible
     {
         const int chunks_per_row = K / 8, total = k * chunks_per_row;
+        const int cpr_shift = (chunks_per_row & (chunks_per_row - 1)) ? -1 : __ffs(chunks_per_row) - 1;
         for (int base = warp * 32; base < total; base += 256) {
             const int idx = base + lane;
-            const int n = idx / chunks_per_row, ck = idx % chunks_per_row;
+            int n, ck;
+            if (cpr_shift >= 0) {                      // the usual case: no division between the wait and the MMAs
+                n = idx >> cpr_shift;
+                ck = idx & (chunks_per_row - 1);
+            } else {
+                n = idx / chunks_per_row;
+                ck = idx - n * chunks_per_row;
+            }
             uint4 v = make_uint4(0, 0, 0, 0);
             if (idx < total) {
                 v = *reinterpret_cast<const uint4*>(act + (size_t)(t * k + n) * K + ck * 8);
@@ -822,7 +837,9 @@ void launch_pair_gateup(const GemmArgs& a, const SmallArgs& sa, const __nv_bfloa
     const size_t smem = (size_t)a.H * 2 + 64 + (size_t)(KS - 1) * PP * 2 * 128 * 4 + (size_t)(a.H / kGroup) * 4;
     static SmemOnce smem_once;
     allow_smem(kern, 100 * 1024, smem_once);
-    kern<<<sa.n_pairs * tiles, 256, smem, st>>>(a, sa, hidden, act, KS);
+    int ks_log2 = 0;
+    while ((1 << ks_log2) < KS) ++ks_log2;
+    kern<<<dim3(tiles, a.top_k, sa.n_pairs / a.top_k), 256, smem, st>>>(a, sa, hidden, act, ks_log2);
     count_launch();
 }
 
@@ -978,7 +995,7 @@ bool launch_token_down_bulk(const GemmArgs& a, const SmallArgs& sa, const __nv_b
     static SmemOnce smem_once;
     allow_smem(kern, 100 * 1024, smem_once);
     cudaLaunchConfig_t lc{};
-    lc.gridDim = dim3(T * (a.H / kPanelRows));
+    lc.gridDim = dim3(a.H / kPanelRows, T);
     lc.blockDim = dim3(256);
     lc.dynamicSmemBytes = smem;
     lc.stream = st;
