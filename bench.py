@@ -572,64 +572,17 @@ def main():
     h_i = [ids[j].cpu().pin_memory() for j in pick]
     h_w = [ws[j].cpu().pin_memory() for j in pick]
     h_out = torch.empty_like(h_h[0]).pin_memory()
-    d_h, d_i, d_w, d_o = torch.empty_like(hs[0]), torch.empty_like(ids[0]), torch.empty_like(ws[0]), torch.empty_like(hs[0])
 
+    # the library's host-buffer entry point: inputs in host memory, result in host memory, synchronous; one call per
+    # step.  (It stages the three inputs, copies them to the device in one copy, runs the layer, copies the result
+    # back and waits; with no host wait inside the layer call it replays a graph recorded per (layer, T).)
     def e2e_step(i):
         j = i % len(h_h)
-        with torch.cuda.stream(stream):
-            d_h.copy_(h_h[j], non_blocking=True)
-            d_i.copy_(h_i[j], non_blocking=True)
-            d_w.copy_(h_w[j], non_blocking=True)
-            cache.forward(i % L, d_h, d_i, d_w, out=d_o, stream=stream)
-            h_out.copy_(d_o, non_blocking=True)
-        stream.synchronize()
+        cache.forward_host(i % L, h_h[j], h_i[j], h_w[j], out=h_out, stream=stream)
 
-    e2e_mode = "per-step launches"
-    if graphable and T <= 64:
-        # serving-loop form: the step's inputs (hidden | ids | weights) sit in ONE pinned staging buffer and go to the
-        # device in ONE copy; per layer one CUDA graph of [H2D copy, forward, D2H copy].  A step writes its inputs
-        # into the staging buffer, replays the graph and waits for the result.
-        def _al(n):
-            return (n + 255) & ~255
-        nb_h, nb_i, nb_w = h_h[0].numel() * 2, h_i[0].numel() * 4, h_w[0].numel() * 4
-        o_i, o_w, nb_all = _al(nb_h), _al(nb_h) + _al(nb_i), _al(nb_h) + _al(nb_i) + _al(nb_w)
-        s_all = torch.empty(nb_all, dtype=torch.uint8).pin_memory()
-        d_all = torch.empty(nb_all, dtype=torch.uint8, device=dev)
-
-        def _views(buf):
-            return (buf[:nb_h].view(torch.bfloat16).view(h_h[0].shape), buf[o_i:o_i + nb_i].view(torch.int32).view(h_i[0].shape),
-                    buf[o_w:o_w + nb_w].view(torch.float32).view(h_w[0].shape))
-        s_h, s_i, s_w = _views(s_all)
-        g_h, g_i, g_w = _views(d_all)
-        graphs = []
-        with torch.cuda.stream(stream):
-            cache.forward(0, d_h, d_i, d_w, out=d_o, stream=stream)
-        stream.synchronize()
-        for l in range(L):
-            g = torch.cuda.CUDAGraph()
-            with torch.cuda.graph(g, stream=stream):
-                d_all.copy_(s_all, non_blocking=True)
-                cache.forward(l, g_h, g_i, g_w, out=d_o, stream=stream)
-                h_out.copy_(d_o, non_blocking=True)
-            graphs.append(g)
-
-        # the host-side inputs of every step are kept in the same packed form (as a caller that owns its request
-        # buffers would lay them out), so a step is one host copy into the staging buffer
-        h_all = []
-        for j in range(len(h_h)):
-            buf = torch.zeros(nb_all, dtype=torch.uint8)
-            vh, vi, vw = _views(buf)
-            vh.copy_(h_h[j]); vi.copy_(h_i[j]); vw.copy_(h_w[j])
-            h_all.append(buf)
-
-        def e2e_step(i):                                   # noqa: F811  (replaces the launch-per-call form)
-            s_all.copy_(h_all[i % len(h_all)])
-            with torch.cuda.stream(stream):
-                graphs[i % L].replay()
-            stream.synchronize()
-        e2e_mode = "one CUDA graph per step (one H2D copy of the packed inputs, forward, D2H copy)"
-
-    for i in range(3):
+    e2e_mode = ("exmoe_moe_forward_host: host tensors in and out, one call per step (recorded graph per (layer, T))"
+                if graphable else "exmoe_moe_forward_host: host tensors in and out, one call per step (plain launches)")
+    for i in range(max(3, 2 * L)):                      # every layer's graph is recorded before the timed calls
         e2e_step(i)
     if world > 1:
         dist.barrier()
@@ -639,8 +592,6 @@ def main():
     dt = time.perf_counter() - t0
     dt = max_over_ranks(dt, world, dev)
     h2d = h_h[0].numel() * 2 + h_i[0].numel() * 4 + h_w[0].numel() * 4
-    if e2e_mode.startswith("one CUDA graph"):
-        h2d = nb_all                                       # the packed staging buffer, padding included
     e2e = {"value": world * n_e2e * T / dt, "unit": UNIT, "h2d_bytes_per_step": int(h2d),
            "d2h_bytes_per_step": int(h_out.numel() * 2), "steps": n_e2e, "mode": e2e_mode}
 

@@ -19,7 +19,7 @@
  *     memory.  `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).
  *   - The caller owns every buffer it passes (tensors, slot memory, workspace, host bank) and
  *     must keep them alive while the cache exists.  The library owns only its host bookkeeping,
- *     one copy stream, its events and a small pinned staging buffer.
+ *     one copy stream, its events, pinned staging buffers and the graphs of exmoe_moe_forward_host.
  *   - BF16 tensors are row-major, dense.  ids are int32, mixture weights are float32.
  *   - All calls on one cache must come from one host thread at a time.
  */
@@ -115,6 +115,19 @@ int exmoe_cache_create(exmoe_cache** out, const exmoe_shape* shape, int num_laye
  * device-initiated miss path the call is fully asynchronous on `stream` as well. */
 int exmoe_moe_forward(exmoe_cache* cache, int layer, const void* hidden_bf16, const int32_t* topk_ids,
                       const float* topk_weights, int T, void* out_bf16, void* stream);
+
+/* The same layer call for a caller whose tensors live in HOST memory (pageable or pinned):
+ *   hidden_host : host, BF16 [T, H]      ids_host : host, int32 [T, k]      weights_host : host, float32 [T, k]
+ *   out_host    : host, BF16 [T, H], fully overwritten
+ * The inputs are copied into the library's pinned staging buffer, go to the device in one copy, the layer runs as
+ * in exmoe_moe_forward, the result comes back in one copy, and the call returns when out_host holds it
+ * (synchronous; `stream` carries the work).  When the call contains no host wait (C = E, or the device-initiated
+ * miss path) its launch sequence is recorded once per (layer, T) in a CUDA graph and later calls are one graph
+ * launch; otherwise every call issues the launches one by one.  Calls of 256 KB of activations or more whose four
+ * tensors are page-locked skip the staging buffer: the device copies use the caller's memory.  Same results, state and errors as
+ * exmoe_moe_forward.  Not to be called while `stream` is being captured by the caller. */
+int exmoe_moe_forward_host(exmoe_cache* cache, int layer, const void* hidden_host, const int32_t* ids_host,
+                           const float* weights_host, int T, void* out_host, void* stream);
 
 /* How the misses of a C < E cache reach their slots (Sec. 3.4 step 3; the paper's runtime issues host copies).
  *   EXMOE_MISS_DEVICE_FETCH (default when every host bank has a 16-byte aligned device-visible address, which

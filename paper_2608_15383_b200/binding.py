@@ -47,6 +47,7 @@ _SIGNATURES = {
     "exmoe_cache_create": (c_int, [POINTER(c_void_p), POINTER(exmoe_shape), c_int, c_int, POINTER(c_void_p), c_void_p,
                                    c_void_p, c_int, c_int]),
     "exmoe_moe_forward": (c_int, [c_void_p, c_int, c_void_p, c_void_p, c_void_p, c_int, c_void_p, c_void_p]),
+    "exmoe_moe_forward_host": (c_int, [c_void_p, c_int, c_void_p, c_void_p, c_void_p, c_int, c_void_p, c_void_p]),
     "exmoe_moe_forward_static": (c_int, [POINTER(exmoe_shape), c_void_p, c_void_p, c_void_p, c_void_p, c_int, c_void_p, c_void_p]),
     "exmoe_route": (c_int, [POINTER(exmoe_shape), c_void_p, c_void_p, c_void_p, c_int, c_void_p, c_void_p, c_void_p]),
     "exmoe_cache_get_state": (c_int, [c_void_p, c_int, c_void_p, c_void_p, c_void_p, c_void_p]),
@@ -241,6 +242,23 @@ class Cache:
                                      _dev(topk_ids, torch.int32, "topk_ids"), _dev(topk_weights, torch.float32, "topk_weights"),
                                      int(T), _dev(out, torch.bfloat16, "out"), _stream_ptr(stream))
         _check(rc, "exmoe_moe_forward")
+        return out
+
+    # exmoe_moe_forward_host
+    def forward_host(self, layer, hidden, topk_ids, topk_weights, out=None, stream=None):
+        """Host tensors in, host tensor out (synchronous): hidden BF16 [T, H], ids int32 [T, k], weights fp32 [T, k]."""
+        T = int(hidden.shape[0])
+        for t, dt, what in ((hidden, torch.bfloat16, "hidden"), (topk_ids, torch.int32, "topk_ids"),
+                            (topk_weights, torch.float32, "topk_weights")):
+            if t.is_cuda or t.dtype != dt or not t.is_contiguous():
+                raise ValueError(f"{what}: need a contiguous CPU tensor of {dt}")
+        if out is None:
+            out = torch.empty((T, self.shape.d_model), dtype=torch.bfloat16)
+        elif out.is_cuda or out.dtype != torch.bfloat16 or not out.is_contiguous():
+            raise ValueError("out: need a contiguous CPU tensor of torch.bfloat16")
+        rc = lib().exmoe_moe_forward_host(self.handle, int(layer), c_void_p(hidden.data_ptr()), c_void_p(topk_ids.data_ptr()),
+                                          c_void_p(topk_weights.data_ptr()), T, c_void_p(out.data_ptr()), _stream_ptr(stream))
+        _check(rc, "exmoe_moe_forward_host")
         return out
 
     def state(self, layer):

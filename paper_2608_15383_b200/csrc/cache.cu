@@ -5,6 +5,7 @@
 #include <atomic>
 #include <cstring>
 #include <new>
+#include <map>
 #include <vector>
 
 #include "common.cuh"
@@ -84,7 +85,21 @@ struct exmoe_cache {
     int prof_only;                            // 0 = all kernels; 1..3 = launch only that kind (timing runs)
     std::vector<cudaEvent_t> prof_ev[5];      // begin/end pairs per kernel kind (4 = miss copies, copy stream)
     size_t prof_used[5];
+    // exmoe_moe_forward_host: staging on both sides and one instantiated graph per (layer, T)
+    uint8_t* d_stage;                         // device: hidden | ids | weights | out, each 256-byte aligned
+    uint8_t* h_stage;                         // pinned host mirror of d_stage
+    size_t stage_in_bytes, stage_out_off, stage_bytes;
+    struct HostGraph {
+        cudaGraphExec_t exec;
+        bool last_small, last_pair;
+    };
+    std::map<long long, HostGraph> host_graphs;
 };
+
+static void drop_host_graphs(exmoe_cache* c) {
+    for (auto& kv : c->host_graphs) cudaGraphExecDestroy(kv.second.exec);
+    c->host_graphs.clear();
+}
 
 enum { PROF_PLAN = 0, PROF_GATEUP = 1, PROF_DOWN = 2, PROF_COMBINE = 3, PROF_COPY = 4 };
 
@@ -155,6 +170,14 @@ static void carve_workspace(exmoe_cache* c, uint8_t* ws, size_t* total) {
     c->saved_ids = k.take<int32_t>(kPairMaxPairs);
     c->tc_scratch = k.take<uint8_t>(prefill_scratch_bytes(c->max_pairs, E));
     c->xg = c->max_pairs > kSmallMaxPairs ? k.take<__nv_bfloat16>((size_t)c->max_pairs * s.d_model) : nullptr;
+    {   // staging of the host-buffer entry point: hidden | ids | weights (one H2D copy), then out (one D2H copy)
+        const size_t nb_h = align_up((size_t)c->max_tokens * s.d_model * 2, 256);
+        const size_t nb_i = align_up((size_t)c->max_pairs * 4, 256);
+        c->stage_in_bytes = nb_h + 2 * nb_i;
+        c->stage_out_off = c->stage_in_bytes;
+        c->stage_bytes = c->stage_in_bytes + nb_h;
+        c->d_stage = k.take<uint8_t>(c->stage_bytes);
+    }
     *total = k.off;
 }
 
@@ -303,6 +326,7 @@ int exmoe_cache_create(exmoe_cache** out, const exmoe_shape* shape, int num_laye
     c->stream_ok = stream_supported(c->shape.d_model, c->shape.d_ff);
     c->miss_path = map_banks(c) ? EXMOE_MISS_DEVICE_FETCH : EXMOE_MISS_HOST_COPIES;
     bool ok = cudaMallocHost(&c->h_plan, c->plan_d2h_bytes) == cudaSuccess;
+    ok = ok && cudaMallocHost(&c->h_stage, c->stage_bytes) == cudaSuccess;
     ok = ok && cudaStreamCreateWithFlags(&c->copy_stream, cudaStreamNonBlocking) == cudaSuccess;
     ok = ok && cudaEventCreateWithFlags(&c->ev_plan, cudaEventDisableTiming) == cudaSuccess;
     for (int i = 0; i < kEventRing && ok; ++i) {
@@ -514,8 +538,89 @@ int exmoe_cache_set_miss_path(exmoe_cache* c, int mode) {
     if (cudaDeviceSynchronize() != cudaSuccess) return EXMOE_ERR_CUDA;     // no wave of the other mode is in flight
     if (mode == EXMOE_MISS_DEVICE_FETCH && !map_banks(c)) return EXMOE_ERR_NOT_PINNED;
     for (auto& v : c->slot_last_seq) std::fill(v.begin(), v.end(), 0);       // everything earlier has completed
+    drop_host_graphs(c);                                                     // they hold the other mode's launch sequence
     c->miss_path = mode;
     return EXMOE_OK;
+}
+
+int exmoe_moe_forward_host(exmoe_cache* c, int layer, const void* hidden_host, const int32_t* ids_host,
+                           const float* weights_host, int T, void* out_host, void* stream) {
+    if (!c || layer < 0 || layer >= c->L || T < 0 || T > c->max_tokens) return EXMOE_ERR_ARG;
+    if (T == 0) return EXMOE_OK;
+    if (!hidden_host || !ids_host || !weights_host || !out_host) return EXMOE_ERR_ARG;
+    cudaStream_t st = (cudaStream_t)stream;
+    const exmoe_shape& s = c->shape;
+    const size_t nb_h = (size_t)T * s.d_model * 2, nb_i = (size_t)T * s.top_k * 4;
+    const size_t off_i = align_up((size_t)c->max_tokens * s.d_model * 2, 256);
+    const size_t off_w = off_i + align_up((size_t)c->max_pairs * 4, 256);
+    void* d_h = c->d_stage;
+    int32_t* d_i = reinterpret_cast<int32_t*>(c->d_stage + off_i);
+    float* d_w = reinterpret_cast<float*>(c->d_stage + off_w);
+    void* d_o = c->d_stage + c->stage_out_off;
+    // Large calls whose tensors are page-locked already skip the staging copies (8 MB each way at 2048 tokens would
+    // cost more than the layer): the device copies read and write the caller's memory, as plain launches.
+    if (nb_h >= ((size_t)256 << 10)) {
+        bool pinned = true;
+        const void* ptrs[4] = {hidden_host, ids_host, weights_host, out_host};
+        for (int i = 0; i < 4 && pinned; ++i) {
+            cudaPointerAttributes attr{};
+            pinned = cudaPointerGetAttributes(&attr, ptrs[i]) == cudaSuccess && attr.type == cudaMemoryTypeHost;
+        }
+        cudaGetLastError();
+        if (pinned) {
+            bool ok = cudaMemcpyAsync(d_h, hidden_host, nb_h, cudaMemcpyHostToDevice, st) == cudaSuccess;
+            ok = ok && cudaMemcpyAsync(d_i, ids_host, nb_i, cudaMemcpyHostToDevice, st) == cudaSuccess;
+            ok = ok && cudaMemcpyAsync(d_w, weights_host, nb_i, cudaMemcpyHostToDevice, st) == cudaSuccess;
+            int rc = ok ? exmoe_moe_forward(c, layer, d_h, d_i, d_w, T, d_o, st) : EXMOE_ERR_CUDA;
+            if (!rc && cudaMemcpyAsync(out_host, d_o, nb_h, cudaMemcpyDeviceToHost, st) != cudaSuccess) rc = EXMOE_ERR_CUDA;
+            if (cudaStreamSynchronize(st) != cudaSuccess) rc = rc ? rc : EXMOE_ERR_CUDA;
+            return rc;
+        }
+    }
+    std::memcpy(c->h_stage, hidden_host, nb_h);
+    std::memcpy(c->h_stage + off_i, ids_host, nb_i);
+    std::memcpy(c->h_stage + off_w, weights_host, nb_i);
+    const size_t in_bytes = off_w + nb_i;                                 // one copy covers the three inputs
+    auto enqueue = [&]() -> int {
+        if (cudaMemcpyAsync(c->d_stage, c->h_stage, in_bytes, cudaMemcpyHostToDevice, st) != cudaSuccess) return EXMOE_ERR_CUDA;
+        const int rc = exmoe_moe_forward(c, layer, d_h, d_i, d_w, T, d_o, st);
+        if (rc) return rc;
+        if (cudaMemcpyAsync(c->h_stage + c->stage_out_off, d_o, nb_h, cudaMemcpyDeviceToHost, st) != cudaSuccess)
+            return EXMOE_ERR_CUDA;
+        return EXMOE_OK;
+    };
+    // The launch sequence of a call is fixed when no host wait sits inside it (all experts resident, or the
+    // device-initiated miss path): it is then captured once per (layer, T) and replayed, one graph launch per call.
+    const bool fixed = (c->C == s.num_experts || c->miss_path == EXMOE_MISS_DEVICE_FETCH) && !c->prof_on && !c->prof_only;
+    const long long key = (long long)layer * ((long long)c->max_tokens + 1) + T;
+    int rc = EXMOE_OK;
+    auto it = fixed ? c->host_graphs.find(key) : c->host_graphs.end();
+    if (it != c->host_graphs.end()) {
+        c->last_layer = layer;
+        c->last_T = T;
+        c->last_small = it->second.last_small;
+        c->last_pair = it->second.last_pair;
+        if (cudaGraphLaunch(it->second.exec, st) != cudaSuccess) rc = EXMOE_ERR_CUDA;
+    } else {
+        rc = enqueue();                                                   // this call runs as plain launches
+    }
+    if (cudaStreamSynchronize(st) != cudaSuccess) rc = rc ? rc : EXMOE_ERR_CUDA;
+    if (!rc) std::memcpy(out_host, c->h_stage + c->stage_out_off, nb_h);
+    if (!rc && fixed && it == c->host_graphs.end() && c->host_graphs.size() < 256) {
+        // ... and the same sequence is recorded for the next call of this (layer, T); recording launches nothing
+        cudaGraph_t g = nullptr;
+        cudaGraphExec_t exec = nullptr;
+        bool ok = cudaStreamBeginCapture(st, cudaStreamCaptureModeThreadLocal) == cudaSuccess;
+        if (ok) {
+            const int crc = enqueue();
+            ok = cudaStreamEndCapture(st, &g) == cudaSuccess && crc == EXMOE_OK && g;
+        }
+        ok = ok && cudaGraphInstantiate(&exec, g, 0) == cudaSuccess;
+        if (g) cudaGraphDestroy(g);
+        if (ok) c->host_graphs[key] = exmoe_cache::HostGraph{exec, c->last_small, c->last_pair};
+        else cudaGetLastError();                                          // stay on plain launches for this key
+    }
+    return rc;
 }
 
 int exmoe_cache_prefetch(exmoe_cache* c, int layer, const int32_t* expert_ids, int n_ids, void* stream) {
@@ -663,7 +768,9 @@ int exmoe_cache_destroy(exmoe_cache* c) {
     cudaDeviceSynchronize();
     for (int k = 0; k < 5; ++k)
         for (cudaEvent_t e : c->prof_ev[k]) cudaEventDestroy(e);
+    drop_host_graphs(c);
     if (c->h_plan) cudaFreeHost(c->h_plan);
+    if (c->h_stage) cudaFreeHost(c->h_stage);
     if (c->copy_stream) cudaStreamDestroy(c->copy_stream);
     if (c->ev_plan) cudaEventDestroy(c->ev_plan);
     for (int i = 0; i < kEventRing; ++i) {
