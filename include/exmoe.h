@@ -120,7 +120,8 @@ int exmoe_moe_forward(exmoe_cache* cache, int layer, const void* hidden_bf16, co
  *   hidden_host : host, BF16 [T, H]      ids_host : host, int32 [T, k]      weights_host : host, float32 [T, k]
  *   out_host    : host, BF16 [T, H], fully overwritten
  * The inputs are copied into the library's pinned staging buffer, go to the device in one copy, the layer runs as
- * in exmoe_moe_forward, the result comes back in one copy, and the call returns when out_host holds it
+ * in exmoe_moe_forward, the result comes back in one copy (results of up to 64 KB are written by the last kernel
+ * straight into the pinned staging buffer), and the call returns when out_host holds it
  * (synchronous; `stream` carries the work).  When the call contains no host wait (C = E, or the device-initiated
  * miss path) its launch sequence is recorded once per (layer, T) in a CUDA graph and later calls are one graph
  * launch; otherwise every call issues the launches one by one.  Calls of 256 KB of activations or more whose four

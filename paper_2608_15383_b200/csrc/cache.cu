@@ -556,7 +556,10 @@ int exmoe_moe_forward_host(exmoe_cache* c, int layer, const void* hidden_host, c
     void* d_h = c->d_stage;
     int32_t* d_i = reinterpret_cast<int32_t*>(c->d_stage + off_i);
     float* d_w = reinterpret_cast<float*>(c->d_stage + off_w);
-    void* d_o = c->d_stage + c->stage_out_off;
+    // Small results are written by the last kernel straight into the pinned staging buffer (mapped into the device's
+    // address space; posted writes over the host link), which saves the copy node after the layer.
+    const bool out_direct = nb_h <= ((size_t)64 << 10);
+    void* d_o = out_direct ? static_cast<void*>(c->h_stage + c->stage_out_off) : static_cast<void*>(c->d_stage + c->stage_out_off);
     // Large calls whose tensors are page-locked already skip the staging copies (8 MB each way at 2048 tokens would
     // cost more than the layer): the device copies read and write the caller's memory, as plain launches.
     if (nb_h >= ((size_t)256 << 10)) {
@@ -585,7 +588,8 @@ int exmoe_moe_forward_host(exmoe_cache* c, int layer, const void* hidden_host, c
         if (cudaMemcpyAsync(c->d_stage, c->h_stage, in_bytes, cudaMemcpyHostToDevice, st) != cudaSuccess) return EXMOE_ERR_CUDA;
         const int rc = exmoe_moe_forward(c, layer, d_h, d_i, d_w, T, d_o, st);
         if (rc) return rc;
-        if (cudaMemcpyAsync(c->h_stage + c->stage_out_off, d_o, nb_h, cudaMemcpyDeviceToHost, st) != cudaSuccess)
+        if (!out_direct &&
+            cudaMemcpyAsync(c->h_stage + c->stage_out_off, d_o, nb_h, cudaMemcpyDeviceToHost, st) != cudaSuccess)
             return EXMOE_ERR_CUDA;
         return EXMOE_OK;
     };
