@@ -574,15 +574,15 @@ def main():
     h_out = torch.empty_like(h_h[0]).pin_memory()
 
     # the library's host-buffer entry point: inputs in host memory, result in host memory, synchronous; one call per
-    # step.  (It stages the three inputs, copies them to the device in one copy, runs the layer, copies the result
-    # back and waits; with no host wait inside the layer call it replays a graph recorded per (layer, T).)
+    # step (it stages the three inputs, copies them to the device in one copy, runs the layer and waits; tiny batches
+    # replay a graph recorded per (layer, T), small results are written straight into pinned host memory, large
+    # page-locked tensors are used in place)
     def e2e_step(i):
         j = i % len(h_h)
         cache.forward_host(i % L, h_h[j], h_i[j], h_w[j], out=h_out, stream=stream)
 
-    e2e_mode = ("exmoe_moe_forward_host: host tensors in and out, one call per step (recorded graph per (layer, T))"
-                if graphable else "exmoe_moe_forward_host: host tensors in and out, one call per step (plain launches)")
-    for i in range(max(3, 2 * L)):                      # every layer's graph is recorded before the timed calls
+    e2e_mode = "exmoe_moe_forward_host: host tensors in and out, one synchronous call per step"
+    for i in range(max(3, 2 * L)):                      # every layer's graph (tiny batches) is recorded before the timed calls
         e2e_step(i)
     if world > 1:
         dist.barrier()

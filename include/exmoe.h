@@ -121,12 +121,12 @@ int exmoe_moe_forward(exmoe_cache* cache, int layer, const void* hidden_bf16, co
  *   out_host    : host, BF16 [T, H], fully overwritten
  * The inputs are copied into the library's pinned staging buffer, go to the device in one copy, the layer runs as
  * in exmoe_moe_forward, the result comes back in one copy (results of up to 64 KB are written by the last kernel
- * straight into the pinned staging buffer), and the call returns when out_host holds it
- * (synchronous; `stream` carries the work).  When the call contains no host wait (C = E, or the device-initiated
- * miss path) its launch sequence is recorded once per (layer, T) in a CUDA graph and later calls are one graph
- * launch; otherwise every call issues the launches one by one.  Calls of 256 KB of activations or more whose four
- * tensors are page-locked skip the staging buffer: the device copies use the caller's memory.  Same results, state and errors as
- * exmoe_moe_forward.  Not to be called while `stream` is being captured by the caller. */
+ * straight into the pinned staging buffer), and the call returns when out_host holds it (synchronous; `stream`
+ * carries the work).  Tiny batches (T * top_k <= 24) whose call contains no host wait (C = E, or the
+ * device-initiated miss path) record their launch sequence once per (layer, T) in a CUDA graph and replay it; all
+ * other calls issue their launches one by one.  Calls of 256 KB of activations or more whose four tensors are
+ * page-locked skip the staging buffer: the device copies use the caller's memory.  Same results, state and errors
+ * as exmoe_moe_forward.  Not to be called while `stream` is being captured by the caller. */
 int exmoe_moe_forward_host(exmoe_cache* cache, int layer, const void* hidden_host, const int32_t* ids_host,
                            const float* weights_host, int T, void* out_host, void* stream);
 

@@ -595,7 +595,11 @@ int exmoe_moe_forward_host(exmoe_cache* c, int layer, const void* hidden_host, c
     };
     // The launch sequence of a call is fixed when no host wait sits inside it (all experts resident, or the
     // device-initiated miss path): it is then captured once per (layer, T) and replayed, one graph launch per call.
-    const bool fixed = (c->C == s.num_experts || c->miss_path == EXMOE_MISS_DEVICE_FETCH) && !c->prof_on && !c->prof_only;
+    // Only for the tiny-batch path: rotating over 16 layer banks, one token per call, the replay gives 30.4 k calls/s
+    // against 28.6 k with plain launches; at 16 tokens (grouping, two GEMM kernels, combine) plain launches win,
+    // 207 k against 197 k tokens/s, and the larger the call the less the launches matter.
+    const bool fixed = (c->C == s.num_experts || c->miss_path == EXMOE_MISS_DEVICE_FETCH) && !c->prof_on && !c->prof_only &&
+                       T * s.top_k <= kSmallMaxPairs;
     const long long key = (long long)layer * ((long long)c->max_tokens + 1) + T;
     int rc = EXMOE_OK;
     auto it = fixed ? c->host_graphs.find(key) : c->host_graphs.end();

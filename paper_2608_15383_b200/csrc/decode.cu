@@ -149,7 +149,7 @@ decode_gemm_kernel(GemmArgs a, SmallArgs sa, const __nv_bfloat16* __restrict__ x
                    __nv_bfloat16* __restrict__ act_out, const float* __restrict__ topk_w, float* __restrict__ y_out,
                    int KS, int blocks_per_warp) {
     constexpr int NM = GATEUP ? 2 : 1;
-    extern __shared__ __align__(16) unsigned char smem[];
+    extern __shared__ __align__(128) unsigned char smem[];
     __shared__ int s_scalars[4];
     const int K = GATEUP ? a.H : a.I;                  // reduction length
     const int NR = GATEUP ? a.I : a.H;                 // output rows of the weight matrix
@@ -447,7 +447,7 @@ template <int NBT>
 __global__ void __launch_bounds__(256)
 token_down_kernel(GemmArgs a, SmallArgs sa, const __nv_bfloat16* __restrict__ act, const float* __restrict__ topk_w,
                   int bpwg) {
-    extern __shared__ __align__(16) unsigned char smem[];
+    extern __shared__ __align__(128) unsigned char smem[];
     const int K = a.I, KB = K / kGroup, k = a.top_k;
     const int x_stride = K * 2 + 64;
     unsigned char* xs = smem;                                          // [k][x_stride]
@@ -679,7 +679,7 @@ __global__ void __launch_bounds__(256, 2)
 pair_gateup_kernel(GemmArgs a, SmallArgs sa, const __nv_bfloat16* __restrict__ hidden,
                    __nv_bfloat16* __restrict__ act_out, int ks_log2) {
     // grid = (tiles of the intermediate dimension, selected expert j, token t): pair p = t * k + j
-    extern __shared__ __align__(16) unsigned char smem[];
+    extern __shared__ __align__(128) unsigned char smem[];
     grid_launch_dependents();
     if ((blockIdx.x | blockIdx.y | blockIdx.z) == 0) keep_pair_ids(sa);
     pair_gateup_item<NB>(a, sa, hidden, act_out, ks_log2, (int)(blockIdx.z * a.top_k + blockIdx.y), (int)blockIdx.z,

@@ -1,8 +1,9 @@
 """exmoe_moe_forward_host: the layer call with host tensors in and out.
 
-It must give the bits of exmoe_moe_forward on the same inputs, on the first call of a (layer, T) (plain launches) and
-on the later ones (replay of the recorded graph), with all experts resident and with a 16-slot cache, where the
-slot map and counters must also stay the oracle's.
+It must give the bits of exmoe_moe_forward on the same inputs: for pageable and page-locked tensors, for tiny batches
+on their first call (plain launches) and on later ones (replay of the recorded graph), for small results (written
+straight into pinned host memory) and large ones, with all experts resident and with a 16-slot cache, where the slot
+map and counters must also stay the oracle's.
 """
 import numpy as np
 import pytest
@@ -37,7 +38,7 @@ def test_host_forward_matches_device_forward(B, olmoe_layer, C):
     host = B.Cache(s, [bank], C, max_tokens=200)
     sc = ocache.SlotCache(64, C, 0, bytes_per_expert=host.bytes_per_expert)
     stream = torch.cuda.Stream()
-    order = [1, 16, 1, 3, 16, 64, 1, 200, 64, 3, 200, 16]              # every size comes back: first call plain, then replays
+    order = [1, 16, 1, 3, 16, 64, 1, 200, 64, 3, 200, 16]              # every size comes back
     for step, T in enumerate(order):
         hidden, ids, p = helpers.routed_inputs(s, T, seed=26000 + step, alpha=0.5)
         want = full.forward(0, hidden.cuda(), ids.cuda(), p.cuda()).cpu()
@@ -76,11 +77,12 @@ def test_host_forward_follows_a_miss_path_switch(B, olmoe_layer):
     sc = ocache.SlotCache(64, 16, 0, bytes_per_expert=host.bytes_per_expert)
     stream = torch.cuda.Stream()
     for step in range(9):
+        T = 2 if step % 3 else 16                                      # T = 2 replays a graph, T = 16 is plain launches
         if step == 3:
             host.set_miss_path(B.MISS_HOST_COPIES)
         if step == 6:
             host.set_miss_path(B.MISS_DEVICE_FETCH)
-        hidden, ids, p = helpers.routed_inputs(s, 16, seed=26200 + step, alpha=1.0)
+        hidden, ids, p = helpers.routed_inputs(s, T, seed=26200 + step, alpha=1.0)
         want = full.forward(0, hidden.cuda(), ids.cuda(), p.cuda()).cpu()
         got = host.forward_host(0, hidden, ids, p, stream=stream)
         assert torch.equal(got.view(torch.int16), want.view(torch.int16)), step
