@@ -494,12 +494,30 @@ gather_rows_kernel(const __nv_bfloat16* __restrict__ hidden, const int32_t* __re
                    const int32_t* __restrict__ n_valid, int top_k, int H, __nv_bfloat16* __restrict__ xg,
                    const int32_t* __restrict__ counts, const int32_t* __restrict__ group_keys,
                    const int32_t* __restrict__ wave_start, Tile* __restrict__ tiles, int32_t* __restrict__ n_tiles, int bn) {
-    const int r = blockIdx.x;
-    if (r == 0 && tiles) build_tile_list(counts, group_keys, wave_start, tiles, n_tiles, bn);
+    if (blockIdx.x == 0 && tiles) build_tile_list(counts, group_keys, wave_start, tiles, n_tiles, bn);
+    // one warp per row, eight rows per CTA; a lane keeps up to eight 16-byte loads in flight before it stores
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int r = blockIdx.x * 8 + warp;
     if (r >= *n_valid) return;
-    const uint4* src = reinterpret_cast<const uint4*>(hidden + (size_t)(perm[r] / top_k) * H);
+    int token = 0;
+    if (lane == 0) token = perm[r] / top_k;
+    token = __shfl_sync(0xffffffffu, token, 0);
+    const uint4* src = reinterpret_cast<const uint4*>(hidden + (size_t)token * H);
     uint4* dst = reinterpret_cast<uint4*>(xg + (size_t)r * H);
-    for (int i = threadIdx.x; i < H / 8; i += 256) dst[i] = src[i];
+    const int n16 = H / 8;
+    for (int base = 0; base < n16; base += 256) {
+        uint4 v[8];
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            const int i = base + lane + 32 * j;
+            if (i < n16) v[j] = src[i];
+        }
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            const int i = base + lane + 32 * j;
+            if (i < n16) dst[i] = v[j];
+        }
+    }
 }
 
 }  // namespace
@@ -550,7 +568,7 @@ void launch_gather_rows(const __nv_bfloat16* hidden, const int32_t* perm, const 
                         bool small_n, cudaStream_t st) {
     int32_t* n_tiles = reinterpret_cast<int32_t*>(scratch);
     Tile* tiles = single_wave ? reinterpret_cast<Tile*>(reinterpret_cast<unsigned char*>(scratch) + 256) : nullptr;
-    gather_rows_kernel<<<n_pairs, 256, 0, st>>>(hidden, perm, n_valid, top_k, H, xg, single_wave ? single_wave->counts : nullptr,
+    gather_rows_kernel<<<(n_pairs + 7) / 8, 256, 0, st>>>(hidden, perm, n_valid, top_k, H, xg, single_wave ? single_wave->counts : nullptr,
                                                  single_wave ? single_wave->group_keys : nullptr, wave_start, tiles, n_tiles,
                                                  small_n ? BN_SMALL : BN);
     count_launch();
