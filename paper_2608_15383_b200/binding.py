@@ -52,6 +52,8 @@ _SIGNATURES = {
     "exmoe_route": (c_int, [POINTER(exmoe_shape), c_void_p, c_void_p, c_void_p, c_int, c_void_p, c_void_p, c_void_p]),
     "exmoe_cache_get_state": (c_int, [c_void_p, c_int, c_void_p, c_void_p, c_void_p, c_void_p]),
     "exmoe_debug_last_plan": (c_int, [c_void_p, c_int] + [c_void_p] * 9),
+    "exmoe_debug_last_path": (c_int, [c_void_p]),
+    "exmoe_debug_force_cluster_size": (c_int, [c_int]),
     "exmoe_debug_read_slot": (c_int, [c_void_p, c_int, c_int, c_void_p]),
     "exmoe_debug_wait_timeout": (c_int, [c_void_p, ctypes.c_longlong, POINTER(c_int)]),
     "exmoe_cache_stats": (c_int, [c_void_p, c_int, POINTER(exmoe_stats)]),
@@ -165,6 +167,11 @@ def exmoe_route(shape, hidden, w_router, bias=None, topk_ids=None, topk_weights=
     return topk_ids, topk_weights
 
 
+def exmoe_debug_force_cluster_size(cluster_size):
+    """Test hook: restrict the one-launch tiny-batch kernel to one cluster size (1, 2, 4, 8); 0 = automatic."""
+    _check(lib().exmoe_debug_force_cluster_size(int(cluster_size)), "exmoe_debug_force_cluster_size")
+
+
 def exmoe_launch_count():
     return int(lib().exmoe_launch_count())
 
@@ -207,6 +214,7 @@ def pad_hidden(hidden, d_model_padded):
 
 
 MISS_HOST_COPIES, MISS_DEVICE_FETCH = 0, 1
+PATH_CLUSTER, PATH_PAIR, PATH_SMALL, PATH_STREAM, PATH_TENSOR_SMALL_N, PATH_TENSOR, PATH_COOP = 1, 2, 3, 4, 5, 6, 7
 
 
 class Cache:
@@ -236,8 +244,6 @@ class Cache:
         T = hidden.shape[0]
         if out is None:
             out = torch.empty_like(hidden)
-        if T == 0:
-            return out
         rc = lib().exmoe_moe_forward(self.handle, int(layer), _dev(hidden, torch.bfloat16, "hidden"),
                                      _dev(topk_ids, torch.int32, "topk_ids"), _dev(topk_weights, torch.float32, "topk_weights"),
                                      int(T), _dev(out, torch.bfloat16, "out"), _stream_ptr(stream))
@@ -291,6 +297,13 @@ class Cache:
                 "offsets": offsets.numpy(), "perm": perm.numpy()[:n_valid],
                 "misses": [tuple(int(x) for x in misses[3 * i:3 * i + 3]) for i in range(nm)]}
 
+    def last_path(self):
+        """PATH_* of the kernel family that served the most recent forward (exmoe_debug_last_path)."""
+        rc = int(lib().exmoe_debug_last_path(self.handle))
+        if rc < 0:
+            raise ExmoeError(rc, "exmoe_debug_last_path")
+        return rc
+
     def read_slot(self, layer, slot):
         out = torch.empty(self.bytes_per_expert, dtype=torch.uint8)
         _check(lib().exmoe_debug_read_slot(self.handle, layer, slot, out.data_ptr()), "exmoe_debug_read_slot")
@@ -309,7 +322,8 @@ class Cache:
 
     # exmoe_cache_set_miss_path
     def set_miss_path(self, mode):
-        """mode: MISS_HOST_COPIES (default) or MISS_DEVICE_FETCH (no host wait; graph-capturable with C < E)."""
+        """mode: MISS_DEVICE_FETCH (the default when the banks are mapped: no host wait, graph-capturable with C < E)
+        or MISS_HOST_COPIES (plan read back once per call, one host-issued copy per miss on the copy stream)."""
         _check(lib().exmoe_cache_set_miss_path(self.handle, int(mode)), "exmoe_cache_set_miss_path")
 
     # exmoe_cache_prefetch

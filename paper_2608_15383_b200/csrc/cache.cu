@@ -62,10 +62,12 @@ struct exmoe_cache {
     size_t plan_d2h_bytes;                    // header | wave_of | slot_of | misses, contiguous
     __nv_bfloat16* act;                       // [max_pairs, I] SwiGLU output, grouped row order
     float* y;                                 // [max_pairs, H] weighted expert outputs, pair order
+    float* yk;                                // partial down results of the one-launch tiny-batch kernel
     int* arrive;                              // fused-combine arrival counters of the small path
     size_t arrive_words;
     bool last_small;
     bool last_pair;
+    int last_path;                            // EXMOE_PATH_* of the most recent forward
     int32_t* saved_ids;                       // ids of the last pairwise call (plan materialised on request)
     bool stream_ok;                           // the shape fits the streaming middle-regime kernels
     void* tc_scratch;                         // tile list of the tensor-core path
@@ -92,6 +94,7 @@ struct exmoe_cache {
     struct HostGraph {
         cudaGraphExec_t exec;
         bool last_small, last_pair;
+        int last_path;
     };
     std::map<long long, HostGraph> host_graphs;
 };
@@ -165,6 +168,7 @@ static void carve_workspace(exmoe_cache* c, uint8_t* ws, size_t* total) {
     }
     c->act = k.take<__nv_bfloat16>((size_t)c->max_pairs * s.d_ff);
     c->y = k.take<float>((size_t)c->max_pairs * s.d_model);
+    c->yk = k.take<float>(cluster_partial_floats(s.d_model, s.d_ff));
     c->arrive_words = (size_t)(kSmallMaxPairs / s.top_k + 1) * (s.d_model / kPanelRows);
     c->arrive = k.take<int>(c->arrive_words);
     c->saved_ids = k.take<int32_t>(kPairMaxPairs);
@@ -423,6 +427,8 @@ int exmoe_moe_forward(exmoe_cache* c, int layer, const void* hidden, const int32
     c->last_pair = pairwise;
     const bool use_stream = !small && c->stream_ok && P <= kStreamMaxPairs;
     const bool small_n = P <= kPrefillSmallNMaxPairs;      // tensor-core path: which kernel shape
+    c->last_path = pairwise ? EXMOE_PATH_PAIR : small ? EXMOE_PATH_SMALL : use_stream ? EXMOE_PATH_STREAM
+                   : small_n ? EXMOE_PATH_TENSOR_SMALL_N : EXMOE_PATH_TENSOR;
     if (!small && build_plan && !use_stream) {
         ProfScope ps(c, PROF_PLAN, st);                  // hidden rows in plan order, once for all waves
         tiles_fused = (n_waves == 1);                    // one wave: its tile list comes out of the same launch
@@ -476,13 +482,18 @@ int exmoe_moe_forward(exmoe_cache* c, int layer, const void* hidden, const int32
             sw.act = c->act;
             sw.topk_w = topk_weights;
             sw.y = c->y;
+            sw.yk = c->yk;
             sw.out = (__nv_bfloat16*)out;
             sw.max_rows = T;
             sw.max_groups = groups;
             sw.pairwise = pairwise;
             sw.saved_ids = c->saved_ids;
-            if (pairwise && !c->prof_only && !c->prof_on) {
-                launch_small_wave(a, sw, st, true, true);                // may fuse both GEMMs into one launch
+            if (pairwise && !c->prof_only && !c->prof_on && !cluster_forced_size() && launch_coop_decode(a, sw, c->d_status + 16, st)) {
+                c->last_path = EXMOE_PATH_COOP;                          // the whole layer in one cooperative launch
+            } else if (pairwise && !c->prof_only && !c->prof_on && launch_cluster_decode(a, sw, st)) {
+                c->last_path = EXMOE_PATH_CLUSTER;                       // the whole layer in one launch
+            } else if (pairwise && !c->prof_only && !c->prof_on) {
+                launch_small_wave(a, sw, st, true, true);
             } else {
                 if (!c->prof_only || c->prof_only == PROF_GATEUP) {
                     ProfScope ps(c, PROF_GATEUP, st);
@@ -608,6 +619,7 @@ int exmoe_moe_forward_host(exmoe_cache* c, int layer, const void* hidden_host, c
         c->last_T = T;
         c->last_small = it->second.last_small;
         c->last_pair = it->second.last_pair;
+        c->last_path = it->second.last_path;
         if (cudaGraphLaunch(it->second.exec, st) != cudaSuccess) rc = EXMOE_ERR_CUDA;
     } else {
         rc = enqueue();                                                   // this call runs as plain launches
@@ -625,7 +637,7 @@ int exmoe_moe_forward_host(exmoe_cache* c, int layer, const void* hidden_host, c
         }
         ok = ok && cudaGraphInstantiate(&exec, g, 0) == cudaSuccess;
         if (g) cudaGraphDestroy(g);
-        if (ok) c->host_graphs[key] = exmoe_cache::HostGraph{exec, c->last_small, c->last_pair};
+        if (ok) c->host_graphs[key] = exmoe_cache::HostGraph{exec, c->last_small, c->last_pair, c->last_path};
         else cudaGetLastError();                                          // stay on plain launches for this key
     }
     return rc;
@@ -704,6 +716,18 @@ int exmoe_debug_last_plan(exmoe_cache* c, int layer, int32_t* n_active, int32_t*
     if (offsets) std::memcpy(offsets, off.data(), off.size() * 4);
     if (perm) ok = ok && cudaMemcpy(perm, c->plan.perm, (size_t)c->last_T * c->shape.top_k * 4, cudaMemcpyDeviceToHost) == cudaSuccess;
     return ok ? EXMOE_OK : EXMOE_ERR_CUDA;
+}
+
+int exmoe_debug_last_path(exmoe_cache* c) {
+    if (!c) return EXMOE_ERR_ARG;
+    if (c->last_layer < 0) return EXMOE_ERR_STATE;
+    return c->last_path;
+}
+
+int exmoe_debug_force_cluster_size(int cluster_size) {
+    if (cluster_size != 0 && cluster_size != 1 && cluster_size != 2 && cluster_size != 4 && cluster_size != 8) return EXMOE_ERR_ARG;
+    cluster_force_size(cluster_size);
+    return EXMOE_OK;
 }
 
 int exmoe_debug_read_slot(exmoe_cache* c, int layer, int slot, void* host_out) {
