@@ -221,24 +221,13 @@ int exmoe_debug_last_plan(exmoe_cache* cache, int layer, int32_t* n_active, int3
  * number of waves and on whether the shape fits the kernel, never on the values of the tensors.  Returns one of
  * EXMOE_PATH_* (positive), EXMOE_ERR_STATE before the first forward.  Does not synchronise. */
 enum {
-    EXMOE_PATH_CLUSTER = 1,        /* one launch, a thread-block cluster per token-expert pair (T*k <= 24, one wave) */
-    EXMOE_PATH_PAIR = 2,           /* per-pair gate/up kernel + by-token down kernel (same sizes, other shapes) */
+    EXMOE_PATH_PAIR = 2,           /* per-pair gate/up kernel + by-token down kernel (T*k <= 24, one wave) */
     EXMOE_PATH_SMALL = 3,          /* grouping rebuilt inside the GEMM CTAs (T*k <= 24, several waves) */
     EXMOE_PATH_STREAM = 4,         /* bulk-copy weight ring + register dequantisation (T*k <= 512) */
     EXMOE_PATH_TENSOR_SMALL_N = 5, /* tcgen05 kernels, 64-row token tiles (T*k <= 1024) */
-    EXMOE_PATH_TENSOR = 6,         /* tcgen05 kernels, 256-row token tiles */
-    EXMOE_PATH_COOP = 7            /* one cooperative launch, a device-wide barrier between the projections (one token) */
+    EXMOE_PATH_TENSOR = 6          /* tcgen05 kernels, 256-row token tiles */
 };
 int exmoe_debug_last_path(exmoe_cache* cache);
-
-/* Test hook of the one-launch tiny-batch kernels (no paper counterpart).  By default a tiny batch whose CTAs can all
- * be resident at once runs the cooperative kernel (EXMOE_PATH_COOP); otherwise, up to 8 pairs, the cluster kernel,
- * which gives each (token-expert pair, K range of the down projection) to a thread-block cluster and picks the
- * smallest cluster size whose CTAs fit their weight slices into shared memory.  cluster_size = 1, 2, 4 or 8 sends
- * every tiny batch (up to 24 pairs) to the cluster kernel with exactly that size (shapes it does not fit fall back
- * to EXMOE_PATH_PAIR); 0 restores the default; EXMOE_ERR_ARG otherwise.  Process-wide; the layer output does not
- * depend on it. */
-int exmoe_debug_force_cluster_size(int cluster_size);
 
 /* Copy one slot's bytes back to the host (test hook for the miss-copy path; synchronises). */
 int exmoe_debug_read_slot(exmoe_cache* cache, int layer, int slot, void* host_out);

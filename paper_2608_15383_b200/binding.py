@@ -53,7 +53,6 @@ _SIGNATURES = {
     "exmoe_cache_get_state": (c_int, [c_void_p, c_int, c_void_p, c_void_p, c_void_p, c_void_p]),
     "exmoe_debug_last_plan": (c_int, [c_void_p, c_int] + [c_void_p] * 9),
     "exmoe_debug_last_path": (c_int, [c_void_p]),
-    "exmoe_debug_force_cluster_size": (c_int, [c_int]),
     "exmoe_debug_read_slot": (c_int, [c_void_p, c_int, c_int, c_void_p]),
     "exmoe_debug_wait_timeout": (c_int, [c_void_p, ctypes.c_longlong, POINTER(c_int)]),
     "exmoe_cache_stats": (c_int, [c_void_p, c_int, POINTER(exmoe_stats)]),
@@ -167,11 +166,6 @@ def exmoe_route(shape, hidden, w_router, bias=None, topk_ids=None, topk_weights=
     return topk_ids, topk_weights
 
 
-def exmoe_debug_force_cluster_size(cluster_size):
-    """Test hook: restrict the one-launch tiny-batch kernel to one cluster size (1, 2, 4, 8); 0 = automatic."""
-    _check(lib().exmoe_debug_force_cluster_size(int(cluster_size)), "exmoe_debug_force_cluster_size")
-
-
 def exmoe_launch_count():
     return int(lib().exmoe_launch_count())
 
@@ -214,7 +208,7 @@ def pad_hidden(hidden, d_model_padded):
 
 
 MISS_HOST_COPIES, MISS_DEVICE_FETCH = 0, 1
-PATH_CLUSTER, PATH_PAIR, PATH_SMALL, PATH_STREAM, PATH_TENSOR_SMALL_N, PATH_TENSOR, PATH_COOP = 1, 2, 3, 4, 5, 6, 7
+PATH_PAIR, PATH_SMALL, PATH_STREAM, PATH_TENSOR_SMALL_N, PATH_TENSOR = 2, 3, 4, 5, 6
 
 
 class Cache:

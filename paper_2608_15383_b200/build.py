@@ -9,7 +9,7 @@ import sys
 PKG = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(PKG, "csrc")
 LIB = os.path.join(PKG, "libexmoe.so")
-SOURCES = ["pack.cu", "plan.cu", "decode.cu", "cluster.cu", "coop.cu", "stream.cu", "prefill.cu", "route.cu", "cache.cu"]
+SOURCES = ["pack.cu", "plan.cu", "decode.cu", "stream.cu", "prefill.cu", "route.cu", "cache.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "--shared"]
 

@@ -62,7 +62,6 @@ struct exmoe_cache {
     size_t plan_d2h_bytes;                    // header | wave_of | slot_of | misses, contiguous
     __nv_bfloat16* act;                       // [max_pairs, I] SwiGLU output, grouped row order
     float* y;                                 // [max_pairs, H] weighted expert outputs, pair order
-    float* yk;                                // partial down results of the one-launch tiny-batch kernel
     int* arrive;                              // fused-combine arrival counters of the small path
     size_t arrive_words;
     bool last_small;
@@ -168,7 +167,6 @@ static void carve_workspace(exmoe_cache* c, uint8_t* ws, size_t* total) {
     }
     c->act = k.take<__nv_bfloat16>((size_t)c->max_pairs * s.d_ff);
     c->y = k.take<float>((size_t)c->max_pairs * s.d_model);
-    c->yk = k.take<float>(cluster_partial_floats(s.d_model, s.d_ff));
     c->arrive_words = (size_t)(kSmallMaxPairs / s.top_k + 1) * (s.d_model / kPanelRows);
     c->arrive = k.take<int>(c->arrive_words);
     c->saved_ids = k.take<int32_t>(kPairMaxPairs);
@@ -482,17 +480,12 @@ int exmoe_moe_forward(exmoe_cache* c, int layer, const void* hidden, const int32
             sw.act = c->act;
             sw.topk_w = topk_weights;
             sw.y = c->y;
-            sw.yk = c->yk;
             sw.out = (__nv_bfloat16*)out;
             sw.max_rows = T;
             sw.max_groups = groups;
             sw.pairwise = pairwise;
             sw.saved_ids = c->saved_ids;
-            if (pairwise && !c->prof_only && !c->prof_on && !cluster_forced_size() && launch_coop_decode(a, sw, c->d_status + 16, st)) {
-                c->last_path = EXMOE_PATH_COOP;                          // the whole layer in one cooperative launch
-            } else if (pairwise && !c->prof_only && !c->prof_on && launch_cluster_decode(a, sw, st)) {
-                c->last_path = EXMOE_PATH_CLUSTER;                       // the whole layer in one launch
-            } else if (pairwise && !c->prof_only && !c->prof_on) {
+            if (pairwise && !c->prof_only && !c->prof_on) {
                 launch_small_wave(a, sw, st, true, true);
             } else {
                 if (!c->prof_only || c->prof_only == PROF_GATEUP) {
@@ -722,12 +715,6 @@ int exmoe_debug_last_path(exmoe_cache* c) {
     if (!c) return EXMOE_ERR_ARG;
     if (c->last_layer < 0) return EXMOE_ERR_STATE;
     return c->last_path;
-}
-
-int exmoe_debug_force_cluster_size(int cluster_size) {
-    if (cluster_size != 0 && cluster_size != 1 && cluster_size != 2 && cluster_size != 4 && cluster_size != 8) return EXMOE_ERR_ARG;
-    cluster_force_size(cluster_size);
-    return EXMOE_OK;
 }
 
 int exmoe_debug_read_slot(exmoe_cache* c, int layer, int slot, void* host_out) {

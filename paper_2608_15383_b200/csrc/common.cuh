@@ -74,7 +74,6 @@ struct SmallWave {
     __nv_bfloat16* act;
     const float* topk_w;
     float* y;
-    float* yk;                  // [kSmallMaxPairs, K ranges of the down projection, H] partial results of the one-launch kernel
     __nv_bfloat16* out;
     int max_rows, max_groups;
     bool pairwise;              // T*k <= kPairMaxPairs and a single wave: per-pair gate/up, by-token down
@@ -86,14 +85,6 @@ constexpr int kPairMaxPairs = 32;
 #endif
 constexpr int kSmallMaxPairs = EXMOE_SMALL_MAX_PAIRS;
 constexpr int kSmallMaxSlots = 1024;
-#ifndef EXMOE_CLUSTER_MAX_PAIRS
-#define EXMOE_CLUSTER_MAX_PAIRS 8
-#endif
-constexpr int kClusterMaxPairs = EXMOE_CLUSTER_MAX_PAIRS;   // one-launch kernel (cluster.cu) up to this many pairs
-#ifndef EXMOE_COOP_MAX_PAIRS
-#define EXMOE_COOP_MAX_PAIRS 32
-#endif
-constexpr int kCoopMaxPairs = EXMOE_COOP_MAX_PAIRS;         // cooperative one-launch kernel (coop.cu), when all CTAs fit the GPU
 
 // launch accounting (exmoe_launch_count)
 void count_launch(int n = 1);
@@ -130,13 +121,6 @@ bool stream_supported(int H, int I);
 bool launch_stream_wave(const GemmArgs& a, const __nv_bfloat16* hidden, __nv_bfloat16* act, const float* topk_w, float* y,
                         int* status, int max_groups, bool gateup, bool down, cudaStream_t st);
 void launch_small_wave(const GemmArgs& a, const SmallWave& w, cudaStream_t st, bool gateup, bool down);
-// One-launch tiny-batch layer (cluster.cu): a thread-block cluster per token-expert pair; false = shape not served, nothing queued.
-bool launch_cluster_decode(const GemmArgs& a, const SmallWave& w, cudaStream_t st);
-// One-launch one-token layer (coop.cu): cooperative kernel, one device-wide barrier; `sync_words` = two zero-initialised ints.
-bool launch_coop_decode(const GemmArgs& a, const SmallWave& w, int* sync_words, cudaStream_t st);
-size_t cluster_partial_floats(int H, int I);      // size of SmallWave::yk
-void cluster_force_size(int cs);                  // test hook: 0 = choose by shape, 1/2/4/8 = only that cluster size
-int cluster_forced_size();
 size_t prefill_scratch_bytes(int max_pairs, int num_experts);
 // CUtensorMap objects of the grouped hidden rows and of the activations: 256-row boxes for the large-N kernel shape,
 // 64-row boxes for the small-N shape

@@ -846,18 +846,8 @@ void launch_pair_gateup(const GemmArgs& a, const SmallArgs& sa, const __nv_bfloa
 // K split over KS warps (KS in {1,2,4,8}, 8/KS panels per CTA) and register depth NB; aims at
 // four blocks per warp so that all of a warp's weights are in flight at once.
 struct DecodeCfg { int NB, KS, bpw; };
-// `down`: the down projection prefers K ranges of at most two blocks (256 intermediates), so that one small
-// thread-block cluster of the one-launch kernel (cluster.cu) can produce exactly the activations a range needs;
-// every kernel of this family then adds the same ranges in the same order.
-DecodeCfg pick_cfg(int K, int rows, bool down) {
+DecodeCfg pick_cfg(int K, int rows) {
     const int KB = K / kGroup;
-    if (down) {
-        for (int bpw = 2; bpw >= 1; --bpw) {
-            if (KB % bpw) continue;
-            const int ksv = KB / bpw;
-            if ((ksv == 1 || ksv == 2 || ksv == 4 || ksv == 8) && rows % (kPanelRows * (8 / ksv)) == 0) return {bpw, ksv, bpw};
-        }
-    }
     int pref = 1;
     while (pref < 8 && KB / (pref * 2) >= 4) pref *= 2;
     const int order[4][4] = {{1, 2, 4, 8}, {2, 1, 4, 8}, {4, 2, 8, 1}, {8, 4, 2, 1}};
@@ -908,7 +898,7 @@ template <bool GATEUP, int MODE>
 void launch_decode(const GemmArgs& a, const SmallArgs& sa, const __nv_bfloat16* x, __nv_bfloat16* act, const float* w,
                    float* y, int max_rows, int max_groups, cudaStream_t st) {
     const int K = GATEUP ? a.H : a.I, NR = GATEUP ? a.I : a.H;
-    const DecodeCfg cfg = pick_cfg(K, NR, !GATEUP);
+    const DecodeCfg cfg = pick_cfg(K, NR);
     // rows per pass: one 8-row chunk covers decode; more chunks amortise the dequantisation
     int nch = max_rows <= 8 ? 1 : (max_rows <= 16 ? 2 : 4);
     while (nch > 1 && (size_t)8 * nch * (K * 2 + 64) > 150 * 1024) nch >>= 1;
@@ -1022,13 +1012,6 @@ bool launch_token_down_bulk(const GemmArgs& a, const SmallArgs& sa, const __nv_b
     return true;
 }
 
-// The K split (ranges per matrix row panel, blocks per range) that fixes the rounding order of every decode kernel.
-void decode_k_split(int K, int rows, bool down, int* ks, int* bpw) {
-    const DecodeCfg cfg = pick_cfg(K, rows, down);
-    *ks = cfg.KS;
-    *bpw = cfg.bpw;
-}
-
 // One wave of the SMALL path: gate/up kernel, then the down kernel with the fused combine.
 void launch_small_wave(const GemmArgs& a, const SmallWave& w, cudaStream_t st, bool gateup, bool down) {
     SmallArgs sa{};
@@ -1048,7 +1031,7 @@ void launch_small_wave(const GemmArgs& a, const SmallWave& w, cudaStream_t st, b
     sa.saved_ids = w.saved_ids;
     if (w.pairwise) {                                   // T*k <= 32, one wave: no grouping, by-token down + combine
         if (gateup) {
-            const DecodeCfg cfg = pick_cfg(a.H, a.I, false);
+            const DecodeCfg cfg = pick_cfg(a.H, a.I);
             if (cfg.bpw == 4) launch_pair_gateup<4>(a, sa, w.hidden, w.act, cfg.KS, st);
             else if (cfg.bpw == 2) launch_pair_gateup<2>(a, sa, w.hidden, w.act, cfg.KS, st);
             else if (cfg.bpw == 1) launch_pair_gateup<1>(a, sa, w.hidden, w.act, cfg.KS, st);
@@ -1056,7 +1039,7 @@ void launch_small_wave(const GemmArgs& a, const SmallWave& w, cudaStream_t st, b
         }
         if (down) {
             const int KB = a.I / kGroup;
-            const int bpwg = pick_cfg(a.I, a.H, true).bpw;    // the grouped kernel's K-split range, replayed for rounding
+            const int bpwg = pick_cfg(a.I, a.H).bpw;    // the grouped kernel's K-split range, replayed for rounding
             const int T = w.n_pairs / a.top_k;
             bool done = false;
 #ifndef EXMOE_NO_BULK_DECODE
