@@ -11,9 +11,14 @@ experts) so that every step's weights come from HBM, not from the 126 MB L2.
 
 Prints ONE JSON line: MoE-layer tokens/s (inputs resident in HBM, CUDA-graph replay, CUDA events),
 the end-to-end number through host buffers, the roofline of the dominant kernel (gate/up GEMM;
-packed weight + scale bytes it must read / its CUDA-event time / measured HBM copy rate), the CPU
-oracle timed on the host cores on a bounded sample, SM clocks sampled during the timed region and
-the number of kernels launched.  `--impl reference` times the CPU oracle alone.
+packed weight + scale bytes it must read / its CUDA-event time / measured HBM copy rate) and of the
+whole step, the CPU oracle timed on the host cores on a bounded sample, SM clocks sampled during the
+timed region and the number of kernels launched.  The timed region is long whatever --steps is: the
+graph of K steps is replayed until a repetition lasts at least 60 ms, five repetitions are taken and
+the median is reported (with the spread), so that the clocks are up and the sampler sees the region.
+The default (decode) run then adds two short legs to the same line: `config.prefill` (config 4,
+tensor-core roofline) and `config.offload` (config 3, host-link roofline), plus the pack throughput.
+`--impl reference` times the CPU oracle alone.
 """
 import argparse
 import json
@@ -40,10 +45,12 @@ WORKLOADS = {
                 "x alpha, alpha cycling over {2, 1, 0.5, 0} in four blocks of steps (1-4 waves per step)"),
     "prefill": (2048, 64, 1, 0.0, "config4: OLMoE-shaped prefill, T=2048, 64 slots resident, uniform routing"),
 }
-# DRAM bytes (read + write) per launch of the dominant kernel, from the committed ncu captures under profiles/
-# (decode: profiles/decode_t1_c64_pair_kernels_ncu_full.md; decode16: profiles/decode16_t16_c64_stream_kernels_ncu_full.md;
-# prefill: profiles/prefill_t2048_c64_tcgen05_ncu_full.md)
-NCU_TRAFFIC_BYTES = {"decode": 17.33e6, "decode16": 62.83e6 + 0.87e6, "prefill": 214.68e6 + 12.51e6}
+# DRAM bytes (read + write) per launch of the dominant kernel, from one ncu capture each (dram__bytes_read.sum +
+# dram__bytes_write.sum, two layer banks = 415 MB resident; per-launch traffic does not depend on the number of banks):
+# (bytes, kernel captured, date of the capture)
+NCU_TRAFFIC = {"decode": (17.33e6, "pair_gateup_kernel<4>, T=1", "2026-11-25"),
+               "decode16": (62.83e6 + 0.87e6, "stream_gemm_kernel<1,true,1>, T=16", "2026-11-25"),
+               "prefill": (214.68e6 + 12.51e6, "prefill_gemm_kernel<true,256,2>, T=2048", "2026-11-25")}
 METRIC = "moe_layer_tokens_per_s"
 UNIT = "tokens/s"
 
@@ -60,7 +67,7 @@ def load_peaks():
 
 class ClockSampler:
     """SM clock and throttle reasons of this rank's GPU while the timed region runs.  Read-only NVML queries from a
-    sampling thread every ~2 ms (the timed region of the decode workload lasts ~13 ms); falls back to
+    sampling thread every ~5 ms (every timed region lasts hundreds of ms); falls back to
     `nvidia-smi -lms 100` when the NVML binding is missing."""
     Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
          "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
@@ -91,7 +98,7 @@ class ClockSampler:
                                 self.reasons.add(n)
                     except Exception:
                         pass
-                    time.sleep(0.002)
+                    time.sleep(0.005)
             self.thread = threading.Thread(target=loop, daemon=True)
             self.thread.start()
             return
@@ -117,7 +124,7 @@ class ClockSampler:
             self.thread.join(timeout=2)
             if self.sm:
                 out.update(sm_mhz=float(np.median(self.sm)), sm_max_mhz=float(max(self.mx)), reasons=sorted(self.reasons),
-                           samples=len(self.sm), source="nvml, 2 ms period")
+                           samples=len(self.sm), source="nvml, 5 ms period")
             return out
         if self.p is None:
             return out
@@ -183,13 +190,29 @@ def make_inputs(shape, T, n_sets, alpha, seed0, device):
     return hs, ids, ws
 
 
+PACK_STATS = {}
+
+
 def build_banks(shape, layers, seed0, device, keep_layer0=False):
-    """Per layer: draw BF16 expert weights on the device, pack them with exmoe_pack into a pinned host bank."""
+    """Per layer: draw BF16 expert weights on the device, pack them with exmoe_pack into a pinned host bank.
+    The last layer's packing (exmoe_pack alone, device buffers in and out, host clock around a synchronised loop) is timed."""
     from paper_2608_15383_b200 import binding
     banks, kept = [], None
     for l in range(layers):
         wg, wu, wd = synth.expert_weights(shape, seed0 + l, device=device)
         banks.append(binding.pack_bank(shape, wg, wu, wd, device=device))
+        if l == layers - 1:
+            buf = torch.empty(binding.exmoe_packed_bytes(shape), dtype=torch.uint8, device=device)
+            torch.cuda.synchronize()
+            t0 = time.perf_counter()
+            for e in range(shape.num_experts):
+                binding.exmoe_pack(shape, wg[e], wu[e], wd[e], buf)
+            torch.cuda.synchronize()
+            dt = time.perf_counter() - t0
+            read = 3 * shape.d_ff * shape.d_model * 2
+            PACK_STATS.update({"experts_per_s": shape.num_experts / dt, "bf16_gb_read_per_s": shape.num_experts * read / dt / 1e9,
+                               "us_per_expert": 1e6 * dt / shape.num_experts,
+                               "note": "exmoe_pack, one synchronous call per expert (the status covers the data)"})
         if l == 0 and keep_layer0:
             kept = (wg.cpu(), wu.cpu(), wd.cpu())
         del wg, wu, wd
@@ -240,7 +263,7 @@ def run_reference(args, rank, world):
     per_step_budget = max(2.0, 120.0 / max(args.steps + args.warmup, 1))
     from oracle import moe as omoe, quant as oquant
     leg = None
-    for _ in range(args.warmup):
+    for _ in range(args.warmup):                         # one bounded-sample step each
         oracle_leg(shape, T, (wg, wu, wd), hs[:1], ids[:1], ws[:1], 0.0)
     t0 = time.perf_counter()
     tokens = 0
@@ -366,6 +389,272 @@ def run_stack_sweep(args, dev, binding):
     return rows
 
 
+MIN_REGION_MS = 60.0      # a timed repetition replays the K-step graph until it lasts at least this long
+REPS = 5                  # repetitions; the median is reported
+
+
+def timed_repetitions(stream, run_once, ms_hint=None):
+    """CUDA-event time of `run_once` (one graph replay of K steps, or K host-driven steps), repeated back to back until
+    a repetition lasts MIN_REGION_MS, REPS repetitions.  Returns (list of ms per call of run_once, calls per repetition)."""
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    with torch.cuda.stream(stream):
+        e0.record(stream)
+        run_once()
+        e1.record(stream)
+    stream.synchronize()
+    one = max(e0.elapsed_time(e1), 1e-3)
+    m = int(min(max(1, np.ceil(MIN_REGION_MS / one)), 20000))
+    out = []
+    for _ in range(REPS):
+        with torch.cuda.stream(stream):
+            e0.record(stream)
+            for _ in range(m):
+                run_once()
+            e1.record(stream)
+        stream.synchronize()
+        out.append(e0.elapsed_time(e1) / m)
+    return out, m
+
+
+def run_leg(name, args, shape, banks, dev, rank, local_rank, world, peaks, K, W, seed0, full):
+    """One workload through the device-timed path (and, if `full`, the per-kernel, end-to-end and copy-link parts).
+    Returns a dict with value, ms_per_step, roofline, kernel_us, clocks, launches and descriptive fields."""
+    import torch.distributed as dist
+    from paper_2608_15383_b200 import binding
+    T, C, L, alpha, desc = WORKLOADS[name]
+    L = min(args.layers or L, len(banks))
+    if full and args.tokens:
+        T, desc = args.tokens, desc + " [tokens per step overridden: %d]" % args.tokens
+    if full and args.slots:
+        C, desc = args.slots, desc + " [slots overridden: %d]" % args.slots
+    if full and args.alpha is not None:
+        alpha, desc = args.alpha, desc + " [routing skew alpha overridden: %g]" % args.alpha
+    cache = binding.Cache(shape, banks[:L], C, max_tokens=T, device=dev)
+    if C < shape.num_experts:
+        cache.set_miss_path(binding.MISS_DEVICE_FETCH if args.miss_path == "device" else binding.MISS_HOST_COPIES)
+        desc += " [miss path: %s]" % ("device-initiated fetch kernel" if args.miss_path == "device" else "host-issued copies")
+    n_sets = min(K + W, 1024) if T <= 64 else 4
+    hs, ids, ws = make_inputs(shape, T, n_sets, alpha, seed0, dev)
+    outs = [torch.empty_like(hs[0]) for _ in range(2)]
+    stream = torch.cuda.Stream(device=dev)
+    identity = (C == shape.num_experts)
+    graphable = identity or args.miss_path == "device"       # no host wait inside the call: the steps replay from a graph
+
+    def step(i, out):
+        cache.forward(i % L, hs[i % n_sets], ids[i % n_sets], ws[i % n_sets], out=out, stream=stream)
+
+    with torch.cuda.stream(stream):
+        for i in range(3):
+            step(i, outs[0])
+    stream.synchronize()
+
+    # ---- device-timed region: CUDA-graph replay of the K steps (no host sync inside), repeated (see timed_repetitions)
+    if graphable:
+        graph_w, graph_k = torch.cuda.CUDAGraph(), torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph_w, stream=stream):
+            for i in range(W):
+                step(i, outs[i & 1])
+        launches0 = binding.exmoe_launch_count()
+        with torch.cuda.graph(graph_k, stream=stream):
+            for i in range(W, W + K):
+                step(i, outs[i & 1])
+        launches = binding.exmoe_launch_count() - launches0
+        with torch.cuda.stream(stream):
+            graph_w.replay()
+            graph_k.replay()          # untimed first replay: uploads the instantiated graph to the device
+        run_once = graph_k.replay
+    else:
+        with torch.cuda.stream(stream):
+            for i in range(W):
+                step(i, outs[i & 1])
+        launches0 = binding.exmoe_launch_count()
+        with torch.cuda.stream(stream):
+            for i in range(W, W + K):
+                step(i, outs[i & 1])
+        launches = binding.exmoe_launch_count() - launches0
+
+        def run_once():
+            for i in range(W, W + K):
+                step(i, outs[i & 1])
+    stream.synchronize()
+    if world > 1:
+        dist.barrier()
+    torch.cuda.synchronize()
+    sampler = ClockSampler(local_rank)
+    stats0 = cache.stats(0) if not identity else None
+    sampler.mark()
+    reps_ms, replays = timed_repetitions(stream, run_once)
+    torch.cuda.synchronize()
+    clocks = sampler.stop()
+    if world > 1:
+        dist.barrier()
+    ms = max_over_ranks(float(np.median(reps_ms)), world, dev)              # ms per K steps, slowest rank's median
+    value = whole_job_tokens_per_s(world, K, T, ms)
+    ms_step = ms / K
+    if clocks.get("sm_mhz"):
+        clocks["us_per_step_x_sm_ghz"] = 1e3 * ms_step * clocks["sm_mhz"] / 1e3   # kcycles per step: compare across clock states
+
+    res = {"name": name, "desc": desc, "T": T, "C": C, "L": L, "K": K, "W": W, "value": value, "ms_per_step": ms_step,
+           "launches": int(launches), "clocks": clocks, "graphable": graphable,
+           "repetitions": {"count": REPS, "replays_of_the_K_step_graph_each": replays,
+                           "ms_per_step_min_median_max": [min(reps_ms) / K, float(np.median(reps_ms)) / K, max(reps_ms) / K],
+                           "region_ms_each": float(np.median(reps_ms)) * replays}}
+
+    # ---- per-kernel times (roofline of the dominant kernel): the same steps with ONLY one kernel kind
+    # launched, timed with CUDA events on the launching stream (graph replay when graphable), same repetition rule
+    n_prof = min(K, 200)
+    kinds = {}
+    for kind, kname in ((1, "gate_up"), (2, "down")):
+        cache.profile_enable(False, only=kind)
+        with torch.cuda.stream(stream):
+            step(0, outs[0])
+        stream.synchronize()
+        if identity:
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g, stream=stream):
+                for i in range(W, W + n_prof):
+                    step(i, outs[i & 1])
+            with torch.cuda.stream(stream):
+                g.replay()
+            kms, _ = timed_repetitions(stream, g.replay)
+        else:
+            def only_once():
+                for i in range(W, W + n_prof):
+                    step(i, outs[i & 1])
+            kms, _ = timed_repetitions(stream, only_once)
+        kinds[kname] = {"us_per_launch": 1e3 * float(np.median(kms)) / n_prof, "launches_per_replay": n_prof}
+    cache.profile_enable(False)
+    bpe = cache.bytes_per_expert
+    w13_bytes = bpe * 2 // 3
+    active = float(np.mean([len(torch.unique(ids[i % n_sets])) for i in range(W, W + n_prof)]))      # the steps timed above
+    active_all = float(np.mean([len(torch.unique(ids[i % n_sets])) for i in range(W, W + K, max(K // 200, 1))]))
+    step_gbs = active_all * bpe / (ms_step * 1e-3) / 1e9
+    flops_step = 2.0 * T * shape.top_k * 3 * shape.d_ff * shape.d_model
+    step_tflops = flops_step / (ms_step * 1e-3) / 1e12
+    traffic = NCU_TRAFFIC.get(name) if not (full and (args.tokens or args.slots)) else None
+    if T * shape.top_k > 512:
+        flops = 2.0 * T * shape.top_k * 2 * shape.d_ff * shape.d_model          # gate/up GEMM of one step
+        achieved = flops / (kinds["gate_up"]["us_per_launch"] * 1e-6) / 1e12
+        roof = {"bound": "tensor", "achieved": achieved, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
+                "frac": achieved / peaks["bf16_tflops"], "traffic": traffic[0] if traffic else None,
+                "traffic_unit": "bytes per launch (ncu dram read + write)",
+                "traffic_source": ("one ncu capture of %s on %s" % traffic[1:]) if traffic else None,
+                "kernel": "gate_up (prefill_gemm_kernel<true>, tcgen05)", "flops_per_launch": flops,
+                "peak_source": peaks["source"] + " cuBLAS bf16, burst",
+                "whole_step": {"achieved": step_tflops, "flops_per_step": flops_step, "frac": step_tflops / peaks["bf16_tflops"],
+                               "frac_of_sustained": step_tflops / peaks["bf16_tflops_sustained"]}}
+    else:
+        gu_bytes = active * w13_bytes                                            # packed gate/up codes + scales
+        achieved = gu_bytes / (kinds["gate_up"]["us_per_launch"] * 1e-6) / 1e9
+        roof = {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                "frac": achieved / peaks["hbm_gbs"], "traffic": traffic[0] if traffic else None,
+                "traffic_unit": "bytes per launch (ncu dram read + write)",
+                "traffic_source": ("one ncu capture of %s on %s" % traffic[1:]) if traffic else None,
+                "kernel": "gate_up (pair_gateup_kernel)" if T * shape.top_k <= 24 else "gate_up (stream_gemm_kernel<1,true,1>)",
+                "bytes_per_launch": gu_bytes, "peak_source": peaks["source"] + " copy rate, burst",
+                "whole_step": {"achieved": step_gbs, "bytes_per_step": active_all * bpe, "frac": step_gbs / peaks["hbm_gbs"]}}
+    if not identity:
+        roof["note"] = ("C < E: the timed launches include resolution and the waves' miss traffic, so this fraction is not a "
+                        "kernel figure; the workload is bound by the host link")
+    res.update({"roofline": roof, "kernel_us": kinds, "active_experts_per_step": active_all,
+                "packed_gb_per_s_whole_step": step_gbs, "tflops_whole_step": step_tflops, "bytes_per_expert": bpe})
+
+    extra = {}
+    if not identity:
+        st = cache.stats(0)
+        extra = {"hit_rate": st["hits"] / max(st["lookups"], 1), "h2d_expert_bytes_per_token":
+                 st["h2d_bytes"] / max(st["forwards"] * T, 1), "waves_per_step": st["waves"] / max(st["forwards"], 1)}
+        # the H2D link is the roofline of this workload: miss-traffic busy time and rate vs a plain pinned copy
+        n_c = min(K, 100)
+        cache.profile_enable(True)
+        b0 = cache.stats(0)["h2d_bytes"]
+        c0, c1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        with torch.cuda.stream(stream):
+            c0.record(stream)
+            for j in range(n_c):                              # steps spread evenly over the timed range (all alpha blocks)
+                i = W + j * max(K // n_c, 1)
+                step(i, outs[i & 1])
+            c1.record(stream)
+        stream.synchronize()
+        copy_ms, _ = cache.profile_read(4)
+        gemm_ms = cache.profile_read(1)[0] + cache.profile_read(2)[0]
+        wall_ms = c0.elapsed_time(c1)
+        moved = cache.stats(0)["h2d_bytes"] - b0
+        cache.profile_enable(False)
+        big = banks[0][:32]                                  # 104 MB of the pinned bank
+        dst = torch.empty_like(big, device=dev)
+        p0, p1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        dst.copy_(big, non_blocking=True)
+        torch.cuda.synchronize()
+        p0.record()
+        dst.copy_(big, non_blocking=True)
+        p1.record()
+        torch.cuda.synchronize()
+        ceiling = big.numel() / p0.elapsed_time(p1) / 1e6
+        rate = moved / max(copy_ms, 1e-9) / 1e6
+        res["roofline_gemm_view"] = res.pop("roofline")      # not a kernel figure here: the step is bound by the host link
+        res["roofline"] = {"bound": "host link", "achieved": rate, "peak": ceiling, "unit": "GB/s", "frac": rate / ceiling,
+                           "kernel": "fetch_misses_kernel (reads of the mapped pinned bank)" if args.miss_path == "device"
+                           else "host-issued cudaMemcpyAsync per miss",
+                           "whole_step_frac": (moved / n_c) / (ms_step * 1e-3) / 1e9 / ceiling,
+                           "miss_traffic_busy_fraction": copy_ms / wall_ms, "gemm_kernels_busy_fraction": gemm_ms / wall_ms,
+                           "h2d_bytes_per_step": moved / n_c,
+                           "peak_source": "one 104 MB pinned-host-to-device copy, measured in this run"}
+        res["kernel_us"] = {"note": "C < E: single-kind launches still carry resolution and miss traffic; see roofline"}
+        del dst
+    res["extra"] = extra
+
+    if full:
+        # ---- end to end: host buffers in, host buffer out, copies inside the timed region
+        n_e2e = min(max(K, 100), 300)
+        n_host = 8 if identity else min(n_sets, 128)
+        pick = [(j * n_sets) // n_host for j in range(n_host)]
+        h_h = [hs[j].cpu().pin_memory() for j in pick]
+        h_i = [ids[j].cpu().pin_memory() for j in pick]
+        h_w = [ws[j].cpu().pin_memory() for j in pick]
+        h_out = torch.empty_like(h_h[0]).pin_memory()
+
+        # the library's host-buffer entry point: inputs in host memory, result in host memory, synchronous; one call per
+        # step (it stages the three inputs, copies them to the device in one copy, runs the layer and waits; tiny batches
+        # replay a graph recorded per (layer, T), small results are written straight into pinned host memory, large
+        # page-locked tensors are used in place)
+        def e2e_step(i):
+            j = i % len(h_h)
+            cache.forward_host(i % L, h_h[j], h_i[j], h_w[j], out=h_out, stream=stream)
+
+        for i in range(max(3, 2 * L)):                      # every layer's graph (tiny batches) is recorded before the timed calls
+            e2e_step(i)
+        if world > 1:
+            dist.barrier()
+        t0 = time.perf_counter()
+        for i in range(n_e2e):
+            e2e_step(i)
+        dt = time.perf_counter() - t0
+        dt = max_over_ranks(dt, world, dev)
+        h2d = h_h[0].numel() * 2 + h_i[0].numel() * 4 + h_w[0].numel() * 4
+        res["e2e"] = {"value": world * n_e2e * T / dt, "unit": UNIT, "h2d_bytes_per_step": int(h2d),
+                      "d2h_bytes_per_step": int(h_out.numel() * 2), "steps": n_e2e,
+                      "mode": "exmoe_moe_forward_host: host tensors in and out, one synchronous call per step"}
+        res["inputs"] = (hs, ids, ws)
+    res["status"] = cache.status()
+    cache.close()
+    del cache
+    torch.cuda.empty_cache()
+    return res
+
+
+def leg_summary(r):
+    """The part of a leg that goes under config.<name> of the main line."""
+    out = {"workload": r["desc"], "tokens_per_step": r["T"], "slots": r["C"], "steps": r["K"], "warmup": r["W"],
+           "value": r["value"], "unit": UNIT, "ms_per_step": r["ms_per_step"], "repetitions": r["repetitions"],
+           "timing": "CUDA graph replay of all steps" if r["graphable"] else "host-driven loop (one plan read-back per step)",
+           "active_experts_per_step": r["active_experts_per_step"], "packed_gb_per_s_whole_step": r["packed_gb_per_s_whole_step"],
+           "tflops_whole_step": r["tflops_whole_step"], "kernel_us": r["kernel_us"], "roofline": r["roofline"],
+           "gpu_launches": r["launches"], "clocks": r["clocks"], "status": r["status"]}
+    out.update(r["extra"])
+    return out
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -384,6 +673,8 @@ def main():
     ap.add_argument("--tokens", type=int, default=0, help="override the workload's tokens per step")
     ap.add_argument("--cpu-budget", type=float, default=15.0, help="seconds of CPU oracle work for cpu_baseline")
     ap.add_argument("--layers", type=int, default=0, help="layer banks to rotate over (0 = the workload's default)")
+    ap.add_argument("--no-extra-legs", action="store_true",
+                    help="decode workload: skip the short prefill (config 4) and offload (config 3) legs")
     args = ap.parse_args()
 
     rank = int(os.environ.get("RANK", "0"))
@@ -394,7 +685,7 @@ def main():
         args.steps_requested = args.steps
         if args.steps > 50:
             args.steps = 50
-        args.warmup = min(args.warmup, 3)
+        args.warmup = min(args.warmup, 20)
         run_reference(args, rank, world)
         return
 
@@ -420,232 +711,45 @@ def main():
                                          "Zipf routing; the step includes the fused router kernel (Eq. 1) and the torch residual update between layers",
                                          "sweep": rows}}), flush=True)
         return
-    T, C, L, alpha, desc = WORKLOADS[args.workload]
-    L = args.layers or L
-    if args.tokens:
-        T, desc = args.tokens, desc + " [tokens per step overridden: %d]" % args.tokens
-    if args.slots:
-        C, desc = args.slots, desc + " [slots overridden: %d]" % args.slots
-    if args.alpha is not None:
-        alpha, desc = args.alpha, desc + " [routing skew alpha overridden: %g]" % args.alpha
     shape = synth.OLMOE
     K, W = args.steps, max(args.warmup, 3)
     peaks = load_peaks()
 
     # ---- data: replicas only, every rank holds the same workload with its own seed offset
     seed0 = 2000 + 100000 * rank
+    L = args.layers or WORKLOADS[args.workload][2]
     banks, w_cpu = build_banks(shape, L, seed0, dev, keep_layer0=(rank == 0))
-    cache = binding.Cache(shape, banks, C, max_tokens=T, device=dev)
-    if C < shape.num_experts:
-        cache.set_miss_path(binding.MISS_DEVICE_FETCH if args.miss_path == "device" else binding.MISS_HOST_COPIES)
-        desc += " [miss path: %s]" % ("device-initiated fetch kernel" if args.miss_path == "device" else "host-issued copies")
-    n_sets = min(K + W, 1024) if T <= 64 else 4
-    hs, ids, ws = make_inputs(shape, T, n_sets, alpha, seed0, dev)
-    outs = [torch.empty_like(hs[0]) for _ in range(2)]
-    stream = torch.cuda.Stream(device=dev)
-    identity = (C == shape.num_experts)
-    graphable = identity or args.miss_path == "device"       # no host wait inside the call: the steps replay from a graph
+    main_leg = run_leg(args.workload, args, shape, banks, dev, rank, local_rank, world, peaks, K, W, seed0, full=True)
+    hs, ids, ws = main_leg.pop("inputs")
+    T = main_leg["T"]
 
-    def step(i, out):
-        cache.forward(i % L, hs[i % n_sets], ids[i % n_sets], ws[i % n_sets], out=out, stream=stream)
-
-    with torch.cuda.stream(stream):
-        for i in range(3):
-            step(i, outs[0])
-    stream.synchronize()
-
-    # ---- device-timed region: CUDA-graph replay when the layer is fully resident (no host sync inside)
-    launches0 = binding.exmoe_launch_count()
-    graph_w = graph_k = None
-    if graphable:
-        graph_w, graph_k = torch.cuda.CUDAGraph(), torch.cuda.CUDAGraph()
-        with torch.cuda.graph(graph_w, stream=stream):
-            for i in range(W):
-                step(i, outs[i & 1])
-        launches0 = binding.exmoe_launch_count()
-        with torch.cuda.graph(graph_k, stream=stream):
-            for i in range(W, W + K):
-                step(i, outs[i & 1])
-        launches = binding.exmoe_launch_count() - launches0
-        with torch.cuda.stream(stream):
-            graph_w.replay()
-            graph_k.replay()          # untimed first replay: uploads the instantiated graph to the device
-    else:
-        with torch.cuda.stream(stream):
-            for i in range(W):
-                step(i, outs[i & 1])
-    stream.synchronize()
-    if world > 1:
-        dist.barrier()
-    torch.cuda.synchronize()
-    sampler = ClockSampler(local_rank)
-    time.sleep(0.15)
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    stats0 = cache.stats(0) if not identity else None
-    sampler.mark()
-    with torch.cuda.stream(stream):
-        e0.record(stream)
-        if graphable:
-            graph_k.replay()
-        else:
-            launches0 = binding.exmoe_launch_count()
-            for i in range(W, W + K):
-                step(i, outs[i & 1])
-            launches = binding.exmoe_launch_count() - launches0
-        e1.record(stream)
-    stream.synchronize()
-    torch.cuda.synchronize()
-    ms = e0.elapsed_time(e1)
-    clocks = sampler.stop()
-    if world > 1:
-        dist.barrier()
-    ms = max_over_ranks(ms, world, dev)
-    value = whole_job_tokens_per_s(world, K, T, ms)
-
-    # ---- per-kernel times (roofline of the dominant kernel): the same steps with ONLY one kernel kind
-    # launched, timed with CUDA events on the launching stream (graph replay when fully resident)
-    n_prof = min(K, 200)
-    kinds = {}
-    for kind, name in ((1, "gate_up"), (2, "down")):
-        cache.profile_enable(False, only=kind)
-        a0, a1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        if identity:
-            g = torch.cuda.CUDAGraph()
-            with torch.cuda.stream(stream):
-                step(0, outs[0])
-            stream.synchronize()
-            with torch.cuda.graph(g, stream=stream):
-                for i in range(W, W + n_prof):
-                    step(i, outs[i & 1])
-            with torch.cuda.stream(stream):
-                g.replay()
-                a0.record(stream)
-                g.replay()
-                a1.record(stream)
-        else:
-            with torch.cuda.stream(stream):
-                for i in range(3):
-                    step(i, outs[0])
-                a0.record(stream)
-                for i in range(W, W + n_prof):
-                    step(i, outs[i & 1])
-                a1.record(stream)
-        stream.synchronize()
-        kinds[name] = {"us_per_launch": 1e3 * a0.elapsed_time(a1) / n_prof, "launches": n_prof}
-    cache.profile_enable(False)
-    bpe = cache.bytes_per_expert
-    w13_bytes = bpe * 2 // 3
-    active = float(np.mean([len(torch.unique(ids[i % n_sets])) for i in range(W, W + n_prof)]))      # the steps timed above
-    active_all = float(np.mean([len(torch.unique(ids[i % n_sets])) for i in range(W, W + K, max(K // 200, 1))]))
-    if args.workload == "prefill":
-        flops = 2.0 * T * shape.top_k * 2 * shape.d_ff * shape.d_model          # gate/up GEMM of one step
-        achieved = flops / (kinds["gate_up"]["us_per_launch"] * 1e-6) / 1e12
-        roof = {"bound": "tensor", "achieved": achieved, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
-                "frac": achieved / peaks["bf16_tflops"],
-                "traffic": NCU_TRAFFIC_BYTES.get(args.workload) if not args.tokens else None,
-                "traffic_unit": "bytes per launch (ncu dram read + write)", "kernel": "gate_up (prefill_gemm_kernel<true>, tcgen05)", "flops_per_launch": flops,
-                "peak_source": peaks["source"] + " cuBLAS bf16, burst"}
-    else:
-        gu_bytes = active * w13_bytes                                            # packed gate/up codes + scales
-        achieved = gu_bytes / (kinds["gate_up"]["us_per_launch"] * 1e-6) / 1e9
-        roof = {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                "frac": achieved / peaks["hbm_gbs"],
-                "traffic": NCU_TRAFFIC_BYTES.get(args.workload) if not args.tokens else None,
-                "traffic_unit": "bytes per launch (ncu dram read + write)",
-                "kernel": "gate_up (pair_gateup_kernel)" if T * shape.top_k <= 24 else
-                "gate_up (stream_gemm_kernel<1,true,1>)" if T * shape.top_k <= 512 else "gate_up",
-                "bytes_per_launch": gu_bytes, "peak_source": peaks["source"] + " copy rate, burst"}
-    if not identity:
-        roof["note"] = ("C < E: the timed launches include resolution and the waves' miss traffic, so this fraction is not a "
-                        "kernel figure; the workload is bound by the host link: compare config.h2d_gb_per_s_during_copies "
-                        "with config.pinned_copy_ceiling_gb_per_s")
-    step_gbs = active_all * bpe / (ms * 1e-3 / K) / 1e9
-    step_tflops = 2.0 * T * shape.top_k * 3 * shape.d_ff * shape.d_model / (ms * 1e-3 / K) / 1e12
-
-    # ---- end to end: host buffers in, host buffer out, copies inside the timed region
-    n_e2e = min(K, 300)
-    # fully resident: eight input sets; with a cache (C < E) the sets are spread over the whole timed range, so that the
-    # end-to-end loop sees the same routing mix (hit rate) as the device-timed one
-    n_host = 8 if identity else min(n_sets, 128)
-    pick = [(j * n_sets) // n_host for j in range(n_host)]
-    h_h = [hs[j].cpu().pin_memory() for j in pick]
-    h_i = [ids[j].cpu().pin_memory() for j in pick]
-    h_w = [ws[j].cpu().pin_memory() for j in pick]
-    h_out = torch.empty_like(h_h[0]).pin_memory()
-
-    # the library's host-buffer entry point: inputs in host memory, result in host memory, synchronous; one call per
-    # step (it stages the three inputs, copies them to the device in one copy, runs the layer and waits; tiny batches
-    # replay a graph recorded per (layer, T), small results are written straight into pinned host memory, large
-    # page-locked tensors are used in place)
-    def e2e_step(i):
-        j = i % len(h_h)
-        cache.forward_host(i % L, h_h[j], h_i[j], h_w[j], out=h_out, stream=stream)
-
-    e2e_mode = "exmoe_moe_forward_host: host tensors in and out, one synchronous call per step"
-    for i in range(max(3, 2 * L)):                      # every layer's graph (tiny batches) is recorded before the timed calls
-        e2e_step(i)
-    if world > 1:
-        dist.barrier()
-    t0 = time.perf_counter()
-    for i in range(n_e2e):
-        e2e_step(i)
-    dt = time.perf_counter() - t0
-    dt = max_over_ranks(dt, world, dev)
-    h2d = h_h[0].numel() * 2 + h_i[0].numel() * 4 + h_w[0].numel() * 4
-    e2e = {"value": world * n_e2e * T / dt, "unit": UNIT, "h2d_bytes_per_step": int(h2d),
-           "d2h_bytes_per_step": int(h_out.numel() * 2), "steps": n_e2e, "mode": e2e_mode}
-
-    status = cache.status()
-    extra = {}
-    if not identity:
-        st = cache.stats(0)
-        extra = {"hit_rate": st["hits"] / max(st["lookups"], 1), "h2d_expert_bytes_per_token":
-                 st["h2d_bytes"] / max(st["forwards"] * T, 1), "waves_per_step": st["waves"] / max(st["forwards"], 1)}
-        # the H2D link is the roofline of this workload: copy-stream busy time and rate vs a plain pinned copy
-        n_c = min(K, 100)
-        cache.profile_enable(True)
-        b0 = cache.stats(0)["h2d_bytes"]
-        c0, c1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        with torch.cuda.stream(stream):
-            c0.record(stream)
-            for j in range(n_c):                              # steps spread evenly over the timed range (all alpha blocks)
-                i = W + j * max(K // n_c, 1)
-                step(i, outs[i & 1])
-            c1.record(stream)
-        stream.synchronize()
-        copy_ms, n_waves_copied = cache.profile_read(4)
-        wall_ms = c0.elapsed_time(c1)
-        moved = cache.stats(0)["h2d_bytes"] - b0
-        cache.profile_enable(False)
-        big = banks[0][:32]                                  # 104 MB of the pinned bank
-        dst = torch.empty_like(big, device=dev)
-        p0, p1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        dst.copy_(big, non_blocking=True)
-        torch.cuda.synchronize()
-        p0.record()
-        dst.copy_(big, non_blocking=True)
-        p1.record()
-        torch.cuda.synchronize()
-        extra.update({"h2d_gb_per_s_during_copies": moved / max(copy_ms, 1e-9) / 1e6,
-                      "copy_stream_busy_fraction": copy_ms / wall_ms,
-                      "pinned_copy_ceiling_gb_per_s": big.numel() / p0.elapsed_time(p1) / 1e6,
-                      "h2d_bytes_per_step": moved / n_c})
+    legs = {}
+    if args.workload == "decode" and not args.no_extra_legs and not (args.tokens or args.slots):
+        # the other two parts of the metric, short: prefill TFLOP/s (config 4) and the offloaded decode (config 3)
+        legs["prefill"] = leg_summary(run_leg("prefill", args, shape, banks, dev, rank, local_rank, world, peaks, 50, 3, seed0 + 7, full=False))
+        legs["offload"] = leg_summary(run_leg("offload", args, shape, banks, dev, rank, local_rank, world, peaks, 100, 5, seed0 + 9, full=False))
 
     if rank == 0:
         cpu = oracle_leg(shape, T, w_cpu, hs, ids, ws, args.cpu_budget)
-        line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
-                "ms_per_step": ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        bpe = main_leg["bytes_per_expert"]
+        Lm = main_leg["L"]
+        config = {"workload": main_leg["desc"], "tokens_per_step": T, "slots": main_leg["C"], "layers_rotated": Lm,
+                  "l2": "inputs larger than L2: steps rotate over %d layer banks (%.2f GB packed)" % (Lm, Lm * 64 * bpe / 1e9)
+                  if Lm > 1 else "single layer bank (%.0f MB packed) vs 126 MB L2" % (64 * bpe / 1e6),
+                  "timing": ("CUDA graph replay of all steps" if main_leg["graphable"] else "host-driven loop (one plan read-back per step)") +
+                            "; the K-step region is repeated back to back (see repetitions), the median repetition is reported",
+                  "repetitions": main_leg["repetitions"],
+                  "active_experts_per_step": main_leg["active_experts_per_step"],
+                  "packed_gb_per_s_whole_step": main_leg["packed_gb_per_s_whole_step"],
+                  "tflops_whole_step": main_leg["tflops_whole_step"],
+                  "kernel_us": main_leg["kernel_us"], "parallelism": "replicas only (no collective)", "status": main_leg["status"],
+                  "pack": dict(PACK_STATS), **main_leg["extra"], **legs}
+        line = {"metric": METRIC, "value": main_leg["value"], "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
+                "ms_per_step": main_leg["ms_per_step"], "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
                 "dtype": "int4 weights x bf16 activations, fp32 accumulate", "data": "synthetic",
-                "config": {"workload": desc, "tokens_per_step": T, "slots": C, "layers_rotated": L,
-                           "l2": "inputs larger than L2: steps rotate over %d layer banks (%.2f GB packed)" % (L, L * 64 * bpe / 1e9)
-                           if L > 1 else "single layer bank (%.0f MB packed) vs 126 MB L2" % (64 * bpe / 1e6),
-                           "timing": "CUDA graph replay of all steps" if graphable else "host-driven loop (one plan read-back per step)",
-                           "active_experts_per_step": active_all, "packed_gb_per_s_whole_step": step_gbs,
-                           "tflops_whole_step": step_tflops,
-                           "kernel_us": kinds, "parallelism": "replicas only (no collective)", "status": status, **extra},
-                "roofline": roof, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": int(launches), "clocks": clocks}
+                "config": config, "roofline": main_leg["roofline"], "cpu_baseline": cpu, "e2e": main_leg["e2e"],
+                "gpu_launches": main_leg["launches"], "clocks": main_leg["clocks"]}
         print(json.dumps(line), flush=True)
-    cache.close()
     if world > 1:
         dist.barrier()
         dist.destroy_process_group()
