@@ -173,8 +173,20 @@ def whole_job_tokens_per_s(world, steps, tokens_per_step, ms_max):
 
 
 def make_inputs(shape, T, n_sets, alpha, seed0, device):
-    """n_sets independent (hidden, ids, weights) batches, generated on the device, routed by Eq. 1.
+    """n_sets independent (hidden, ids, weights) batches, generated on the device and routed by Eq. 1: by the library's
+    router kernel (exmoe_route) on a GPU, by the oracle's router on the CPU (the reference arm runs without a GPU).
     alpha = "cycle": the sets fall into four consecutive blocks with alpha = 2, 1, 0.5, 0 (same rank permutation)."""
+    if str(device) == "cpu":
+        from oracle import router as orouter
+
+        def route(h, wr, k, bias):
+            ids, p, _ = orouter.route(h.float().numpy(), wr.float().numpy(), k, None if bias is None else bias.numpy())
+            return torch.from_numpy(ids), torch.from_numpy(p.astype(np.float32))
+    else:
+        from paper_2608_15383_b200 import binding
+
+        def route(h, wr, k, bias):
+            return binding.exmoe_route(shape, h, wr, None if bias is None else bias.float().contiguous())
     wr = synth.router_weights(shape, seed0 + 1, device=device)
     cycle = (2.0, 1.0, 0.5, 0.0)
     base = synth.zipf_bias(shape.num_experts, 1.0, seed0 + 2).to(device)
@@ -183,7 +195,7 @@ def make_inputs(shape, T, n_sets, alpha, seed0, device):
         al = cycle[min(3, i * 4 // max(n_sets, 1))] if alpha == "cycle" else float(alpha)
         bias = base * al if al else None
         h = synth.hidden_states(shape, T, seed0 + 10 + i, device=device)
-        a, b = synth.route(h, wr, shape.top_k, bias)
+        a, b = route(h, wr, shape.top_k, bias)
         hs.append(h)
         ids.append(a)
         ws.append(b)

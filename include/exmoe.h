@@ -21,7 +21,10 @@
  *     must keep them alive while the cache exists.  The library owns only its host bookkeeping,
  *     one copy stream, its events, pinned staging buffers and the graphs of exmoe_moe_forward_host.
  *   - BF16 tensors are row-major, dense.  ids are int32, mixture weights are float32.
- *   - All calls on one cache must come from one host thread at a time.
+ *   - All calls on one cache must come from one host thread at a time, and all forwards (and prefetches of the same
+ *     layer) on one cache must be issued to ONE stream or be ordered by the caller with events: the workspace
+ *     (plan, activations, pair buffer) is shared by the layers, and the host-copy miss path orders slot reuse against
+ *     the stream that ran the earlier wave.
  */
 #ifndef EXMOE_H
 #define EXMOE_H
@@ -36,8 +39,9 @@ extern "C" {
 enum {
     EXMOE_OK = 0,
     EXMOE_ERR_ARG = -1,           /* null pointer, negative size, T > max_tokens, layer out of range */
-    EXMOE_ERR_SHAPE = -2,         /* d_model or d_ff not a multiple of 128, group_size != 128,
-                                     top_k > num_slots, num_slots > num_experts, ... (Sec. 3.3, Sec. 7) */
+    EXMOE_ERR_SHAPE = -2,         /* d_model or d_ff not a multiple of 128 (Sec. 7 leaves such shapes to padding), group_size
+                                     != 128, top_k > num_slots, num_slots > num_experts (Sec. 3.3), a size beyond a kernel's
+                                     shared memory */
     EXMOE_ERR_NOT_PINNED = -3,    /* a host bank pointer is not page-locked host memory (Sec. 3.3) */
     EXMOE_ERR_CUDA = -4,          /* a CUDA runtime call failed */
     EXMOE_ERR_NONFINITE = -5,     /* exmoe_pack: a weight is NaN/Inf or a scale overflows FP16 */
@@ -55,8 +59,8 @@ typedef struct {
     int group_size;   /* 128 (Eq. 3) */
 } exmoe_shape;
 
-/* Runtime counters of one layer's cache (Sec. 4.2 "cache events, transferred bytes").
- * All zero while the layer is fully resident (C = E): lookup accounting is bypassed (Sec. 5.1). */
+/* Runtime counters of one layer's cache: the quantities the cache reports in Sec. 4.2 and Table 1 (hit rate, host-to-
+ * device traffic).  All zero while the layer is fully resident (C = E): no lookups happen then (Sec. 3.3, Fig. 2 caption). */
 typedef struct {
     uint64_t lookups;    /* active experts looked up, summed over calls */
     uint64_t hits;
@@ -68,6 +72,7 @@ typedef struct {
 
 typedef struct exmoe_cache exmoe_cache; /* opaque */
 
+/* Name of a status code (no paper counterpart: part of this ABI's error convention).  Never NULL. */
 const char* exmoe_strerror(int code);
 
 /* Eq. 4: bytes of one packed expert = 3*I*H * (4/8 + 16/(128*8)); 3,244,032 for OLMoE.
@@ -161,7 +166,7 @@ int exmoe_cache_set_miss_path(exmoe_cache* cache, int mode);
  * EXMOE_ERR_BAD_EXPERT_ID. */
 int exmoe_cache_prefetch(exmoe_cache* cache, int layer, const int32_t* expert_ids, int n_ids, void* stream);
 
-/* Router of one sparse block (Eq. 1; Sec. 3.4 "router weights are ... not renormalized"): logits z_t = W_r h_t in
+/* Router of one sparse block (Eq. 1; the selected probabilities are used as they are, Sec. 3.4): logits z_t = W_r h_t in
  * binary32 (BF16 products, fixed summation order), plus `bias` if given, softmax over all E experts, the k
  * largest, equal values ordered by ascending expert id.  Writes exmoe_moe_forward's inputs on the device.
  *   hidden_bf16  : dev, BF16 [T, H], 16-byte aligned     router_bf16 : dev, BF16 [E, H], 16-byte aligned
@@ -191,17 +196,27 @@ int exmoe_route(const exmoe_shape* shape, const void* hidden_bf16, const void* r
  *                  its streaming kernels, which split K differently, and the two agree within the output
  *                  tolerance (a few BF16 roundings), not bit for bit.
  *
- * Limits (fixed by the size of the scratch): T * top_k <= 32 and d_ff <= 4096; anything larger is refused
- * with EXMOE_ERR_SHAPE before any work is queued.  T = 0 is a no-op.
+ * Limits: T * top_k <= 32 and d_ff <= 4096 (the size of the scratch), and the shared memory of the two kernels:
+ * top_k * (2 * d_ff + 132 + d_ff / 32) <= 204,800 bytes and 2 * d_model + d_model / 32 + 7,232 <= 102,400 bytes
+ * (d_ff = 4096 allows top_k <= 24; OLMoE's 1024 allows 32); anything larger is refused with EXMOE_ERR_SHAPE before
+ * any work is queued.  T = 0 is a no-op.
  * First call on a device: looks up the device address of the scratch array (cudaGetSymbolAddress, with that
  * device current) and keeps it; make this first call outside any stream capture.
  * The scratch is shared by all calls and keeps the previous call's contents; the function clears the one word
  * that must start at zero.  Calls on one device that may overlap on the GPU (different streams without
  * ordering between them) race on it: order them, or use exmoe_moe_forward with separate workspaces.
- * An id outside [0, E) contributes nothing; it is not reported by this entry point. */
+ * An id outside [0, E) contributes nothing.  What the kernels find on the device - such an id
+ * (EXMOE_ERR_BAD_EXPERT_ID) or a bounded wait that expired (EXMOE_ERR_TIMEOUT, output rows then unwritten) - cannot be
+ * returned by this asynchronous call: it is kept in a sticky word of the scratch and read with
+ * exmoe_moe_forward_static_status(). */
 int exmoe_moe_forward_static(const exmoe_shape* shape, const void* experts_dev, const void* hidden_bf16,
                              const int32_t* topk_ids, const float* topk_weights, int T, void* out_bf16,
                              void* stream);
+
+/* Sticky device-side status of exmoe_moe_forward_static on the current device (the paper has no counterpart):
+ * synchronises the device, returns EXMOE_OK or the last EXMOE_ERR_BAD_EXPERT_ID / EXMOE_ERR_TIMEOUT recorded since the
+ * previous call of this function, and clears it.  Allocates nothing. */
+int exmoe_moe_forward_static_status(void);
 
 /* Test hooks (synchronise).  Sec. 3.3 state of one layer: expert_slot [E] (-1 = not resident),
  * slot_expert [C] (-1 = empty), slot_stamp [C], all host pointers, any may be NULL. */
@@ -229,6 +244,10 @@ enum {
 };
 int exmoe_debug_last_path(exmoe_cache* cache);
 
+/* Bytes of the staged host-to-device input copy of the most recent exmoe_moe_forward_host (test hook; no paper
+ * counterpart): T * d_model * 2 + 2 * T * top_k * 4 rounded up to 16-byte pieces, whatever max_tokens is. */
+int exmoe_debug_last_host_copy_bytes(exmoe_cache* cache, size_t* h2d_bytes);
+
 /* Copy one slot's bytes back to the host (test hook for the miss-copy path; synchronises). */
 int exmoe_debug_read_slot(exmoe_cache* cache, int layer, int slot, void* host_out);
 
@@ -240,9 +259,16 @@ int exmoe_debug_read_slot(exmoe_cache* cache, int layer, int slot, void* host_ou
  * raised; exmoe_status() then reports EXMOE_ERR_TIMEOUT.  Synchronous. */
 int exmoe_debug_wait_timeout(exmoe_cache* cache, long long budget_cycles, int* gave_up);
 
-int exmoe_cache_stats(exmoe_cache* cache, int layer, exmoe_stats* out);   /* synchronises */
-int exmoe_cache_reset(exmoe_cache* cache, int layer);                     /* empty cache, zero counters */
-int exmoe_status(exmoe_cache* cache);   /* synchronises; returns and clears the sticky device status */
+/* Counters of one layer's cache (Sec. 4.2: hit rate and transferred bytes are reported per configuration).  Synchronises. */
+int exmoe_cache_stats(exmoe_cache* cache, int layer, exmoe_stats* out);
+/* Back to the state after exmoe_cache_create: empty cache (C < E), zero stamps and counters (Sec. 3.3 start state;
+ * the paper's runs start each configuration from a fresh cache, Sec. 4.2).  Synchronises. */
+int exmoe_cache_reset(exmoe_cache* cache, int layer);
+/* Sticky device-side status of the cache's kernels (no paper counterpart): synchronises, returns EXMOE_OK or the last
+ * EXMOE_ERR_BAD_EXPERT_ID / EXMOE_ERR_TIMEOUT raised on the device since the previous call, and clears it. */
+int exmoe_status(exmoe_cache* cache);
+/* Releases the library's own resources (events, copy stream, pinned staging, recorded graphs); the caller's buffers
+ * stay the caller's (Sec. 3.3: slots and bank outlive individual requests).  Synchronises the device first. */
 int exmoe_cache_destroy(exmoe_cache* cache);
 
 /* Measurement hooks (the paper has no counterpart).  While enabled, every exmoe_moe_forward brackets
@@ -258,7 +284,7 @@ int exmoe_cache_destroy(exmoe_cache* cache);
 int exmoe_profile_enable(exmoe_cache* cache, int on);
 int exmoe_profile_read(exmoe_cache* cache, int kind, double* total_ms, uint64_t* launches);
 
-/* Kernels launched by this library since it was loaded (all streams, all caches). */
+/* Kernels launched by this library since it was loaded (all streams, all caches); measurement hook, no paper counterpart. */
 uint64_t exmoe_launch_count(void);
 
 #ifdef __cplusplus

@@ -48,6 +48,8 @@ _SIGNATURES = {
                                    c_void_p, c_int, c_int]),
     "exmoe_moe_forward": (c_int, [c_void_p, c_int, c_void_p, c_void_p, c_void_p, c_int, c_void_p, c_void_p]),
     "exmoe_moe_forward_host": (c_int, [c_void_p, c_int, c_void_p, c_void_p, c_void_p, c_int, c_void_p, c_void_p]),
+    "exmoe_moe_forward_static_status": (c_int, []),
+    "exmoe_debug_last_host_copy_bytes": (c_int, [c_void_p, POINTER(c_size_t)]),
     "exmoe_moe_forward_static": (c_int, [POINTER(exmoe_shape), c_void_p, c_void_p, c_void_p, c_void_p, c_int, c_void_p, c_void_p]),
     "exmoe_route": (c_int, [POINTER(exmoe_shape), c_void_p, c_void_p, c_void_p, c_int, c_void_p, c_void_p, c_void_p]),
     "exmoe_cache_get_state": (c_int, [c_void_p, c_int, c_void_p, c_void_p, c_void_p, c_void_p]),
@@ -150,6 +152,11 @@ def exmoe_moe_forward_static(shape, experts_dev, hidden, topk_ids, topk_weights,
     return out
 
 
+def exmoe_moe_forward_static_status():
+    """Sticky device-side status of exmoe_moe_forward_static on the current device (synchronises, clears)."""
+    return int(lib().exmoe_moe_forward_static_status())
+
+
 def exmoe_route(shape, hidden, w_router, bias=None, topk_ids=None, topk_weights=None, stream=None):
     """Eq. 1 on the device: logits, softmax over all experts, top-k.  Returns (ids int32 [T, k], weights fp32 [T, k])."""
     T = int(hidden.shape[0])
@@ -214,15 +221,30 @@ PATH_PAIR, PATH_SMALL, PATH_STREAM, PATH_TENSOR_SMALL_N, PATH_TENSOR = 2, 3, 4, 
 class Cache:
     """exmoe_cache handle plus the torch buffers it borrows (slot memory, workspace, host banks)."""
 
-    def __init__(self, shape, banks, num_slots, max_tokens, wave_cap=0, device="cuda"):
+    GUARD_BYTE = 0xA5
+
+    def __init__(self, shape, banks, num_slots, max_tokens, wave_cap=0, device="cuda", guard_bytes=0):
+        """guard_bytes > 0 (a multiple of 256): slot memory and workspace are carved out of larger tensors whose
+        margins on both sides are filled with GUARD_BYTE; guards_intact() tells whether any kernel wrote there."""
         self.shape, self.C, self.L = shape, int(num_slots), len(banks)
         self.max_tokens = int(max_tokens)
         self.wave_cap = int(wave_cap) if wave_cap else int(num_slots)
         self.bytes_per_expert = exmoe_packed_bytes(shape)
         slot_bytes, ws_bytes = exmoe_cache_workspace_bytes(shape, self.L, self.C, self.max_tokens)
         self.banks = list(banks)
-        self.slot_mem = torch.empty(slot_bytes, dtype=torch.uint8, device=device)
-        self.workspace = torch.empty(ws_bytes, dtype=torch.uint8, device=device)
+        g = int(guard_bytes)
+        if g % 256:
+            raise ValueError("guard_bytes must be a multiple of 256")
+        self._guarded = []
+        bufs = []
+        for n in (slot_bytes, ws_bytes):
+            n_al = -(-n // 256) * 256
+            whole = torch.full((n_al + 2 * g,), self.GUARD_BYTE, dtype=torch.uint8, device=device) if g else \
+                torch.empty(n_al, dtype=torch.uint8, device=device)
+            if g:
+                self._guarded.append((whole, g, n))
+            bufs.append(whole[g:g + n])
+        self.slot_mem, self.workspace = bufs
         ptrs = (c_void_p * self.L)(*[c_void_p(b.data_ptr()) for b in self.banks])
         h = c_void_p()
         rc = lib().exmoe_cache_create(byref(h), byref(_shape(shape)), self.L, self.C, ptrs,
@@ -297,6 +319,19 @@ class Cache:
         if rc < 0:
             raise ExmoeError(rc, "exmoe_debug_last_path")
         return rc
+
+    def last_host_copy_bytes(self):
+        n = c_size_t()
+        _check(lib().exmoe_debug_last_host_copy_bytes(self.handle, byref(n)), "exmoe_debug_last_host_copy_bytes")
+        return n.value
+
+    def guards_intact(self):
+        """True if every guard byte around slot memory and workspace still holds GUARD_BYTE (synchronises)."""
+        torch.cuda.synchronize()
+        for whole, g, n in self._guarded:
+            if not bool((whole[:g] == self.GUARD_BYTE).all()) or not bool((whole[g + n:] == self.GUARD_BYTE).all()):
+                return False
+        return True
 
     def read_slot(self, layer, slot):
         out = torch.empty(self.bytes_per_expert, dtype=torch.uint8)

@@ -69,6 +69,7 @@ struct exmoe_cache {
     int last_path;                            // EXMOE_PATH_* of the most recent forward
     int32_t* saved_ids;                       // ids of the last pairwise call (plan materialised on request)
     bool stream_ok;                           // the shape fits the streaming middle-regime kernels
+    bool pair_ok, small_ok;                   // ... the per-pair kernels / the in-CTA-grouping kernels (shared memory)
     void* tc_scratch;                         // tile list of the tensor-core path
     __nv_bfloat16* xg;                        // [max_pairs, H] hidden rows in plan order (tensor-core path only)
     PrefillMaps tc_maps;                      // TMA descriptors of xg and act
@@ -90,6 +91,7 @@ struct exmoe_cache {
     uint8_t* d_stage;                         // device: hidden | ids | weights | out, each 256-byte aligned
     uint8_t* h_stage;                         // pinned host mirror of d_stage
     size_t stage_in_bytes, stage_out_off, stage_bytes;
+    size_t last_host_h2d_bytes;               // bytes of the staged input copy of the last exmoe_moe_forward_host
     struct HostGraph {
         cudaGraphExec_t exec;
         bool last_small, last_pair;
@@ -171,7 +173,7 @@ static void carve_workspace(exmoe_cache* c, uint8_t* ws, size_t* total) {
     c->arrive = k.take<int>(c->arrive_words);
     c->saved_ids = k.take<int32_t>(kPairMaxPairs);
     c->tc_scratch = k.take<uint8_t>(prefill_scratch_bytes(c->max_pairs, E));
-    c->xg = c->max_pairs > kSmallMaxPairs ? k.take<__nv_bfloat16>((size_t)c->max_pairs * s.d_model) : nullptr;
+    c->xg = (c->max_pairs > kSmallMaxPairs || !c->small_ok) ? k.take<__nv_bfloat16>((size_t)c->max_pairs * s.d_model) : nullptr;
     {   // staging of the host-buffer entry point: hidden | ids | weights (one H2D copy), then out (one D2H copy)
         const size_t nb_h = align_up((size_t)c->max_tokens * s.d_model * 2, 256);
         const size_t nb_i = align_up((size_t)c->max_pairs * 4, 256);
@@ -201,6 +203,8 @@ static int fill_dims(exmoe_cache* c, const exmoe_shape* shape, int num_layers, i
     c->n_keys = c->max_waves * c->C;
     if (c->n_keys > kMaxKeys) return EXMOE_ERR_SHAPE;
     c->bpe = packed_bytes(*shape);
+    c->pair_ok = pair_path_fits(shape->d_model, shape->d_ff, shape->top_k);
+    c->small_ok = small_path_fits(shape->d_model, shape->d_ff, c->C, kSmallMaxPairs);
     return EXMOE_OK;
 }
 
@@ -273,15 +277,14 @@ int exmoe_pack(const exmoe_shape* shape, const void* w_gate, const void* w_up, c
          reinterpret_cast<uintptr_t>(w_up) | reinterpret_cast<uintptr_t>(w_down)) & 15)
         return EXMOE_ERR_ARG;
     cudaStream_t st = (cudaStream_t)stream;
-    int* d_flag = nullptr;
-    if (cudaMalloc(&d_flag, sizeof(int)) != cudaSuccess) return EXMOE_ERR_CUDA;
+    int* d_flag = pack_flag_word();
+    if (!d_flag) return EXMOE_ERR_CUDA;
     int flag = 0;
     rc = EXMOE_OK;
     if (cudaMemsetAsync(d_flag, 0, sizeof(int), st) != cudaSuccess) rc = EXMOE_ERR_CUDA;
     if (!rc) rc = launch_pack(*shape, w_gate, w_up, w_down, packed_out, d_flag, st);
     if (!rc && cudaMemcpyAsync(&flag, d_flag, sizeof(int), cudaMemcpyDeviceToHost, st) != cudaSuccess) rc = EXMOE_ERR_CUDA;
     if (cudaStreamSynchronize(st) != cudaSuccess) rc = EXMOE_ERR_CUDA;
-    cudaFree(d_flag);
     if (!rc && flag) rc = EXMOE_ERR_NONFINITE;
     return rc;
 }
@@ -370,7 +373,7 @@ int exmoe_moe_forward(exmoe_cache* c, int layer, const void* hidden, const int32
     c->last_layer = layer;
     c->last_T = T;
 
-    const bool small = (P <= kSmallMaxPairs && C <= kSmallMaxSlots);   // decode: grouping fused into the GEMM kernels
+    const bool small = (P <= kSmallMaxPairs && C <= kSmallMaxSlots && c->small_ok);   // decode: grouping fused into the GEMM kernels
     c->last_small = small;
     if (!identity) {
         ProfScope ps(c, PROF_PLAN, st);
@@ -421,7 +424,7 @@ int exmoe_moe_forward(exmoe_cache* c, int layer, const void* hidden, const int32
     a.I = s.d_ff;
 
     bool tiles_fused = false;
-    const bool pairwise = small && P <= kPairMaxPairs && n_waves == 1;
+    const bool pairwise = small && P <= kPairMaxPairs && n_waves == 1 && c->pair_ok;
     c->last_pair = pairwise;
     const bool use_stream = !small && c->stream_ok && P <= kStreamMaxPairs;
     const bool small_n = P <= kPrefillSmallNMaxPairs;      // tensor-core path: which kernel shape
@@ -449,8 +452,10 @@ int exmoe_moe_forward(exmoe_cache* c, int layer, const void* hidden, const int32
             if (wave_has_miss) prof_mark(c, PROF_COPY, c->copy_stream);       // begin of the wave's copies
             for (; mi < n_miss && h_miss[3 * mi + 2] == w; ++mi) {
                 const int e = h_miss[3 * mi], v = h_miss[3 * mi + 1];
+                // the wave that last read the slot; once the ring has wrapped its entry belongs to a later wave, so the
+                // most recent compute event stands in (all forwards of a cache share one stream order: see exmoe.h)
                 const uint64_t last = c->slot_last_seq[layer][v];
-                if (last) cudaStreamWaitEvent(c->copy_stream, c->ev_compute[last % kEventRing], 0);
+                if (last) cudaStreamWaitEvent(c->copy_stream, c->ev_compute[(c->seq - last >= kEventRing ? c->seq : last) % kEventRing], 0);
                 if (cudaMemcpyAsync(const_cast<uint8_t*>(a.slots) + (size_t)v * c->bpe, c->bank[layer] + (size_t)e * c->bpe,
                                     c->bpe, cudaMemcpyHostToDevice, c->copy_stream) != cudaSuccess)
                     return EXMOE_ERR_CUDA;
@@ -555,8 +560,10 @@ int exmoe_moe_forward_host(exmoe_cache* c, int layer, const void* hidden_host, c
     cudaStream_t st = (cudaStream_t)stream;
     const exmoe_shape& s = c->shape;
     const size_t nb_h = (size_t)T * s.d_model * 2, nb_i = (size_t)T * s.top_k * 4;
-    const size_t off_i = align_up((size_t)c->max_tokens * s.d_model * 2, 256);
-    const size_t off_w = off_i + align_up((size_t)c->max_pairs * 4, 256);
+    // hidden | ids | weights back to back (16-byte aligned pieces), so that the one H2D copy moves what this call needs
+    // and not what max_tokens would; the recorded graphs are keyed by T, so T-dependent offsets are safe
+    const size_t off_i = align_up(nb_h, 16);
+    const size_t off_w = off_i + align_up(nb_i, 16);
     void* d_h = c->d_stage;
     int32_t* d_i = reinterpret_cast<int32_t*>(c->d_stage + off_i);
     float* d_w = reinterpret_cast<float*>(c->d_stage + off_w);
@@ -575,6 +582,7 @@ int exmoe_moe_forward_host(exmoe_cache* c, int layer, const void* hidden_host, c
         }
         cudaGetLastError();
         if (pinned) {
+            c->last_host_h2d_bytes = nb_h + 2 * nb_i;
             bool ok = cudaMemcpyAsync(d_h, hidden_host, nb_h, cudaMemcpyHostToDevice, st) == cudaSuccess;
             ok = ok && cudaMemcpyAsync(d_i, ids_host, nb_i, cudaMemcpyHostToDevice, st) == cudaSuccess;
             ok = ok && cudaMemcpyAsync(d_w, weights_host, nb_i, cudaMemcpyHostToDevice, st) == cudaSuccess;
@@ -588,6 +596,7 @@ int exmoe_moe_forward_host(exmoe_cache* c, int layer, const void* hidden_host, c
     std::memcpy(c->h_stage + off_i, ids_host, nb_i);
     std::memcpy(c->h_stage + off_w, weights_host, nb_i);
     const size_t in_bytes = off_w + nb_i;                                 // one copy covers the three inputs
+    c->last_host_h2d_bytes = in_bytes;
     auto enqueue = [&]() -> int {
         if (cudaMemcpyAsync(c->d_stage, c->h_stage, in_bytes, cudaMemcpyHostToDevice, st) != cudaSuccess) return EXMOE_ERR_CUDA;
         const int rc = exmoe_moe_forward(c, layer, d_h, d_i, d_w, T, d_o, st);
@@ -715,6 +724,12 @@ int exmoe_debug_last_path(exmoe_cache* c) {
     if (!c) return EXMOE_ERR_ARG;
     if (c->last_layer < 0) return EXMOE_ERR_STATE;
     return c->last_path;
+}
+
+int exmoe_debug_last_host_copy_bytes(exmoe_cache* c, size_t* h2d_bytes) {
+    if (!c || !h2d_bytes) return EXMOE_ERR_ARG;
+    *h2d_bytes = c->last_host_h2d_bytes;
+    return EXMOE_OK;
 }
 
 int exmoe_debug_read_slot(exmoe_cache* c, int layer, int slot, void* host_out) {

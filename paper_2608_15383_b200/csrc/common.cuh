@@ -103,6 +103,7 @@ inline bool allow_smem(F kern, int bytes, SmemOnce& once) {
 }
 
 // ---- kernel launchers (defined in the .cu files) ------------------------------------------------
+int* pack_flag_word();      // a device word for one exmoe_pack call's non-finite flag (no allocation)
 int launch_pack(const exmoe_shape& s, const void* wg, const void* wu, const void* wd, void* out,
                 int* d_flag, cudaStream_t st);
 void launch_resolve(const exmoe_shape& s, int C, int Cw, size_t bytes_per_expert, const int32_t* ids, int n_pairs,
@@ -121,6 +122,8 @@ bool stream_supported(int H, int I);
 bool launch_stream_wave(const GemmArgs& a, const __nv_bfloat16* hidden, __nv_bfloat16* act, const float* topk_w, float* y,
                         int* status, int max_groups, bool gateup, bool down, cudaStream_t st);
 void launch_small_wave(const GemmArgs& a, const SmallWave& w, cudaStream_t st, bool gateup, bool down);
+bool pair_path_fits(int H, int I, int top_k);                           // shared memory of the per-pair kernels within limits
+bool small_path_fits(int H, int I, int num_slots, int n_pairs);         // ... of the in-CTA-grouping kernels
 size_t prefill_scratch_bytes(int max_pairs, int num_experts);
 // CUtensorMap objects of the grouped hidden rows and of the activations: 256-row boxes for the large-N kernel shape,
 // 64-row boxes for the small-N shape

@@ -1012,6 +1012,28 @@ bool launch_token_down_bulk(const GemmArgs& a, const SmallArgs& sa, const __nv_b
     return true;
 }
 
+// Shared memory the per-pair kernels ask for (launch_pair_gateup, launch_token_down): false when either exceeds its
+// opt-in limit, so that callers can refuse or take another path BEFORE anything is queued.
+bool pair_path_fits(int H, int I, int top_k) {
+    const DecodeCfg cfg = pick_cfg(H, I);
+    const int PP = 8 / cfg.KS;
+    const size_t gu = (size_t)H * 2 + 64 + (size_t)(cfg.KS - 1) * PP * 2 * 128 * 4 + (size_t)(H / kGroup) * 4;
+    const size_t dn = (size_t)top_k * (I * 2 + 64) + (size_t)top_k * 17 * 4 + (size_t)(I / kGroup) * top_k * 4;
+    return gu <= 100 * 1024 && dn <= 200 * 1024 && (cfg.bpw == 1 || cfg.bpw == 2 || cfg.bpw == 4);
+}
+// ... and the in-CTA-grouping kernels with one 8-row chunk per pass (their smallest footprint)
+bool small_path_fits(int H, int I, int num_slots, int n_pairs) {
+    for (int g = 0; g < 2; ++g) {
+        const int K = g ? I : H, NR = g ? H : I;
+        const DecodeCfg cfg = pick_cfg(K, NR);
+        const int PP = 8 / cfg.KS, NM = g ? 1 : 2;
+        const size_t smem = (size_t)8 * (K * 2 + 64) + (size_t)(cfg.KS - 1) * PP * NM * 128 * 4 + (size_t)(K / kGroup) * 8 * 4 +
+                            (size_t)(3 * num_slots + 1 + 2 * n_pairs) * 4;
+        if (smem > 200 * 1024) return false;
+    }
+    return true;
+}
+
 // One wave of the SMALL path: gate/up kernel, then the down kernel with the fused combine.
 void launch_small_wave(const GemmArgs& a, const SmallWave& w, cudaStream_t st, bool gateup, bool down) {
     SmallArgs sa{};
@@ -1073,7 +1095,7 @@ void launch_small_wave(const GemmArgs& a, const SmallWave& w, cudaStream_t st, b
 // ------------------------------------------------------------------------------------------------
 constexpr int kStaticMaxPairs = kPairMaxPairs;           // T * top_k <= 32
 constexpr int kStaticMaxDff = 4096;                      // d_ff <= 4096
-constexpr size_t kStaticCtrlBytes = 256;                 // [0,4) status word, [64,192) kept ids
+constexpr size_t kStaticCtrlBytes = 256;                 // [32,36) sticky status word, [64,192) kept ids
 constexpr size_t kStaticScratchBytes = kStaticCtrlBytes + (size_t)kStaticMaxPairs * kStaticMaxDff * 2;   // 262,400 B
 
 static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
@@ -1081,6 +1103,34 @@ static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBy
 }  // namespace exmoe
 
 #include <mutex>
+
+// Device address of the scratch on the current device (set-up once per device, see exmoe_moe_forward_static).
+static unsigned char* static_scratch_ptr() {
+    static std::mutex mu;
+    static unsigned char* dev_ptr[64] = {};
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+    std::lock_guard<std::mutex> lock(mu);
+    if (!dev_ptr[dev]) {
+        void* p = nullptr;
+        if (cudaGetSymbolAddress(&p, exmoe::g_static_scratch) != cudaSuccess || !p) {
+            cudaGetLastError();
+            return nullptr;
+        }
+        dev_ptr[dev] = static_cast<unsigned char*>(p);
+    }
+    return dev_ptr[dev];
+}
+
+extern "C" int exmoe_moe_forward_static_status(void) {
+    unsigned char* scratch = static_scratch_ptr();
+    if (!scratch) return EXMOE_ERR_CUDA;
+    if (cudaDeviceSynchronize() != cudaSuccess) return EXMOE_ERR_CUDA;
+    int v = 0;
+    if (cudaMemcpy(&v, scratch + 32, 4, cudaMemcpyDeviceToHost) != cudaSuccess) return EXMOE_ERR_CUDA;
+    if (v && cudaMemset(scratch + 32, 0, 4) != cudaSuccess) return EXMOE_ERR_CUDA;
+    return v;
+}
 
 extern "C" int exmoe_moe_forward_static(const exmoe_shape* shape, const void* experts_dev, const void* hidden_bf16,
                                         const int32_t* topk_ids, const float* topk_weights, int T, void* out_bf16,
@@ -1092,6 +1142,8 @@ extern "C" int exmoe_moe_forward_static(const exmoe_shape* shape, const void* ex
         return EXMOE_ERR_SHAPE;
     // the fixed scratch bounds the problem: reject anything larger instead of overrunning it
     if ((long long)T * shape->top_k > kStaticMaxPairs || shape->d_ff > kStaticMaxDff) return EXMOE_ERR_SHAPE;
+    // ... and so does the shared memory of the two kernels (e.g. top_k = 32 with d_ff = 4096 would ask for 264 KB)
+    if (!pair_path_fits(shape->d_model, shape->d_ff, shape->top_k)) return EXMOE_ERR_SHAPE;
     if (T == 0) return EXMOE_OK;
     if (!experts_dev || !hidden_bf16 || !topk_ids || !topk_weights || !out_bf16) return EXMOE_ERR_ARG;
     if ((reinterpret_cast<uintptr_t>(experts_dev) | reinterpret_cast<uintptr_t>(hidden_bf16) |
@@ -1100,28 +1152,14 @@ extern "C" int exmoe_moe_forward_static(const exmoe_shape* shape, const void* ex
 
     // Set-up, once per device, with that device current: in host code `g_static_scratch` is only a
     // stand-in for the symbol, not a device address; the address a kernel may use comes from
-    // cudaGetSymbolAddress.
-    static std::mutex mu;
-    static unsigned char* dev_ptr[64] = {};
-    int dev = -1;
-    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return EXMOE_ERR_CUDA;
-    unsigned char* scratch = nullptr;
-    {
-        std::lock_guard<std::mutex> lock(mu);
-        if (!dev_ptr[dev]) {
-            void* p = nullptr;
-            if (cudaGetSymbolAddress(&p, g_static_scratch) != cudaSuccess || !p) {
-                cudaGetLastError();
-                return EXMOE_ERR_CUDA;
-            }
-            dev_ptr[dev] = static_cast<unsigned char*>(p);
-        }
-        scratch = dev_ptr[dev];
-    }
+    // cudaGetSymbolAddress (static_scratch_ptr).
+    unsigned char* scratch = static_scratch_ptr();
+    if (!scratch) return EXMOE_ERR_CUDA;
 
     cudaStream_t st = (cudaStream_t)stream;
-    // the array keeps the previous call's contents: the status word must start at zero
-    if (cudaMemsetAsync(scratch, 0, kStaticCtrlBytes, st) != cudaSuccess) return EXMOE_ERR_CUDA;
+    // the array keeps the previous call's contents: the kept ids must start clean; the status word at [32, 36) is
+    // sticky on purpose (exmoe_moe_forward_static_status reads and clears it)
+    if (cudaMemsetAsync(scratch + 64, 0, kStaticCtrlBytes - 64, st) != cudaSuccess) return EXMOE_ERR_CUDA;
 
     GemmArgs a{};
     a.slots = static_cast<const uint8_t*>(experts_dev);
@@ -1135,7 +1173,7 @@ extern "C" int exmoe_moe_forward_static(const exmoe_shape* shape, const void* ex
     w.n_pairs = T * shape->top_k;
     w.E = shape->num_experts;
     w.wave = 0;
-    w.status = reinterpret_cast<int*>(scratch);
+    w.status = reinterpret_cast<int*>(scratch + 32);
     w.saved_ids = reinterpret_cast<int32_t*>(scratch + 64);
     w.hidden = static_cast<const __nv_bfloat16*>(hidden_bf16);
     w.act = reinterpret_cast<__nv_bfloat16*>(scratch + kStaticCtrlBytes);

@@ -6,6 +6,8 @@
 // word of codes.  HBM-bound: 2 bytes read and 0.516 bytes written per weight.
 #include "common.cuh"
 
+#include <mutex>
+
 namespace exmoe {
 
 __global__ void __launch_bounds__(256)
@@ -69,6 +71,29 @@ pack_kernel(const __nv_bfloat16* __restrict__ wg, const __nv_bfloat16* __restric
     const int h = oct >> 3, set = (oct >> 2) & 1, c = oct & 3, q = row & 7, rr = row >> 3;
     *reinterpret_cast<uint32_t*>(blk + h * 512 + (4 * q + c) * 16 + (2 * set + rr) * 4) = word;
     if (oct == 0) *reinterpret_cast<__half*>(blk + kCodeBytes + (2 * q + rr) * 2) = zero ? __float2half_rn(0.f) : s16;
+}
+
+// Non-finite flags of the calls in flight: a ring of words inside the library (exmoe_pack allocates nothing), one word
+// per call, so that calls from several host threads on several streams do not share a flag.
+constexpr int kPackFlags = 64;
+static __device__ int g_pack_flags[kPackFlags];
+
+int* pack_flag_word() {
+    static std::mutex mu;
+    static int* base[64] = {};
+    static unsigned next[64] = {};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+    std::lock_guard<std::mutex> lock(mu);
+    if (!base[dev]) {
+        void* p = nullptr;                                  // the symbol's device address (host code only holds a stand-in)
+        if (cudaGetSymbolAddress(&p, g_pack_flags) != cudaSuccess || !p) {
+            cudaGetLastError();
+            return nullptr;
+        }
+        base[dev] = static_cast<int*>(p);
+    }
+    return base[dev] + (next[dev]++ % kPackFlags);
 }
 
 int launch_pack(const exmoe_shape& s, const void* wg, const void* wu, const void* wd, void* out, int* d_flag,

@@ -1,7 +1,7 @@
 // Device-side expert-ID resolution with LRU slot replacement (Section 3.3), wave assignment and
 // expert map with sentinel (Section 3.4 steps 1-2), and token grouping by (wave, slot): histogram,
-// exclusive prefix sum and stable permutation of token-expert pairs (Figure 1, "tokens are grouped
-// by selected expert").  Integer work only; every result is deterministic and bit-exact.
+// exclusive prefix sum and stable permutation of token-expert pairs (the grouping step of Figure 1's caption).
+// Integer work only; every result is deterministic and bit-exact.
 #include "common.cuh"
 
 namespace exmoe {
@@ -284,7 +284,7 @@ __device__ __forceinline__ void scan_keys_warp0(const int32_t* cnt, int n_keys, 
     }
 }
 
-// Small problems (up to 1024 pairs): one CTA does histogram, scan and the stable permutation.
+// Small problems (up to 2048 pairs): one CTA does histogram, scan and the stable permutation.
 __global__ void __launch_bounds__(256)
 group_small_kernel(const int32_t* __restrict__ ids, int n_pairs, int E, int C, int n_keys, int max_waves,
                    bool identity, PlanPtrs plan, int* __restrict__ status) {

@@ -1,17 +1,16 @@
 """Seeded synthetic inputs shared by the tests, the smoke check and the benchmark.
 
-This module only draws random tensors and runs the router (Eq. 1 of the paper: logits,
-softmax, top-k) that produces the layer's inputs `topk_ids` / `topk_weights`.  It holds
-none of the layer's own arithmetic (no quantiser, no expert MLP, no cache logic), so both
-the CUDA path and the CPU oracle can be fed from it without sharing code.
+This module only draws random tensors.  It holds none of the method's arithmetic (no quantiser,
+no expert MLP, no cache logic, no router: Eq. 1 is `exmoe_route` in the library, `oracle/router.py`
+in the oracle and a torch restatement in the test helpers), so both the CUDA path and the CPU
+oracle can be fed from it without sharing code.
 
 Recipe (stand-in for the OLMoE checkpoint and prompts the paper measures on):
   expert weights  N(0, 0.02) rounded to BF16          W_g, W_u: [E, I, H]   W_d: [E, H, I]
   hidden states   N(0, 1)    rounded to BF16          [T, H]
   router          N(0, 0.02) rounded to BF16          [E, H]
-  routing         fp32 logits (+ optional per-expert bias), softmax over all E experts,
-                  top-k by descending probability, ties to the lower expert id,
-                  weights NOT renormalised over the selected k.
+  routing         (by the caller's router) logits + optional per-expert bias, softmax over all
+                  E experts, top-k, ties to the lower expert id, weights NOT renormalised.
   Zipf skew       bias_e = alpha * (-1.1 * ln rank_e), rank a seeded permutation of 1..E.
 """
 from dataclasses import dataclass
@@ -69,21 +68,10 @@ def zipf_bias(num_experts, alpha, seed):
     return alpha * (-1.1 * torch.log(rank))
 
 
-def route(hidden, w_router, top_k, bias=None):
-    """Eq. 1: logits -> softmax over all experts -> top-k.  Returns (ids int32 [T,k], p fp32 [T,k])."""
-    logits = hidden.float() @ w_router.float().t()
-    if bias is not None:
-        logits = logits + bias.to(logits.device)
-    p = torch.softmax(logits, dim=-1)
-    order = torch.sort(-p, dim=-1, stable=True).indices[:, :top_k]     # ties -> lower id
-    w = torch.gather(p, 1, order)
-    return order.to(torch.int32).contiguous(), w.contiguous()
-
-
 class SyntheticStack:
-    """Stand-in for a 16-layer sparse model around the MoE layers (config 5): per layer a BF16 router
-    (Eq. 1 with an optional Zipf bias), and between layers the dense parts abstracted to
-    h <- bf16(h + moe_out + N(0, 0.1)).  Only input generation: the MoE layer itself is `layer_fn`."""
+    """Stand-in for a 16-layer sparse model around the MoE layers (config 5): per layer BF16 router weights and an
+    optional Zipf bias, and between layers the dense parts abstracted to h <- bf16(h + moe_out + N(0, 0.1)).
+    Only input generation: the MoE layer is `layer_fn`, the router (Eq. 1) is `route_fn`, both the caller's."""
 
     def __init__(self, shape: Shape, num_layers, seed, alpha=1.0, device="cpu"):
         self.shape, self.L, self.device = shape, int(num_layers), device
@@ -97,19 +85,16 @@ class SyntheticStack:
         return [torch.randn((T, self.shape.d_model), generator=self.gen, device=self.device, dtype=torch.float32) * 0.1
                 for _ in range(self.L)]
 
-    def step(self, layer_fn, hidden, record=None, noise=None, route_fn=None, lookahead_fn=None):
+    def step(self, layer_fn, hidden, route_fn, record=None, noise=None, lookahead_fn=None):
         """layer_fn(layer, hidden, ids, weights) -> moe output.  Returns the hidden state after all layers.
         `noise`: per-layer residual tensors to use instead of drawing fresh ones.
-        `route_fn(layer, hidden) -> (ids, weights)`: a router to use instead of this module's `route` (it gets
-        this stack's `routers[layer]` and `bias[layer]` from the caller).
+        `route_fn(layer, hidden) -> (ids, weights)`: the router (Eq. 1), applied by the caller to this stack's
+        `routers[layer]` and `bias[layer]`.
         `lookahead_fn(next_layer, hidden)`: called before layer l runs, with layer l's input and l + 1 (a prefetch
         policy can guess layer l + 1's experts from it); its result is ignored."""
         h = hidden
         for l in range(self.L):
-            if route_fn is not None:
-                ids, w = route_fn(l, h)
-            else:
-                ids, w = route(h, self.routers[l], self.shape.top_k, self.bias[l])
+            ids, w = route_fn(l, h)
             if lookahead_fn is not None and l + 1 < self.L:
                 lookahead_fn(l + 1, h)
             out = layer_fn(l, h, ids, w)

@@ -64,11 +64,24 @@ def make_layer(shape, seed, device="cuda"):
     return OracleLayer(shape, wg, wu, wd), bank
 
 
+def route(hidden, w_router, top_k, bias=None):
+    """Harness router, Eq. 1 restated with torch ops in binary32: logits -> softmax over all experts -> top-k, ties
+    to the lower id, no renormalisation.  Returns (ids int32 [T,k], p fp32 [T,k]).  It only makes layer INPUTS for
+    the tests (the product's router is exmoe_route, the oracle's is oracle/router.py)."""
+    logits = hidden.float() @ w_router.float().t()
+    if bias is not None:
+        logits = logits + bias.to(logits.device)
+    p = torch.softmax(logits, dim=-1)
+    order = torch.sort(-p, dim=-1, stable=True).indices[:, :top_k]
+    w = torch.gather(p, 1, order)
+    return order.to(torch.int32).contiguous(), w.contiguous()
+
+
 def routed_inputs(shape, T, seed, alpha=0.0, device="cuda"):
     hidden = synth.hidden_states(shape, T, seed)
     wr = synth.router_weights(shape, seed + 7919)
     bias = synth.zipf_bias(shape.num_experts, alpha, seed + 31) if alpha else None
-    ids, p = synth.route(hidden, wr, shape.top_k, bias)
+    ids, p = route(hidden, wr, shape.top_k, bias)
     return hidden, ids, p
 
 

@@ -337,7 +337,8 @@ def test_config5_stack_teacher_forced(B):
     h = synth.hidden_states(s, 5, seed=3).cuda()
     for step in range(3):
         rec = []
-        h = stack.step(lambda l, x, ids, w: cache.forward(l, x, ids, w).clone(), h, record=rec)
+        h = stack.step(lambda l, x, ids, w: cache.forward(l, x, ids, w).clone(), h,
+                       lambda l, x: helpers.route(x, stack.routers[l], s.top_k, stack.bias[l]), record=rec)
         for (l, x, ids, w, out) in rec:
             y, ref = layers[l][0].forward(x.cpu(), ids.cpu(), w.cpu())
             helpers.check_output(out, y, ref, f"step {step} layer {l}")

@@ -57,7 +57,7 @@ def test_router_matches_oracle(B, shape, T, alpha):
     n_diff = check(shape, hidden, w_router, bias, ids, w)
     assert n_diff <= max(1, T // 50)                      # near-ties are rare with random inputs
     # the harness router (torch, binary32) makes the same choices up to the same near-ties
-    ids_t, w_t = synth.route(hidden.cuda(), w_router.cuda(), shape.top_k, None if bias is None else bias.cuda())
+    ids_t, w_t = helpers.route(hidden.cuda(), w_router.cuda(), shape.top_k, None if bias is None else bias.cuda())
     same = (ids_t == ids).all(dim=1).float().mean().item()
     assert same >= 0.95
 

@@ -6,6 +6,8 @@ import torch
 from oracle import moe, quant
 from paper_2608_15383_b200 import synth
 
+import helpers
+
 SHAPE = synth.Shape(d_model=256, d_ff=128, num_experts=8, top_k=2)
 
 
@@ -20,7 +22,7 @@ def layer():
             mats.append(quant.dequantize_g128(q, s))
         deq.append(tuple(mats))
     hidden = synth.hidden_states(SHAPE, 16, seed=1)
-    ids, p = synth.route(hidden, synth.router_weights(SHAPE, seed=2), SHAPE.top_k)
+    ids, p = helpers.route(hidden, synth.router_weights(SHAPE, seed=2), SHAPE.top_k)
     return deq, hidden.float().numpy(), ids.numpy(), p.numpy()
 
 

@@ -187,6 +187,31 @@ def test_layout_by_hand_single_code():
     assert np.array_equal(blob, expect)
 
 
+def test_layout_by_hand_second_code_first_half_word_zero_even_t():
+    """A second hand-placed code on the other branch of every rule: first half (h = 0), word 0 (first 32-wide set,
+    row q), an even t (low nibbles 0-3), panel 0, block 0, plus a neighbour with odd t in the same word: the byte
+    offsets and nibbles below are worked out from the written layout, not from the index tables."""
+    q = np.zeros((16, 128), dtype=np.int8)
+    s = np.zeros((16, 1), dtype=np.float16)
+    # row 5 (q = 5, r = 0), k = 8*3 + 4: h = 0, set 0, c = 3, t = 4 -> chunk 4*5 + 3 = 23, word 0, nibble (4 >> 1) = 2
+    q[5, 28] = 7
+    # same word, t = 1 (k = 25): nibble (1 >> 1) + 4 = 4
+    q[5, 25] = -8
+    s[5, 0] = 2.0
+    blob = layout.pack_matrix(q, s)
+    expect = np.full(1056, 0x88, dtype=np.uint8)
+    expect[1024:] = 0
+    word_off = 16 * 23 + 4 * 0
+    expect[word_off + 1] = 0x80 | (7 + 8)            # nibble 2 = low nibble of byte 1; its high nibble keeps code 0
+    expect[word_off + 2] = 0x80 | (-8 + 8)           # nibble 4 = low nibble of byte 2
+    expect[1024 + 2 * (2 * 5 + 0):1024 + 2 * (2 * 5 + 0) + 2] = np.array([2.0], dtype="<f2").view(np.uint8)
+    assert np.array_equal(blob, expect)
+    # and the whole word as the kernels read it: eight codes at shifts 0, 16, 4, 20, 8, 24, 12, 28 for t = 0..7
+    word = int(blob[word_off:word_off + 4].view("<u4")[0])
+    codes = [((word >> (4 * ((t >> 1) + 4 * (t & 1)))) & 0xF) - 8 for t in range(8)]
+    assert codes == [0, -8, 0, 0, 7, 0, 0, 0]
+
+
 def test_expert_blob_order_and_determinism():
     wg, wu, wd = bf16_weights((128, 256), 1), bf16_weights((128, 256), 2), bf16_weights((256, 128), 3)
     blob = layout.pack_expert(wg, wu, wd)
