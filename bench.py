@@ -590,6 +590,7 @@ def run_leg(name, args, shape, banks, dev, rank, local_rank, world, peaks, K, W,
         stream.synchronize()
         copy_ms, _ = cache.profile_read(4)
         gemm_ms = cache.profile_read(1)[0] + cache.profile_read(2)[0]
+        fetch_ms, fetch_with_gemm_ms = cache.profile_overlap()   # device timestamps of the brackets on both streams
         wall_ms = c0.elapsed_time(c1)
         moved = cache.stats(0)["h2d_bytes"] - b0
         cache.profile_enable(False)
@@ -610,6 +611,9 @@ def run_leg(name, args, shape, banks, dev, rank, local_rank, world, peaks, K, W,
                            else "host-issued cudaMemcpyAsync per miss",
                            "whole_step_frac": (moved / n_c) / (ms_step * 1e-3) / 1e9 / ceiling,
                            "miss_traffic_busy_fraction": copy_ms / wall_ms, "gemm_kernels_busy_fraction": gemm_ms / wall_ms,
+                           "fetch_time_overlapped_with_gemm_kernels": {"ms": fetch_with_gemm_ms, "of_fetch_ms": fetch_ms,
+                                                                       "fraction": fetch_with_gemm_ms / max(fetch_ms, 1e-9),
+                                                                       "of_gemm_time": fetch_with_gemm_ms / max(gemm_ms, 1e-9)},
                            "h2d_bytes_per_step": moved / n_c,
                            "peak_source": "one 104 MB pinned-host-to-device copy, measured in this run"}
         res["kernel_us"] = {"note": "C < E: single-kind launches still carry resolution and miss traffic; see roofline"}

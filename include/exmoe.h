@@ -141,8 +141,10 @@ int exmoe_moe_forward_host(exmoe_cache* cache, int layer, const void* hidden_hos
  *       wave's GEMM kernels a kernel on the caller's stream reads the wave's missed experts straight out of the
  *       pinned host bank (through its mapped address, over PCIe) into their slots.  The host waits for nothing and
  *       exmoe_moe_forward is a fixed launch sequence that may be captured in a CUDA graph.  It launches
- *       ceil(min(T*k, E) / wave_cap) waves whatever the ids turn out to be (a wave without work finds none), and
- *       within one call copies do not overlap kernels.
+ *       ceil(min(T*k, E) / wave_cap) waves whatever the ids turn out to be (a wave without work finds none).  For
+ *       24 < T*k <= 512 the fetch kernel runs on the library's side stream while the wave's GEMM kernels run over the
+ *       groups whose experts were already resident; the kernels over the fetched groups wait for it (events in both
+ *       directions, inside the capture too).  Smaller and larger calls fetch and compute in stream order.
  *   EXMOE_MISS_HOST_COPIES: the resolution kernel's miss plan is read back once per call (the paper's single
  *       batched id transfer) and the host waits for it, then issues one copy per missed expert on the library's
  *       copy stream, ordered against the compute stream by events; the copies of a wave overlap the kernels of
@@ -283,6 +285,10 @@ int exmoe_cache_destroy(exmoe_cache* cache);
  * restores normal operation. */
 int exmoe_profile_enable(exmoe_cache* cache, int on);
 int exmoe_profile_read(exmoe_cache* cache, int kind, double* total_ms, uint64_t* launches);
+/* Evidence for Sec. 3.3's asynchronous miss copies: of the time the bracketed miss traffic (kind 4) was running since the
+ * last enable, how much fell inside a bracketed GEMM interval (kinds 1 and 2) on the other stream.  Device timestamps of
+ * the brackets' events; synchronises.  Both zero when nothing was bracketed. */
+int exmoe_profile_overlap(exmoe_cache* cache, double* fetch_ms, double* fetch_during_gemm_ms);
 
 /* Kernels launched by this library since it was loaded (all streams, all caches); measurement hook, no paper counterpart. */
 uint64_t exmoe_launch_count(void);

@@ -65,6 +65,7 @@ _SIGNATURES = {
     "exmoe_cache_destroy": (c_int, [c_void_p]),
     "exmoe_profile_enable": (c_int, [c_void_p, c_int]),
     "exmoe_profile_read": (c_int, [c_void_p, c_int, POINTER(ctypes.c_double), POINTER(c_uint64)]),
+    "exmoe_profile_overlap": (c_int, [c_void_p, POINTER(ctypes.c_double), POINTER(ctypes.c_double)]),
     "exmoe_launch_count": (c_uint64, []),
 }
 
@@ -375,6 +376,12 @@ class Cache:
         ms, n = ctypes.c_double(), c_uint64()
         _check(lib().exmoe_profile_read(self.handle, int(kind), byref(ms), byref(n)), "exmoe_profile_read")
         return ms.value, int(n.value)
+
+    def profile_overlap(self):
+        """(ms of bracketed miss traffic, ms of it that ran while a bracketed GEMM kernel ran) since profile_enable."""
+        a, b = ctypes.c_double(), ctypes.c_double()
+        _check(lib().exmoe_profile_overlap(self.handle, byref(a), byref(b)), "exmoe_profile_overlap")
+        return a.value, b.value
 
     def close(self):
         if getattr(self, "handle", None):

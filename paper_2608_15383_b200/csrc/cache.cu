@@ -145,12 +145,16 @@ static void carve_workspace(exmoe_cache* c, uint8_t* ws, size_t* total) {
     c->plan.slot_of = p ? p + HDR_WORDS + E : nullptr;
     c->plan.misses = p ? p + HDR_WORDS + 2 * E : nullptr;
     c->plan_d2h_bytes = (HDR_WORDS + 5 * (size_t)E) * 4;
+    c->plan.key_miss = k.take<int32_t>(c->n_keys);
+    c->plan.n_keys = c->n_keys;
     int32_t* pf = k.take<int32_t>(HDR_WORDS + 5 * (size_t)E);
     c->plan_pf = PlanPtrs{};
     c->plan_pf.header = pf;
     c->plan_pf.wave_of = pf ? pf + HDR_WORDS : nullptr;
     c->plan_pf.slot_of = pf ? pf + HDR_WORDS + E : nullptr;
     c->plan_pf.misses = pf ? pf + HDR_WORDS + 2 * E : nullptr;
+    c->plan_pf.key_miss = nullptr;                        // a prefetch runs no GEMM kernels
+    c->plan_pf.n_keys = 0;
     c->plan.counts = k.take<int32_t>(c->n_keys);
     c->plan.offsets = k.take<int32_t>(c->n_keys + 1);
     c->plan.group_keys = k.take<int32_t>(c->n_keys);
@@ -418,6 +422,8 @@ int exmoe_moe_forward(exmoe_cache* c, int layer, const void* hidden, const int32
     a.offsets = c->plan.offsets;
     a.group_keys = c->plan.group_keys;
     a.perm = c->plan.perm;
+    a.key_miss = c->plan.key_miss;
+    a.group_filter = 0;
     a.num_slots = C;
     a.top_k = k;
     a.H = s.d_model;
@@ -441,9 +447,30 @@ int exmoe_moe_forward(exmoe_cache* c, int layer, const void* hidden, const int32
     int mi = 0;
     for (int w = 0; w < n_waves; ++w) {
         int groups = identity ? (E < P ? E : P) : 0;
+        bool split = false;                              // the wave's kernels run twice: resident groups, then fetched ones
         if (dev_fetch) {
-            ProfScope ps(c, PROF_COPY, st);
-            launch_fetch_misses(c->plan, w, c->bank_dev[layer], const_cast<uint8_t*>(a.slots), c->bpe, E, C, st);
+#ifndef EXMOE_NO_FETCH_OVERLAP
+            split = use_stream && !c->prof_only;
+#endif
+            if (split) {
+                // Sec. 3.3's asynchronous miss copy, Sec. 3.4 steps 3-5: the wave's fetch kernel runs on the library's side
+                // stream, behind everything that may still read the slots it overwrites (resolution and grouping for the
+                // first wave, the previous wave's kernels after that); meanwhile the wave's kernels run over the groups
+                // whose experts were resident (a miss only evicts slots the wave does not use), then wait for the fetch
+                // and run over the fetched groups.  Ordered by events in both directions: no kernel polls another.
+                cudaEvent_t fork = c->ev_compute[(++c->seq) % kEventRing];
+                cudaEventRecord(fork, st);
+                cudaStreamWaitEvent(c->copy_stream, fork, 0);
+                {
+                    ProfScope ps(c, PROF_COPY, c->copy_stream);
+                    launch_fetch_misses(c->plan, w, c->bank_dev[layer], const_cast<uint8_t*>(a.slots), c->bpe, E, C, c->copy_stream,
+                                        false, /*follows_resolve=*/false);
+                }
+                cudaEventRecord(c->ev_copy[(++c->copy_seq) % kEventRing], c->copy_stream);
+            } else {
+                ProfScope ps(c, PROF_COPY, st);
+                launch_fetch_misses(c->plan, w, c->bank_dev[layer], const_cast<uint8_t*>(a.slots), c->bpe, E, C, st);
+            }
             groups = c->Cw < P ? c->Cw : P;              // upper bound of the wave's groups (sizes the grids only)
             if (groups > E) groups = E;
         } else if (!identity) {
@@ -504,7 +531,20 @@ int exmoe_moe_forward(exmoe_cache* c, int layer, const void* hidden, const int32
             }
         } else if (use_stream) {
             // a few to a few dozen rows per expert: bulk-copy weight ring + register dequantisation, pair buffer + combine
-            if (!c->prof_only) {
+            if (split) {
+                a.group_filter = 1;
+                {
+                    ProfScope ps(c, PROF_GATEUP, st);
+                    launch_stream_wave(a, (const __nv_bfloat16*)hidden, c->act, topk_weights, c->y, c->d_status, groups, true, true, st);
+                }
+                cudaStreamWaitEvent(st, c->ev_copy[c->copy_seq % kEventRing], 0);     // the wave's fetched experts are in their slots
+                a.group_filter = 2;
+                {
+                    ProfScope ps(c, PROF_GATEUP, st);
+                    launch_stream_wave(a, (const __nv_bfloat16*)hidden, c->act, topk_weights, c->y, c->d_status, groups, true, true, st);
+                }
+                a.group_filter = 0;
+            } else if (!c->prof_only) {
                 ProfScope ps(c, PROF_GATEUP, st);    // both kernels: the down kernel is a programmatic dependent
                 launch_stream_wave(a, (const __nv_bfloat16*)hidden, c->act, topk_weights, c->y, c->d_status, groups, true, true,
                                    st);
@@ -785,6 +825,38 @@ int exmoe_profile_read(exmoe_cache* c, int kind, double* total_ms, uint64_t* lau
     }
     *total_ms = sum;
     *launches = n;
+    return EXMOE_OK;
+}
+
+int exmoe_profile_overlap(exmoe_cache* c, double* fetch_ms, double* fetch_during_gemm_ms) {
+    if (!c || !fetch_ms || !fetch_during_gemm_ms) return EXMOE_ERR_ARG;
+    if (cudaDeviceSynchronize() != cudaSuccess) return EXMOE_ERR_CUDA;
+    // device timestamps of every bracketed interval, relative to the first GEMM bracket (all events are on one device)
+    auto intervals = [&](int kind, cudaEvent_t ref, std::vector<std::pair<double, double>>& out) -> bool {
+        for (size_t i = 0; i + 1 < c->prof_used[kind]; i += 2) {
+            float t0 = 0.f, t1 = 0.f;
+            if (cudaEventElapsedTime(&t0, ref, c->prof_ev[kind][i]) != cudaSuccess ||
+                cudaEventElapsedTime(&t1, ref, c->prof_ev[kind][i + 1]) != cudaSuccess)
+                return false;
+            out.emplace_back((double)t0, (double)t1);
+        }
+        return true;
+    };
+    *fetch_ms = *fetch_during_gemm_ms = 0.0;
+    if (c->prof_used[PROF_COPY] < 2 || c->prof_used[PROF_GATEUP] < 2) return EXMOE_OK;
+    cudaEvent_t ref = c->prof_ev[PROF_GATEUP][0];
+    std::vector<std::pair<double, double>> f, g;
+    if (!intervals(PROF_COPY, ref, f) || !intervals(PROF_GATEUP, ref, g) || !intervals(PROF_DOWN, ref, g)) {
+        cudaGetLastError();
+        return EXMOE_ERR_CUDA;
+    }
+    for (const auto& fi : f) {
+        *fetch_ms += fi.second - fi.first;
+        for (const auto& gi : g) {
+            const double lo = std::max(fi.first, gi.first), hi = std::min(fi.second, gi.second);
+            if (hi > lo) *fetch_during_gemm_ms += hi - lo;
+        }
+    }
     return EXMOE_OK;
 }
 

@@ -30,6 +30,8 @@ struct PlanPtrs {
     int32_t* wave_of;       // [E]
     int32_t* slot_of;       // [E]
     int32_t* misses;        // [3*E] (expert, slot, wave)
+    int32_t* key_miss;      // [n_keys] 1 where the group (wave, slot) holds an expert that missed in this call
+    int n_keys;
     int32_t* counts;        // [n_keys]
     int32_t* offsets;       // [n_keys + 1]
     int32_t* group_keys;    // [n_keys] active keys, ascending
@@ -56,6 +58,8 @@ struct GemmArgs {
     const int32_t* group_keys;
     const int32_t* wave_start;  // already offset to the wave: [0] first group, [1] end
     const int32_t* perm;
+    const int32_t* key_miss;    // [n_keys] (see PlanPtrs); may be null
+    int group_filter;           // 0 all groups of the wave; 1 only groups whose expert was resident; 2 only the missed ones
     int num_slots;              // C (key % C = slot)
     int top_k;
     int H, I;
@@ -110,7 +114,7 @@ void launch_resolve(const exmoe_shape& s, int C, int Cw, size_t bytes_per_expert
                     LayerState state, PlanPtrs plan, int* d_status, cudaStream_t st);
 // Device-initiated miss path: one kernel copies wave `wave`'s missed experts from the mapped host bank into their slots.
 void launch_fetch_misses(const PlanPtrs& plan, int wave, const uint8_t* bank_dev, uint8_t* slots, size_t bpe, int E, int C,
-                         cudaStream_t st, bool small_grid = false);
+                         cudaStream_t st, bool small_grid = false, bool follows_resolve = true);
 void launch_group(const exmoe_shape& s, int C, int n_keys, int max_waves, bool identity, const int32_t* ids,
                   int n_pairs, PlanPtrs plan, int* d_status, cudaStream_t st);
 // Streaming kernels (bulk-copy weight ring in shared memory) for kSmallMaxPairs < T*k <= kStreamMaxPairs.

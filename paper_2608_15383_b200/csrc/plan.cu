@@ -41,6 +41,8 @@ resolve_kernel(const int32_t* __restrict__ ids, int n_pairs, int E, int C, int C
         s_sexp[v] = st.slot_expert[v];
         s_stamp[v] = st.slot_stamp[v];
     }
+    if (plan.key_miss)
+        for (int i = tid; i < plan.n_keys; i += blockDim.x) plan.key_miss[i] = 0;
     __syncthreads();
     for (int p = tid; p < n_pairs; p += blockDim.x) {
         const int id = ids[p];
@@ -102,6 +104,7 @@ resolve_kernel(const int32_t* __restrict__ ids, int n_pairs, int E, int C, int C
                     plan.misses[3 * nm + 0] = e;
                     plan.misses[3 * nm + 1] = s;
                     plan.misses[3 * nm + 2] = w;
+                    if (plan.key_miss) plan.key_miss[w * C + s] = 1;      // this group's weights arrive with the wave's fetch
                 }
                 ++nm;
                 ++misses;
@@ -204,7 +207,7 @@ fetch_misses_kernel(const int32_t* __restrict__ header, const int32_t* __restric
 }
 
 void launch_fetch_misses(const PlanPtrs& plan, int wave, const uint8_t* bank_dev, uint8_t* slots, size_t bpe, int E, int C,
-                         cudaStream_t st, bool small_grid) {
+                         cudaStream_t st, bool small_grid, bool follows_resolve) {
     int sms = 0, dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0)
         sms = 148;
@@ -218,7 +221,7 @@ void launch_fetch_misses(const PlanPtrs& plan, int wave, const uint8_t* bank_dev
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     lc.attrs = attr;
-    lc.numAttrs = (wave == 0) ? 1 : 0;                 // wave 0 directly follows the resolution kernel
+    lc.numAttrs = (wave == 0 && follows_resolve) ? 1 : 0;   // wave 0 directly follows the resolution kernel (same stream)
 #ifdef EXMOE_DISABLE_PDL
     lc.numAttrs = 0;
 #endif

@@ -203,6 +203,12 @@ stream_gemm_kernel(const StreamArgs p) {
                 rrow0[j] = a.offsets[rkey[j]];
             }
         }
+        // group filter (miss fetch overlapped with compute): a launch takes only the groups whose expert was resident
+        // (1) or only those that were fetched for this wave (2); the others count as empty
+        const int filter = a.key_miss ? a.group_filter : 0;
+#pragma unroll
+        for (int j = 0; j < kScanChunks; ++j)
+            if (filter && 32 * j + lane < n_groups && (a.key_miss[rkey[j]] != 0) != (filter == 2)) rrows[j] = 0;
         auto entry = [&](int chunk, int& key, int& rows, int& row0) {
             key = rows = row0 = 0;
             bool have = false;
@@ -218,6 +224,7 @@ stream_gemm_kernel(const StreamArgs p) {
                 key = a.group_keys[g0 + 32 * chunk + lane];
                 rows = a.counts[key];
                 row0 = a.offsets[key];
+                if (filter && (a.key_miss[key] != 0) != (filter == 2)) rows = 0;
             }
         };
         int total = 0;

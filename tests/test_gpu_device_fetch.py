@@ -195,3 +195,31 @@ def test_prefetch_of_the_next_layer_overlaps_a_forward(B):
         assert torch.equal(out1.view(torch.int16), want[1].view(torch.int16)), step
     assert cache.status() == 0
     cache.close(); full.close()
+
+
+def test_miss_fetch_overlaps_the_resident_groups_kernels(B, olmoe_layer):
+    """Config 3's path (16 tokens, 16 slots): the wave's fetch kernel runs on the side stream while the GEMM kernels run
+    over the groups whose experts were resident.  Device timestamps show fetch time inside GEMM intervals; the output
+    stays bit-identical to the resident run and the plan, state and counters to the oracle."""
+    ora, bank = olmoe_layer
+    s = synth.OLMOE
+    full = B.Cache(s, [bank], 64, max_tokens=16)
+    part = B.Cache(s, [bank], 16, max_tokens=16)
+    sc = ocache.SlotCache(64, 16, 0, bytes_per_expert=part.bytes_per_expert)
+    part.profile_enable(True)
+    for step in range(8):
+        hidden, ids, p = helpers.routed_inputs(s, 16, seed=8800 + step, alpha=2.0)     # strong skew: many hits per step
+        h, i, w = hidden.cuda(), ids.cuda(), p.cuda()
+        a = full.forward(0, h, i, w)
+        b = part.forward(0, h, i, w)
+        assert part.last_path() == B.PATH_STREAM
+        helpers.compare_plan(part, sc, ids)
+        assert torch.equal(a.view(torch.int16), b.view(torch.int16)), step
+    fetch_ms, both_ms = part.profile_overlap()
+    part.profile_enable(False)
+    st = part.stats(0)
+    assert st["hits"] > 0 and st["misses"] > 0
+    assert fetch_ms > 0 and 0 < both_ms <= fetch_ms
+    assert part.status() == 0 and full.status() == 0
+    full.close()
+    part.close()
