@@ -102,7 +102,7 @@ int exmoe_cache_workspace_bytes(const exmoe_shape* shape, int num_layers, int nu
  *   host_bank[l] : host, pinned, E * bytes_per_expert bytes: expert e of layer l at offset
  *                  e * bytes_per_expert, exactly as exmoe_pack wrote it.
  *   slot_mem     : dev, slot_bytes_total, 256-byte aligned.   workspace : dev, workspace_bytes, 256-aligned.
- *   wave_cap     : experts per wave, 1..num_slots; 0 means num_slots (Sec. 3.4 "at most C").
+ *   wave_cap     : experts per wave, 1..num_slots; 0 means num_slots (a wave never exceeds C, Sec. 3.4).
  * C = E: all experts are copied into their slots here (slot = expert id) and later calls do no
  * lookups.  C < E: the cache starts empty.  Synchronous. */
 int exmoe_cache_create(exmoe_cache** out, const exmoe_shape* shape, int num_layers, int num_slots,

@@ -192,7 +192,7 @@ def pack_bank(shape, w_gate, w_up, w_down, device="cuda"):
 
 
 def padded_dims(d_model, d_ff, group=128):
-    """Section 3.2 asks for dims that are multiples of the group size (other shapes "may require padding"): the
+    """Section 3.2 asks for dims that are multiples of the group size and Section 7 leaves other shapes to padding: the
     next multiples of 128."""
     up = lambda n: -(-int(n) // group) * group
     return up(d_model), up(d_ff)

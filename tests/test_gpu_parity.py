@@ -544,7 +544,7 @@ def test_shared_expert_geometry(B, T):
 
 
 def test_padding_of_dims_that_are_not_multiples_of_128(B):
-    """Section 3.2: other shapes "may require padding".  d_model = 200, d_ff = 300 padded with zeros to 256 / 384:
+    """Section 7 leaves shapes that are not multiples of the group size to padding.  d_model = 200, d_ff = 300 padded with zeros to 256 / 384:
     the padded layer matches the oracle on the padded weights, its extra output columns are exactly zero, and the
     first 200 columns agree, up to int4 quantisation noise, with the unquantised layer (Eq. 2) on the unpadded weights."""
     raw = synth.Shape(d_model=200, d_ff=300, num_experts=4, top_k=2)
