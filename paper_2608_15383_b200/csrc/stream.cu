@@ -140,7 +140,11 @@ struct Cursor {
 };
 
 // NMW: matrices held by one warp (2 = gate and up of the same panel; 1 = one matrix, gate/up split over warps)
-template <int NCH, bool GATEUP, int NMW>
+// KBc, PPc, KSc: blocks along K, panels per tile and K ranges per panel as COMPILE-TIME constants (0 = taken from the
+// arguments).  With run-time values about a third of the executed instructions were address arithmetic, predicates and
+// loop control around the conversion and the MMAs; the shapes that matter (OLMoE's two matrices) get their own
+// instantiations with the block loop unrolled and every stride a literal, all others run the generic one.
+template <int NCH, bool GATEUP, int NMW, int KBc = 0, int PPc = 0, int KSc = 0>
 __global__ void __launch_bounds__(kStreamThreads, 1)
 stream_gemm_kernel(const StreamArgs p) {
     constexpr int NM = GATEUP ? 2 : 1;                                // matrices per tile
@@ -149,8 +153,13 @@ stream_gemm_kernel(const StreamArgs p) {
     constexpr int CHN = (NMW * NCH >= 2) ? 1 : 2;                          // accumulator chains per (matrix, chunk): two independent MMA chains per warp at least
     extern __shared__ __align__(128) unsigned char smem[];
     const GemmArgs& a = p.a;
-    const int K = GATEUP ? a.H : a.I, NR = GATEUP ? a.I : a.H;
-    const int KB = K / kGroup, PP = p.PP, KS = p.KS, bpw = KB / KS;
+    constexpr bool FIXED = KBc > 0;
+    constexpr int BPWc = KSc > 0 ? KBc / (KSc > 0 ? KSc : 1) : 0;     // blocks per K range when the geometry is fixed
+    const int NR = GATEUP ? a.I : a.H;
+    const int KB = FIXED ? KBc : (GATEUP ? a.H : a.I) / kGroup, K = KB * kGroup;
+    const int PP = FIXED ? PPc : p.PP, KS = FIXED ? KSc : p.KS, bpw = KB / KS;
+    const uint32_t x_stride = FIXED ? (uint32_t)(KBc * kGroup * 2 + 64) : p.x_stride;
+    const uint32_t stage_bytes = FIXED ? (uint32_t)((GATEUP ? 2 : 1) * PPc * KBc * kBlockBytes) : p.stage_bytes;
     const int tiles = NR / (kPanelRows * PP);
     const int S = p.n_stages, NX = p.n_xbuf;
     unsigned char* wst = smem;
@@ -291,9 +300,9 @@ stream_gemm_kernel(const StreamArgs p) {
             if (n >= S && !warp_wait(&w_empty[s], ph, abort_flag, p.status)) break;
             const int4 gm = meta[cur.gi];
             if (lane == 0) {
-                const uint8_t* src = a.slots + (size_t)gm.x * a.slot_stride + mat_off + (size_t)cur.tile * p.stage_bytes;
-                mbar_expect_tx(&w_full[s], p.stage_bytes);
-                bulk_load(wst + (size_t)s * p.stage_bytes, src, p.stage_bytes, &w_full[s]);
+                const uint8_t* src = a.slots + (size_t)gm.x * a.slot_stride + mat_off + (size_t)cur.tile * stage_bytes;
+                mbar_expect_tx(&w_full[s], stage_bytes);
+                bulk_load(wst + (size_t)s * stage_bytes, src, stage_bytes, &w_full[s]);
             }
             __syncwarp();
             cur.advance(tiles, (gm.y + R - 1) / R);
@@ -324,7 +333,7 @@ stream_gemm_kernel(const StreamArgs p) {
                 if (lane < rows_here) {
                     const size_t src_row = GATEUP ? (size_t)(a.perm[gm.z + pass0 + lane] / a.top_k)
                                                   : (size_t)(gm.z + pass0 + lane);
-                    bulk_load(xs + ((size_t)b * R + lane) * p.x_stride, p.x_src + src_row * K, (uint32_t)K * 2, &x_full[b]);
+                    bulk_load(xs + ((size_t)b * R + lane) * x_stride, p.x_src + src_row * K, (uint32_t)K * 2, &x_full[b]);
                 }
                 __syncwarp();
                 ++n;
@@ -373,7 +382,7 @@ stream_gemm_kernel(const StreamArgs p) {
             const int rows_here = min(R, m_rows - pass0);
             if (++s == S) s = 0;
             if (s == 0) w_ph ^= 1u;
-            const unsigned char* xbuf = xs + (size_t)xb * R * p.x_stride;
+            const unsigned char* xbuf = xs + (size_t)xb * R * x_stride;
             float* adjb = adjg + (size_t)xb * KB * R;
             if (fresh) {                               // new rows: each group forms its own copy of the corrections
                 if (!mbar_wait(&x_full[xb], x_ph, abort_flag, p.status)) ok = false;
@@ -381,7 +390,7 @@ stream_gemm_kernel(const StreamArgs p) {
                 // a block is 16 chunks of 8 values: the 16 lanes of a half-warp hold one block of one row
                 const int chunks_per_row = K >> 3;
                 for (int nn = 0; nn < rows_here; ++nn) {
-                    const unsigned char* xrow = xbuf + (size_t)nn * p.x_stride;
+                    const unsigned char* xrow = xbuf + (size_t)nn * x_stride;
                     for (int base = cw * 32; base < chunks_per_row; base += kGroupThreads) {
                         const int ck = base + lane;
                         uint4 v = make_uint4(0, 0, 0, 0);
@@ -396,7 +405,7 @@ stream_gemm_kernel(const StreamArgs p) {
                 // each reads them only after its own barrier below; no copy targets these rows until every warp
                 // has released the buffer), so the fragment loads of the MMA loop need no row predicate
                 for (int nn = rows_here; nn < R; ++nn) {
-                    unsigned char* xrow = const_cast<unsigned char*>(xbuf) + (size_t)nn * p.x_stride;
+                    unsigned char* xrow = const_cast<unsigned char*>(xbuf) + (size_t)nn * x_stride;
                     for (int ck = cw * 32 + lane; ck < chunks_per_row; ck += kGroupThreads)
                         *reinterpret_cast<uint4*>(xrow + ck * 16) = make_uint4(0, 0, 0, 0);
                 }
@@ -412,7 +421,7 @@ stream_gemm_kernel(const StreamArgs p) {
                 }
                 continue;
             }
-            const unsigned char* stage = wst + (size_t)s * p.stage_bytes;
+            const unsigned char* stage = wst + (size_t)s * stage_bytes;
             float tot[NMW][NCH][4];
 #pragma unroll
             for (int m = 0; m < NMW; ++m)
@@ -420,7 +429,8 @@ stream_gemm_kernel(const StreamArgs p) {
                 for (int ch = 0; ch < NCH; ++ch)
 #pragma unroll
                     for (int i = 0; i < 4; ++i) tot[m][ch][i] = 0.f;
-            for (int b = 0; b < bpw; ++b) {
+#pragma unroll
+            for (int b = 0; b < (FIXED ? BPWc : bpw); ++b) {
                 const int kb = ks * bpw + b;
                 uint4 wv[NMW][2];
                 uint32_t sv[NMW];
@@ -452,7 +462,7 @@ stream_gemm_kernel(const StreamArgs p) {
                         uint4 xv[NCH];
 #pragma unroll
                         for (int ch = 0; ch < NCH; ++ch) {
-                            xv[ch] = *reinterpret_cast<const uint4*>(xbuf + (size_t)(8 * ch + q) * p.x_stride + k0 * 2);
+                            xv[ch] = *reinterpret_cast<const uint4*>(xbuf + (size_t)(8 * ch + q) * x_stride + k0 * 2);
                         }
 #pragma unroll
                         for (int m = 0; m < NMW; ++m) {
@@ -570,9 +580,25 @@ bool launch_stream_cfg(const GemmArgs& a, const __nv_bfloat16* x, __nv_bfloat16*
     StreamGeom g;
     if (!stream_geometry(GATEUP ? a.H : a.I, GATEUP ? a.I : a.H, NM, NCH, &g)) return false;
     void (*kern)(const StreamArgs) = stream_gemm_kernel<NCH, GATEUP, 1>;
-    if (GATEUP && g.NMW == 2) kern = stream_gemm_kernel<NCH, GATEUP, GATEUP ? 2 : 1>;
-    static SmemOnce smem_once[2];
-    allow_smem(kern, (int)kSmemLimit, smem_once[g.NMW - 1]);
+    int variant = 0;
+    if (GATEUP && g.NMW == 2) {
+        kern = stream_gemm_kernel<NCH, GATEUP, GATEUP ? 2 : 1>;
+        variant = 1;
+    }
+#ifndef EXMOE_STREAM_GENERIC_ONLY
+    // OLMoE's two matrices with their geometry as literals (d_model 2048: 16 blocks, one panel pair per tile, K in four
+    // ranges; d_ff 1024: 8 blocks, four panels per tile, K in two ranges)
+    const int KBv = (GATEUP ? a.H : a.I) / kGroup;
+    if (GATEUP && g.NMW == 1 && KBv == 16 && g.PP == 1 && g.KS == 4) {
+        kern = stream_gemm_kernel<NCH, GATEUP, 1, 16, 1, 4>;
+        variant = 2;
+    } else if (!GATEUP && KBv == 8 && g.PP == 4 && g.KS == 2) {
+        kern = stream_gemm_kernel<NCH, GATEUP, 1, 8, 4, 2>;
+        variant = 2;
+    }
+#endif
+    static SmemOnce smem_once[3];
+    allow_smem(kern, (int)kSmemLimit, smem_once[variant]);
     int sms = 0, dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0)
         sms = 148;
