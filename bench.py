@@ -622,7 +622,7 @@ def run_leg(name, args, shape, banks, dev, rank, local_rank, world, peaks, K, W,
 
     if full:
         # ---- end to end: host buffers in, host buffer out, copies inside the timed region
-        n_e2e = min(max(K, 100), 300)
+        n_e2e = 4 if args.profile_run else min(max(K, 100), 300)
         n_host = 8 if identity else min(n_sets, 128)
         pick = [(j * n_sets) // n_host for j in range(n_host)]
         h_h = [hs[j].cpu().pin_memory() for j in pick]
@@ -691,6 +691,9 @@ def main():
     ap.add_argument("--layers", type=int, default=0, help="layer banks to rotate over (0 = the workload's default)")
     ap.add_argument("--no-extra-legs", action="store_true",
                     help="decode workload: skip the short prefill (config 4) and offload (config 3) legs")
+    ap.add_argument("--profile-run", action="store_true",
+                    help="for captures under a profiler: one repetition of one replay per timed region, no extra legs, no "
+                         "CPU oracle leg, a short end-to-end loop (the printed numbers are then not bench values)")
     args = ap.parse_args()
 
     rank = int(os.environ.get("RANK", "0"))
@@ -730,6 +733,10 @@ def main():
     shape = synth.OLMOE
     K, W = args.steps, max(args.warmup, 3)
     peaks = load_peaks()
+    if args.profile_run:
+        global MIN_REGION_MS, REPS
+        MIN_REGION_MS, REPS = 0.0, 1
+        args.no_extra_legs, args.cpu_budget = True, 0.0
 
     # ---- data: replicas only, every rank holds the same workload with its own seed offset
     seed0 = 2000 + 100000 * rank

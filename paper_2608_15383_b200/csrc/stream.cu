@@ -653,9 +653,12 @@ bool launch_stream_wave(const GemmArgs& a, const __nv_bfloat16* hidden, __nv_bfl
 #else
     const bool entry_dependent = false;
 #endif
-    if (gateup) ok = launch_stream_cfg<1, true>(a, hidden, act, topk_w, y, status, max_groups, entry_dependent, st);
+#ifndef EXMOE_STREAM_NCH
+#define EXMOE_STREAM_NCH 1
+#endif
+    if (gateup) ok = launch_stream_cfg<EXMOE_STREAM_NCH, true>(a, hidden, act, topk_w, y, status, max_groups, entry_dependent, st);
     // a programmatic dependent only when the gate/up kernel of the same wave was launched just before it
-    if (down && ok) ok = launch_stream_cfg<1, false>(a, act, act, topk_w, y, status, max_groups, gateup, st);
+    if (down && ok) ok = launch_stream_cfg<EXMOE_STREAM_NCH, false>(a, act, act, topk_w, y, status, max_groups, gateup, st);
     return ok;
 }
 
