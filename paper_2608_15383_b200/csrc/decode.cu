@@ -687,6 +687,142 @@ pair_gateup_kernel(GemmArgs a, SmallArgs sa, const __nv_bfloat16* __restrict__ h
 }
 
 // ------------------------------------------------------------------------------------------------
+// Wide variant of the per-pair gate/up kernel: ONE CTA of 16 warps per SM instead of two of 8, each warp one
+// (panel pair, K range) unit held in registers, and every warp a pipeline of its own: its K range of the hidden
+// row goes into a private piece of shared memory, it forms the range's block corrections itself (same chunk ->
+// lane mapping and butterfly as the staging loops above: same bits), requests its blocks AHEAD blocks before it
+// needs them and starts on a block as soon as that block's registers have arrived.  No CTA-wide barrier before the
+// K-range partials meet, so the conversion of the early blocks runs while the late ones are still in flight.
+// Arithmetic and summation orders are those of pair_gateup_item.
+// ------------------------------------------------------------------------------------------------
+constexpr int kWideWarps = 16;
+#ifndef EXMOE_WIDE_MAX_PAIRS
+#define EXMOE_WIDE_MAX_PAIRS 32
+#endif
+constexpr int kWideMaxPairs = EXMOE_WIDE_MAX_PAIRS;     // pairs up to which the wide gate/up kernel is taken
+#ifndef EXMOE_WIDE_AHEAD
+#define EXMOE_WIDE_AHEAD 4
+#endif
+
+// one 128-wide block of a unit: gate and up words in registers, activations of the warp's K range in `xr`
+__device__ __forceinline__ void wide_block(const uint4 (&wb)[2][2], const uint32_t (&sb)[2], float adj, int b,
+                                           const unsigned char* xr, int lane, float (&tot)[2][2]) {
+    const int q = lane >> 2, c = lane & 3;
+    float acc[2][4];
+#pragma unroll
+    for (int m = 0; m < 2; ++m)
+#pragma unroll
+        for (int i = 0; i < 4; ++i) acc[m][i] = 0.f;
+#pragma unroll
+    for (int h = 0; h < 2; ++h)
+#pragma unroll
+        for (int set = 0; set < 2; ++set) {
+            const int k0 = b * kGroup + 64 * h + 32 * set + 8 * c;
+            uint4 xb = make_uint4(0, 0, 0, 0);
+            if (q == 0) xb = *reinterpret_cast<const uint4*>(xr + k0 * 2);
+#pragma unroll
+            for (int m = 0; m < 2; ++m) {
+                const uint32_t wq = set ? wb[m][h].z : wb[m][h].x;
+                const uint32_t wq8 = set ? wb[m][h].w : wb[m][h].y;
+                mma_m16n8k16(acc[m], code_pair(wq, 0), code_pair(wq8, 0), code_pair(wq, 4), code_pair(wq8, 4), xb.x, xb.y);
+                mma_m16n8k16(acc[m], code_pair(wq, 8), code_pair(wq8, 8), code_pair(wq, 12), code_pair(wq8, 12), xb.z, xb.w);
+            }
+        }
+#pragma unroll
+    for (int m = 0; m < 2; ++m) {
+        const __half2 sc = *reinterpret_cast<const __half2*>(&sb[m]);
+        tot[m][0] = fmaf(__low2float(sc), acc[m][0] + adj, tot[m][0]);
+        tot[m][1] = fmaf(__high2float(sc), acc[m][2] + adj, tot[m][1]);
+    }
+}
+
+template <int NB>
+__global__ void __launch_bounds__(32 * kWideWarps, 1)
+pair_gateup_wide_kernel(GemmArgs a, SmallArgs sa, const __nv_bfloat16* __restrict__ hidden,
+                        __nv_bfloat16* __restrict__ act_out, int ks_log2) {
+    // grid = (slices of 16 >> ks_log2 panel pairs, selected expert j, token t): pair p = t * k + j
+    extern __shared__ __align__(128) unsigned char smem[];
+    grid_launch_dependents();
+    if ((blockIdx.x | blockIdx.y | blockIdx.z) == 0) keep_pair_ids(sa);
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int q = lane >> 2, c = lane & 3;
+    const int p = blockIdx.z * a.top_k + blockIdx.y;
+    const int KB = a.H / kGroup, KS = 1 << ks_log2, PP = kWideWarps >> ks_log2;
+    const int ks = warp & (KS - 1), pp = warp >> ks_log2;
+    unsigned char* xw = smem + (size_t)warp * NB * kGroup * 2;                  // this warp's K range of the hidden row
+    float* red = reinterpret_cast<float*>(smem + (size_t)kWideWarps * NB * kGroup * 2);   // [PP][KS][2][16]
+
+    // the hidden row does not depend on the ids: request this warp's K range of it first
+    constexpr int XL = (NB * 16 + 31) / 32;                                      // 16-byte chunks per lane
+    const unsigned char* xrow = reinterpret_cast<const unsigned char*>(hidden + (size_t)blockIdx.z * a.H) + (size_t)ks * NB * kGroup * 2;
+    uint4 xpre[XL];
+#pragma unroll
+    for (int i = 0; i < XL; ++i) {
+        xpre[i] = make_uint4(0, 0, 0, 0);
+        if (i * 32 + lane < NB * 16) xpre[i] = ldg_early128(xrow + (size_t)(i * 32 + lane) * 16);
+    }
+    const int id = sa.ids[p];
+    if (id < 0 || id >= sa.E) return;                  // uniform over the CTA; the pair contributes nothing
+    const int slot = sa.slot_of ? sa.slot_of[id] : id;
+    const int panel = blockIdx.x * PP + pp;
+    const uint8_t* base = a.slots + (size_t)slot * a.slot_stride + ((size_t)(2 * panel) * KB + (size_t)ks * NB) * kBlockBytes;
+    uint4 wreg[NB][2][2];
+    uint32_t sreg[NB][2];
+    auto issue_block = [&](int b) {
+#pragma unroll
+        for (int m = 0; m < 2; ++m) {
+            const uint8_t* blk = base + ((size_t)m * KB + b) * kBlockBytes;
+            wreg[b][m][0] = ldg_stream128(blk + lane * 16);
+            wreg[b][m][1] = ldg_stream128(blk + 512 + lane * 16);
+            sreg[b][m] = ldg_stream32(blk + kCodeBytes + q * 4);
+        }
+    };
+    constexpr int AHEAD = EXMOE_WIDE_AHEAD < NB ? EXMOE_WIDE_AHEAD : NB;         // blocks requested before the arithmetic starts
+#pragma unroll
+    for (int b = 0; b < AHEAD; ++b) issue_block(b);
+    float adjv[NB];
+#pragma unroll
+    for (int i = 0; i < XL; ++i) {
+        const int ck = i * 32 + lane;
+        if (ck < NB * 16) *reinterpret_cast<uint4*>(xw + ck * 16) = xpre[i];
+        float sx = sum8_bf16(xpre[i]);
+#pragma unroll
+        for (int m = 8; m >= 1; m >>= 1) sx += __shfl_xor_sync(0xffffffffu, sx, m);
+        const float lo = __shfl_sync(0xffffffffu, sx, 0), hi = __shfl_sync(0xffffffffu, sx, 16);
+        // __fmul_rn: the product is rounded on its own, as where pair_gateup_item keeps it in shared memory (left to the
+        // compiler it would be contracted into the accumulator addition that consumes it: different bits)
+        if (2 * i < NB) adjv[2 * i] = __fmul_rn(-136.f, lo);
+        if (2 * i + 1 < NB) adjv[2 * i + 1] = __fmul_rn(-136.f, hi);
+    }
+    __syncwarp();
+    float tot[2][2] = {{0.f, 0.f}, {0.f, 0.f}};
+#pragma unroll
+    for (int b = 0; b < NB; ++b) {
+        if (b + AHEAD < NB) issue_block(b + AHEAD);
+        wide_block(wreg[b], sreg[b], adjv[b], b, xw, lane, tot);
+    }
+    if (c == 0) {
+        float* r = red + (size_t)warp * 32;            // warp = pp * KS + ks
+        r[q] = tot[0][0];
+        r[q + 8] = tot[0][1];
+        r[16 + q] = tot[1][0];
+        r[16 + q + 8] = tot[1][1];
+    }
+    __syncthreads();
+    // K ranges added in ascending order, SwiGLU, one rounding to BF16
+    if (tid < PP * kPanelRows) {
+        const int spp = tid >> 4, r = tid & 15;
+        const float* rb = red + ((size_t)spp << ks_log2) * 32;
+        float g = rb[r], u = rb[16 + r];
+        for (int s2 = 1; s2 < KS; ++s2) {
+            g += rb[s2 * 32 + r];
+            u += rb[s2 * 32 + 16 + r];
+        }
+        act_out[(size_t)p * a.I + (size_t)(blockIdx.x * PP + spp) * kPanelRows + r] = __float2bfloat16_rn(g / (1.f + __expf(-g)) * u);
+    }
+}
+
+// ------------------------------------------------------------------------------------------------
 // Bulk-copy variant of the by-token down kernel, used for two or more tokens.  Each expert warp brings its
 // panel (one contiguous range of the packed image) into SHARED MEMORY with one cp.async.bulk, completion counted
 // in bytes on an mbarrier, instead of into registers: the CTA is light in registers, all of its weight bytes are
@@ -841,6 +977,26 @@ void launch_pair_gateup(const GemmArgs& a, const SmallArgs& sa, const __nv_bfloa
     while ((1 << ks_log2) < KS) ++ks_log2;
     kern<<<dim3(tiles, a.top_k, sa.n_pairs / a.top_k), 256, smem, st>>>(a, sa, hidden, act, ks_log2);
     count_launch();
+}
+
+// false when the shape does not fit the wide kernel (the caller then takes pair_gateup_kernel)
+template <int NB>
+bool launch_pair_gateup_wide(const GemmArgs& a, const SmallArgs& sa, const __nv_bfloat16* hidden, __nv_bfloat16* act, int KS,
+                             cudaStream_t st) {
+#ifdef EXMOE_NO_WIDE_GATEUP
+    return false;
+#endif
+    int ks_log2 = 0;
+    while ((1 << ks_log2) < KS) ++ks_log2;
+    const int PP = kWideWarps >> ks_log2;
+    if ((1 << ks_log2) != KS || PP < 1 || a.I % (kPanelRows * PP)) return false;
+    auto kern = pair_gateup_wide_kernel<NB>;
+    const size_t smem = (size_t)kWideWarps * NB * kGroup * 2 + (size_t)kWideWarps * 32 * 4;
+    static SmemOnce smem_once;
+    allow_smem(kern, 100 * 1024, smem_once);
+    kern<<<dim3(a.I / (kPanelRows * PP), a.top_k, sa.n_pairs / a.top_k), 32 * kWideWarps, smem, st>>>(a, sa, hidden, act, ks_log2);
+    count_launch();
+    return true;
 }
 
 // K split over KS warps (KS in {1,2,4,8}, 8/KS panels per CTA) and register depth NB; aims at
@@ -1054,7 +1210,12 @@ void launch_small_wave(const GemmArgs& a, const SmallWave& w, cudaStream_t st, b
     if (w.pairwise) {                                   // T*k <= 32, one wave: no grouping, by-token down + combine
         if (gateup) {
             const DecodeCfg cfg = pick_cfg(a.H, a.I);
-            if (cfg.bpw == 4) launch_pair_gateup<4>(a, sa, w.hidden, w.act, cfg.KS, st);
+            // one token: the wide kernel (one 16-warp CTA per SM, every warp its own load/convert pipeline)
+            const bool wide = w.n_pairs <= kWideMaxPairs;
+            if (cfg.bpw == 4 && wide && launch_pair_gateup_wide<4>(a, sa, w.hidden, w.act, cfg.KS, st)) {}
+            else if (cfg.bpw == 2 && wide && launch_pair_gateup_wide<2>(a, sa, w.hidden, w.act, cfg.KS, st)) {}
+            else if (cfg.bpw == 1 && wide && launch_pair_gateup_wide<1>(a, sa, w.hidden, w.act, cfg.KS, st)) {}
+            else if (cfg.bpw == 4) launch_pair_gateup<4>(a, sa, w.hidden, w.act, cfg.KS, st);
             else if (cfg.bpw == 2) launch_pair_gateup<2>(a, sa, w.hidden, w.act, cfg.KS, st);
             else if (cfg.bpw == 1) launch_pair_gateup<1>(a, sa, w.hidden, w.act, cfg.KS, st);
             else launch_decode<true, MODE_PAIR>(a, sa, w.hidden, w.act, nullptr, nullptr, 1, w.n_pairs, st);
