@@ -12,6 +12,8 @@ import torch
 from oracle import router as orouter
 from paper_2608_15383_b200 import synth
 
+import helpers
+
 pytestmark = pytest.mark.gpu
 
 NEAR_TIE = 2e-5          # logit gap below which binary32 and binary64 may order two experts differently
