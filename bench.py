@@ -48,7 +48,7 @@ WORKLOADS = {
 # DRAM bytes (read + write) per launch of the dominant kernel, from one ncu capture each (dram__bytes_read.sum +
 # dram__bytes_write.sum, two layer banks = 415 MB resident; per-launch traffic does not depend on the number of banks):
 # (bytes, kernel captured, date of the capture)
-NCU_TRAFFIC = {"decode": (17.33e6, "pair_gateup_kernel<4>, T=1", "2026-11-25"),
+NCU_TRAFFIC = {"decode": (17.33e6, "pair_gateup_kernel<4>, T=1 (pair_gateup_wide_kernel<4> reads the same bytes)", "2026-11-25"),
                "decode16": (62.83e6 + 0.87e6, "stream_gemm_kernel<1,true,1>, T=16", "2026-11-25"),
                "prefill": (214.68e6 + 12.51e6, "prefill_gemm_kernel<true,256,2>, T=2048", "2026-11-25")}
 METRIC = "moe_layer_tokens_per_s"
@@ -544,7 +544,7 @@ def run_leg(name, args, shape, banks, dev, rank, local_rank, world, peaks, K, W,
     flops_step = 2.0 * T * shape.top_k * 3 * shape.d_ff * shape.d_model
     step_tflops = flops_step / (ms_step * 1e-3) / 1e12
     traffic = NCU_TRAFFIC.get(name) if not (full and (args.tokens or args.slots)) else None
-    if T * shape.top_k > 512:
+    if T * shape.top_k > 640:
         flops = 2.0 * T * shape.top_k * 2 * shape.d_ff * shape.d_model          # gate/up GEMM of one step
         achieved = flops / (kinds["gate_up"]["us_per_launch"] * 1e-6) / 1e12
         roof = {"bound": "tensor", "achieved": achieved, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
@@ -562,7 +562,7 @@ def run_leg(name, args, shape, banks, dev, rank, local_rank, world, peaks, K, W,
                 "frac": achieved / peaks["hbm_gbs"], "traffic": traffic[0] if traffic else None,
                 "traffic_unit": "bytes per launch (ncu dram read + write)",
                 "traffic_source": ("one ncu capture of %s on %s" % traffic[1:]) if traffic else None,
-                "kernel": "gate_up (pair_gateup_kernel)" if T * shape.top_k <= 24 else "gate_up (stream_gemm_kernel<1,true,1>)",
+                "kernel": "gate_up (pair_gateup_wide_kernel)" if T * shape.top_k <= 24 else "gate_up (stream_gemm_kernel<1,true,1>)",
                 "bytes_per_launch": gu_bytes, "peak_source": peaks["source"] + " copy rate, burst",
                 "whole_step": {"achieved": step_gbs, "bytes_per_step": active_all * bpe, "frac": step_gbs / peaks["hbm_gbs"]}}
     if not identity:

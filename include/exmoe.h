@@ -142,7 +142,7 @@ int exmoe_moe_forward_host(exmoe_cache* cache, int layer, const void* hidden_hos
  *       pinned host bank (through its mapped address, over PCIe) into their slots.  The host waits for nothing and
  *       exmoe_moe_forward is a fixed launch sequence that may be captured in a CUDA graph.  It launches
  *       ceil(min(T*k, E) / wave_cap) waves whatever the ids turn out to be (a wave without work finds none).  For
- *       24 < T*k <= 512 the fetch kernel runs on the library's side stream while the wave's GEMM kernels run over the
+ *       24 < T*k <= 640 the fetch kernel runs on the library's side stream while the wave's GEMM kernels run over the
  *       groups whose experts were already resident; the kernels over the fetched groups wait for it (events in both
  *       directions, inside the capture too).  Smaller and larger calls fetch and compute in stream order.
  *   EXMOE_MISS_HOST_COPIES: the resolution kernel's miss plan is read back once per call (the paper's single
@@ -240,7 +240,7 @@ int exmoe_debug_last_plan(exmoe_cache* cache, int layer, int32_t* n_active, int3
 enum {
     EXMOE_PATH_PAIR = 2,           /* per-pair gate/up kernel + by-token down kernel (T*k <= 24, one wave) */
     EXMOE_PATH_SMALL = 3,          /* grouping rebuilt inside the GEMM CTAs (T*k <= 24, several waves) */
-    EXMOE_PATH_STREAM = 4,         /* bulk-copy weight ring + register dequantisation (T*k <= 512) */
+    EXMOE_PATH_STREAM = 4,         /* bulk-copy weight ring + register dequantisation (T*k <= 640) */
     EXMOE_PATH_TENSOR_SMALL_N = 5, /* tcgen05 kernels, 64-row token tiles (T*k <= 1024) */
     EXMOE_PATH_TENSOR = 6          /* tcgen05 kernels, 256-row token tiles */
 };

@@ -119,7 +119,7 @@ void launch_group(const exmoe_shape& s, int C, int n_keys, int max_waves, bool i
                   int n_pairs, PlanPtrs plan, int* d_status, cudaStream_t st);
 // Streaming kernels (bulk-copy weight ring in shared memory) for kSmallMaxPairs < T*k <= kStreamMaxPairs.
 #ifndef EXMOE_STREAM_MAX_PAIRS
-#define EXMOE_STREAM_MAX_PAIRS 512
+#define EXMOE_STREAM_MAX_PAIRS 640
 #endif
 constexpr int kStreamMaxPairs = EXMOE_STREAM_MAX_PAIRS;   // above: tensor-core path
 bool stream_supported(int H, int I);

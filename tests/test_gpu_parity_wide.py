@@ -87,10 +87,10 @@ def test_small_n_tensor_core_kernels_at_olmoe_shape(B, olmoe_layer, T):
     cache.close()
 
 
-@pytest.mark.parametrize("M", [513, 600, 1025, 1300])
+@pytest.mark.parametrize("M", [641, 800, 1025, 1300])
 def test_group_size_sweep_reaches_the_tensor_core_kernels(B, M):
     """One expert, k = 1, group sizes past the streaming kernels' range: both tensor-core kernel shapes on a single
-    group with ragged tiles (513 = 8 tiles of 64 rows + 1 row; 1300 = 6 tiles of 224 rows, the last one short),
+    group with ragged tiles (641 = 10 tiles of 64 rows + 1 row; 1300 = 6 tiles of 224 rows, the last one short),
     every row against the dequantised reference (Sec. 5.3 checks group sizes against such a reference)."""
     s = synth.Shape(d_model=2048, d_ff=1024, num_experts=2, top_k=1)
     if not hasattr(test_group_size_sweep_reaches_the_tensor_core_kernels, "layer"):
