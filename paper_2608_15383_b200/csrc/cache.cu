@@ -72,7 +72,7 @@ struct exmoe_cache {
     bool pair_ok, small_ok;                   // ... the per-pair kernels / the in-CTA-grouping kernels (shared memory)
     void* tc_scratch;                         // tile list of the tensor-core path
     __nv_bfloat16* xg;                        // [max_pairs, H] hidden rows in plan order (tensor-core path only)
-    PrefillMaps tc_maps;                      // TMA descriptors of xg and act
+    PrefillMaps tc_maps;                      // TMA descriptors of xg and act (a device array carved from the workspace)
     int32_t* h_plan;                          // pinned staging of the plan
     cudaStream_t copy_stream;
     cudaEvent_t ev_plan;
@@ -178,6 +178,7 @@ static void carve_workspace(exmoe_cache* c, uint8_t* ws, size_t* total) {
     c->saved_ids = k.take<int32_t>(kPairMaxPairs);
     c->tc_scratch = k.take<uint8_t>(prefill_scratch_bytes(c->max_pairs, E));
     c->xg = (c->max_pairs > kSmallMaxPairs || !c->small_ok) ? k.take<__nv_bfloat16>((size_t)c->max_pairs * s.d_model) : nullptr;
+    c->tc_maps.dev = c->xg ? k.take<uint8_t>(kPrefillMapBytes) : nullptr;
     {   // staging of the host-buffer entry point: hidden | ids | weights (one H2D copy), then out (one D2H copy)
         const size_t nb_h = align_up((size_t)c->max_tokens * s.d_model * 2, 256);
         const size_t nb_i = align_up((size_t)c->max_pairs * 4, 256);

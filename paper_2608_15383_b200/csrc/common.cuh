@@ -129,9 +129,10 @@ void launch_small_wave(const GemmArgs& a, const SmallWave& w, cudaStream_t st, b
 bool pair_path_fits(int H, int I, int top_k);                           // shared memory of the per-pair kernels within limits
 bool small_path_fits(int H, int I, int num_slots, int n_pairs);         // ... of the in-CTA-grouping kernels
 size_t prefill_scratch_bytes(int max_pairs, int num_experts);
-// CUtensorMap objects of the grouped hidden rows and of the activations: 256-row boxes for the large-N kernel shape,
-// 64-row boxes for the small-N shape
-struct alignas(64) PrefillMaps { unsigned char x[128], act[128], x_small[128], act_small[128]; };
+// CUtensorMap objects of the grouped hidden rows and of the activations, in device memory: per matrix a family of 16
+// maps whose boxes hold 16, 32, ..., 256 rows (a tile's box holds exactly the rows its MMAs read); x family, then act
+constexpr size_t kPrefillMapBytes = 2 * 16 * 128;
+struct PrefillMaps { unsigned char* dev; };
 int prefill_setup(PrefillMaps* maps, const __nv_bfloat16* xg, const __nv_bfloat16* act, int max_pairs, int H, int I);
 void launch_wait_selftest(int* status, long long budget_cycles, int* result, cudaStream_t st);
 // grouped copy of the hidden rows; when `single_wave` is given its CTA 0 also builds that wave's tile list in `scratch`
@@ -139,7 +140,7 @@ void launch_gather_rows(const __nv_bfloat16* hidden, const int32_t* perm, const 
                         int H, __nv_bfloat16* xg, const GemmArgs* single_wave, const int32_t* wave_start, void* scratch,
                         bool small_n, cudaStream_t st);
 // which: bit 0 = gate/up GEMM + SwiGLU, bit 1 = down GEMM x routing weight, bit 2 = (re)build the wave's tile list
-// small_n: the 64-row, four-stage kernel shape (a few dozen rows per expert) instead of the 256-row, two-stage one
+// small_n: the 64-row, eight-stage kernel shape (a few dozen rows per expert) instead of the 256-row, four-stage one
 void launch_prefill_wave(const GemmArgs& g, const int32_t* wave_start, void* scratch, int* status, const PrefillMaps* maps,
                          __nv_bfloat16* act, const float* topk_w, float* y, int which, bool small_n, cudaStream_t st);
 #ifndef EXMOE_PREFILL_SMALL_N_MAX_PAIRS

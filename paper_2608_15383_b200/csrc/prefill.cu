@@ -41,14 +41,16 @@ namespace {
 constexpr int BM = 128;            // weight rows per tile
 constexpr int BN = 256;            // max grouped rows (tokens) per tile of the large-N kernel shape
 constexpr int BN_SMALL = 64;       // ... and of the small-N shape (a few dozen rows per expert: four stages fit)
-constexpr int BK = 128;            // K per stage = one packed block / one scale group
+constexpr int BK = 128;            // one packed block / one scale group
+constexpr int BKS = 64;            // K per ring stage = half a packed block (the half one dequantisation warp converts)
 // A (dequantised weights): no swizzle; core matrix = 8 rows x 16 B; k-chunks 160 B apart (128 + 32 pad, so that
-// the 8 lanes of a quarter warp, 2 rows x 4 k-chunks, hit 8 different 16-byte bank groups), row groups 2560 B apart
+// the 8 lanes of a quarter warp, 2 rows x 4 k-chunks, hit 8 different 16-byte bank groups), row groups 1280 B apart
 constexpr int A_LBO = 160;
-constexpr int A_SBO = 16 * A_LBO;
-constexpr int A_STAGE_BYTES = 16 * A_SBO;      // 40 KB
-// B (tokens): TMA 128-byte swizzle; two halves of 64 columns, each 256 rows x 128 B; 8-row atoms of 1024 B
+constexpr int A_SBO = (BKS / 8) * A_LBO;
+constexpr int A_STAGE_BYTES = 16 * A_SBO;      // 20 KB
+// B (tokens): TMA 128-byte swizzle; 64 columns x up to 256 rows of 128 B; 8-row atoms of 1024 B
 constexpr int B_SBO = 1024;
+constexpr int N_MAPS = 16;         // tensor maps per operand: boxes of 16, 32, ..., 256 rows
 constexpr int NUM_THREADS = 896;   // 28 warps: MMA, TMA, 2 idle, 4 + 4 epilogue, 8 + 8 dequant
 
 struct Tile { int key, n0, nrows, pad; };
@@ -167,20 +169,21 @@ struct PrefillArgs {
     int* status;
 };
 
-// BN_T = token rows per tile (256 or 64), STAGES = ring depth (2 or 4).  The round trip of one stage (MMAs
-// complete -> commit -> dequantisation warps refill -> MMA issuer wakes) is about 2000 cycles whatever the tile
-// holds, so with few rows per expert (tiny MMAs) the ring depth sets the rate: the small-N shape spends the
-// shared memory it saves on the token tile on two more stages.
+// BN_T = token rows per tile (256 or 64), STAGES = ring depth.  One ring stage holds 64 of K: half a packed block
+// of the weights (the half one dequantisation warp converts) and a [rows x 64] box of tokens.  The round trip of one
+// stage (MMAs complete -> commit -> token box fetched from L2, weights converted -> MMA issuer wakes) is 2000-3000
+// cycles, far more than the stage's MMAs take, so the ring depth sets the rate: 64-wide stages give the large shape
+// four of them and the small shape eight in the same shared memory.  The token box holds exactly the tile's rows
+// (rounded up to 16): `maps` is a family of tensor maps over the same matrix with boxes of 16, 32, ..., 256 rows.
 template <bool GATEUP, int BN_T, int STAGES>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
-prefill_gemm_kernel(PrefillArgs a, const __grid_constant__ CUtensorMap tmap_b, __nv_bfloat16* __restrict__ act_out,
+prefill_gemm_kernel(PrefillArgs a, const CUtensorMap* __restrict__ maps, __nv_bfloat16* __restrict__ act_out,
                     const float* __restrict__ topk_w, const int32_t* __restrict__ offsets, float* __restrict__ y_out) {
     extern __shared__ unsigned char smem_raw[];
     unsigned char* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);   // swizzled tiles need 1 KB alignment
-    constexpr int B_HALF_BYTES = BN_T * 128;                      // BN_T rows x 64 columns
-    constexpr int B_STAGE_BYTES = 2 * B_HALF_BYTES;
+    constexpr int B_STAGE_BYTES = BN_T * 128;                     // BN_T rows x 64 columns
     unsigned char* sB = smem;                                     // [STAGES][B_STAGE_BYTES]
-    unsigned char* sA = smem + STAGES * B_STAGE_BYTES;            // [STAGES][40 KB]
+    unsigned char* sA = smem + STAGES * B_STAGE_BYTES;            // [STAGES][20 KB]
     uint64_t* bars = reinterpret_cast<uint64_t*>(sA + STAGES * A_STAGE_BYTES);
     uint64_t* full = bars;                          // [STAGES]  producers -> MMA
     uint64_t* empty = bars + STAGES;                // [STAGES]  MMA -> producers (tcgen05.commit)
@@ -198,7 +201,7 @@ prefill_gemm_kernel(PrefillArgs a, const __grid_constant__ CUtensorMap tmap_b, _
 
     if (tid == 0) {
         for (int s = 0; s < STAGES; ++s) {
-            mbar_init(&full[s], 17);          // 16 A-producer warps + the TMA thread's expect_tx arrive
+            mbar_init(&full[s], 9);           // the 8 A-producer warps of this k-half + the TMA thread's expect_tx arrive
             mbar_init(&empty[s], 1);
         }
         for (int b = 0; b < 2; ++b) {
@@ -220,7 +223,7 @@ prefill_gemm_kernel(PrefillArgs a, const __grid_constant__ CUtensorMap tmap_b, _
     if (warp == 0) {
         // ------------------------------------------------------------------ MMA issuer
         // the whole warp walks the loop (so it stays converged for the block-wide teardown); lane 0 issues
-        int it = 0;                                                // running k-block counter (stage/phase)
+        int s = 0, ph = 0;                                         // ring position of the next stage to consume
         int tcount = 0;
         bool ok = true;
         PROF_DECL;
@@ -236,11 +239,10 @@ prefill_gemm_kernel(PrefillArgs a, const __grid_constant__ CUtensorMap tmap_b, _
             if (!ok) break;
             tc_fence_after();
             const uint32_t d_tmem = tmem_base + buf * BN_T;
-            for (int kb = 0; kb < KB; ++kb, ++it) {
-                const int s = it % STAGES;
+            for (int ks = 0; ks < 2 * KB; ++ks) {
                 {
                     PROF_WAIT_BEGIN;
-                    ok = mbar_wait(&full[s], (it / STAGES) & 1, abort_flag, a.status);
+                    ok = mbar_wait(&full[s], ph, abort_flag, a.status);
                     PROF_WAIT_END;
                 }
                 ok = __all_sync(0xffffffffu, ok);
@@ -250,14 +252,15 @@ prefill_gemm_kernel(PrefillArgs a, const __grid_constant__ CUtensorMap tmap_b, _
                     const uint64_t da = make_desc_a(smem_u32(sA + s * A_STAGE_BYTES));
                     const uint64_t db = make_desc_b(smem_u32(sB + s * B_STAGE_BYTES));
 #pragma unroll
-                    for (int j = 0; j < BK / 16; ++j) {            // K16 step j: A two k-chunks on, B 32 bytes on in its half
+                    for (int j = 0; j < BKS / 16; ++j) {           // K16 step j: A two k-chunks on, B 32 bytes on
                         const uint64_t aj = da + (uint64_t)(j * 2 * A_LBO >> 4);
-                        const uint64_t bj = db + (uint64_t)(((j >> 2) * B_HALF_BYTES + (j & 3) * 32) >> 4);
-                        tc_mma(d_tmem, aj, bj, idesc, (kb | j) ? 1u : 0u);
+                        const uint64_t bj = db + (uint64_t)((j * 32) >> 4);
+                        tc_mma(d_tmem, aj, bj, idesc, (ks | j) ? 1u : 0u);
                     }
                     tc_commit(&empty[s]);                          // stage reusable once these MMAs have read it
                 }
                 __syncwarp();
+                if (++s == STAGES) { s = 0; ph ^= 1; }
             }
             if (ok && lane == 0) tc_commit(&acc_full[buf]);        // accumulator complete
             __syncwarp();
@@ -323,37 +326,37 @@ prefill_gemm_kernel(PrefillArgs a, const __grid_constant__ CUtensorMap tmap_b, _
         PROF_REPORT("epilogue");
     } else if (warp == 1) {
         // ------------------------------------------------------------------ B producer (TMA, one thread issues)
-        int it = 0;
+        int s = 0, ph = 0;
         bool ok = true;
         PROF_DECL;
         for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
             const Tile tl = a.tiles[t / MT];
             const int row0 = offsets[tl.key] + tl.n0;
-            for (int kb = 0; kb < KB; ++kb, ++it) {
-                const int s = it % STAGES;
+            const int n_mma = (tl.nrows + 15) & ~15;               // rows of the box = rows the MMAs read
+            const CUtensorMap* map = maps + (n_mma / 16 - 1);
+            for (int ks = 0; ks < 2 * KB; ++ks) {
                 {
                     PROF_WAIT_BEGIN;
-                    ok = mbar_wait(&empty[s], ((it / STAGES) & 1) ^ 1, abort_flag, a.status);
+                    ok = mbar_wait(&empty[s], ph ^ 1, abort_flag, a.status);
                     PROF_WAIT_END;
                 }
                 ok = __all_sync(0xffffffffu, ok);
                 if (!ok) break;
                 if (lane == 0) {
-                    const uint32_t dst = smem_u32(sB + s * B_STAGE_BYTES);
-                    mbar_expect_tx(&full[s], B_STAGE_BYTES);
-                    tma_load_2d(dst, &tmap_b, kb * BK, row0, &full[s]);                   // columns kb*128 .. +63
-                    tma_load_2d(dst + B_HALF_BYTES, &tmap_b, kb * BK + 64, row0, &full[s]);
+                    mbar_expect_tx(&full[s], n_mma * 128);
+                    tma_load_2d(smem_u32(sB + s * B_STAGE_BYTES), map, ks * BKS, row0, &full[s]);
                 }
                 __syncwarp();
+                if (++s == STAGES) { s = 0; ph ^= 1; }
             }
         }
         PROF_REPORT("B producer");
     } else if (warp >= 8 && !(warp >= 16 && warp < 20)) {
         // ------------------------------------------------------------------ A producers (dequantise)
         const int pw = warp & 7;                                   // panel of the tile = 8-row groups 2*pw, 2*pw+1
-        const int hh = warp >= 20 ? 1 : 0;                         // 64-wide k-half of every block
+        const int hh = warp >= 20 ? 1 : 0;                         // 64-wide k-half of every block = every second stage
         const int q = lane >> 2, c = lane & 3;
-        int it = 0;
+        int s = hh % STAGES, ph = 0;                               // ring position of this warp's next stage (2 * blocks + hh)
         bool ok = true;
         PROF_DECL;
         for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
@@ -377,7 +380,6 @@ prefill_gemm_kernel(PrefillArgs a, const __grid_constant__ CUtensorMap tmap_b, _
                 for (int u = 0; u < PF; ++u) {
                     const int kb = kb0 + u;
                     if (kb >= KB) break;
-                    const int s = it % STAGES;
                     constexpr int nx_off = PF - 1;
                     if (kb + nx_off < KB) {                        // keep two blocks of codes in flight
                         const uint8_t* blk = pn + (size_t)(kb + nx_off) * kBlockBytes;
@@ -386,7 +388,7 @@ prefill_gemm_kernel(PrefillArgs a, const __grid_constant__ CUtensorMap tmap_b, _
                     }
                     {
                         PROF_WAIT_BEGIN;
-                        ok = mbar_wait(&empty[s], ((it / STAGES) & 1) ^ 1, abort_flag, a.status);
+                        ok = mbar_wait(&empty[s], ph ^ 1, abort_flag, a.status);
                         PROF_WAIT_END;
                     }
                     ok = __all_sync(0xffffffffu, ok);
@@ -399,14 +401,15 @@ prefill_gemm_kernel(PrefillArgs a, const __grid_constant__ CUtensorMap tmap_b, _
 #pragma unroll
                     for (int wi = 0; wi < 4; ++wi) {
                         const int r = wi & 1, set = wi >> 1;
-                        const int kc = 8 * hh + 4 * set + c;                              // 16-byte k-chunk
+                        const int kc = 4 * set + c;                                       // 16-byte k-chunk of the stage
                         const uint4 val = dequant_word(words[wi], r ? s_hi : s_lo);
                         *reinterpret_cast<uint4*>(dst + (2 * pw + r) * A_SBO + kc * A_LBO + q * 16) = val;
                     }
                     fence_proxy_async();
                     __syncwarp();
                     if (lane == 0) mbar_arrive(&full[s]);
-                    ++it;
+                    s += 2;                                        // this warp's next stage is two on
+                    if (s >= STAGES) { s -= STAGES; ph ^= 1; }
                 }
                 if (!ok) break;
             }
@@ -551,10 +554,14 @@ static int encode_map(CUtensorMap* out, const void* base, int rows, int cols, in
 }
 
 int prefill_setup(PrefillMaps* maps, const __nv_bfloat16* xg, const __nv_bfloat16* act, int max_pairs, int H, int I) {
-    int rc = encode_map(reinterpret_cast<CUtensorMap*>(maps->x), xg, max_pairs, H, BN);
-    if (!rc) rc = encode_map(reinterpret_cast<CUtensorMap*>(maps->act), act, max_pairs, I, BN);
-    if (!rc) rc = encode_map(reinterpret_cast<CUtensorMap*>(maps->x_small), xg, max_pairs, H, BN_SMALL);
-    if (!rc) rc = encode_map(reinterpret_cast<CUtensorMap*>(maps->act_small), act, max_pairs, I, BN_SMALL);
+    static_assert(kPrefillMapBytes == 2 * N_MAPS * sizeof(CUtensorMap), "map families of the two operands");
+    alignas(64) CUtensorMap host[2 * N_MAPS];
+    int rc = EXMOE_OK;
+    for (int i = 0; i < N_MAPS && !rc; ++i) {
+        rc = encode_map(&host[i], xg, max_pairs, H, 16 * (i + 1));
+        if (!rc) rc = encode_map(&host[N_MAPS + i], act, max_pairs, I, 16 * (i + 1));
+    }
+    if (!rc && cudaMemcpy(maps->dev, host, sizeof(host), cudaMemcpyHostToDevice) != cudaSuccess) rc = EXMOE_ERR_CUDA;
     return rc;
 }
 
@@ -590,9 +597,9 @@ void launch_prefill_wave(const GemmArgs& g, const int32_t* wave_start, void* scr
     a.H = g.H;
     a.I = g.I;
     a.status = status;
-    constexpr int kStagesLarge = 2, kStagesSmall = 4;
-    const size_t smem_large = (size_t)kStagesLarge * (A_STAGE_BYTES + 2 * BN * 128) + 256 + 1024;
-    const size_t smem_small = (size_t)kStagesSmall * (A_STAGE_BYTES + 2 * BN_SMALL * 128) + 256 + 1024;
+    constexpr int kStagesLarge = 4, kStagesSmall = 8;
+    const size_t smem_large = (size_t)kStagesLarge * (A_STAGE_BYTES + BN * 128) + 256 + 1024;
+    const size_t smem_small = (size_t)kStagesSmall * (A_STAGE_BYTES + BN_SMALL * 128) + 256 + 1024;
     static SmemOnce once[4];
     allow_smem(prefill_gemm_kernel<true, BN, kStagesLarge>, (int)smem_large, once[0]);
     allow_smem(prefill_gemm_kernel<false, BN, kStagesLarge>, (int)smem_large, once[1]);
@@ -601,24 +608,24 @@ void launch_prefill_wave(const GemmArgs& g, const int32_t* wave_start, void* scr
     int dev = 0, sms = 148;
     cudaGetDevice(&dev);
     cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-    const CUtensorMap* mx = reinterpret_cast<const CUtensorMap*>(small_n ? maps->x_small : maps->x);
-    const CUtensorMap* ma = reinterpret_cast<const CUtensorMap*>(small_n ? maps->act_small : maps->act);
+    const CUtensorMap* mx = reinterpret_cast<const CUtensorMap*>(maps->dev);
+    const CUtensorMap* ma = mx + N_MAPS;
     if (which & 4) {
         tile_list_kernel<<<1, 1024, 0, st>>>(g.counts, g.group_keys, wave_start, tiles, n_tiles, small_n ? BN_SMALL : BN);
         count_launch();
     }
     if (which & 1) {
         if (small_n)
-            prefill_gemm_kernel<true, BN_SMALL, kStagesSmall><<<sms, NUM_THREADS, smem_small, st>>>(a, *mx, act, nullptr, g.offsets, nullptr);
+            prefill_gemm_kernel<true, BN_SMALL, kStagesSmall><<<sms, NUM_THREADS, smem_small, st>>>(a, mx, act, nullptr, g.offsets, nullptr);
         else
-            prefill_gemm_kernel<true, BN, kStagesLarge><<<sms, NUM_THREADS, smem_large, st>>>(a, *mx, act, nullptr, g.offsets, nullptr);
+            prefill_gemm_kernel<true, BN, kStagesLarge><<<sms, NUM_THREADS, smem_large, st>>>(a, mx, act, nullptr, g.offsets, nullptr);
         count_launch();
     }
     if (which & 2) {
         if (small_n)
-            prefill_gemm_kernel<false, BN_SMALL, kStagesSmall><<<sms, NUM_THREADS, smem_small, st>>>(a, *ma, nullptr, topk_w, g.offsets, y);
+            prefill_gemm_kernel<false, BN_SMALL, kStagesSmall><<<sms, NUM_THREADS, smem_small, st>>>(a, ma, nullptr, topk_w, g.offsets, y);
         else
-            prefill_gemm_kernel<false, BN, kStagesLarge><<<sms, NUM_THREADS, smem_large, st>>>(a, *ma, nullptr, topk_w, g.offsets, y);
+            prefill_gemm_kernel<false, BN, kStagesLarge><<<sms, NUM_THREADS, smem_large, st>>>(a, ma, nullptr, topk_w, g.offsets, y);
         count_launch();
     }
 }
