@@ -251,55 +251,92 @@ prefill_gemm_kernel(PrefillArgs a, const CUtensorMap* __restrict__ maps, __nv_bf
 
     if (warp == 0) {
         // ------------------------------------------------------------------ MMA issuer
-        // the whole warp walks the loop (so it stays converged for the block-wide teardown); lane 0 issues
-        int sb = 0, phb = 0, sa = 0, pha = 0;                      // ring positions of the next stage to consume
-        int tcount = 0;
-        bool ok = true;
+        // ONE thread runs the loop (the other lanes wait at the warp barrier below).  tcgen05.mma issue blocks while
+        // the tensor pipe is busy, and the pipe holds little beyond the MMA it executes: every instruction this
+        // thread spends between two MMAs is time the pipe may drain, and with six busy warps on the same scheduler
+        // each instruction takes many cycles to issue (measured alone: the same four MMAs per stage run at N / 2
+        // cycles each with compile-time operands, at 150-160 cycles each, whatever N, behind run-time ring
+        // arithmetic and a barrier test).  So the ring is unrolled (stage index, barrier addresses and operand offsets
+        // are compile-time constants) and the NEXT stage's barriers are tested before this stage's MMAs are issued,
+        // the answer being read after them.  Shapes whose stage count per tile is not a multiple of the ring depth
+        // take the plain loop.
+        static_assert(SB == 2 * SA, "the unrolled issue loop walks the A ring twice per turn of the B ring");
         PROF_DECL;
-        for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x, ++tcount) {
-            const Tile tl = a.tiles[t / MT];
-            const int n_mma = (tl.nrows + 15) & ~15;
-            const uint32_t idesc = make_idesc(n_mma);
-            const int buf = tcount & 1;
-            PROF_WAIT_BEGIN;
-            ok = mbar_wait(&acc_empty[buf], ((tcount >> 1) & 1) ^ 1, abort_flag, a.status);
-            PROF_WAIT_END;
-            ok = __all_sync(0xffffffffu, ok);
-            if (!ok) break;
-            tc_fence_after();
-            const uint32_t d_tmem = tmem_base + buf * BN_T;
-            for (int ks = 0; ks < 2 * KB; ++ks) {
-                {
-                    PROF_WAIT_BEGIN;
-                    ok = mbar_wait(&fullA[sa], pha, abort_flag, a.status);
-                    PROF_WAIT_END;
-                }
-                {
-                    PROF_WAIT_BEGIN;
-                    if (ok) ok = mbar_wait(&fullB[sb], phb, abort_flag, a.status);
-                    PROF_WAIT2_END;
-                }
-                ok = __all_sync(0xffffffffu, ok);
-                if (!ok) break;
-                tc_fence_after();
-                if (lane == 0) {
-                    PROF_WAIT_BEGIN;
-                    const uint64_t db = make_desc_b(smem_u32(sB + sb * B_STAGE_BYTES));
-                    const uint32_t ta = tmem_a + sa * A_STAGE_COLS;
+        if (lane == 0) {
+            int tcount = 0;
+            bool ok = true;
+            const uint64_t db0 = make_desc_b(smem_u32(sB));
+            if ((2 * KB) % SB == 0) {
+                int pb = 0;                                        // parity of the B ring's current turn; the A ring's is 0, 1 in every turn
+                bool ready = false;                                // next stage's barriers already seen complete
+                for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x, ++tcount) {
+                    const Tile tl = a.tiles[t / MT];
+                    const int n_mma = (tl.nrows + 15) & ~15;
+                    const uint32_t idesc = make_idesc(n_mma);
+                    const int buf = tcount & 1;
+                    if (!mbar_try(&acc_empty[buf], ((tcount >> 1) & 1) ^ 1)) {
+                        PROF_WAIT_BEGIN;
+                        ok = mbar_wait(&acc_empty[buf], ((tcount >> 1) & 1) ^ 1, abort_flag, a.status);
+                        PROF_WAIT_END;
+                        if (!ok) break;
+                    }
+                    const uint32_t d_tmem = tmem_base + buf * BN_T;
+                    for (int ks0 = 0; ks0 < 2 * KB && ok; ks0 += SB) {
 #pragma unroll
-                    for (int j = 0; j < BKS / 16; ++j)             // K16 step j: A 8 columns on, B 32 bytes on
-                        tc_mma_ta(d_tmem, ta + 8 * j, db + (uint64_t)((j * 32) >> 4), idesc, (ks | j) ? 1u : 0u);
-                    tc_commit(&emptyB[sb]);                        // both stages reusable once these MMAs have read them
-                    tc_commit(&emptyA[sa]);
-                    PROF_WAIT3_END;
+                        for (int st = 0; st < SB; ++st) {
+                            const int sa = st % SA, pa = st / SA;
+                            if (!ready) {
+                                PROF_WAIT_BEGIN;
+                                ok = mbar_wait(&fullA[sa], pa, abort_flag, a.status) && mbar_wait(&fullB[st], pb, abort_flag, a.status);
+                                PROF_WAIT_END;
+                                if (!ok) break;
+                            }
+                            const int nst = (st + 1) % SB;
+                            const bool ready_next = mbar_try(&fullA[nst % SA], nst / SA) && mbar_try(&fullB[nst], nst ? pb : pb ^ 1);
+                            tc_fence_after();                      // the A stage was written with tcgen05.st by other threads
+                            const uint64_t db = db0 + (uint64_t)(st * (B_STAGE_BYTES >> 4));
+                            const uint32_t ta = tmem_a + sa * A_STAGE_COLS;
+#pragma unroll
+                            for (int j = 0; j < BKS / 16; ++j)     // K16 step j: A 8 columns on, B 32 bytes on
+                                tc_mma_ta(d_tmem, ta + 8 * j, db + (uint64_t)((j * 32) >> 4), idesc, (ks0 | st | j) ? 1u : 0u);
+                            tc_commit(&emptyB[st]);                // both stages reusable once these MMAs have read them
+                            tc_commit(&emptyA[sa]);
+                            ready = ready_next;
+                        }
+                        pb ^= 1;
+                    }
+                    if (ok) tc_commit(&acc_full[buf]);             // accumulator complete
                 }
-                __syncwarp();
-                if (++sb == SB) { sb = 0; phb ^= 1; }
-                if (++sa == SA) { sa = 0; pha ^= 1; }
+            } else {
+                int sb = 0, phb = 0, sa = 0, pha = 0;              // ring positions of the next stage to consume
+                for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x, ++tcount) {
+                    const Tile tl = a.tiles[t / MT];
+                    const int n_mma = (tl.nrows + 15) & ~15;
+                    const uint32_t idesc = make_idesc(n_mma);
+                    const int buf = tcount & 1;
+                    ok = mbar_wait(&acc_empty[buf], ((tcount >> 1) & 1) ^ 1, abort_flag, a.status);
+                    if (!ok) break;
+                    const uint32_t d_tmem = tmem_base + buf * BN_T;
+                    for (int ks = 0; ks < 2 * KB; ++ks) {
+                        if (!mbar_try(&fullA[sa], pha)) ok = mbar_wait(&fullA[sa], pha, abort_flag, a.status);
+                        if (ok && !mbar_try(&fullB[sb], phb)) ok = mbar_wait(&fullB[sb], phb, abort_flag, a.status);
+                        if (!ok) break;
+                        tc_fence_after();
+                        const uint64_t db = db0 + (uint64_t)(sb * (B_STAGE_BYTES >> 4));
+                        const uint32_t ta = tmem_a + sa * A_STAGE_COLS;
+#pragma unroll
+                        for (int j = 0; j < BKS / 16; ++j)
+                            tc_mma_ta(d_tmem, ta + 8 * j, db + (uint64_t)((j * 32) >> 4), idesc, (ks | j) ? 1u : 0u);
+                        tc_commit(&emptyB[sb]);
+                        tc_commit(&emptyA[sa]);
+                        if (++sb == SB) { sb = 0; phb ^= 1; }
+                        if (++sa == SA) { sa = 0; pha ^= 1; }
+                    }
+                    if (ok) tc_commit(&acc_full[buf]);
+                }
             }
-            if (ok && lane == 0) tc_commit(&acc_full[buf]);        // accumulator complete
-            __syncwarp();
         }
+        __syncwarp();
         PROF_REPORT("mma");
     } else if ((warp >= 4 && warp < 8) || (warp >= 16 && warp < 20)) {
         // ------------------------------------------------------------------ epilogue
