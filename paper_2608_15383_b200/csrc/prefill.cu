@@ -2,43 +2,29 @@
 // GEMMs per wave of Section 3.4 / Eq. 2 when every expert has many rows).
 //
 // Swap-AB: the WEIGHTS are the UMMA A operand (M = 128 rows = 8 consecutive 16-row panels of the
-// packed matrix), the TOKENS are the B operand (N <= 192 grouped rows), the accumulator D[128 x N]
+// packed matrix), the TOKENS are the B operand (N <= 256 grouped rows), the accumulator D[128 x N]
 // lives in TMEM (fp32, lane = weight row, column = token).  For gate/up the 8 panels are
 // gate p, up p, gate p+1, ... so one accumulator holds 64 intermediates' gate rows and up rows
 // 16 lanes apart: SwiGLU is one shuffle away in the epilogue.
 //
-// The dequantised weights never touch shared memory: the conversion warps write them into TENSOR MEMORY
-// (tcgen05.st) and the MMAs take A from there.  With A and B both in shared memory the kernel was bound by the
-// shared-memory data pipe (operand reads of the MMAs + the conversion warps' stores + the TMA writes asked for
-// about 190 B per clock of a 128 B per clock pipe: tensor pipe 45 % busy); A through tensor memory leaves the
-// token tile's write and its read.
-//
-// A persistent CTA (one per SM, 28 warps) is specialised by warp:
-//   warp 0        allocates TMEM, then one elected thread issues tcgen05.mma (4 x K16 per 64-wide stage, A from
-//                 TMEM, B through a shared-memory descriptor) and tcgen05.commit to the stage-empty /
-//                 accumulator-full mbarriers.
+// A persistent CTA (one per SM, 16 warps) is specialised by warp:
+//   warp 0        allocates TMEM, then one elected thread issues tcgen05.mma (8 x K16 per 128-wide
+//                 block) and tcgen05.commit to the stage-empty / accumulator-full mbarriers.
 //   warps 4-7,    epilogue (two groups, even / odd 32-column chunks): tcgen05.ld the accumulator (warp w
 //   16-19         reads TMEM lanes 32(w%4)..), SwiGLU -> BF16 activations, or routing weight -> fp32
-//                 pair buffer; two accumulators let the epilogue of tile i overlap the MMAs of tile i+1.
-//   warp 1        B producer: one thread issues one TMA tile load (cp.async.bulk.tensor.2d, 128-byte swizzle,
-//                 the tile's rows x 64 columns) per stage from the grouped activation matrix; completion is
-//                 counted in bytes on the stage's full barrier.  No multicast.
-//   warps 8-15,   A producers, one 16-row panel and one 64-wide k-half each (warp w owns TMEM lanes
-//   20-27         32(w%4) + 16((w/4)%2) ..+15): stream packed int4 (128-bit loads, two blocks ahead in registers),
-//                 dequantise to BF16 (shift/lop3 -> 128+u, subtract 136, multiply by the exactly split group
-//                 scale: one rounding) and store the 16 x 64 piece with one tcgen05.st.16x256b.x4: that shape
-//                 hands every lane exactly the cells its mma-fragment-ordered codes belong to, up to a fixed
-//                 permutation of K inside every 64 (below), which the token matrices are stored in as well.
-// TMEM columns: accumulators [0, 2 BN), A ring [2 BN, 2 BN + 32 SA).  The A ring (SA stages of 32 columns) and
-// the B ring (SB stages of shared memory) advance together, one stage of each per 64 of K.
-// Producers -> MMA through fullA / fullB mbarriers (tcgen05.wait::st + tcgen05.fence::before_thread_sync before
-// the A arrive), MMA -> producers through tcgen05.commit on emptyA / emptyB.
-//
-// K order.  Lane (q, c) of a conversion warp holds, for rows q and q + 8, the true k = 32 s + 8 c + (0..7) of the
-// stage (s = 0, 1); tcgen05.st.16x256b gives it the cells of positions 16 i + 4 c + (0..3), i = 0..3.  So position
-// P = 4 U + e of every 64 holds true k = 4 u + e with U = 8 (u / 8) + 4 (u % 2) + (u % 8) / 2.  Both B matrices
-// are written in that order: the grouped copy of the hidden rows by gather_rows_kernel, the activations by the
-// gate/up epilogue (perm64 below).  A sum over k does not care, as long as both operands agree.
+//                 pair buffer; two accumulators (2 x 256 columns) let the epilogue of tile i overlap
+//                 the MMAs of tile i+1.
+//   warp 1        B producer: one thread issues two TMA tile loads (cp.async.bulk.tensor.2d, 128-byte
+//                 swizzle, 256 rows x 64 columns each) per stage from the grouped activation matrix;
+//                 completion is counted in bytes on the stage's full barrier.  No multicast.
+//   warps 8-15,   A producers, one 16-row panel and one 64-wide k-half each: stream packed int4 (128-bit
+//   20-27         loads, two blocks ahead in registers), dequantise to BF16 (shift/lop3 -> 128+u, subtract 136,
+//                 multiply by the exactly split group scale: one rounding) and store the canonical no-swizzle K-major
+//                 core-matrix layout (k-chunk stride padded to 160 bytes: conflict-free stores).
+// Producers -> MMA through full[stage] mbarriers (generic-proxy writes are fenced with
+// fence.proxy.async before the arrive), MMA -> producers through tcgen05.commit on empty[stage].
+// The gate/up GEMM reads its tokens from a grouped copy of the hidden states (rows in plan order),
+// written once per call by gather_rows_kernel, so that both GEMMs load B with plain tiled TMA.
 // Every wait is bounded: on expiry the CTA raises EXMOE_ERR_TIMEOUT, all roles drain, TMEM is freed.
 #include <cuda.h>
 
@@ -53,37 +39,31 @@ namespace exmoe {
 namespace {
 
 constexpr int BM = 128;            // weight rows per tile
-constexpr int BN = 192;            // max grouped rows (tokens) per tile of the large-N kernel shape
-constexpr int BN_SMALL = 64;       // ... and of the small-N shape (a few dozen rows per expert)
+constexpr int BN = 256;            // max grouped rows (tokens) per tile of the large-N kernel shape
+constexpr int BN_SMALL = 64;       // ... and of the small-N shape (a few dozen rows per expert: four stages fit)
 constexpr int BK = 128;            // one packed block / one scale group
 constexpr int BKS = 64;            // K per ring stage = half a packed block (the half one dequantisation warp converts)
-constexpr int A_STAGE_COLS = BKS / 2;   // TMEM columns of one A stage (two BF16 per 32-bit cell)
-// B (tokens): TMA 128-byte swizzle; 64 columns x up to 192 rows of 128 B; 8-row atoms of 1024 B
+// A (dequantised weights): no swizzle; core matrix = 8 rows x 16 B; k-chunks 160 B apart (128 + 32 pad, so that
+// the 8 lanes of a quarter warp, 2 rows x 4 k-chunks, hit 8 different 16-byte bank groups), row groups 1280 B apart
+constexpr int A_LBO = 160;
+constexpr int A_SBO = (BKS / 8) * A_LBO;
+constexpr int A_STAGE_BYTES = 16 * A_SBO;      // 20 KB
+// B (tokens): TMA 128-byte swizzle; 64 columns x up to 256 rows of 128 B; 8-row atoms of 1024 B
 constexpr int B_SBO = 1024;
 constexpr int N_MAPS = 16;         // tensor maps per operand: boxes of 16, 32, ..., 256 rows
 constexpr int NUM_THREADS = 896;   // 28 warps: MMA, TMA, 2 idle, 4 + 4 epilogue, 8 + 8 dequant
 
-// position inside a 64-wide K group where true element w is stored (see "K order" above)
-__host__ __device__ __forceinline__ int perm64(int w) {
-    const int u = w >> 2;
-    return (((u & 8) | ((u & 1) << 2) | ((u & 7) >> 1)) << 2) | (w & 3);
-}
-
 struct Tile { int key, n0, nrows, pad; };
 
 #ifdef EXMOE_PREFILL_PROF
-#define PROF_DECL long long prof_t0 = clock64(), prof_wait = 0, prof_wait2 = 0, prof_wait3 = 0
+#define PROF_DECL long long prof_t0 = clock64(), prof_wait = 0
 #define PROF_WAIT_BEGIN long long prof_w0 = clock64()
 #define PROF_WAIT_END prof_wait += clock64() - prof_w0
-#define PROF_WAIT2_END prof_wait2 += clock64() - prof_w0
-#define PROF_WAIT3_END prof_wait3 += clock64() - prof_w0
-#define PROF_REPORT(name) if (blockIdx.x == 7 && lane == 0) printf("%s warp %d: total %lld wait %lld wait2 %lld wait3 %lld\n", name, warp, clock64() - prof_t0, prof_wait, prof_wait2, prof_wait3)
+#define PROF_REPORT(name) if (blockIdx.x == 7 && lane == 0) printf("%s warp %d: total %lld wait %lld\n", name, warp, clock64() - prof_t0, prof_wait)
 #else
 #define PROF_DECL
 #define PROF_WAIT_BEGIN
 #define PROF_WAIT_END
-#define PROF_WAIT2_END
-#define PROF_WAIT3_END
 #define PROF_REPORT(name)
 #endif
 
@@ -93,24 +73,14 @@ __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::
 __device__ __forceinline__ void tc_commit(uint64_t* bar) {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
-// D[tmem] (+)= A[tmem] x B[smem descriptor]; A: 128 lanes x 8 columns (K = 16 BF16, two per cell)
-__device__ __forceinline__ void tc_mma_ta(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+__device__ __forceinline__ void tc_mma(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
         "setp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
-        ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
         : "memory");
 }
-// 16 lanes x 32 columns: lane (q, c) of the warp gives, for i = 0..3, r[4i], r[4i+1] = row q, columns 8i + 2c, +1 and
-// r[4i+2], r[4i+3] = row q + 8, same columns
-__device__ __forceinline__ void tc_st_16x256b_x4(uint32_t taddr, const uint32_t (&r)[16]) {
-    asm volatile("tcgen05.st.sync.aligned.16x256b.x4.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16};"
-                 ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]),
-                   "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15])
-                 : "memory");
-}
-__device__ __forceinline__ void tc_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tc_ld32(uint32_t taddr, uint32_t (&r)[32]) {
     asm volatile(
         "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
@@ -123,7 +93,15 @@ __device__ __forceinline__ void tc_ld32(uint32_t taddr, uint32_t (&r)[32]) {
 }
 __device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
-// shared-memory matrix descriptor, K-major, version 1 (sm_100)
+// shared-memory matrix descriptors, K-major, version 1 (sm_100)
+__device__ __forceinline__ uint64_t make_desc_a(uint32_t saddr) {            // no swizzle
+    uint64_t d = 0;
+    d |= (uint64_t)((saddr >> 4) & 0x3fff);
+    d |= (uint64_t)((A_LBO >> 4) & 0x3fff) << 16;
+    d |= (uint64_t)((A_SBO >> 4) & 0x3fff) << 32;
+    d |= (uint64_t)1 << 46;
+    return d;
+}
 __device__ __forceinline__ uint64_t make_desc_b(uint32_t saddr) {            // 128-byte swizzle
     uint64_t d = 0;
     d |= (uint64_t)((saddr >> 4) & 0x3fff);
@@ -191,29 +169,72 @@ struct PrefillArgs {
     int* status;
 };
 
-// BN_T = token rows per tile (192 or 64), SB = depth of the token ring in shared memory, SA = depth of the weight
-// ring in tensor memory.  One stage of each holds 64 of K: half a packed block of the weights (the half one
-// dequantisation warp converts) and a [rows x 64] box of tokens.  The round trip of a token stage (MMAs complete ->
-// commit -> box fetched from L2 -> MMA issuer wakes) is 2000-3000 cycles, several times what the stage's MMAs take,
-// so the token ring is as deep as shared memory allows.  The token box holds exactly the tile's rows (rounded up to
-// 16): `maps` is a family of tensor maps over the same matrix with boxes of 16, 32, ..., 256 rows.
-template <bool GATEUP, int BN_T, int SB, int SA>
+// Epilogue of one tile by one warp: TMEM lanes 32e .. 32e+31 of the accumulator at `tmem_acc`, the 32-column chunks
+// c0 = first, first + 64, ...  Gate/up: SwiGLU -> BF16 activations; down: routing weight -> fp32 pair buffer.
+template <bool GATEUP>
+__device__ __forceinline__ void epilogue_tile(const PrefillArgs& a, const Tile& tl, int mt, int e, int first, int lane,
+                                              uint32_t tmem_acc, const int32_t* __restrict__ offsets,
+                                              __nv_bfloat16* __restrict__ act_out, const float* __restrict__ topk_w,
+                                              float* __restrict__ y_out) {
+    const int row0 = offsets[tl.key] + tl.n0;
+    const uint32_t taddr = tmem_acc + ((uint32_t)(32 * e) << 16);
+    for (int c0 = first; c0 < tl.nrows; c0 += 64) {
+        uint32_t v[32];
+        tc_ld32(taddr + c0, v);
+        tc_wait_ld();
+        if (GATEUP) {
+            // lanes 0-15: gate rows, lanes 16-31: up rows of the same 16 intermediates
+            const int interm = (mt * 4 + e) * 16 + (lane & 15);
+#pragma unroll
+            for (int j = 0; j < 16; ++j) {
+                const uint32_t send = (lane < 16) ? v[j + 16] : v[j];
+                const uint32_t recv = __shfl_xor_sync(0xffffffffu, send, 16);
+                const int col = (lane < 16) ? j : j + 16;
+                const float g = __uint_as_float((lane < 16) ? v[j] : recv);
+                const float u = __uint_as_float((lane < 16) ? recv : v[j + 16]);
+                const int n = c0 + col;
+                if (n < tl.nrows)
+                    act_out[(size_t)(row0 + n) * a.I + interm] = __float2bfloat16_rn(__fdividef(g, 1.f + __expf(-g)) * u);
+            }
+        } else {
+            const int h = mt * BM + 32 * e + lane;
+            int my_pair = 0;                               // lane j holds pair and weight of column c0 + j
+            float my_w = 0.f;
+            if (c0 + lane < tl.nrows) {
+                my_pair = a.perm[row0 + c0 + lane];
+                my_w = topk_w[my_pair];
+            }
+#pragma unroll
+            for (int j = 0; j < 32; ++j) {
+                const int pair = __shfl_sync(0xffffffffu, my_pair, j);
+                const float wj = __shfl_sync(0xffffffffu, my_w, j);
+                if (c0 + j < tl.nrows) y_out[(size_t)pair * a.H + h] = wj * __uint_as_float(v[j]);
+            }
+        }
+    }
+}
+
+// BN_T = token rows per tile (256 or 64), STAGES = ring depth.  One ring stage holds 64 of K: half a packed block
+// of the weights (the half one dequantisation warp converts) and a [rows x 64] box of tokens.  The round trip of one
+// stage (MMAs complete -> commit -> token box fetched from L2, weights converted -> MMA issuer wakes) is 2000-3000
+// cycles, far more than the stage's MMAs take, so the ring depth sets the rate: 64-wide stages give the large shape
+// four of them and the small shape eight in the same shared memory.  The token box holds exactly the tile's rows
+// (rounded up to 16): `maps` is a family of tensor maps over the same matrix with boxes of 16, 32, ..., 256 rows.
+template <bool GATEUP, int BN_T, int STAGES>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 prefill_gemm_kernel(PrefillArgs a, const CUtensorMap* __restrict__ maps, __nv_bfloat16* __restrict__ act_out,
                     const float* __restrict__ topk_w, const int32_t* __restrict__ offsets, float* __restrict__ y_out) {
-    static_assert(2 * BN_T + SA * A_STAGE_COLS <= 512, "accumulators and the A ring share the 512 TMEM columns");
     extern __shared__ unsigned char smem_raw[];
     unsigned char* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);   // swizzled tiles need 1 KB alignment
     constexpr int B_STAGE_BYTES = BN_T * 128;                     // BN_T rows x 64 columns
-    unsigned char* sB = smem;                                     // [SB][B_STAGE_BYTES]
-    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + SB * B_STAGE_BYTES);
-    uint64_t* fullB = bars;                         // [SB]  TMA -> MMA
-    uint64_t* emptyB = bars + SB;                   // [SB]  MMA -> TMA thread (tcgen05.commit)
-    uint64_t* fullA = bars + 2 * SB;                // [SA]  conversion warps -> MMA
-    uint64_t* emptyA = bars + 2 * SB + SA;          // [SA]  MMA -> conversion warps (tcgen05.commit)
-    uint64_t* acc_full = bars + 2 * SB + 2 * SA;    // [2]   MMA -> epilogue
-    uint64_t* acc_empty = acc_full + 2;             // [2]   epilogue -> MMA (8 warp arrivals)
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_empty + 2);
+    unsigned char* sB = smem;                                     // [STAGES][B_STAGE_BYTES]
+    unsigned char* sA = smem + STAGES * B_STAGE_BYTES;            // [STAGES][20 KB]
+    uint64_t* bars = reinterpret_cast<uint64_t*>(sA + STAGES * A_STAGE_BYTES);
+    uint64_t* full = bars;                          // [STAGES]  producers -> MMA
+    uint64_t* empty = bars + STAGES;                // [STAGES]  MMA -> producers (tcgen05.commit)
+    uint64_t* acc_full = bars + 2 * STAGES;         // [2]       MMA -> epilogue
+    uint64_t* acc_empty = bars + 2 * STAGES + 2;    // [2]       epilogue -> MMA (8 warp arrivals)
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * STAGES + 4);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -224,13 +245,9 @@ prefill_gemm_kernel(PrefillArgs a, const CUtensorMap* __restrict__ maps, __nv_bf
     const int total_tiles = (*a.n_tiles) * MT;
 
     if (tid == 0) {
-        for (int s = 0; s < SB; ++s) {
-            mbar_init(&fullB[s], 1);          // the TMA thread's expect_tx arrive (+ the bytes)
-            mbar_init(&emptyB[s], 1);
-        }
-        for (int s = 0; s < SA; ++s) {
-            mbar_init(&fullA[s], 8);          // the 8 conversion warps of this k-half
-            mbar_init(&emptyA[s], 1);
+        for (int s = 0; s < STAGES; ++s) {
+            mbar_init(&full[s], 9);           // the 8 A-producer warps of this k-half + the TMA thread's expect_tx arrive
+            mbar_init(&empty[s], 1);
         }
         for (int b = 0; b < 2; ++b) {
             mbar_init(&acc_full[b], 1);
@@ -247,7 +264,6 @@ prefill_gemm_kernel(PrefillArgs a, const CUtensorMap* __restrict__ maps, __nv_bf
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
-    const uint32_t tmem_a = tmem_base + 2 * BN_T;                  // first column of the A ring
 
     if (warp == 0) {
         // ------------------------------------------------------------------ MMA issuer
@@ -257,18 +273,17 @@ prefill_gemm_kernel(PrefillArgs a, const CUtensorMap* __restrict__ maps, __nv_bf
         // each instruction takes many cycles to issue (measured alone: the same four MMAs per stage run at N / 2
         // cycles each with compile-time operands, at 150-160 cycles each, whatever N, behind run-time ring
         // arithmetic and a barrier test).  So the ring is unrolled (stage index, barrier addresses and operand offsets
-        // are compile-time constants) and the NEXT stage's barriers are tested before this stage's MMAs are issued,
+        // are compile-time constants) and the NEXT stage's barrier is tested before this stage's MMAs are issued,
         // the answer being read after them.  Shapes whose stage count per tile is not a multiple of the ring depth
         // take the plain loop.
-        static_assert(SB == 2 * SA, "the unrolled issue loop walks the A ring twice per turn of the B ring");
         PROF_DECL;
         if (lane == 0) {
             int tcount = 0;
             bool ok = true;
-            const uint64_t db0 = make_desc_b(smem_u32(sB));
-            if ((2 * KB) % SB == 0) {
-                int pb = 0;                                        // parity of the B ring's current turn; the A ring's is 0, 1 in every turn
-                bool ready = false;                                // next stage's barriers already seen complete
+            const uint64_t da0 = make_desc_a(smem_u32(sA)), db0 = make_desc_b(smem_u32(sB));
+            if ((2 * KB) % STAGES == 0) {
+                int ph = 0;                                        // parity of the ring's current turn
+                bool ready = false;                                // next stage's barrier already seen complete
                 for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x, ++tcount) {
                     const Tile tl = a.tiles[t / MT];
                     const int n_mma = (tl.nrows + 15) & ~15;
@@ -280,35 +295,33 @@ prefill_gemm_kernel(PrefillArgs a, const CUtensorMap* __restrict__ maps, __nv_bf
                         PROF_WAIT_END;
                         if (!ok) break;
                     }
+                    tc_fence_after();
                     const uint32_t d_tmem = tmem_base + buf * BN_T;
-                    for (int ks0 = 0; ks0 < 2 * KB && ok; ks0 += SB) {
+                    for (int ks0 = 0; ks0 < 2 * KB && ok; ks0 += STAGES) {
 #pragma unroll
-                        for (int st = 0; st < SB; ++st) {
-                            const int sa = st % SA, pa = st / SA;
+                        for (int st = 0; st < STAGES; ++st) {
                             if (!ready) {
                                 PROF_WAIT_BEGIN;
-                                ok = mbar_wait(&fullA[sa], pa, abort_flag, a.status) && mbar_wait(&fullB[st], pb, abort_flag, a.status);
+                                ok = mbar_wait(&full[st], ph, abort_flag, a.status);
                                 PROF_WAIT_END;
                                 if (!ok) break;
                             }
-                            const int nst = (st + 1) % SB;
-                            const bool ready_next = mbar_try(&fullA[nst % SA], nst / SA) && mbar_try(&fullB[nst], nst ? pb : pb ^ 1);
-                            tc_fence_after();                      // the A stage was written with tcgen05.st by other threads
+                            const int nst = (st + 1) % STAGES;
+                            const bool ready_next = mbar_try(&full[nst], nst ? ph : ph ^ 1);
+                            const uint64_t da = da0 + (uint64_t)(st * (A_STAGE_BYTES >> 4));
                             const uint64_t db = db0 + (uint64_t)(st * (B_STAGE_BYTES >> 4));
-                            const uint32_t ta = tmem_a + sa * A_STAGE_COLS;
 #pragma unroll
-                            for (int j = 0; j < BKS / 16; ++j)     // K16 step j: A 8 columns on, B 32 bytes on
-                                tc_mma_ta(d_tmem, ta + 8 * j, db + (uint64_t)((j * 32) >> 4), idesc, (ks0 | st | j) ? 1u : 0u);
-                            tc_commit(&emptyB[st]);                // both stages reusable once these MMAs have read them
-                            tc_commit(&emptyA[sa]);
+                            for (int j = 0; j < BKS / 16; ++j)     // K16 step j: A two k-chunks on, B 32 bytes on
+                                tc_mma(d_tmem, da + (uint64_t)(j * 2 * A_LBO >> 4), db + (uint64_t)((j * 32) >> 4), idesc, (ks0 | st | j) ? 1u : 0u);
+                            tc_commit(&empty[st]);                 // stage reusable once these MMAs have read it
                             ready = ready_next;
                         }
-                        pb ^= 1;
+                        ph ^= 1;
                     }
                     if (ok) tc_commit(&acc_full[buf]);             // accumulator complete
                 }
             } else {
-                int sb = 0, phb = 0, sa = 0, pha = 0;              // ring positions of the next stage to consume
+                int s = 0, ph = 0;                                 // ring position of the next stage to consume
                 for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x, ++tcount) {
                     const Tile tl = a.tiles[t / MT];
                     const int n_mma = (tl.nrows + 15) & ~15;
@@ -316,21 +329,18 @@ prefill_gemm_kernel(PrefillArgs a, const CUtensorMap* __restrict__ maps, __nv_bf
                     const int buf = tcount & 1;
                     ok = mbar_wait(&acc_empty[buf], ((tcount >> 1) & 1) ^ 1, abort_flag, a.status);
                     if (!ok) break;
+                    tc_fence_after();
                     const uint32_t d_tmem = tmem_base + buf * BN_T;
                     for (int ks = 0; ks < 2 * KB; ++ks) {
-                        if (!mbar_try(&fullA[sa], pha)) ok = mbar_wait(&fullA[sa], pha, abort_flag, a.status);
-                        if (ok && !mbar_try(&fullB[sb], phb)) ok = mbar_wait(&fullB[sb], phb, abort_flag, a.status);
+                        if (!mbar_try(&full[s], ph)) ok = mbar_wait(&full[s], ph, abort_flag, a.status);
                         if (!ok) break;
-                        tc_fence_after();
-                        const uint64_t db = db0 + (uint64_t)(sb * (B_STAGE_BYTES >> 4));
-                        const uint32_t ta = tmem_a + sa * A_STAGE_COLS;
+                        const uint64_t da = da0 + (uint64_t)(s * (A_STAGE_BYTES >> 4));
+                        const uint64_t db = db0 + (uint64_t)(s * (B_STAGE_BYTES >> 4));
 #pragma unroll
                         for (int j = 0; j < BKS / 16; ++j)
-                            tc_mma_ta(d_tmem, ta + 8 * j, db + (uint64_t)((j * 32) >> 4), idesc, (ks | j) ? 1u : 0u);
-                        tc_commit(&emptyB[sb]);
-                        tc_commit(&emptyA[sa]);
-                        if (++sb == SB) { sb = 0; phb ^= 1; }
-                        if (++sa == SA) { sa = 0; pha ^= 1; }
+                            tc_mma(d_tmem, da + (uint64_t)(j * 2 * A_LBO >> 4), db + (uint64_t)((j * 32) >> 4), idesc, (ks | j) ? 1u : 0u);
+                        tc_commit(&empty[s]);
+                        if (++s == STAGES) { s = 0; ph ^= 1; }
                     }
                     if (ok) tc_commit(&acc_full[buf]);
                 }
@@ -355,44 +365,7 @@ prefill_gemm_kernel(PrefillArgs a, const CUtensorMap* __restrict__ maps, __nv_bf
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
             tc_fence_after();
-            const int row0 = offsets[tl.key] + tl.n0;
-            const uint32_t taddr = tmem_base + buf * BN_T + ((uint32_t)(32 * e) << 16);
-            for (int c0 = odd; c0 < tl.nrows; c0 += 64) {
-                uint32_t v[32];
-                tc_ld32(taddr + c0, v);
-                tc_wait_ld();
-                if (GATEUP) {
-                    // lanes 0-15: gate rows, lanes 16-31: up rows of the same 16 intermediates; the activation row is
-                    // the down GEMM's token operand: stored in the K order of that kernel's weights (perm64)
-                    const int interm = (mt * 4 + e) * 16 + (lane & 15);
-                    const int pos = (interm & ~63) | perm64(interm & 63);
-#pragma unroll
-                    for (int j = 0; j < 16; ++j) {
-                        const uint32_t send = (lane < 16) ? v[j + 16] : v[j];
-                        const uint32_t recv = __shfl_xor_sync(0xffffffffu, send, 16);
-                        const int col = (lane < 16) ? j : j + 16;
-                        const float g = __uint_as_float((lane < 16) ? v[j] : recv);
-                        const float u = __uint_as_float((lane < 16) ? recv : v[j + 16]);
-                        const int n = c0 + col;
-                        if (n < tl.nrows)
-                            act_out[(size_t)(row0 + n) * a.I + pos] = __float2bfloat16_rn(__fdividef(g, 1.f + __expf(-g)) * u);
-                    }
-                } else {
-                    const int h = mt * BM + 32 * e + lane;
-                    int my_pair = 0;                               // lane j holds pair and weight of column c0 + j
-                    float my_w = 0.f;
-                    if (c0 + lane < tl.nrows) {
-                        my_pair = a.perm[row0 + c0 + lane];
-                        my_w = topk_w[my_pair];
-                    }
-#pragma unroll
-                    for (int j = 0; j < 32; ++j) {
-                        const int pair = __shfl_sync(0xffffffffu, my_pair, j);
-                        const float wj = __shfl_sync(0xffffffffu, my_w, j);
-                        if (c0 + j < tl.nrows) y_out[(size_t)pair * a.H + h] = wj * __uint_as_float(v[j]);
-                    }
-                }
-            }
+            epilogue_tile<GATEUP>(a, tl, mt, e, odd, lane, tmem_base + buf * BN_T, offsets, act_out, topk_w, y_out);
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(&acc_empty[buf]);
@@ -411,27 +384,26 @@ prefill_gemm_kernel(PrefillArgs a, const CUtensorMap* __restrict__ maps, __nv_bf
             for (int ks = 0; ks < 2 * KB; ++ks) {
                 {
                     PROF_WAIT_BEGIN;
-                    ok = mbar_wait(&emptyB[s], ph ^ 1, abort_flag, a.status);
+                    ok = mbar_wait(&empty[s], ph ^ 1, abort_flag, a.status);
                     PROF_WAIT_END;
                 }
                 ok = __all_sync(0xffffffffu, ok);
                 if (!ok) break;
                 if (lane == 0) {
-                    mbar_expect_tx(&fullB[s], n_mma * 128);
-                    tma_load_2d(smem_u32(sB + s * B_STAGE_BYTES), map, ks * BKS, row0, &fullB[s]);
+                    mbar_expect_tx(&full[s], n_mma * 128);
+                    tma_load_2d(smem_u32(sB + s * B_STAGE_BYTES), map, ks * BKS, row0, &full[s]);
                 }
                 __syncwarp();
-                if (++s == SB) { s = 0; ph ^= 1; }
+                if (++s == STAGES) { s = 0; ph ^= 1; }
             }
         }
         PROF_REPORT("B producer");
     } else if (warp >= 8 && !(warp >= 16 && warp < 20)) {
-        // ------------------------------------------------------------------ A producers (dequantise into TMEM)
-        const int pw = 2 * (warp & 3) + ((warp >> 2) & 1);         // panel of the tile: TMEM lanes 16 pw .. 16 pw + 15,
-                                                                   // inside the lane quarter (warp % 4) this warp may access
+        // ------------------------------------------------------------------ A producers (dequantise)
+        const int pw = warp & 7;                                   // panel of the tile = 8-row groups 2*pw, 2*pw+1
         const int hh = warp >= 20 ? 1 : 0;                         // 64-wide k-half of every block = every second stage
-        const int q = lane >> 2;
-        int s = hh % SA, ph = 0;                                   // ring position of this warp's next stage (2 * blocks + hh)
+        const int q = lane >> 2, c = lane & 3;
+        int s = hh % STAGES, ph = 0;                               // ring position of this warp's next stage (2 * blocks + hh)
         bool ok = true;
         PROF_DECL;
         for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
@@ -461,34 +433,30 @@ prefill_gemm_kernel(PrefillArgs a, const CUtensorMap* __restrict__ maps, __nv_bf
                         w[(u + nx_off) % PF] = ldg_stream128(blk + hh * 512 + lane * 16);
                         sc[(u + nx_off) % PF] = ldg_stream32(blk + kCodeBytes + q * 4);
                     }
-                    // convert first (registers only), then wait for the stage to be free
-                    const __half2 sh = *reinterpret_cast<const __half2*>(&sc[u]);
-                    const ScaleSplit s_lo = split_scale(__low2float(sh));                 // row q
-                    const ScaleSplit s_hi = split_scale(__high2float(sh));                // row q + 8
-                    // words: x = row q, k 8c.. ; y = row q + 8, k 8c.. ; z = row q, k 32 + 8c.. ; w = row q + 8, k 32 + 8c..
-                    const uint4 x0 = dequant_word(w[u].x, s_lo), x1 = dequant_word(w[u].y, s_hi);
-                    const uint4 x2 = dequant_word(w[u].z, s_lo), x3 = dequant_word(w[u].w, s_hi);
-                    const uint32_t r[16] = {x0.x, x0.y, x1.x, x1.y, x0.z, x0.w, x1.z, x1.w,
-                                            x2.x, x2.y, x3.x, x3.y, x2.z, x2.w, x3.z, x3.w};
                     {
                         PROF_WAIT_BEGIN;
-                        ok = mbar_wait(&emptyA[s], ph ^ 1, abort_flag, a.status);
+                        ok = mbar_wait(&empty[s], ph ^ 1, abort_flag, a.status);
                         PROF_WAIT_END;
                     }
                     ok = __all_sync(0xffffffffu, ok);
                     if (!ok) break;
-                    tc_fence_after();
-                    {
-                        PROF_WAIT_BEGIN;
-                        tc_st_16x256b_x4(tmem_a + s * A_STAGE_COLS + ((uint32_t)(16 * pw) << 16), r);
-                        tc_wait_st();
-                        PROF_WAIT2_END;
+                    unsigned char* dst = sA + s * A_STAGE_BYTES;
+                    const __half2 sh = *reinterpret_cast<const __half2*>(&sc[u]);
+                    const ScaleSplit s_lo = split_scale(__low2float(sh));                 // row q
+                    const ScaleSplit s_hi = split_scale(__high2float(sh));                // row q + 8
+                    const uint32_t words[4] = {w[u].x, w[u].y, w[u].z, w[u].w};
+#pragma unroll
+                    for (int wi = 0; wi < 4; ++wi) {
+                        const int r = wi & 1, set = wi >> 1;
+                        const int kc = 4 * set + c;                                       // 16-byte k-chunk of the stage
+                        const uint4 val = dequant_word(words[wi], r ? s_hi : s_lo);
+                        *reinterpret_cast<uint4*>(dst + (2 * pw + r) * A_SBO + kc * A_LBO + q * 16) = val;
                     }
-                    tc_fence_before();
+                    fence_proxy_async();
                     __syncwarp();
-                    if (lane == 0) mbar_arrive(&fullA[s]);
+                    if (lane == 0) mbar_arrive(&full[s]);
                     s += 2;                                        // this warp's next stage is two on
-                    if (s >= SA) { s -= SA; ph ^= 1; }
+                    if (s >= STAGES) { s -= STAGES; ph ^= 1; }
                 }
                 if (!ok) break;
             }
@@ -501,6 +469,270 @@ prefill_gemm_kernel(PrefillArgs a, const CUtensorMap* __restrict__ maps, __nv_bf
     __syncthreads();
     tc_fence_after();
     if (warp == 0) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512));
+}
+
+// ---------------------------------------------------------------------------------------------------------------
+// The same GEMM on CTA PAIRS (tcgen05 cta_group::2): one MMA of M = 256 weight rows x N <= 256 tokens spans two SMs.
+// CTA r of the pair dequantises the 128 weight rows of m-tile 2 mp + r into ITS shared memory and fetches HALF of the
+// token tile (rows r N/2 .. (r+1) N/2); the tensor cores of both SMs read both halves.  Per SM that halves the token
+// bytes written into and read from shared memory, which is what bounds the one-CTA kernel at 256-row tiles (its MMA
+// operand reads, dequantisation stores and TMA writes ask for ~190 B per clock of a 128 B per clock pipe), and one
+// thread issues for two SMs.  Stage = one packed block (128 of K): 40 KB of weights + two [N/2 x 64] token boxes.
+//   CTA 0, warp 0: waits for its own stage (full) and the peer's (full_peer, which the peer's warp 0 relays), issues
+//                  8 MMAs and one tcgen05.commit that arrives on empty[s] of BOTH CTAs (.multicast::cluster on the
+//                  commit only; every load is a plain TMA load of this GPU's memory into the issuing CTA).
+//   CTA 1, warp 0: relay: waits for its CTA's full[s], arrives on CTA 0's full_peer[s].
+//   epilogue warps of both CTAs read their own TMEM (lanes = their 128 weight rows); the peer's arrive on CTA 0's
+//   acc_empty through the cluster's shared-memory window.
+// All waits are bounded as in the one-CTA kernel; the two CTAs leave together through a cluster barrier.
+constexpr int P_STAGES = 3;
+constexpr int PA_SBO = 16 * A_LBO;                 // 16 k-chunks of 160 B per 8-row group
+constexpr int PA_STAGE_BYTES = 16 * PA_SBO;        // 40 KB
+constexpr int PB_HALF_BYTES = 128 * 128;           // up to 128 rows x 64 columns
+constexpr int PB_STAGE_BYTES = 2 * PB_HALF_BYTES;  // 32 KB
+
+__device__ __forceinline__ uint64_t make_desc_a_pair(uint32_t saddr) {       // no swizzle, 128-wide stage
+    uint64_t d = 0;
+    d |= (uint64_t)((saddr >> 4) & 0x3fff);
+    d |= (uint64_t)((A_LBO >> 4) & 0x3fff) << 16;
+    d |= (uint64_t)((PA_SBO >> 4) & 0x3fff) << 32;
+    d |= (uint64_t)1 << 46;
+    return d;
+}
+__device__ __forceinline__ void tc_mma_pair(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+// arrives (once the MMAs issued so far are complete) on the barrier at this offset in both CTAs of the pair
+__device__ __forceinline__ void tc_commit_pair(uint64_t* bar) {
+    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+                 ::"r"(smem_u32(bar)), "h"((uint16_t)3) : "memory");
+}
+__device__ __forceinline__ void cluster_sync_all() {
+    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// instruction descriptor of the pair MMA: D fp32, A/B BF16, both K-major, M = 256, N = n
+__device__ __forceinline__ uint32_t make_idesc_pair(int n) {
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(256 >> 4) << 24);
+}
+
+template <bool GATEUP>
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NUM_THREADS, 1)
+prefill_pair_gemm_kernel(PrefillArgs a, const CUtensorMap* __restrict__ maps8, __nv_bfloat16* __restrict__ act_out,
+                         const float* __restrict__ topk_w, const int32_t* __restrict__ offsets, float* __restrict__ y_out) {
+    extern __shared__ unsigned char smem_raw[];
+    unsigned char* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);   // the same offset in both CTAs
+    unsigned char* sB = smem;                                     // [P_STAGES][32 KB]
+    unsigned char* sA = smem + P_STAGES * PB_STAGE_BYTES;         // [P_STAGES][40 KB]
+    uint64_t* bars = reinterpret_cast<uint64_t*>(sA + P_STAGES * PA_STAGE_BYTES);
+    uint64_t* full = bars;                          // [P_STAGES]  this CTA's producers -> warp 0
+    uint64_t* empty = bars + P_STAGES;              // [P_STAGES]  MMA -> producers of both CTAs (multicast commit)
+    uint64_t* full_peer = bars + 2 * P_STAGES;      // [P_STAGES]  CTA 1's relay -> CTA 0's MMA issuer
+    uint64_t* acc_full = bars + 3 * P_STAGES;       // [2]         MMA -> epilogues of both CTAs (multicast commit)
+    uint64_t* acc_empty = acc_full + 2;             // [2]         epilogues of both CTAs -> CTA 0's MMA issuer (16 arrivals)
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_empty + 2);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    uint32_t rank;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(rank));
+    const int pair_id = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
+    const int K = GATEUP ? a.H : a.I;
+    const int KB = K / BK;
+    const int MP = (GATEUP ? 2 * a.I : a.H) / (2 * BM);           // pairs of m-tiles of the packed matrix
+    const size_t w13_bytes = matrix_bytes(2 * a.I, a.H);
+    const int total_tiles = (*a.n_tiles) * MP;
+
+    if (tid == 0) {
+        for (int s = 0; s < P_STAGES; ++s) {
+            mbar_init(&full[s], 17);          // 16 A-producer warps + the TMA thread's expect_tx arrive
+            mbar_init(&empty[s], 1);
+            mbar_init(&full_peer[s], 1);
+        }
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(&acc_full[b], 1);
+            mbar_init(&acc_empty[b], 16);     // 8 epilogue warps of each CTA
+        }
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 0) {
+        asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(512));
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::);
+    }
+    tc_fence_before();
+    __syncthreads();
+    cluster_sync_all();                       // the peer's barriers exist before anything arrives on them
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    if (warp == 0 && rank == 0) {
+        // ------------------------------------------------------------------ MMA issuer of the pair (one thread)
+        if (lane == 0) {
+            int s = 0, ph = 0, tcount = 0;
+            bool ok = true;
+            const uint64_t da0 = make_desc_a_pair(smem_u32(sA)), db0 = make_desc_b(smem_u32(sB));
+            for (int t = pair_id; t < total_tiles && ok; t += n_pairs, ++tcount) {
+                const Tile tl = a.tiles[t / MP];
+                const int n_mma = (tl.nrows + 15) & ~15;
+                const uint32_t idesc = make_idesc_pair(n_mma);
+                const int buf = tcount & 1;
+                ok = mbar_wait<true>(&acc_empty[buf], ((tcount >> 1) & 1) ^ 1, abort_flag, a.status);
+                if (!ok) break;
+                tc_fence_after();
+                const uint32_t d_tmem = tmem_base + buf * BN;
+                for (int kb = 0; kb < KB; ++kb) {
+                    if (!mbar_try(&full[s], ph)) ok = mbar_wait(&full[s], ph, abort_flag, a.status);
+                    if (ok && !mbar_try_cluster(&full_peer[s], ph)) ok = mbar_wait<true>(&full_peer[s], ph, abort_flag, a.status);
+                    if (!ok) break;
+                    const uint64_t da = da0 + (uint64_t)(s * (PA_STAGE_BYTES >> 4));
+                    const uint64_t db = db0 + (uint64_t)(s * (PB_STAGE_BYTES >> 4));
+#pragma unroll
+                    for (int j = 0; j < BK / 16; ++j) {            // K16 step j: A two k-chunks on, B 32 bytes on in its half
+                        const uint64_t aj = da + (uint64_t)(j * 2 * A_LBO >> 4);
+                        const uint64_t bj = db + (uint64_t)(((j >> 2) * PB_HALF_BYTES + (j & 3) * 32) >> 4);
+                        tc_mma_pair(d_tmem, aj, bj, idesc, (kb | j) ? 1u : 0u);
+                    }
+                    tc_commit_pair(&empty[s]);                     // stage reusable in both CTAs once these MMAs have read it
+                    if (++s == P_STAGES) { s = 0; ph ^= 1; }
+                }
+                if (ok) tc_commit_pair(&acc_full[buf]);            // accumulators of both CTAs complete
+            }
+        }
+        __syncwarp();
+    } else if (warp == 0) {
+        // ------------------------------------------------------------------ relay (CTA 1): stage full here -> tell CTA 0
+        int s = 0, ph = 0;
+        bool ok = true;
+        for (int t = pair_id; t < total_tiles && ok; t += n_pairs) {
+            for (int kb = 0; kb < KB; ++kb) {
+                ok = mbar_wait(&full[s], ph, abort_flag, a.status);
+                ok = __all_sync(0xffffffffu, ok);
+                if (!ok) break;
+                if (lane == 0) {
+                    fence_proxy_async();
+                    mbar_arrive_remote(&full_peer[s], 0);
+                }
+                __syncwarp();
+                if (++s == P_STAGES) { s = 0; ph ^= 1; }
+            }
+        }
+    } else if ((warp >= 4 && warp < 8) || (warp >= 16 && warp < 20)) {
+        // ------------------------------------------------------------------ epilogue (own 128 weight rows)
+        const int e = warp & 3;
+        const int odd = warp >= 16 ? 32 : 0;
+        int tcount = 0;
+        bool ok = true;
+        for (int t = pair_id; t < total_tiles && ok; t += n_pairs, ++tcount) {
+            const Tile tl = a.tiles[t / MP];
+            const int mt = 2 * (t % MP) + (int)rank;
+            const int buf = tcount & 1;
+            ok = mbar_wait(&acc_full[buf], (tcount >> 1) & 1, abort_flag, a.status);
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) break;
+            tc_fence_after();
+            epilogue_tile<GATEUP>(a, tl, mt, e, odd, lane, tmem_base + buf * BN, offsets, act_out, topk_w, y_out);
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) {
+                if (rank == 0) mbar_arrive(&acc_empty[buf]);
+                else mbar_arrive_remote(&acc_empty[buf], 0);
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------------ B producer: this CTA's half of the token tile
+        int s = 0, ph = 0;
+        bool ok = true;
+        for (int t = pair_id; t < total_tiles && ok; t += n_pairs) {
+            const Tile tl = a.tiles[t / MP];
+            const int n_half = ((tl.nrows + 15) & ~15) >> 1;       // multiple of 8: whole swizzle atoms
+            const int row0 = offsets[tl.key] + tl.n0 + (int)rank * n_half;
+            const CUtensorMap* map = maps8 + (n_half / 8 - 1);
+            for (int kb = 0; kb < KB; ++kb) {
+                ok = mbar_wait(&empty[s], ph ^ 1, abort_flag, a.status);
+                ok = __all_sync(0xffffffffu, ok);
+                if (!ok) break;
+                if (lane == 0) {
+                    const uint32_t dst = smem_u32(sB + s * PB_STAGE_BYTES);
+                    mbar_expect_tx(&full[s], 2 * n_half * 128);
+                    tma_load_2d(dst, map, kb * BK, row0, &full[s]);                       // columns kb*128 .. +63
+                    tma_load_2d(dst + PB_HALF_BYTES, map, kb * BK + 64, row0, &full[s]);
+                }
+                __syncwarp();
+                if (++s == P_STAGES) { s = 0; ph ^= 1; }
+            }
+        }
+    } else if (warp >= 8 && !(warp >= 16 && warp < 20)) {
+        // ------------------------------------------------------------------ A producers (dequantise this CTA's m-tile)
+        const int pw = warp & 7;                                   // panel of the tile = 8-row groups 2*pw, 2*pw+1
+        const int hh = warp >= 20 ? 1 : 0;                         // 64-wide k-half of every block
+        const int q = lane >> 2, c = lane & 3;
+        int s = 0, ph = 0;
+        bool ok = true;
+        for (int t = pair_id; t < total_tiles && ok; t += n_pairs) {
+            const Tile tl = a.tiles[t / MP];
+            const int mt = 2 * (t % MP) + (int)rank;
+            const int slot = tl.key % a.num_slots;
+            const uint8_t* mat = a.slots + (size_t)slot * a.slot_stride + (GATEUP ? 0 : w13_bytes);
+            const uint8_t* pn = mat + (size_t)(mt * 8 + pw) * KB * kBlockBytes;
+            constexpr int PF = 3;                                  // blocks in flight per lane (this one + 2 ahead)
+            uint4 w[PF];
+            uint32_t sc[PF];
+#pragma unroll
+            for (int i = 0; i < PF - 1; ++i)
+                if (i < KB) {
+                    const uint8_t* blk = pn + (size_t)i * kBlockBytes;
+                    w[i] = ldg_stream128(blk + hh * 512 + lane * 16);
+                    sc[i] = ldg_stream32(blk + kCodeBytes + q * 4);
+                }
+            for (int kb0 = 0; kb0 < KB; kb0 += PF) {
+#pragma unroll
+                for (int u = 0; u < PF; ++u) {
+                    const int kb = kb0 + u;
+                    if (kb >= KB) break;
+                    constexpr int nx_off = PF - 1;
+                    if (kb + nx_off < KB) {                        // keep two blocks of codes in flight
+                        const uint8_t* blk = pn + (size_t)(kb + nx_off) * kBlockBytes;
+                        w[(u + nx_off) % PF] = ldg_stream128(blk + hh * 512 + lane * 16);
+                        sc[(u + nx_off) % PF] = ldg_stream32(blk + kCodeBytes + q * 4);
+                    }
+                    ok = mbar_wait(&empty[s], ph ^ 1, abort_flag, a.status);
+                    ok = __all_sync(0xffffffffu, ok);
+                    if (!ok) break;
+                    tc_fence_after();
+                    unsigned char* dst = sA + s * PA_STAGE_BYTES;
+                    const __half2 sh = *reinterpret_cast<const __half2*>(&sc[u]);
+                    const ScaleSplit s_lo = split_scale(__low2float(sh));                 // row q
+                    const ScaleSplit s_hi = split_scale(__high2float(sh));                // row q + 8
+                    const uint32_t words[4] = {w[u].x, w[u].y, w[u].z, w[u].w};
+#pragma unroll
+                    for (int wi = 0; wi < 4; ++wi) {
+                        const int r = wi & 1, set = wi >> 1;
+                        const int kc = 8 * hh + 4 * set + c;                              // 16-byte k-chunk
+                        const uint4 val = dequant_word(words[wi], r ? s_hi : s_lo);
+                        *reinterpret_cast<uint4*>(dst + (2 * pw + r) * PA_SBO + kc * A_LBO + q * 16) = val;
+                    }
+                    fence_proxy_async();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(&full[s]);
+                    if (++s == P_STAGES) { s = 0; ph ^= 1; }
+                }
+                if (!ok) break;
+            }
+        }
+    }
+
+    // ---------------------------------------------------------------------- teardown (all roles, abort or not)
+    tc_fence_before();
+    __syncthreads();
+    cluster_sync_all();                       // neither CTA leaves while the other may still read its memory or signal it
+    tc_fence_after();
+    if (warp == 0) asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512));
 }
 
 // Self-test of the bounded wait: one warp waits on an mbarrier that nothing will ever complete, with a short
@@ -577,9 +809,7 @@ gather_rows_kernel(const __nv_bfloat16* __restrict__ hidden, const int32_t* __re
                    const int32_t* __restrict__ counts, const int32_t* __restrict__ group_keys,
                    const int32_t* __restrict__ wave_start, Tile* __restrict__ tiles, int32_t* __restrict__ n_tiles, int bn) {
     if (blockIdx.x == 0 && tiles) build_tile_list(counts, group_keys, wave_start, tiles, n_tiles, bn);
-    // one warp per row, eight rows per CTA; a lane moves pairs of 16-byte chunks, four pairs in flight before it
-    // stores.  The copy is written in the K order of the tensor-core kernels' weights: inside every 32 elements, the
-    // low halves of the four 16-byte chunks first (chunk pairs side by side), then the high halves (perm64).
+    // one warp per row, eight rows per CTA; a lane keeps up to eight 16-byte loads in flight before it stores
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int r = blockIdx.x * 8 + warp;
     if (r >= *n_valid) return;
@@ -588,25 +818,18 @@ gather_rows_kernel(const __nv_bfloat16* __restrict__ hidden, const int32_t* __re
     token = __shfl_sync(0xffffffffu, token, 0);
     const uint4* src = reinterpret_cast<const uint4*>(hidden + (size_t)token * H);
     uint4* dst = reinterpret_cast<uint4*>(xg + (size_t)r * H);
-    const int n_pairs = H / 16;                                   // pairs of chunks = 16 elements each
-    for (int base = 0; base < n_pairs; base += 128) {
-        uint4 va[4], vb[4];
+    const int n16 = H / 8;
+    for (int base = 0; base < n16; base += 256) {
+        uint4 v[8];
 #pragma unroll
-        for (int j = 0; j < 4; ++j) {
-            const int p = base + lane + 32 * j;
-            if (p < n_pairs) {
-                va[j] = src[2 * p];
-                vb[j] = src[2 * p + 1];
-            }
+        for (int j = 0; j < 8; ++j) {
+            const int i = base + lane + 32 * j;
+            if (i < n16) v[j] = src[i];
         }
 #pragma unroll
-        for (int j = 0; j < 4; ++j) {
-            const int p = base + lane + 32 * j;
-            if (p < n_pairs) {
-                const int o = 4 * (p >> 1) + (p & 1);             // 32-element group, first or second chunk pair
-                dst[o] = make_uint4(va[j].x, va[j].y, vb[j].x, vb[j].y);
-                dst[o + 2] = make_uint4(va[j].z, va[j].w, vb[j].z, vb[j].w);
-            }
+        for (int j = 0; j < 8; ++j) {
+            const int i = base + lane + 32 * j;
+            if (i < n16) dst[i] = v[j];
         }
     }
 }
@@ -642,12 +865,14 @@ static int encode_map(CUtensorMap* out, const void* base, int rows, int cols, in
 }
 
 int prefill_setup(PrefillMaps* maps, const __nv_bfloat16* xg, const __nv_bfloat16* act, int max_pairs, int H, int I) {
-    static_assert(kPrefillMapBytes == 2 * N_MAPS * sizeof(CUtensorMap), "map families of the two operands");
-    alignas(64) CUtensorMap host[2 * N_MAPS];
+    static_assert(kPrefillMapBytes == 4 * N_MAPS * sizeof(CUtensorMap), "two map families of each operand");
+    alignas(64) CUtensorMap host[4 * N_MAPS];
     int rc = EXMOE_OK;
     for (int i = 0; i < N_MAPS && !rc; ++i) {
         rc = encode_map(&host[i], xg, max_pairs, H, 16 * (i + 1));
         if (!rc) rc = encode_map(&host[N_MAPS + i], act, max_pairs, I, 16 * (i + 1));
+        if (!rc) rc = encode_map(&host[2 * N_MAPS + i], xg, max_pairs, H, 8 * (i + 1));       // half tiles of the pair kernel
+        if (!rc) rc = encode_map(&host[3 * N_MAPS + i], act, max_pairs, I, 8 * (i + 1));
     }
     if (!rc && cudaMemcpy(maps->dev, host, sizeof(host), cudaMemcpyHostToDevice) != cudaSuccess) rc = EXMOE_ERR_CUDA;
     return rc;
@@ -685,35 +910,50 @@ void launch_prefill_wave(const GemmArgs& g, const int32_t* wave_start, void* scr
     a.H = g.H;
     a.I = g.I;
     a.status = status;
-    constexpr int kSBLarge = 8, kSALarge = 4, kSBSmall = 16, kSASmall = 8;
-    const size_t smem_large = (size_t)kSBLarge * (BN * 128) + 512 + 1024;
-    const size_t smem_small = (size_t)kSBSmall * (BN_SMALL * 128) + 512 + 1024;
+    constexpr int kStagesLarge = 4, kStagesSmall = 8;
+    const size_t smem_large = (size_t)kStagesLarge * (A_STAGE_BYTES + BN * 128) + 256 + 1024;
+    const size_t smem_small = (size_t)kStagesSmall * (A_STAGE_BYTES + BN_SMALL * 128) + 256 + 1024;
     static SmemOnce once[4];
-    allow_smem(prefill_gemm_kernel<true, BN, kSBLarge, kSALarge>, (int)smem_large, once[0]);
-    allow_smem(prefill_gemm_kernel<false, BN, kSBLarge, kSALarge>, (int)smem_large, once[1]);
-    allow_smem(prefill_gemm_kernel<true, BN_SMALL, kSBSmall, kSASmall>, (int)smem_small, once[2]);
-    allow_smem(prefill_gemm_kernel<false, BN_SMALL, kSBSmall, kSASmall>, (int)smem_small, once[3]);
+    allow_smem(prefill_gemm_kernel<true, BN, kStagesLarge>, (int)smem_large, once[0]);
+    allow_smem(prefill_gemm_kernel<false, BN, kStagesLarge>, (int)smem_large, once[1]);
+    allow_smem(prefill_gemm_kernel<true, BN_SMALL, kStagesSmall>, (int)smem_small, once[2]);
+    allow_smem(prefill_gemm_kernel<false, BN_SMALL, kStagesSmall>, (int)smem_small, once[3]);
     int dev = 0, sms = 148;
     cudaGetDevice(&dev);
     cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
     const CUtensorMap* mx = reinterpret_cast<const CUtensorMap*>(maps->dev);
     const CUtensorMap* ma = mx + N_MAPS;
+    // CTA pairs for the large shape when both matrices have an even number of 128-row tiles
+#ifdef EXMOE_NO_PAIR_GEMM
+    const bool pair = false;
+#else
+    const bool pair = !small_n && (2 * g.I / BM) % 2 == 0 && (g.H / BM) % 2 == 0 && sms >= 2;
+#endif
+    const size_t smem_pair = (size_t)P_STAGES * (PA_STAGE_BYTES + PB_STAGE_BYTES) + 512 + 1024;
+    static SmemOnce once_pair[2];
+    allow_smem(prefill_pair_gemm_kernel<true>, (int)smem_pair, once_pair[0]);
+    allow_smem(prefill_pair_gemm_kernel<false>, (int)smem_pair, once_pair[1]);
+    const int grid_pair = sms & ~1;
     if (which & 4) {
         tile_list_kernel<<<1, 1024, 0, st>>>(g.counts, g.group_keys, wave_start, tiles, n_tiles, small_n ? BN_SMALL : BN);
         count_launch();
     }
     if (which & 1) {
         if (small_n)
-            prefill_gemm_kernel<true, BN_SMALL, kSBSmall, kSASmall><<<sms, NUM_THREADS, smem_small, st>>>(a, mx, act, nullptr, g.offsets, nullptr);
+            prefill_gemm_kernel<true, BN_SMALL, kStagesSmall><<<sms, NUM_THREADS, smem_small, st>>>(a, mx, act, nullptr, g.offsets, nullptr);
+        else if (pair)
+            prefill_pair_gemm_kernel<true><<<grid_pair, NUM_THREADS, smem_pair, st>>>(a, mx + 2 * N_MAPS, act, nullptr, g.offsets, nullptr);
         else
-            prefill_gemm_kernel<true, BN, kSBLarge, kSALarge><<<sms, NUM_THREADS, smem_large, st>>>(a, mx, act, nullptr, g.offsets, nullptr);
+            prefill_gemm_kernel<true, BN, kStagesLarge><<<sms, NUM_THREADS, smem_large, st>>>(a, mx, act, nullptr, g.offsets, nullptr);
         count_launch();
     }
     if (which & 2) {
         if (small_n)
-            prefill_gemm_kernel<false, BN_SMALL, kSBSmall, kSASmall><<<sms, NUM_THREADS, smem_small, st>>>(a, ma, nullptr, topk_w, g.offsets, y);
+            prefill_gemm_kernel<false, BN_SMALL, kStagesSmall><<<sms, NUM_THREADS, smem_small, st>>>(a, ma, nullptr, topk_w, g.offsets, y);
+        else if (pair)
+            prefill_pair_gemm_kernel<false><<<grid_pair, NUM_THREADS, smem_pair, st>>>(a, ma + 2 * N_MAPS, nullptr, topk_w, g.offsets, y);
         else
-            prefill_gemm_kernel<false, BN, kSBLarge, kSALarge><<<sms, NUM_THREADS, smem_large, st>>>(a, ma, nullptr, topk_w, g.offsets, y);
+            prefill_gemm_kernel<false, BN, kStagesLarge><<<sms, NUM_THREADS, smem_large, st>>>(a, ma, nullptr, topk_w, g.offsets, y);
         count_launch();
     }
 }
