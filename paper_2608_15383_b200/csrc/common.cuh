@@ -130,9 +130,8 @@ bool pair_path_fits(int H, int I, int top_k);                           // share
 bool small_path_fits(int H, int I, int num_slots, int n_pairs);         // ... of the in-CTA-grouping kernels
 size_t prefill_scratch_bytes(int max_pairs, int num_experts);
 // CUtensorMap objects of the grouped hidden rows and of the activations, in device memory: per matrix a family of 16
-// maps whose boxes hold 16, 32, ..., 256 rows (a tile's box holds exactly the rows its MMAs read) and one of 8, 16,
-// ..., 128 rows (half tiles of the CTA-pair kernel); order: x, act (16-row steps), x, act (8-row steps)
-constexpr size_t kPrefillMapBytes = 4 * 16 * 128;
+// maps whose boxes hold 16, 32, ..., 256 rows (a tile's box holds exactly the rows its MMAs read); x family, then act
+constexpr size_t kPrefillMapBytes = 2 * 16 * 128;
 struct PrefillMaps { unsigned char* dev; };
 int prefill_setup(PrefillMaps* maps, const __nv_bfloat16* xg, const __nv_bfloat16* act, int max_pairs, int H, int I);
 void launch_wait_selftest(int* status, long long budget_cycles, int* result, cudaStream_t st);

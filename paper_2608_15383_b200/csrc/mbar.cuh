@@ -33,32 +33,13 @@ __device__ __forceinline__ bool mbar_try(uint64_t* bar, uint32_t parity) {
         : "memory");
     return ok != 0;
 }
-// the same test with acquire semantics at cluster scope: for a barrier of this CTA that threads of the peer CTA arrive on
-__device__ __forceinline__ bool mbar_try_cluster(uint64_t* bar, uint32_t parity) {
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok)
-        : "r"(smem_u32(bar)), "r"(parity)
-        : "memory");
-    return ok != 0;
-}
-// arrive (release at cluster scope) on the barrier at the same shared-memory offset in CTA `rank` of the cluster
-__device__ __forceinline__ void mbar_arrive_remote(uint64_t* bar, uint32_t rank) {
-    uint32_t remote;
-    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(smem_u32(bar)), "r"(rank));
-    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(remote) : "memory");
-}
 // bounded wait; returns false when the CTA is aborting (and raises the abort on expiry)
-template <bool CLUSTER = false>
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag, int* status,
                                           long long budget = kWaitBudget) {
-    if (CLUSTER ? mbar_try_cluster(bar, parity) : mbar_try(bar, parity)) return true;
+    if (mbar_try(bar, parity)) return true;
     const long long t0 = clock64();
     unsigned polls = 0;
-    while (!(CLUSTER ? mbar_try_cluster(bar, parity) : mbar_try(bar, parity))) {
+    while (!mbar_try(bar, parity)) {
         if ((++polls & 15u) == 0) {                    // the bookkeeping of the bound is amortised over 16 polls
             if (*abort_flag) return false;
             if (clock64() - t0 > budget) {

@@ -7,25 +7,37 @@
 // gate p, up p, gate p+1, ... so one accumulator holds 64 intermediates' gate rows and up rows
 // 16 lanes apart: SwiGLU is one shuffle away in the epilogue.
 //
-// A persistent CTA (one per SM, 16 warps) is specialised by warp:
-//   warp 0        allocates TMEM, then one elected thread issues tcgen05.mma (8 x K16 per 128-wide
-//                 block) and tcgen05.commit to the stage-empty / accumulator-full mbarriers.
+// A persistent CTA (one per SM, 28 warps) is specialised by warp:
+//   warp 0        allocates TMEM, then ONE thread issues tcgen05.mma (4 x K16 per 64-wide ring stage) and
+//                 tcgen05.commit to the stage-empty / accumulator-full mbarriers, from an unrolled ring
+//                 (see the note at the issue loop: what bounds this kernel is what that thread does between MMAs).
 //   warps 4-7,    epilogue (two groups, even / odd 32-column chunks): tcgen05.ld the accumulator (warp w
 //   16-19         reads TMEM lanes 32(w%4)..), SwiGLU -> BF16 activations, or routing weight -> fp32
 //                 pair buffer; two accumulators (2 x 256 columns) let the epilogue of tile i overlap
 //                 the MMAs of tile i+1.
-//   warp 1        B producer: one thread issues two TMA tile loads (cp.async.bulk.tensor.2d, 128-byte
-//                 swizzle, 256 rows x 64 columns each) per stage from the grouped activation matrix;
+//   warp 1        B producer: one thread issues one TMA tile load (cp.async.bulk.tensor.2d, 128-byte
+//                 swizzle, the tile's rows x 64 columns) per stage from the grouped activation matrix;
 //                 completion is counted in bytes on the stage's full barrier.  No multicast.
-//   warps 8-15,   A producers, one 16-row panel and one 64-wide k-half each: stream packed int4 (128-bit
-//   20-27         loads, two blocks ahead in registers), dequantise to BF16 (shift/lop3 -> 128+u, subtract 136,
-//                 multiply by the exactly split group scale: one rounding) and store the canonical no-swizzle K-major
-//                 core-matrix layout (k-chunk stride padded to 160 bytes: conflict-free stores).
+//   warps 8-15,   A producers, one 16-row panel and one 64-wide k-half (= every second stage) each: stream
+//   20-27         packed int4 (128-bit loads, two blocks ahead in registers), dequantise to BF16 (shift/lop3 ->
+//                 128+u, subtract 136, multiply by the exactly split group scale: one rounding) and store the
+//                 canonical no-swizzle K-major core-matrix layout (k-chunk stride padded to 160 bytes:
+//                 conflict-free stores).
 // Producers -> MMA through full[stage] mbarriers (generic-proxy writes are fenced with
 // fence.proxy.async before the arrive), MMA -> producers through tcgen05.commit on empty[stage].
 // The gate/up GEMM reads its tokens from a grouped copy of the hidden states (rows in plan order),
 // written once per call by gather_rows_kernel, so that both GEMMs load B with plain tiled TMA.
 // Every wait is bounded: on expiry the CTA raises EXMOE_ERR_TIMEOUT, all roles drain, TMEM is freed.
+//
+// Measured alone on one SM (one CTA, operands in place): an MMA of this shape takes N / 2 cycles issued back to
+// back, from shared-memory A as from tensor-memory A, and its issue blocks while the pipe is busy.  Two variants
+// of this kernel were built, are parity-green and are in the history, not in the tree: the dequantised weights
+// written to TENSOR MEMORY (tcgen05.st.16x256b hands every lane the cells of its mma-fragment-ordered codes up to
+// a K permutation inside every 64, which the token matrices were stored in as well) with A taken from there, and
+// CTA PAIRS (cta_group::2: M = 256, each CTA dequantises its 128 rows and fetches half of the token tile, one
+// commit multicast to both).  On config 4 they measured 338 and 344 us per step against 323 us for this one:
+// tensor memory leaves room for 192-row tiles only (more tiles, more conversion work), the pair halves neither
+// the conversion work nor, it turned out, the time.
 #include <cuda.h>
 
 #include "common.cuh"
@@ -471,270 +483,6 @@ prefill_gemm_kernel(PrefillArgs a, const CUtensorMap* __restrict__ maps, __nv_bf
     if (warp == 0) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512));
 }
 
-// ---------------------------------------------------------------------------------------------------------------
-// The same GEMM on CTA PAIRS (tcgen05 cta_group::2): one MMA of M = 256 weight rows x N <= 256 tokens spans two SMs.
-// CTA r of the pair dequantises the 128 weight rows of m-tile 2 mp + r into ITS shared memory and fetches HALF of the
-// token tile (rows r N/2 .. (r+1) N/2); the tensor cores of both SMs read both halves.  Per SM that halves the token
-// bytes written into and read from shared memory, which is what bounds the one-CTA kernel at 256-row tiles (its MMA
-// operand reads, dequantisation stores and TMA writes ask for ~190 B per clock of a 128 B per clock pipe), and one
-// thread issues for two SMs.  Stage = one packed block (128 of K): 40 KB of weights + two [N/2 x 64] token boxes.
-//   CTA 0, warp 0: waits for its own stage (full) and the peer's (full_peer, which the peer's warp 0 relays), issues
-//                  8 MMAs and one tcgen05.commit that arrives on empty[s] of BOTH CTAs (.multicast::cluster on the
-//                  commit only; every load is a plain TMA load of this GPU's memory into the issuing CTA).
-//   CTA 1, warp 0: relay: waits for its CTA's full[s], arrives on CTA 0's full_peer[s].
-//   epilogue warps of both CTAs read their own TMEM (lanes = their 128 weight rows); the peer's arrive on CTA 0's
-//   acc_empty through the cluster's shared-memory window.
-// All waits are bounded as in the one-CTA kernel; the two CTAs leave together through a cluster barrier.
-constexpr int P_STAGES = 3;
-constexpr int PA_SBO = 16 * A_LBO;                 // 16 k-chunks of 160 B per 8-row group
-constexpr int PA_STAGE_BYTES = 16 * PA_SBO;        // 40 KB
-constexpr int PB_HALF_BYTES = 128 * 128;           // up to 128 rows x 64 columns
-constexpr int PB_STAGE_BYTES = 2 * PB_HALF_BYTES;  // 32 KB
-
-__device__ __forceinline__ uint64_t make_desc_a_pair(uint32_t saddr) {       // no swizzle, 128-wide stage
-    uint64_t d = 0;
-    d |= (uint64_t)((saddr >> 4) & 0x3fff);
-    d |= (uint64_t)((A_LBO >> 4) & 0x3fff) << 16;
-    d |= (uint64_t)((PA_SBO >> 4) & 0x3fff) << 32;
-    d |= (uint64_t)1 << 46;
-    return d;
-}
-__device__ __forceinline__ void tc_mma_pair(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "setp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
-        : "memory");
-}
-// arrives (once the MMAs issued so far are complete) on the barrier at this offset in both CTAs of the pair
-__device__ __forceinline__ void tc_commit_pair(uint64_t* bar) {
-    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
-                 ::"r"(smem_u32(bar)), "h"((uint16_t)3) : "memory");
-}
-__device__ __forceinline__ void cluster_sync_all() {
-    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
-    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
-}
-// instruction descriptor of the pair MMA: D fp32, A/B BF16, both K-major, M = 256, N = n
-__device__ __forceinline__ uint32_t make_idesc_pair(int n) {
-    return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(256 >> 4) << 24);
-}
-
-template <bool GATEUP>
-__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NUM_THREADS, 1)
-prefill_pair_gemm_kernel(PrefillArgs a, const CUtensorMap* __restrict__ maps8, __nv_bfloat16* __restrict__ act_out,
-                         const float* __restrict__ topk_w, const int32_t* __restrict__ offsets, float* __restrict__ y_out) {
-    extern __shared__ unsigned char smem_raw[];
-    unsigned char* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);   // the same offset in both CTAs
-    unsigned char* sB = smem;                                     // [P_STAGES][32 KB]
-    unsigned char* sA = smem + P_STAGES * PB_STAGE_BYTES;         // [P_STAGES][40 KB]
-    uint64_t* bars = reinterpret_cast<uint64_t*>(sA + P_STAGES * PA_STAGE_BYTES);
-    uint64_t* full = bars;                          // [P_STAGES]  this CTA's producers -> warp 0
-    uint64_t* empty = bars + P_STAGES;              // [P_STAGES]  MMA -> producers of both CTAs (multicast commit)
-    uint64_t* full_peer = bars + 2 * P_STAGES;      // [P_STAGES]  CTA 1's relay -> CTA 0's MMA issuer
-    uint64_t* acc_full = bars + 3 * P_STAGES;       // [2]         MMA -> epilogues of both CTAs (multicast commit)
-    uint64_t* acc_empty = acc_full + 2;             // [2]         epilogues of both CTAs -> CTA 0's MMA issuer (16 arrivals)
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_empty + 2);
-    volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
-
-    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    uint32_t rank;
-    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(rank));
-    const int pair_id = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
-    const int K = GATEUP ? a.H : a.I;
-    const int KB = K / BK;
-    const int MP = (GATEUP ? 2 * a.I : a.H) / (2 * BM);           // pairs of m-tiles of the packed matrix
-    const size_t w13_bytes = matrix_bytes(2 * a.I, a.H);
-    const int total_tiles = (*a.n_tiles) * MP;
-
-    if (tid == 0) {
-        for (int s = 0; s < P_STAGES; ++s) {
-            mbar_init(&full[s], 17);          // 16 A-producer warps + the TMA thread's expect_tx arrive
-            mbar_init(&empty[s], 1);
-            mbar_init(&full_peer[s], 1);
-        }
-        for (int b = 0; b < 2; ++b) {
-            mbar_init(&acc_full[b], 1);
-            mbar_init(&acc_empty[b], 16);     // 8 epilogue warps of each CTA
-        }
-        *abort_flag = 0;
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    }
-    if (warp == 0) {
-        asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(512));
-        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::);
-    }
-    tc_fence_before();
-    __syncthreads();
-    cluster_sync_all();                       // the peer's barriers exist before anything arrives on them
-    tc_fence_after();
-    const uint32_t tmem_base = *tmem_slot;
-
-    if (warp == 0 && rank == 0) {
-        // ------------------------------------------------------------------ MMA issuer of the pair (one thread)
-        if (lane == 0) {
-            int s = 0, ph = 0, tcount = 0;
-            bool ok = true;
-            const uint64_t da0 = make_desc_a_pair(smem_u32(sA)), db0 = make_desc_b(smem_u32(sB));
-            for (int t = pair_id; t < total_tiles && ok; t += n_pairs, ++tcount) {
-                const Tile tl = a.tiles[t / MP];
-                const int n_mma = (tl.nrows + 15) & ~15;
-                const uint32_t idesc = make_idesc_pair(n_mma);
-                const int buf = tcount & 1;
-                ok = mbar_wait<true>(&acc_empty[buf], ((tcount >> 1) & 1) ^ 1, abort_flag, a.status);
-                if (!ok) break;
-                tc_fence_after();
-                const uint32_t d_tmem = tmem_base + buf * BN;
-                for (int kb = 0; kb < KB; ++kb) {
-                    if (!mbar_try(&full[s], ph)) ok = mbar_wait(&full[s], ph, abort_flag, a.status);
-                    if (ok && !mbar_try_cluster(&full_peer[s], ph)) ok = mbar_wait<true>(&full_peer[s], ph, abort_flag, a.status);
-                    if (!ok) break;
-                    const uint64_t da = da0 + (uint64_t)(s * (PA_STAGE_BYTES >> 4));
-                    const uint64_t db = db0 + (uint64_t)(s * (PB_STAGE_BYTES >> 4));
-#pragma unroll
-                    for (int j = 0; j < BK / 16; ++j) {            // K16 step j: A two k-chunks on, B 32 bytes on in its half
-                        const uint64_t aj = da + (uint64_t)(j * 2 * A_LBO >> 4);
-                        const uint64_t bj = db + (uint64_t)(((j >> 2) * PB_HALF_BYTES + (j & 3) * 32) >> 4);
-                        tc_mma_pair(d_tmem, aj, bj, idesc, (kb | j) ? 1u : 0u);
-                    }
-                    tc_commit_pair(&empty[s]);                     // stage reusable in both CTAs once these MMAs have read it
-                    if (++s == P_STAGES) { s = 0; ph ^= 1; }
-                }
-                if (ok) tc_commit_pair(&acc_full[buf]);            // accumulators of both CTAs complete
-            }
-        }
-        __syncwarp();
-    } else if (warp == 0) {
-        // ------------------------------------------------------------------ relay (CTA 1): stage full here -> tell CTA 0
-        int s = 0, ph = 0;
-        bool ok = true;
-        for (int t = pair_id; t < total_tiles && ok; t += n_pairs) {
-            for (int kb = 0; kb < KB; ++kb) {
-                ok = mbar_wait(&full[s], ph, abort_flag, a.status);
-                ok = __all_sync(0xffffffffu, ok);
-                if (!ok) break;
-                if (lane == 0) {
-                    fence_proxy_async();
-                    mbar_arrive_remote(&full_peer[s], 0);
-                }
-                __syncwarp();
-                if (++s == P_STAGES) { s = 0; ph ^= 1; }
-            }
-        }
-    } else if ((warp >= 4 && warp < 8) || (warp >= 16 && warp < 20)) {
-        // ------------------------------------------------------------------ epilogue (own 128 weight rows)
-        const int e = warp & 3;
-        const int odd = warp >= 16 ? 32 : 0;
-        int tcount = 0;
-        bool ok = true;
-        for (int t = pair_id; t < total_tiles && ok; t += n_pairs, ++tcount) {
-            const Tile tl = a.tiles[t / MP];
-            const int mt = 2 * (t % MP) + (int)rank;
-            const int buf = tcount & 1;
-            ok = mbar_wait(&acc_full[buf], (tcount >> 1) & 1, abort_flag, a.status);
-            ok = __all_sync(0xffffffffu, ok);
-            if (!ok) break;
-            tc_fence_after();
-            epilogue_tile<GATEUP>(a, tl, mt, e, odd, lane, tmem_base + buf * BN, offsets, act_out, topk_w, y_out);
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) {
-                if (rank == 0) mbar_arrive(&acc_empty[buf]);
-                else mbar_arrive_remote(&acc_empty[buf], 0);
-            }
-        }
-    } else if (warp == 1) {
-        // ------------------------------------------------------------------ B producer: this CTA's half of the token tile
-        int s = 0, ph = 0;
-        bool ok = true;
-        for (int t = pair_id; t < total_tiles && ok; t += n_pairs) {
-            const Tile tl = a.tiles[t / MP];
-            const int n_half = ((tl.nrows + 15) & ~15) >> 1;       // multiple of 8: whole swizzle atoms
-            const int row0 = offsets[tl.key] + tl.n0 + (int)rank * n_half;
-            const CUtensorMap* map = maps8 + (n_half / 8 - 1);
-            for (int kb = 0; kb < KB; ++kb) {
-                ok = mbar_wait(&empty[s], ph ^ 1, abort_flag, a.status);
-                ok = __all_sync(0xffffffffu, ok);
-                if (!ok) break;
-                if (lane == 0) {
-                    const uint32_t dst = smem_u32(sB + s * PB_STAGE_BYTES);
-                    mbar_expect_tx(&full[s], 2 * n_half * 128);
-                    tma_load_2d(dst, map, kb * BK, row0, &full[s]);                       // columns kb*128 .. +63
-                    tma_load_2d(dst + PB_HALF_BYTES, map, kb * BK + 64, row0, &full[s]);
-                }
-                __syncwarp();
-                if (++s == P_STAGES) { s = 0; ph ^= 1; }
-            }
-        }
-    } else if (warp >= 8 && !(warp >= 16 && warp < 20)) {
-        // ------------------------------------------------------------------ A producers (dequantise this CTA's m-tile)
-        const int pw = warp & 7;                                   // panel of the tile = 8-row groups 2*pw, 2*pw+1
-        const int hh = warp >= 20 ? 1 : 0;                         // 64-wide k-half of every block
-        const int q = lane >> 2, c = lane & 3;
-        int s = 0, ph = 0;
-        bool ok = true;
-        for (int t = pair_id; t < total_tiles && ok; t += n_pairs) {
-            const Tile tl = a.tiles[t / MP];
-            const int mt = 2 * (t % MP) + (int)rank;
-            const int slot = tl.key % a.num_slots;
-            const uint8_t* mat = a.slots + (size_t)slot * a.slot_stride + (GATEUP ? 0 : w13_bytes);
-            const uint8_t* pn = mat + (size_t)(mt * 8 + pw) * KB * kBlockBytes;
-            constexpr int PF = 3;                                  // blocks in flight per lane (this one + 2 ahead)
-            uint4 w[PF];
-            uint32_t sc[PF];
-#pragma unroll
-            for (int i = 0; i < PF - 1; ++i)
-                if (i < KB) {
-                    const uint8_t* blk = pn + (size_t)i * kBlockBytes;
-                    w[i] = ldg_stream128(blk + hh * 512 + lane * 16);
-                    sc[i] = ldg_stream32(blk + kCodeBytes + q * 4);
-                }
-            for (int kb0 = 0; kb0 < KB; kb0 += PF) {
-#pragma unroll
-                for (int u = 0; u < PF; ++u) {
-                    const int kb = kb0 + u;
-                    if (kb >= KB) break;
-                    constexpr int nx_off = PF - 1;
-                    if (kb + nx_off < KB) {                        // keep two blocks of codes in flight
-                        const uint8_t* blk = pn + (size_t)(kb + nx_off) * kBlockBytes;
-                        w[(u + nx_off) % PF] = ldg_stream128(blk + hh * 512 + lane * 16);
-                        sc[(u + nx_off) % PF] = ldg_stream32(blk + kCodeBytes + q * 4);
-                    }
-                    ok = mbar_wait(&empty[s], ph ^ 1, abort_flag, a.status);
-                    ok = __all_sync(0xffffffffu, ok);
-                    if (!ok) break;
-                    tc_fence_after();
-                    unsigned char* dst = sA + s * PA_STAGE_BYTES;
-                    const __half2 sh = *reinterpret_cast<const __half2*>(&sc[u]);
-                    const ScaleSplit s_lo = split_scale(__low2float(sh));                 // row q
-                    const ScaleSplit s_hi = split_scale(__high2float(sh));                // row q + 8
-                    const uint32_t words[4] = {w[u].x, w[u].y, w[u].z, w[u].w};
-#pragma unroll
-                    for (int wi = 0; wi < 4; ++wi) {
-                        const int r = wi & 1, set = wi >> 1;
-                        const int kc = 8 * hh + 4 * set + c;                              // 16-byte k-chunk
-                        const uint4 val = dequant_word(words[wi], r ? s_hi : s_lo);
-                        *reinterpret_cast<uint4*>(dst + (2 * pw + r) * PA_SBO + kc * A_LBO + q * 16) = val;
-                    }
-                    fence_proxy_async();
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(&full[s]);
-                    if (++s == P_STAGES) { s = 0; ph ^= 1; }
-                }
-                if (!ok) break;
-            }
-        }
-    }
-
-    // ---------------------------------------------------------------------- teardown (all roles, abort or not)
-    tc_fence_before();
-    __syncthreads();
-    cluster_sync_all();                       // neither CTA leaves while the other may still read its memory or signal it
-    tc_fence_after();
-    if (warp == 0) asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512));
-}
-
 // Self-test of the bounded wait: one warp waits on an mbarrier that nothing will ever complete, with a short
 // budget; the wait must give up, raise the abort flag and the status word, and the kernel must return normally.
 __global__ void wait_timeout_selftest_kernel(int* status, long long budget, int* result) {
@@ -865,14 +613,12 @@ static int encode_map(CUtensorMap* out, const void* base, int rows, int cols, in
 }
 
 int prefill_setup(PrefillMaps* maps, const __nv_bfloat16* xg, const __nv_bfloat16* act, int max_pairs, int H, int I) {
-    static_assert(kPrefillMapBytes == 4 * N_MAPS * sizeof(CUtensorMap), "two map families of each operand");
-    alignas(64) CUtensorMap host[4 * N_MAPS];
+    static_assert(kPrefillMapBytes == 2 * N_MAPS * sizeof(CUtensorMap), "map families of the two operands");
+    alignas(64) CUtensorMap host[2 * N_MAPS];
     int rc = EXMOE_OK;
     for (int i = 0; i < N_MAPS && !rc; ++i) {
         rc = encode_map(&host[i], xg, max_pairs, H, 16 * (i + 1));
         if (!rc) rc = encode_map(&host[N_MAPS + i], act, max_pairs, I, 16 * (i + 1));
-        if (!rc) rc = encode_map(&host[2 * N_MAPS + i], xg, max_pairs, H, 8 * (i + 1));       // half tiles of the pair kernel
-        if (!rc) rc = encode_map(&host[3 * N_MAPS + i], act, max_pairs, I, 8 * (i + 1));
     }
     if (!rc && cudaMemcpy(maps->dev, host, sizeof(host), cudaMemcpyHostToDevice) != cudaSuccess) rc = EXMOE_ERR_CUDA;
     return rc;
@@ -923,17 +669,6 @@ void launch_prefill_wave(const GemmArgs& g, const int32_t* wave_start, void* scr
     cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
     const CUtensorMap* mx = reinterpret_cast<const CUtensorMap*>(maps->dev);
     const CUtensorMap* ma = mx + N_MAPS;
-    // CTA pairs for the large shape when both matrices have an even number of 128-row tiles
-#ifdef EXMOE_NO_PAIR_GEMM
-    const bool pair = false;
-#else
-    const bool pair = !small_n && (2 * g.I / BM) % 2 == 0 && (g.H / BM) % 2 == 0 && sms >= 2;
-#endif
-    const size_t smem_pair = (size_t)P_STAGES * (PA_STAGE_BYTES + PB_STAGE_BYTES) + 512 + 1024;
-    static SmemOnce once_pair[2];
-    allow_smem(prefill_pair_gemm_kernel<true>, (int)smem_pair, once_pair[0]);
-    allow_smem(prefill_pair_gemm_kernel<false>, (int)smem_pair, once_pair[1]);
-    const int grid_pair = sms & ~1;
     if (which & 4) {
         tile_list_kernel<<<1, 1024, 0, st>>>(g.counts, g.group_keys, wave_start, tiles, n_tiles, small_n ? BN_SMALL : BN);
         count_launch();
@@ -941,8 +676,6 @@ void launch_prefill_wave(const GemmArgs& g, const int32_t* wave_start, void* scr
     if (which & 1) {
         if (small_n)
             prefill_gemm_kernel<true, BN_SMALL, kStagesSmall><<<sms, NUM_THREADS, smem_small, st>>>(a, mx, act, nullptr, g.offsets, nullptr);
-        else if (pair)
-            prefill_pair_gemm_kernel<true><<<grid_pair, NUM_THREADS, smem_pair, st>>>(a, mx + 2 * N_MAPS, act, nullptr, g.offsets, nullptr);
         else
             prefill_gemm_kernel<true, BN, kStagesLarge><<<sms, NUM_THREADS, smem_large, st>>>(a, mx, act, nullptr, g.offsets, nullptr);
         count_launch();
@@ -950,8 +683,6 @@ void launch_prefill_wave(const GemmArgs& g, const int32_t* wave_start, void* scr
     if (which & 2) {
         if (small_n)
             prefill_gemm_kernel<false, BN_SMALL, kStagesSmall><<<sms, NUM_THREADS, smem_small, st>>>(a, ma, nullptr, topk_w, g.offsets, y);
-        else if (pair)
-            prefill_pair_gemm_kernel<false><<<grid_pair, NUM_THREADS, smem_pair, st>>>(a, ma + 2 * N_MAPS, nullptr, topk_w, g.offsets, y);
         else
             prefill_gemm_kernel<false, BN, kStagesLarge><<<sms, NUM_THREADS, smem_large, st>>>(a, ma, nullptr, topk_w, g.offsets, y);
         count_launch();
