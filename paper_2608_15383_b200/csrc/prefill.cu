@@ -181,16 +181,45 @@ struct PrefillArgs {
     int* status;
 };
 
+// What an epilogue warp can fetch before the tile's accumulator is complete: the tile's first grouped row and, for the
+// down GEMM, the (pair, routing weight) of each of its columns (two dependent global loads per 32-column chunk, which
+// cost more than the chunk's stores when they were issued after the wait).
+template <int CHUNKS>
+struct EpiloguePre {
+    int row0;
+    int pair[CHUNKS];
+    float w[CHUNKS];
+};
+template <bool GATEUP, int CHUNKS>
+__device__ __forceinline__ EpiloguePre<CHUNKS> epilogue_prefetch(const PrefillArgs& a, const Tile& tl, int first, int lane,
+                                                                 const int32_t* __restrict__ offsets,
+                                                                 const float* __restrict__ topk_w) {
+    EpiloguePre<CHUNKS> p;
+    p.row0 = offsets[tl.key] + tl.n0;
+#pragma unroll
+    for (int i = 0; i < CHUNKS; ++i) {
+        p.pair[i] = 0;
+        p.w[i] = 0.f;
+        const int c = first + 64 * i + lane;
+        if (!GATEUP && c < tl.nrows) {
+            p.pair[i] = a.perm[p.row0 + c];
+            p.w[i] = topk_w[p.pair[i]];
+        }
+    }
+    return p;
+}
 // Epilogue of one tile by one warp: TMEM lanes 32e .. 32e+31 of the accumulator at `tmem_acc`, the 32-column chunks
 // c0 = first, first + 64, ...  Gate/up: SwiGLU -> BF16 activations; down: routing weight -> fp32 pair buffer.
-template <bool GATEUP>
+template <bool GATEUP, int CHUNKS>
 __device__ __forceinline__ void epilogue_tile(const PrefillArgs& a, const Tile& tl, int mt, int e, int first, int lane,
-                                              uint32_t tmem_acc, const int32_t* __restrict__ offsets,
-                                              __nv_bfloat16* __restrict__ act_out, const float* __restrict__ topk_w,
-                                              float* __restrict__ y_out) {
-    const int row0 = offsets[tl.key] + tl.n0;
+                                              uint32_t tmem_acc, const EpiloguePre<CHUNKS>& pre,
+                                              __nv_bfloat16* __restrict__ act_out, float* __restrict__ y_out) {
+    const int row0 = pre.row0;
     const uint32_t taddr = tmem_acc + ((uint32_t)(32 * e) << 16);
-    for (int c0 = first; c0 < tl.nrows; c0 += 64) {
+#pragma unroll
+    for (int i = 0; i < CHUNKS; ++i) {
+        const int c0 = first + 64 * i;
+        if (c0 >= tl.nrows) break;
         uint32_t v[32];
         tc_ld32(taddr + c0, v);
         tc_wait_ld();
@@ -210,16 +239,10 @@ __device__ __forceinline__ void epilogue_tile(const PrefillArgs& a, const Tile& 
             }
         } else {
             const int h = mt * BM + 32 * e + lane;
-            int my_pair = 0;                               // lane j holds pair and weight of column c0 + j
-            float my_w = 0.f;
-            if (c0 + lane < tl.nrows) {
-                my_pair = a.perm[row0 + c0 + lane];
-                my_w = topk_w[my_pair];
-            }
 #pragma unroll
-            for (int j = 0; j < 32; ++j) {
-                const int pair = __shfl_sync(0xffffffffu, my_pair, j);
-                const float wj = __shfl_sync(0xffffffffu, my_w, j);
+            for (int j = 0; j < 32; ++j) {                 // lane j holds pair and weight of column c0 + j
+                const int pair = __shfl_sync(0xffffffffu, pre.pair[i], j);
+                const float wj = __shfl_sync(0xffffffffu, pre.w[i], j);
                 if (c0 + j < tl.nrows) y_out[(size_t)pair * a.H + h] = wj * __uint_as_float(v[j]);
             }
         }
@@ -371,13 +394,15 @@ prefill_gemm_kernel(PrefillArgs a, const CUtensorMap* __restrict__ maps, __nv_bf
             const Tile tl = a.tiles[t / MT];
             const int mt = t % MT;
             const int buf = tcount & 1;
+            constexpr int CHUNKS = (BN_T + 63) / 64;               // 32-column chunks of this warp in a full tile
+            const EpiloguePre<CHUNKS> pre = epilogue_prefetch<GATEUP, CHUNKS>(a, tl, odd, lane, offsets, topk_w);
             PROF_WAIT_BEGIN;
             ok = mbar_wait(&acc_full[buf], (tcount >> 1) & 1, abort_flag, a.status);
             PROF_WAIT_END;
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
             tc_fence_after();
-            epilogue_tile<GATEUP>(a, tl, mt, e, odd, lane, tmem_base + buf * BN_T, offsets, act_out, topk_w, y_out);
+            epilogue_tile<GATEUP, CHUNKS>(a, tl, mt, e, odd, lane, tmem_base + buf * BN_T, pre, act_out, y_out);
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(&acc_empty[buf]);
