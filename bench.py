@@ -48,9 +48,9 @@ WORKLOADS = {
 # DRAM bytes (read + write) per launch of the dominant kernel, from one ncu capture each (dram__bytes_read.sum +
 # dram__bytes_write.sum, two layer banks = 415 MB resident; per-launch traffic does not depend on the number of banks):
 # (bytes, kernel captured, date of the capture)
-NCU_TRAFFIC = {"decode": (17.33e6, "pair_gateup_kernel<4>, T=1 (pair_gateup_wide_kernel<4> reads the same bytes)", "2026-11-25"),
+NCU_TRAFFIC = {"decode": (17.33e6, "pair_gateup_wide_kernel<4>, T=1", "2026-11-25"),
                "decode16": (62.83e6 + 0.87e6, "stream_gemm_kernel<1,true,1>, T=16", "2026-11-25"),
-               "prefill": (214.68e6 + 12.51e6, "prefill_gemm_kernel<true,256,2>, T=2048", "2026-11-25")}
+               "prefill": (212.95e6 + 12.03e6, "prefill_gemm_kernel<true,256,4>, T=2048", "2026-11-25")}
 METRIC = "moe_layer_tokens_per_s"
 UNIT = "tokens/s"
 
