@@ -52,7 +52,7 @@ namespace {
 
 constexpr int BM = 128;            // weight rows per tile
 constexpr int BN = 256;            // max grouped rows (tokens) per tile of the large-N kernel shape
-constexpr int BN_SMALL = 64;       // ... and of the small-N shape (a few dozen rows per expert: four stages fit)
+constexpr int BN_SMALL = 64;       // ... and of the small-N shape (a few dozen rows per expert: eight stages fit)
 constexpr int BK = 128;            // one packed block / one scale group
 constexpr int BKS = 64;            // K per ring stage = half a packed block (the half one dequantisation warp converts)
 // A (dequantised weights): no swizzle; core matrix = 8 rows x 16 B; k-chunks 160 B apart (128 + 32 pad, so that

@@ -73,7 +73,7 @@ def test_config4_prefill_olmoe_sampled_from_the_plan(B, olmoe_layer, alpha):
 
 @pytest.mark.parametrize("T", [96, 128])
 def test_small_n_tensor_core_kernels_at_olmoe_shape(B, olmoe_layer, T):
-    """Batched decode with 768 and 1024 pairs at OLMoE shape: the 64-row, four-stage tensor-core kernel shape, every
+    """Batched decode with 768 and 1024 pairs at OLMoE shape: the 64-row, eight-stage tensor-core kernel shape, every
     token against the oracle."""
     ora, bank = olmoe_layer
     s = synth.OLMOE
