@@ -443,59 +443,72 @@ prefill_gemm_kernel(PrefillArgs a, const CUtensorMap* __restrict__ maps, __nv_bf
         int s = hh % STAGES, ph = 0;                               // ring position of this warp's next stage (2 * blocks + hh)
         bool ok = true;
         PROF_DECL;
-        for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
-            const Tile tl = a.tiles[t / MT];
-            const int mt = t % MT;
-            const int slot = tl.key % a.num_slots;
-            const uint8_t* mat = a.slots + (size_t)slot * a.slot_stride + (GATEUP ? 0 : w13_bytes);
-            const uint8_t* pn = mat + (size_t)(mt * 8 + pw) * KB * kBlockBytes;
-            constexpr int PF = 3;                                  // blocks in flight per lane (this one + 2 ahead)
-            uint4 w[PF];
-            uint32_t sc[PF];
-#pragma unroll
-            for (int i = 0; i < PF - 1; ++i)
-                if (i < KB) {
-                    const uint8_t* blk = pn + (size_t)i * kBlockBytes;
-                    w[i] = ldg_stream128(blk + hh * 512 + lane * 16);
-                    sc[i] = ldg_stream32(blk + kCodeBytes + q * 4);
+        // The conversion side needs nothing of a tile but its weights, so the warp walks ONE stream of blocks over all
+        // of the CTA's tiles, its loads two blocks ahead of the conversion ACROSS tile boundaries (a tile's first loads
+        // issued only when the tile began cost one memory latency per tile, 8 or 16 blocks).  The load cursor knows its
+        // tile's key one tile early, so entering a tile costs no dependent load either.
+        const int my_tiles = blockIdx.x < total_tiles ? (total_tiles - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x : 0;
+        const int total_blocks = my_tiles * KB;
+        auto panel_row = [&](int t, int key) -> const uint8_t* {
+            const uint8_t* mat = a.slots + (size_t)(key % a.num_slots) * a.slot_stride + (GATEUP ? 0 : w13_bytes);
+            return mat + (size_t)((t % MT) * 8 + pw) * KB * kBlockBytes + hh * 512 + lane * 16;
+        };
+        int c_t = blockIdx.x, c_kb = 0, issued = 0;                // load cursor: tile, block of it, blocks requested so far
+        int c_key_next = 0;
+        const uint8_t* c_pn = nullptr;
+        if (my_tiles) {
+            c_pn = panel_row(c_t, a.tiles[c_t / MT].key);
+            if (c_t + (int)gridDim.x < total_tiles) c_key_next = a.tiles[(c_t + gridDim.x) / MT].key;
+        }
+        constexpr int PF = 3;                                      // blocks in flight per lane (this one + 2 ahead)
+        uint4 w[PF];
+        uint32_t sc[PF];
+        auto fetch = [&](uint4& wv, uint32_t& sv) {                // request the cursor's block, move the cursor on
+            const uint8_t* blk = c_pn + (size_t)c_kb * kBlockBytes;
+            wv = ldg_stream128(blk);
+            sv = ldg_stream32(blk - (hh * 512 + lane * 16) + kCodeBytes + q * 4);
+            ++issued;
+            if (++c_kb == KB) {
+                c_kb = 0;
+                c_t += gridDim.x;
+                if (c_t < total_tiles) {
+                    c_pn = panel_row(c_t, c_key_next);
+                    if (c_t + (int)gridDim.x < total_tiles) c_key_next = a.tiles[(c_t + gridDim.x) / MT].key;
                 }
-            for (int kb0 = 0; kb0 < KB; kb0 += PF) {
+            }
+        };
 #pragma unroll
-                for (int u = 0; u < PF; ++u) {
-                    const int kb = kb0 + u;
-                    if (kb >= KB) break;
-                    constexpr int nx_off = PF - 1;
-                    if (kb + nx_off < KB) {                        // keep two blocks of codes in flight
-                        const uint8_t* blk = pn + (size_t)(kb + nx_off) * kBlockBytes;
-                        w[(u + nx_off) % PF] = ldg_stream128(blk + hh * 512 + lane * 16);
-                        sc[(u + nx_off) % PF] = ldg_stream32(blk + kCodeBytes + q * 4);
-                    }
-                    {
-                        PROF_WAIT_BEGIN;
-                        ok = mbar_wait(&empty[s], ph ^ 1, abort_flag, a.status);
-                        PROF_WAIT_END;
-                    }
-                    ok = __all_sync(0xffffffffu, ok);
-                    if (!ok) break;
-                    unsigned char* dst = sA + s * A_STAGE_BYTES;
-                    const __half2 sh = *reinterpret_cast<const __half2*>(&sc[u]);
-                    const ScaleSplit s_lo = split_scale(__low2float(sh));                 // row q
-                    const ScaleSplit s_hi = split_scale(__high2float(sh));                // row q + 8
-                    const uint32_t words[4] = {w[u].x, w[u].y, w[u].z, w[u].w};
+        for (int i = 0; i < PF - 1; ++i)
+            if (issued < total_blocks) fetch(w[i], sc[i]);
+        for (int g0 = 0; g0 < total_blocks && ok; g0 += PF) {
 #pragma unroll
-                    for (int wi = 0; wi < 4; ++wi) {
-                        const int r = wi & 1, set = wi >> 1;
-                        const int kc = 4 * set + c;                                       // 16-byte k-chunk of the stage
-                        const uint4 val = dequant_word(words[wi], r ? s_hi : s_lo);
-                        *reinterpret_cast<uint4*>(dst + (2 * pw + r) * A_SBO + kc * A_LBO + q * 16) = val;
-                    }
-                    fence_proxy_async();
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(&full[s]);
-                    s += 2;                                        // this warp's next stage is two on
-                    if (s >= STAGES) { s -= STAGES; ph ^= 1; }
+            for (int u = 0; u < PF; ++u) {
+                if (g0 + u >= total_blocks) break;
+                if (issued < total_blocks) fetch(w[(u + PF - 1) % PF], sc[(u + PF - 1) % PF]);   // keep two blocks in flight
+                {
+                    PROF_WAIT_BEGIN;
+                    ok = mbar_wait(&empty[s], ph ^ 1, abort_flag, a.status);
+                    PROF_WAIT_END;
                 }
+                ok = __all_sync(0xffffffffu, ok);
                 if (!ok) break;
+                unsigned char* dst = sA + s * A_STAGE_BYTES;
+                const __half2 sh = *reinterpret_cast<const __half2*>(&sc[u]);
+                const ScaleSplit s_lo = split_scale(__low2float(sh));                 // row q
+                const ScaleSplit s_hi = split_scale(__high2float(sh));                // row q + 8
+                const uint32_t words[4] = {w[u].x, w[u].y, w[u].z, w[u].w};
+#pragma unroll
+                for (int wi = 0; wi < 4; ++wi) {
+                    const int r = wi & 1, set = wi >> 1;
+                    const int kc = 4 * set + c;                                       // 16-byte k-chunk of the stage
+                    const uint4 val = dequant_word(words[wi], r ? s_hi : s_lo);
+                    *reinterpret_cast<uint4*>(dst + (2 * pw + r) * A_SBO + kc * A_LBO + q * 16) = val;
+                }
+                fence_proxy_async();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&full[s]);
+                s += 2;                                            // this warp's next stage is two on
+                if (s >= STAGES) { s -= STAGES; ph ^= 1; }
             }
         }
         PROF_REPORT("A producer");

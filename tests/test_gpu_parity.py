@@ -170,10 +170,12 @@ def test_mid_shape_ragged_groups(B, mid_layer, T):
     cache2.close()
 
 
-@pytest.mark.parametrize("T", [1, 7, 16, 30, 90, 400])
+@pytest.mark.parametrize("T", [1, 7, 16, 30, 90, 250, 400])
 def test_odd_block_counts(B, T):
     """d_model = 3 * 128 and d_ff = 5 * 128: block counts that are not powers of two take the generic kernel
-    bodies (no K split, one block per step) on every path; 3 experts per token, ragged groups."""
+    bodies (no K split, one block per step) on every path; 3 experts per token, ragged groups.  On the tensor-core
+    path (T = 250: 64-row tiles, T = 400: 256-row tiles) 6 and 10 ring stages per tile are no multiple of the ring
+    depth, so the MMA issue loop is the plain one, not the unrolled one."""
     s = synth.Shape(d_model=384, d_ff=640, num_experts=8, top_k=3)
     if not hasattr(test_odd_block_counts, "layer"):
         test_odd_block_counts.layer = helpers.make_layer(s, seed=123)
@@ -183,6 +185,8 @@ def test_odd_block_counts(B, T):
     cache = B.Cache(s, [bank], s.num_experts, max_tokens=400)
     out = cache.forward(0, hidden.cuda(), ids.cuda(), p.cuda())
     helpers.check_output(out, y, ref, f"T={T}")
+    if T >= 250:
+        assert cache.last_path() == (B.PATH_TENSOR_SMALL_N if T == 250 else B.PATH_TENSOR)
     cache2 = B.Cache(s, [bank], 4, max_tokens=400, wave_cap=3)          # several waves, misses
     sc = ocache.SlotCache(s.num_experts, 4, 3, bytes_per_expert=cache2.bytes_per_expert)
     out2 = cache2.forward(0, hidden.cuda(), ids.cuda(), p.cuda())
