@@ -256,3 +256,34 @@ def test_zero_tokens_through_the_abi_and_host_copy_bytes(B):
     assert cache.last_host_copy_bytes() == s.d_model * 2 + 2 * s.top_k * 4       # 1056 bytes, not 2 MB
     assert cache.status() == 0
     cache.close()
+
+
+@pytest.mark.parametrize("T", [16, 128, 2048])
+def test_graph_replay_of_the_larger_paths_is_bit_identical_to_plain_launches(B, olmoe_layer, T):
+    """bench.py times every leg as a CUDA-graph replay: the streaming kernels (T = 16), the 64-row tensor-core shape
+    (T = 128) and the 256-row one (T = 2048, config 4) must give, replayed from a graph over two rotating input sets,
+    the very bits of their plain launches (which the other tests hold to the oracle)."""
+    _, bank = olmoe_layer
+    s = synth.OLMOE
+    cache = B.Cache(s, [bank], 64, max_tokens=T)
+    inputs = [tuple(x.cuda() for x in helpers.routed_inputs(s, T, seed=8800 + T + i, alpha=0.5)) for i in range(2)]
+    plain = [cache.forward(0, h, i, w).clone() for h, i, w in inputs]
+    want = {16: B.PATH_STREAM, 128: B.PATH_TENSOR_SMALL_N, 2048: B.PATH_TENSOR}[T]
+    assert cache.last_path() == want
+    outs = [torch.zeros_like(plain[0]) for _ in inputs]
+    stream = torch.cuda.Stream()
+    stream.wait_stream(torch.cuda.current_stream())
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g, stream=stream):
+        for (h, i, w), o in zip(inputs, outs):
+            cache.forward(0, h, i, w, out=o, stream=stream)
+    for rep in range(2):
+        for o in outs:
+            o.zero_()
+        with torch.cuda.stream(stream):
+            g.replay()
+        stream.synchronize()
+        for o, p in zip(outs, plain):
+            assert torch.equal(o.view(torch.int16), p.view(torch.int16)), f"T={T} replay {rep}"
+    assert cache.status() == 0
+    cache.close()
