@@ -451,6 +451,7 @@ __global__ void __launch_bounds__(256)
 token_down_kernel(GemmArgs a, SmallArgs sa, const __nv_bfloat16* __restrict__ act, const float* __restrict__ topk_w,
                   int bpwg) {
     extern __shared__ __align__(128) unsigned char smem[];
+    grid_launch_dependents();                          // the next kernel in the stream may be placed (it waits for this one)
     const int K = a.I, KB = K / kGroup, k = a.top_k;
     const int x_stride = K * 2 + 64;
     unsigned char* xs = smem;                                          // [k][x_stride]
@@ -702,6 +703,7 @@ pair_gateup_kernel(GemmArgs a, SmallArgs sa, const __nv_bfloat16* __restrict__ h
                    __nv_bfloat16* __restrict__ act_out, int ks_log2) {
     // grid = (tiles of the intermediate dimension, selected expert j, token t): pair p = t * k + j
     extern __shared__ __align__(128) unsigned char smem[];
+    grid_dependency_wait();                            // launched as a programmatic dependent of whatever precedes it in the stream
     grid_launch_dependents();
     if ((blockIdx.x | blockIdx.y | blockIdx.z) == 0) keep_pair_ids(sa);
     pair_gateup_item<NB>(a, sa, hidden, act_out, ks_log2, (int)(blockIdx.z * a.top_k + blockIdx.y), (int)blockIdx.z,
@@ -764,6 +766,10 @@ pair_gateup_wide_kernel(GemmArgs a, SmallArgs sa, const __nv_bfloat16* __restric
                         __nv_bfloat16* __restrict__ act_out, int ks_log2) {
     // grid = (slices of 16 >> ks_log2 panel pairs, selected expert j, token t): pair p = t * k + j
     extern __shared__ __align__(128) unsigned char smem[];
+    // Launched as a programmatic dependent of whatever precedes it in the stream (in a decode loop the previous layer
+    // call's down kernel, which releases its dependents when it starts): the CTAs are placed and wait here, so the
+    // launch latency is off the step; nothing is read or written before the wait.
+    grid_dependency_wait();
     grid_launch_dependents();
     if ((blockIdx.x | blockIdx.y | blockIdx.z) == 0) keep_pair_ids(sa);
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -871,6 +877,7 @@ __global__ void __launch_bounds__(256, 1)
 token_down_bulk_kernel(GemmArgs a, SmallArgs sa, const __nv_bfloat16* __restrict__ act, const float* __restrict__ topk_w,
                        int bpwg) {
     extern __shared__ __align__(128) unsigned char smem[];
+    grid_launch_dependents();                          // the next kernel in the stream may be placed (it waits for this one)
     const int K = a.I, KB = K / kGroup, k = a.top_k;                     // k <= 8: one warp per selected expert
     const uint32_t panel_bytes = (uint32_t)KB * kBlockBytes;
     const int x_stride = K * 2 + 64;
@@ -995,6 +1002,26 @@ token_down_bulk_kernel(GemmArgs a, SmallArgs sa, const __nv_bfloat16* __restrict
     if (!ok && tid == 0) drain_bar(bar, 0);
 }
 
+// launch with programmatic stream serialisation: the grid may be placed while its predecessor in the stream still runs
+// (once that has released its dependents); the kernel itself waits (griddepcontrol.wait) before it touches memory
+template <typename Kern, typename... Args>
+static void launch_pdl(Kern kern, dim3 grid, int block, size_t smem, cudaStream_t st, Args... args) {
+    cudaLaunchConfig_t lc{};
+    lc.gridDim = grid;
+    lc.blockDim = dim3(block);
+    lc.dynamicSmemBytes = smem;
+    lc.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    lc.attrs = attr;
+    lc.numAttrs = 1;
+#ifdef EXMOE_DISABLE_PDL
+    lc.numAttrs = 0;
+#endif
+    cudaLaunchKernelEx(&lc, kern, args...);
+}
+
 template <int NB>
 void launch_pair_gateup(const GemmArgs& a, const SmallArgs& sa, const __nv_bfloat16* hidden, __nv_bfloat16* act, int KS,
                         cudaStream_t st) {
@@ -1005,7 +1032,7 @@ void launch_pair_gateup(const GemmArgs& a, const SmallArgs& sa, const __nv_bfloa
     allow_smem(kern, 100 * 1024, smem_once);
     int ks_log2 = 0;
     while ((1 << ks_log2) < KS) ++ks_log2;
-    kern<<<dim3(tiles, a.top_k, sa.n_pairs / a.top_k), 256, smem, st>>>(a, sa, hidden, act, ks_log2);
+    launch_pdl(kern, dim3(tiles, a.top_k, sa.n_pairs / a.top_k), 256, smem, st, a, sa, hidden, act, ks_log2);
     count_launch();
 }
 
@@ -1024,7 +1051,8 @@ bool launch_pair_gateup_wide(const GemmArgs& a, const SmallArgs& sa, const __nv_
     const size_t smem = (size_t)kWideWarps * NB * kGroup * 2 + (size_t)kWideWarps * 32 * 4;
     static SmemOnce smem_once;
     allow_smem(kern, 100 * 1024, smem_once);
-    kern<<<dim3(a.I / (kPanelRows * PP), a.top_k, sa.n_pairs / a.top_k), 32 * kWideWarps, smem, st>>>(a, sa, hidden, act, ks_log2);
+    launch_pdl(kern, dim3(a.I / (kPanelRows * PP), a.top_k, sa.n_pairs / a.top_k), 32 * kWideWarps, smem, st, a, sa, hidden, act,
+               ks_log2);
     count_launch();
     return true;
 }
