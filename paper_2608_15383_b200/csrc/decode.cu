@@ -1131,6 +1131,7 @@ void launch_decode(const GemmArgs& a, const SmallArgs& sa, const __nv_bfloat16* 
 __global__ void __launch_bounds__(256)
 combine_kernel(const float* __restrict__ y, const int32_t* __restrict__ ids, int E, int T, int k, int H,
                __nv_bfloat16* __restrict__ out) {
+    grid_launch_dependents();                          // the next kernel in the stream may be placed (it waits for this one)
     const int per_row = H / 4;
     const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
     grid_dependency_wait();                            // launched as a programmatic dependent of the down kernel

@@ -297,6 +297,9 @@ group_small_kernel(const int32_t* __restrict__ ids, int n_pairs, int E, int C, i
     int* s_key = s_off + n_keys + 1;       // [n_pairs]
     __shared__ int s_bad;
     const int tid = threadIdx.x;
+    // launched as a programmatic dependent of whatever precedes it in the stream (in a decode loop the previous layer
+    // call's combine kernel): placed early, it waits here before it reads the ids
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     // a kernel launched behind this one as a programmatic dependent may be placed now; it waits for this grid's
     // completion before it reads the plan
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
@@ -514,7 +517,20 @@ void launch_group(const exmoe_shape& s, int C, int n_keys, int max_waves, bool i
         const size_t smem = (size_t)(2 * n_keys + 1 + n_pairs) * 4;
         static SmemOnce smem_once;
         allow_smem(group_small_kernel, 64 * 1024, smem_once);
-        group_small_kernel<<<1, 256, smem, st>>>(ids, n_pairs, E, C, n_keys, max_waves, identity, plan, d_status);
+        cudaLaunchConfig_t lc{};
+        lc.gridDim = dim3(1);
+        lc.blockDim = dim3(256);
+        lc.dynamicSmemBytes = smem;
+        lc.stream = st;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        lc.attrs = attr;
+        lc.numAttrs = 1;
+#ifdef EXMOE_DISABLE_PDL
+        lc.numAttrs = 0;
+#endif
+        cudaLaunchKernelEx(&lc, group_small_kernel, ids, n_pairs, E, C, n_keys, max_waves, identity, plan, d_status);
         count_launch();
         return;
     }
