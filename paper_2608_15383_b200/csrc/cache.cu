@@ -425,6 +425,7 @@ int exmoe_moe_forward(exmoe_cache* c, int layer, const void* hidden, const int32
     a.perm = c->plan.perm;
     a.key_miss = c->plan.key_miss;
     a.group_filter = 0;
+    a.direct_keys = (C == E && c->n_keys <= 128) ? c->n_keys : 0;
     a.num_slots = C;
     a.top_k = k;
     a.H = s.d_model;

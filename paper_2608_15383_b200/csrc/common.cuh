@@ -60,6 +60,9 @@ struct GemmArgs {
     const int32_t* perm;
     const int32_t* key_miss;    // [n_keys] (see PlanPtrs); may be null
     int group_filter;           // 0 all groups of the wave; 1 only groups whose expert was resident; 2 only the missed ones
+    int direct_keys;            // > 0: every key 0 .. direct_keys-1 is a (possibly empty) group of the call's only wave
+                                // (all experts resident, key = expert id): kernels may read counts / offsets by key at
+                                // once instead of going through wave_start and group_keys first
     int num_slots;              // C (key % C = slot)
     int top_k;
     int H, I;

@@ -197,12 +197,16 @@ stream_gemm_kernel(const StreamArgs p) {
         // This CTA's share of the wave's units, and the plan entries of the groups it touches (usually one or
         // two).  The plan entries of up to 32 * kScanChunks active groups are fetched in one go and kept in
         // registers for both steps (count the units; find the overlapping groups); beyond that they are re-read.
-        const int g0 = a.wave_start[0], n_groups = a.wave_start[1] - g0;
+        // With every expert resident the keys are the expert ids and the wave is the whole call: counts and offsets are
+        // then read by key at once (empty keys are empty groups), one round trip to L2 instead of three dependent ones
+        // (wave_start, then group_keys, then counts / offsets) before the first weight copy can be issued.
+        const bool direct = a.direct_keys > 0 && a.direct_keys <= 32 * kScanChunks;
+        const int g0 = direct ? 0 : a.wave_start[0], n_groups = direct ? a.direct_keys : a.wave_start[1] - g0;
         int rkey[kScanChunks], rrows[kScanChunks], rrow0[kScanChunks];
 #pragma unroll
         for (int j = 0; j < kScanChunks; ++j) {
             rkey[j] = 0;
-            if (32 * j + lane < n_groups) rkey[j] = a.group_keys[g0 + 32 * j + lane];
+            if (32 * j + lane < n_groups) rkey[j] = direct ? 32 * j + lane : a.group_keys[g0 + 32 * j + lane];
         }
 #pragma unroll
         for (int j = 0; j < kScanChunks; ++j) {
