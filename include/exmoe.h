@@ -118,7 +118,8 @@ int exmoe_cache_create(exmoe_cache** out, const exmoe_shape* shape, int num_laye
  * nothing and sets the sticky status EXMOE_ERR_BAD_EXPERT_ID (see exmoe_status).
  * C = E: fully asynchronous on `stream`.  C < E: see exmoe_cache_set_miss_path; with the default
  * device-initiated miss path the call is fully asynchronous on `stream` as well.
- * The call's first kernel is launched with programmatic stream serialisation: its blocks may be placed while the
+ * With all experts resident and T * k <= 2048 the call's first kernel (gate/up of the smallest calls, grouping of the
+ * others) is launched with programmatic stream serialisation: its blocks may be placed while the
  * kernel before it in `stream` still runs (if that kernel releases its dependents early, as this library's last
  * kernels do), but it reads and writes nothing before that kernel has completed: stream order holds for memory. */
 int exmoe_moe_forward(exmoe_cache* cache, int layer, const void* hidden_bf16, const int32_t* topk_ids,
