@@ -437,39 +437,30 @@ prefill_gemm_kernel(PrefillArgs a, const CUtensorMap* __restrict__ maps, __nv_bf
         PROF_REPORT("B producer");
     } else if (warp >= 8 && !(warp >= 16 && warp < 20)) {
         // ------------------------------------------------------------------ A producers (dequantise)
+        // A warp converts WHOLE packed blocks of one 16-row panel: both 64-wide halves, that is two consecutive ring
+        // stages, with the block's scales split once (converting one half per warp, each half's warp split the same
+        // scales and paid the loop's fixed instructions per 64 of K: these warps bound the kernel).  Warps 8-15 take
+        // the even blocks of the CTA's block stream, warps 20-27 the odd ones.
         const int pw = warp & 7;                                   // panel of the tile = 8-row groups 2*pw, 2*pw+1
-        const int hh = warp >= 20 ? 1 : 0;                         // 64-wide k-half of every block = every second stage
+        const int par = warp >= 20 ? 1 : 0;                        // parity of this warp's blocks in the CTA's block stream
         const int q = lane >> 2, c = lane & 3;
-        int s = hh % STAGES, ph = 0;                               // ring position of this warp's next stage (2 * blocks + hh)
         bool ok = true;
         PROF_DECL;
         // The conversion side needs nothing of a tile but its weights, so the warp walks ONE stream of blocks over all
-        // of the CTA's tiles, its loads two blocks ahead of the conversion ACROSS tile boundaries (a tile's first loads
-        // issued only when the tile began cost one memory latency per tile, 8 or 16 blocks).  The load cursor knows its
-        // tile's key one tile early, so entering a tile costs no dependent load either.
+        // of the CTA's tiles, its loads one of its blocks (two of the stream) ahead of the conversion ACROSS tile
+        // boundaries.  The load cursor knows its tile's key one tile early, so entering a tile costs no dependent load.
         const int my_tiles = blockIdx.x < total_tiles ? (total_tiles - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x : 0;
-        const int total_blocks = my_tiles * KB;
+        const int total_blocks = my_tiles * KB;                    // of the stream; this warp converts par, par + 2, ...
         auto panel_row = [&](int t, int key) -> const uint8_t* {
             const uint8_t* mat = a.slots + (size_t)(key % a.num_slots) * a.slot_stride + (GATEUP ? 0 : w13_bytes);
-            return mat + (size_t)((t % MT) * 8 + pw) * KB * kBlockBytes + hh * 512 + lane * 16;
+            return mat + (size_t)((t % MT) * 8 + pw) * KB * kBlockBytes + lane * 16;
         };
-        int c_t = blockIdx.x, c_kb = 0, issued = 0;                // load cursor: tile, block of it, blocks requested so far
+        int c_t = blockIdx.x, c_kb = par, c_g = par;               // load cursor: tile, block of it, index in the stream
         int c_key_next = 0;
         const uint8_t* c_pn = nullptr;
-        if (my_tiles) {
-            c_pn = panel_row(c_t, a.tiles[c_t / MT].key);
-            if (c_t + (int)gridDim.x < total_tiles) c_key_next = a.tiles[(c_t + gridDim.x) / MT].key;
-        }
-        constexpr int PF = 3;                                      // blocks in flight per lane (this one + 2 ahead)
-        uint4 w[PF];
-        uint32_t sc[PF];
-        auto fetch = [&](uint4& wv, uint32_t& sv) {                // request the cursor's block, move the cursor on
-            const uint8_t* blk = c_pn + (size_t)c_kb * kBlockBytes;
-            wv = ldg_stream128(blk);
-            sv = ldg_stream32(blk - (hh * 512 + lane * 16) + kCodeBytes + q * 4);
-            ++issued;
-            if (++c_kb == KB) {
-                c_kb = 0;
+        auto enter_tiles = [&]() {                                 // bring the cursor's block index back inside a tile
+            while (c_kb >= KB && c_t < total_tiles) {
+                c_kb -= KB;
                 c_t += gridDim.x;
                 if (c_t < total_tiles) {
                     c_pn = panel_row(c_t, c_key_next);
@@ -477,37 +468,59 @@ prefill_gemm_kernel(PrefillArgs a, const CUtensorMap* __restrict__ maps, __nv_bf
                 }
             }
         };
-#pragma unroll
-        for (int i = 0; i < PF - 1; ++i)
-            if (issued < total_blocks) fetch(w[i], sc[i]);
-        for (int g0 = 0; g0 < total_blocks && ok; g0 += PF) {
+        if (my_tiles) {
+            c_pn = panel_row(c_t, a.tiles[c_t / MT].key);
+            if (c_t + (int)gridDim.x < total_tiles) c_key_next = a.tiles[(c_t + gridDim.x) / MT].key;
+            enter_tiles();                                         // KB == 1 and par == 1: the first block is the next tile's
+        }
+        constexpr int PF = 2;                                      // blocks in flight per lane (this one + 1 ahead)
+        uint4 w[PF][2];
+        uint32_t sc[PF];
+        auto fetch = [&](uint4 (&wv)[2], uint32_t& sv) {           // request the cursor's block, move the cursor two on
+            const uint8_t* blk = c_pn + (size_t)c_kb * kBlockBytes;
+            wv[0] = ldg_stream128(blk);
+            wv[1] = ldg_stream128(blk + 512);
+            sv = ldg_stream32(blk - lane * 16 + kCodeBytes + q * 4);
+            c_g += 2;
+            c_kb += 2;
+            enter_tiles();
+        };
+        if (c_g < total_blocks) fetch(w[0], sc[0]);
+        // ring position of this warp's next stage: stage index of (block g, half h) = 2 g + h
+        int s = (2 * par) % STAGES, ph = ((2 * par) / STAGES) & 1;
+        for (int g0 = par; g0 < total_blocks && ok; g0 += 2 * PF) {
 #pragma unroll
             for (int u = 0; u < PF; ++u) {
-                if (g0 + u >= total_blocks) break;
-                if (issued < total_blocks) fetch(w[(u + PF - 1) % PF], sc[(u + PF - 1) % PF]);   // keep two blocks in flight
-                {
-                    PROF_WAIT_BEGIN;
-                    ok = mbar_wait(&empty[s], ph ^ 1, abort_flag, a.status);
-                    PROF_WAIT_END;
-                }
-                ok = __all_sync(0xffffffffu, ok);
-                if (!ok) break;
-                unsigned char* dst = sA + s * A_STAGE_BYTES;
+                if (g0 + 2 * u >= total_blocks) break;
+                if (c_g < total_blocks) fetch(w[(u + 1) % PF], sc[(u + 1) % PF]);       // keep one block in flight
                 const __half2 sh = *reinterpret_cast<const __half2*>(&sc[u]);
                 const ScaleSplit s_lo = split_scale(__low2float(sh));                 // row q
                 const ScaleSplit s_hi = split_scale(__high2float(sh));                // row q + 8
-                const uint32_t words[4] = {w[u].x, w[u].y, w[u].z, w[u].w};
 #pragma unroll
-                for (int wi = 0; wi < 4; ++wi) {
-                    const int r = wi & 1, set = wi >> 1;
-                    const int kc = 4 * set + c;                                       // 16-byte k-chunk of the stage
-                    const uint4 val = dequant_word(words[wi], r ? s_hi : s_lo);
-                    *reinterpret_cast<uint4*>(dst + (2 * pw + r) * A_SBO + kc * A_LBO + q * 16) = val;
+                for (int h = 0; h < 2; ++h) {                                         // the block's two halves = two stages
+                    {
+                        PROF_WAIT_BEGIN;
+                        ok = mbar_wait(&empty[s], ph ^ 1, abort_flag, a.status);
+                        PROF_WAIT_END;
+                    }
+                    ok = __all_sync(0xffffffffu, ok);
+                    if (!ok) break;
+                    unsigned char* dst = sA + s * A_STAGE_BYTES;
+                    const uint32_t words[4] = {w[u][h].x, w[u][h].y, w[u][h].z, w[u][h].w};
+#pragma unroll
+                    for (int wi = 0; wi < 4; ++wi) {
+                        const int r = wi & 1, set = wi >> 1;
+                        const int kc = 4 * set + c;                                   // 16-byte k-chunk of the stage
+                        const uint4 val = dequant_word(words[wi], r ? s_hi : s_lo);
+                        *reinterpret_cast<uint4*>(dst + (2 * pw + r) * A_SBO + kc * A_LBO + q * 16) = val;
+                    }
+                    fence_proxy_async();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(&full[s]);
+                    if (++s == STAGES) { s = 0; ph ^= 1; }
                 }
-                fence_proxy_async();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(&full[s]);
-                s += 2;                                            // this warp's next stage is two on
+                if (!ok) break;
+                s += 2;                                            // skip the other parity's block (two stages)
                 if (s >= STAGES) { s -= STAGES; ph ^= 1; }
             }
         }
