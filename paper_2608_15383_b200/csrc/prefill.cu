@@ -486,8 +486,24 @@ prefill_gemm_kernel(PrefillArgs a, const CUtensorMap* __restrict__ maps, __nv_bf
             enter_tiles();
         };
         if (c_g < total_blocks) fetch(w[0], sc[0]);
-        // ring position of this warp's next stage: stage index of (block g, half h) = 2 g + h
-        int s = (2 * par) % STAGES, ph = ((2 * par) / STAGES) & 1;
+        // Stage index of (block g, half h) = 2 g + h; this warp's blocks are g = par + 2 i, so the stage count is
+        // n = 2 par + 4 i + h.  With the ring depth a power of two (4 or 8) and the loop unrolled by two blocks, the ring
+        // position of (u = i mod 2, h) is loop-invariant: ((2 par + 4 u) mod STAGES) + h.  Store addresses and barrier
+        // addresses are therefore formed once, outside the loop (the address arithmetic of a run-time ring position was a
+        // tenth of this loop's instructions).
+        static_assert(STAGES == 4 || STAGES == 8, "ring positions of the conversion warps are precomputed for these depths");
+        constexpr int LOG_STAGES = STAGES == 4 ? 2 : 3;
+        unsigned char* stage_ptr[2];
+        uint64_t* full_ptr[2];
+        uint64_t* empty_ptr[2];
+#pragma unroll
+        for (int u = 0; u < 2; ++u) {
+            const int sb = (2 * par + 4 * u) & (STAGES - 1);
+            stage_ptr[u] = sA + sb * A_STAGE_BYTES + (2 * pw) * A_SBO + c * A_LBO + q * 16;
+            full_ptr[u] = &full[sb];
+            empty_ptr[u] = &empty[sb];
+        }
+        int n = 2 * par;                                           // stage count of the next block's first half
         for (int g0 = par; g0 < total_blocks && ok; g0 += 2 * PF) {
 #pragma unroll
             for (int u = 0; u < PF; ++u) {
@@ -496,32 +512,30 @@ prefill_gemm_kernel(PrefillArgs a, const CUtensorMap* __restrict__ maps, __nv_bf
                 const __half2 sh = *reinterpret_cast<const __half2*>(&sc[u]);
                 const ScaleSplit s_lo = split_scale(__low2float(sh));                 // row q
                 const ScaleSplit s_hi = split_scale(__high2float(sh));                // row q + 8
+                const uint32_t ph = (n >> LOG_STAGES) & 1;                            // the same for both halves
 #pragma unroll
                 for (int h = 0; h < 2; ++h) {                                         // the block's two halves = two stages
                     {
                         PROF_WAIT_BEGIN;
-                        ok = mbar_wait(&empty[s], ph ^ 1, abort_flag, a.status);
+                        ok = mbar_wait(empty_ptr[u] + h, ph ^ 1, abort_flag, a.status);
                         PROF_WAIT_END;
                     }
                     ok = __all_sync(0xffffffffu, ok);
                     if (!ok) break;
-                    unsigned char* dst = sA + s * A_STAGE_BYTES;
+                    unsigned char* dst = stage_ptr[u] + h * A_STAGE_BYTES;
                     const uint32_t words[4] = {w[u][h].x, w[u][h].y, w[u][h].z, w[u][h].w};
 #pragma unroll
                     for (int wi = 0; wi < 4; ++wi) {
                         const int r = wi & 1, set = wi >> 1;
-                        const int kc = 4 * set + c;                                   // 16-byte k-chunk of the stage
                         const uint4 val = dequant_word(words[wi], r ? s_hi : s_lo);
-                        *reinterpret_cast<uint4*>(dst + (2 * pw + r) * A_SBO + kc * A_LBO + q * 16) = val;
+                        *reinterpret_cast<uint4*>(dst + r * A_SBO + 4 * set * A_LBO) = val;   // k-chunk 4 set + c of row group 2 pw + r
                     }
                     fence_proxy_async();
                     __syncwarp();
-                    if (lane == 0) mbar_arrive(&full[s]);
-                    if (++s == STAGES) { s = 0; ph ^= 1; }
+                    if (lane == 0) mbar_arrive(full_ptr[u] + h);
                 }
                 if (!ok) break;
-                s += 2;                                            // skip the other parity's block (two stages)
-                if (s >= STAGES) { s -= STAGES; ph ^= 1; }
+                n += 4;
             }
         }
         PROF_REPORT("A producer");
