@@ -50,7 +50,7 @@ WORKLOADS = {
 # (bytes, kernel captured, date of the capture)
 NCU_TRAFFIC = {"decode": (17.33e6, "pair_gateup_wide_kernel<4>, T=1", "2026-11-25"),
                "decode16": (62.83e6 + 0.87e6, "stream_gemm_kernel<1,true,1>, T=16", "2026-11-25"),
-               "prefill": (212.95e6 + 12.03e6, "prefill_gemm_kernel<true,256,4>, T=2048", "2026-11-25")}
+               "prefill": (215.63e6 + 11.33e6, "prefill_gemm_kernel<true,256,4>, T=2048", "2026-11-25")}
 METRIC = "moe_layer_tokens_per_s"
 UNIT = "tokens/s"
 
